@@ -1,0 +1,203 @@
+"""Seeded synthetic inputs for the integer-only encoder layer.
+
+This module only *makes inputs*: random tensors of the shapes and
+distributions the workloads call for, quantized once to integers with
+Eq. 1 (uniform symmetric, ``S = alpha / (2^(b-1) - 1)``), and the static
+activation scales of a layer (Sec. 3.1: fixed offline).  None of the
+method's integer arithmetic (requantization, i-exp, i-GELU, i-LayerNorm)
+lives here, so the CPU oracle and the CUDA path can both be fed from it.
+
+Generators are ``numpy.random.Generator(PCG64(seed))`` with
+``seed = 21010000 + 1000*config + 10*layer + tensor_id``.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+
+import numpy as np
+
+SEED_BASE = 21010000
+
+# tensor ids inside one layer
+_T_X, _T_WQKV, _T_BQKV, _T_WO, _T_BO, _T_WF1, _T_BF1, _T_WF2, _T_BF2 = range(9)
+# gamma1, beta1, gamma2, beta2 share id 9 (drawn in that order from one stream)
+_T_LN = 9
+
+
+@dataclass(frozen=True)
+class ModelConfig:
+    name: str
+    H: int
+    heads: int
+    F: int
+    layers: int
+    L: int
+    config_id: int
+
+
+CONFIGS = {
+    0: ModelConfig("roberta-base-1layer", 768, 12, 3072, 1, 128, 0),
+    2: ModelConfig("roberta-base-12layer", 768, 12, 3072, 12, 128, 2),
+    3: ModelConfig("roberta-large-24layer-L256", 1024, 16, 4096, 24, 256, 3),
+    4: ModelConfig("roberta-large-24layer-L512", 1024, 16, 4096, 24, 512, 4),
+}
+
+
+def rng_for(config_id: int, layer: int, tensor_id: int) -> np.random.Generator:
+    return np.random.Generator(np.random.PCG64(SEED_BASE + 1000 * config_id + 10 * layer + tensor_id))
+
+
+def quantize_sym(x: np.ndarray, S, qmax: int) -> np.ndarray:
+    """Eq. 1 with Int = round-to-nearest-even and clip to +-qmax."""
+    return np.clip(np.rint(x / S), -qmax, qmax)
+
+
+def _quantize_weight(rng: np.random.Generator, n_out: int, n_in: int, std: float = 0.02):
+    """W ~ N(0, std^2), per-output-channel symmetric int8."""
+    W = rng.standard_normal((n_out, n_in), dtype=np.float32).astype(np.float64) * std
+    S_w = np.abs(W).max(axis=1) / 127.0
+    w = quantize_sym(W, S_w[:, None], 127).astype(np.int8)
+    return w, S_w
+
+
+def _quantize_bias(rng: np.random.Generator, S_x: float, S_w: np.ndarray, std: float = 0.02):
+    """float bias ~ N(0, std^2) held as int32 at scale S_x * S_w[n]."""
+    bias = rng.standard_normal(S_w.shape[0]) * std
+    return np.rint(bias / (S_x * S_w)).astype(np.int32)
+
+
+def _gelu_second_moment(sigma: float) -> float:
+    """E[GELU(z)^2] for z ~ N(0, sigma^2), by a plain Riemann sum."""
+    z = np.linspace(-8.0 * sigma, 8.0 * sigma, 20001)
+    erf = np.vectorize(math.erf)
+    g = z * 0.5 * (1.0 + erf(z / math.sqrt(2.0)))
+    pdf = np.exp(-0.5 * (z / sigma) ** 2) / (sigma * math.sqrt(2.0 * math.pi))
+    return float(np.sum(g * g * pdf) * (z[1] - z[0]))
+
+
+def static_activation_scales(H: int, F: int, L: int, S_x: float, w_std: float = 0.02) -> dict:
+    """The 11 static activation scales of a layer, from the input distributions.
+
+    The layer input has (close to) unit variance -- N(0,1) for the first
+    layer, a LayerNorm output with gamma ~ N(1, 0.1^2), beta ~ N(0, 0.1^2)
+    afterwards -- so every site's standard deviation follows from the weight
+    distribution.  int8 sites clip at 4 (context: 5) standard deviations,
+    Q16 sites (held in int32) at 8.
+    """
+    ln_var = 1.0 * (1.0 + 0.1 ** 2) + 0.1 ** 2            # E[(gamma n + beta)^2], n ~ N(0,1)
+    sd_qkv = w_std * math.sqrt(H * 1.0 + 1.0)
+    sd_ctx = w_std * math.sqrt(H / L + 1.0)                # ~ mean of L value rows (+ bias)
+    sd_o = w_std * math.sqrt(H * sd_ctx ** 2 + 1.0)
+    sd_f1 = w_std * math.sqrt(H * ln_var + 1.0)
+    sd_f2 = w_std * math.sqrt(F * _gelu_second_moment(sd_f1) + 1.0)
+    s = {
+        "S_x": float(S_x),
+        "S_q": 4.0 * sd_qkv / 127.0,
+        "S_k": 4.0 * sd_qkv / 127.0,
+        "S_v": 4.0 * sd_qkv / 127.0,
+        "S_ctx": 5.0 * sd_ctx / 127.0,
+        "S_r1": 8.0 * math.sqrt(ln_var + sd_o ** 2) / 32767.0,
+        "S_h1": 4.0 * math.sqrt(ln_var) / 127.0,
+        "S_gi": 8.0 * sd_f1 / 32767.0,
+        "S_go": 4.0 * sd_f1 / 127.0,
+        "S_r2": 8.0 * math.sqrt(ln_var + sd_f2 ** 2) / 32767.0,
+        "S_out": 4.0 * math.sqrt(ln_var) / 127.0,
+    }
+    return s
+
+
+def make_input(config_id: int, B: int, L: int, H: int):
+    """x ~ N(0,1) as int8 with S_x = max|x| / 127.  Returns (x_q [B*L, H], S_x)."""
+    rng = rng_for(config_id, 0, _T_X)
+    x = rng.standard_normal((B * L, H), dtype=np.float32).astype(np.float64)
+    S_x = float(np.abs(x).max() / 127.0)
+    return quantize_sym(x, S_x, 127).astype(np.int8), S_x
+
+
+def make_layer(config_id: int, layer: int, H: int, heads: int, F: int, L: int, S_x: float,
+               p_max: int = 255) -> dict:
+    """One layer's integer parameters and static scales (a plain dict of numpy arrays)."""
+    assert H == heads * 64
+    p = {"H": H, "heads": heads, "F": F, "p_max": p_max}
+    p.update(static_activation_scales(H, F, L, S_x))
+    in_scale = {"qkv": p["S_x"], "o": p["S_ctx"], "f1": p["S_h1"], "f2": p["S_go"]}
+    shapes = {"qkv": (3 * H, H), "o": (H, H), "f1": (F, H), "f2": (H, F)}
+    tids = {"qkv": (_T_WQKV, _T_BQKV), "o": (_T_WO, _T_BO), "f1": (_T_WF1, _T_BF1), "f2": (_T_WF2, _T_BF2)}
+    for nm in ("qkv", "o", "f1", "f2"):
+        w, S_w = _quantize_weight(rng_for(config_id, layer, tids[nm][0]), *shapes[nm])
+        p[f"w_{nm}"] = w
+        p[f"S_w_{nm}"] = S_w
+        p[f"bias_{nm}"] = _quantize_bias(rng_for(config_id, layer, tids[nm][1]), in_scale[nm], S_w)
+    rng = rng_for(config_id, layer, _T_LN)
+    p["gamma1"] = 1.0 + 0.1 * rng.standard_normal(H)
+    p["beta1"] = 0.1 * rng.standard_normal(H)
+    p["gamma2"] = 1.0 + 0.1 * rng.standard_normal(H)
+    p["beta2"] = 0.1 * rng.standard_normal(H)
+    return p
+
+
+def make_model(config_id: int, B: int, layers: int | None = None, H: int | None = None,
+               heads: int | None = None, F: int | None = None, L: int | None = None):
+    """Input and per-layer parameters of one of the encoder configs (0, 2, 3, 4).
+    Layer l+1 consumes layer l's int8 output, so its S_x is layer l's S_out."""
+    cfg = CONFIGS[config_id]
+    H = H or cfg.H
+    heads = heads or cfg.heads
+    F = F or cfg.F
+    L = L or cfg.L
+    layers = layers or cfg.layers
+    x, S_x = make_input(config_id, B, L, H)
+    params = []
+    s_in = S_x
+    for l in range(layers):
+        p = make_layer(config_id, l, H, heads, F, L, s_in)
+        params.append(p)
+        s_in = p["S_out"]
+    return x, params
+
+
+# ---------------------------------------------------------------------------
+# standalone non-linearity sweeps (config 1)
+# ---------------------------------------------------------------------------
+
+def gelu_inputs(n: int, sigma: float, tensor_id: int = 0):
+    """x ~ N(0, sigma^2) as Q16 held in int32; S = max|x|/32767, S_out = max|x|/127."""
+    rng = rng_for(1, 0, tensor_id)
+    x = rng.standard_normal(n, dtype=np.float32).astype(np.float64) * sigma
+    amax = float(np.abs(x).max())
+    S = amax / 32767.0
+    return quantize_sym(x, S, 32767).astype(np.int32), S, amax / 127.0
+
+
+def softmax_inputs(rows: int, L: int, sigma: float, tensor_id: int = 1):
+    """score-like int32 rows: x ~ N(0, sigma^2), S = sigma/16384 (|q| up to ~2^17)."""
+    rng = rng_for(1, 1, tensor_id)
+    x = rng.standard_normal((rows, L), dtype=np.float32).astype(np.float64) * sigma
+    S = sigma / 16384.0
+    return np.rint(x / S).astype(np.int32), S
+
+
+def layernorm_inputs(rows: int, C: int, sigma: float, tensor_id: int = 2, with_residual: bool = True):
+    """Q16 rows with a per-row offset, an int8 residual, gamma/beta and an output scale.
+
+    x ~ N(0, sigma^2) + row offset N(0, (sigma/2)^2); S = max|x|/32767.
+    The residual is N(0, (sigma/4)^2) as int8.  S_out covers 4.5 standard
+    deviations of the normalized, affine-transformed output.
+    """
+    rng = rng_for(1, 2, tensor_id)
+    x = rng.standard_normal((rows, C), dtype=np.float32).astype(np.float64) * sigma
+    x += rng.standard_normal((rows, 1)) * (sigma / 2.0)
+    gamma = 1.0 + 0.1 * rng.standard_normal(C)
+    beta = 0.1 * rng.standard_normal(C)
+    r = S_r = None
+    total = x
+    if with_residual:
+        res = rng.standard_normal((rows, C), dtype=np.float32).astype(np.float64) * (sigma / 4.0)
+        S_r = float(np.abs(res).max() / 127.0)
+        r = quantize_sym(res, S_r, 127).astype(np.int8)
+        total = x + res
+    S = float(np.abs(total).max() / 32767.0)
+    q = quantize_sym(x, S, 32767).astype(np.int32)
+    S_out = 4.5 * math.sqrt(1.0 * (1.0 + 0.1 ** 2) + 0.1 ** 2) / 127.0
+    return q, S, r, S_r, gamma, beta, S_out

@@ -1,0 +1,132 @@
+"""Pins for the oracle's i-exp and i-softmax (Algorithm 3, Eq. 11-15)."""
+import math
+import random
+from fractions import Fraction
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLD = {}
+for line in (Path(__file__).parent / "golden" / "paper_values.txt").read_text().splitlines():
+    if "=" in line and not line.startswith("#"):
+        k, v = line.split("#")[0].split("=")
+        GOLD[k.strip()] = float(v)
+
+# The paper states 1.9e-3 (Sec. 3.5); its printed 4-digit coefficients of Eq. 14
+# give 2.13e-3 in real arithmetic, so the bound used here is 2.2e-3 plus one
+# input step S' for the integer floors.
+IEXP_TOL = 2.2e-3
+
+
+def test_paper_gap_figure_vs_printed_coefficients():
+    a, b, c = GOLD["exp_a"], GOLD["exp_b"], GOLD["exp_c"]
+    p = np.linspace(-math.log(2.0), 0.0, 200001)
+    gap = np.abs(a * (p + b) ** 2 + c - np.exp(p)).max()
+    assert GOLD["iexp_max_gap"] < gap < IEXP_TOL      # 2.128e-3, not 1.9e-3
+    assert abs(gap - 2.128e-3) < 2e-6
+
+
+@pytest.mark.parametrize("S", [1e-8, 3.3e-7, 2e-5, 4.5e-5, 1e-4, 1e-3, 1e-2, 2e-2])
+def test_iexp_tracks_exp_within_the_paper_gap(S):
+    k = oracle.exp_consts(S)
+    Sp = S * 2 ** k["s_in"]
+    # dense near 0, then out to where exp underflows the fixed-point grid
+    d = np.unique(np.concatenate([
+        np.arange(0, min(int(40.0 / S), 200000)),
+        (np.linspace(0.0, 25.0, 100001) / S).astype(np.int64)]))
+    e, S_e = oracle.iexp(-d, S)
+    err = np.abs(e * S_e - np.exp(-d * S))
+    assert err.max() <= IEXP_TOL + Sp
+    # value at zero is the polynomial's L(0) = 1.00027...
+    assert 0.9995 - Sp <= e[0] * S_e <= 1.0005 + Sp
+    # non-increasing inside each halving interval; where z steps, Eq. 14's L(0)/2 sits
+    # 4.2e-5 above L(-ln2), so a rise of at most that much (plus a floor) is the polynomial's own
+    assert (np.diff(e) * S_e <= 5e-5 + S_e).all()
+    inside = np.diff((d >> k["s_in"]) // k["q_ln2"]) == 0
+    assert (np.diff(e)[inside] <= 0).all()
+    # never negative, and 21-bit
+    assert e.min() >= 0 and e.max() < 2 ** 21
+
+
+def test_iexp_is_exactly_zero_beyond_31_halvings():
+    for S in (1e-3, 4.5e-5):
+        k = oracle.exp_consts(S)
+        far = -(31 * k["q_ln2"] << k["s_in"])
+        e, _ = oracle.iexp(np.array([far, far - 12345, -2 ** 31, -2 ** 32 + 1]), S)
+        assert (e == 0).all()
+
+
+def test_exp_constants_follow_algorithm_1():
+    for S in (1e-3, 4.5e-5, 2e-5, 7e-2):
+        k = oracle.exp_consts(S)
+        Sp = S * 2 ** k["s_in"]
+        assert k["q_b"] <= 32767 and (k["s_in"] == 0 or math.floor(1.353 / (Sp / 2)) > 32767)
+        assert k["q_ln2"] == math.floor(math.log(2.0) / Sp)
+        assert k["q_b"] == math.floor(1.353 / Sp)
+        assert abs(k["q_c"] - 0.344 / (0.3585 * Sp * Sp)) < 1.0 + 1e-6 * k["q_c"]
+        assert k["e_top"] == k["q_b"] ** 2 + k["q_c"] < 2 ** 31
+        assert (k["e_top"] >> k["s_out"]) < 2 ** 21
+        assert k["s_out"] == 0 or (k["e_top"] >> (k["s_out"] - 1)) >= 2 ** 21
+    with pytest.raises(oracle.OracleError):
+        oracle.exp_consts(0.7)          # q_ln2 would be 0
+    with pytest.raises(oracle.OracleError):
+        oracle.exp_consts(-1.0)
+
+
+def _float_softmax(x):
+    x = x - x.max(axis=-1, keepdims=True)
+    e = np.exp(x)
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+@pytest.mark.parametrize("L,sigma,M", [(128, 1.0, 255), (512, 1.0, 255), (128, 4.0, 255),
+                                       (37, 4.0, 127), (1, 1.0, 255), (1024, 2.0, 255)])
+def test_softmax_rows_sum_to_fixed_point_one_and_track_float_softmax(L, sigma, M):
+    rng = np.random.default_rng(10 + L)
+    S = sigma / 16384.0
+    q = np.rint(rng.standard_normal((64, L)) * sigma / S).astype(np.int32)
+    p, S_p = oracle.softmax(q, S, M)
+    assert S_p == 1.0 / M
+    sums = p.astype(np.int64).sum(axis=1)
+    # floor division loses less than one unit per element
+    assert (sums <= M).all() and (sums > M - L).all()
+    ref = _float_softmax(q.astype(np.float64) * S)
+    assert np.abs(p * S_p - ref).max() <= 1.0 / M + 3e-3
+    # a larger score never loses more than one step (the polynomial pieces meet 4.2e-5 apart)
+    order = np.argsort(q, axis=1)
+    assert (np.diff(np.take_along_axis(p.astype(np.int64), order, axis=1), axis=1) >= -1).all()
+
+
+def test_softmax_equal_scores_and_one_hot_rows():
+    p, _ = oracle.softmax(np.full((1, 4), 7), 1e-3, 255)
+    assert p.tolist() == [[63, 63, 63, 63]]                 # floor(255/4), sum in (251, 255]
+    q = np.array([[0, -10 ** 6, -10 ** 6, -2 * 10 ** 9]], dtype=np.int64).clip(-2 ** 31, 2 ** 31 - 1)
+    p, _ = oracle.softmax(q, 1e-3, 255)
+    assert p.tolist() == [[255, 0, 0, 0]]
+    p, _ = oracle.softmax(np.array([[2 ** 31 - 1, -2 ** 31]]), 1e-3, 127)
+    assert p.tolist() == [[127, 0]]
+
+
+def test_softmax_brute_force_length_two_against_exact_rationals():
+    # every pair on a grid: p = floor(e * M / (e0 + e1)) in exact rationals, e from i-exp
+    S = 5e-3
+    grid = np.arange(-700, 1, 7)
+    e_of, _ = oracle.iexp(grid, S)
+    lut = dict(zip(grid.tolist(), e_of.tolist()))
+    rows = np.array([[0, g] for g in grid.tolist()] + [[g, 0] for g in grid.tolist()])
+    for M in (255, 127):
+        p, _ = oracle.softmax(rows + 12345, S, M)     # softmax is shift invariant
+        for (a, b), (pa, pb) in zip(rows.tolist(), p.tolist()):
+            ea, eb = lut[a], lut[b]
+            assert pa == math.floor(Fraction(ea * M, ea + eb))
+            assert pb == math.floor(Fraction(eb * M, ea + eb))
+
+
+def test_softmax_argument_checks():
+    with pytest.raises(oracle.OracleError):
+        oracle.softmax(np.zeros((1, 1025), np.int32), 1e-3, 255)
+    with pytest.raises(oracle.OracleError):
+        oracle.softmax(np.zeros((1, 8), np.int32), 1e-3, 200)

@@ -1,0 +1,143 @@
+/*
+ * ibert.h -- C ABI of the B200 (sm_100a) integer-only Transformer encoder layer
+ * of I-BERT (Kim et al., "I-BERT: Integer-only BERT Quantization").
+ *
+ * Every call takes quantized tensors in the paper's (q, S) convention
+ * (Sec. 3.1: real value = S * q, S fixed offline) and returns (q', S').
+ * Kernels never see a scale: the host turns scales into integer constants
+ * before the launch (static quantization; footnote of Algorithm 1).
+ *
+ * General rules
+ *   - Tensor pointers are DEVICE pointers owned by the caller, 16-byte
+ *     aligned, row-major and contiguous unless stated otherwise.
+ *     Scale arrays, gamma/beta and everything inside ibert_layer_desc are
+ *     HOST pointers, read during the call and not retained.
+ *   - Work is enqueued on the stream given to ibert_create(); calls return
+ *     without synchronizing (ibert_last_status() synchronizes).
+ *   - Every function returns IBERT_OK (0) or a negative IBERT_ERR_* code;
+ *     nothing throws, aborts, or falls back to a CPU path.  Invalid
+ *     arguments are rejected on the host before anything is launched.
+ *   - Device-side waits are bounded; if one expires the kernel records
+ *     IBERT_ERR_TIMEOUT in the context's status word and returns normally.
+ *   - Value formats: "int8" = [-127,127] in int8_t; "Q16" = [-32767,32767]
+ *     in an int32_t container; "u8" = [0,255] in uint8_t.
+ *   - Requantization (Appendix C.1, dyadic form b / 2^c):
+ *       requant(v; b, c, qmax) = clamp((v*b + (c>0 ? 2^(c-1) : 0)) >> c, +-qmax)
+ *     with the product in 64 bits, >> arithmetic, 0 <= c <= 31, |b| < 2^31.
+ */
+#ifndef IBERT_H_
+#define IBERT_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define IBERT_OK 0
+#define IBERT_ERR_ARG (-1)         /* null pointer, bad enum, negative size      */
+#define IBERT_ERR_SHAPE (-2)       /* size outside the supported range           */
+#define IBERT_ERR_SCALE_RANGE (-3) /* scale not finite/positive or not dyadic-representable */
+#define IBERT_ERR_ALIGN (-4)       /* pointer or row pitch not 16-byte aligned   */
+#define IBERT_ERR_NOMEM (-5)       /* device or host allocation failed           */
+#define IBERT_ERR_CUDA (-6)        /* a CUDA runtime / driver call failed        */
+#define IBERT_ERR_TIMEOUT (-7)     /* a bounded device-side wait expired         */
+#define IBERT_ERR_VALUE_RANGE (-8) /* an integer left the range the method assumes */
+
+typedef struct ibert_ctx ibert_ctx;     /* device, stream, workspace, status word        */
+typedef struct ibert_layer ibert_layer; /* one layer's device-resident integer parameters */
+
+/* Creates a context on `device` that launches on `cuda_stream` (a cudaStream_t; NULL =
+   the legacy default stream).  The context owns a small device status word and caches of
+   derived constant tables. */
+int ibert_create(ibert_ctx** out, int device, void* cuda_stream);
+int ibert_destroy(ibert_ctx* ctx);
+/* Synchronizes the context's stream and returns the first device-side error recorded since
+   the last call (IBERT_OK if none), or IBERT_ERR_CUDA if the stream is in error. */
+int ibert_last_status(ibert_ctx* ctx);
+const char* ibert_strerror(int code);
+
+/* Host, pure.  Real multiplier m -> (b, c) with m ~= b / 2^c (Appendix C.1; the dyadic
+   form of the cited requantization scheme): c = min(31, 31 - exponent(m)),
+   b = round-half-up(|m| * 2^c) with the sign of m, renormalized if it reaches 2^31.
+   IBERT_ERR_SCALE_RANGE if |m| >= 2^31 or m is not finite. */
+int ibert_dyadic_from_double(double m, int32_t* b, int32_t* c);
+
+/* INT8 MatMul with INT32 accumulation (Sec. 2, Appendix C.1), bias add and requantization:
+     acc[m,n] = sum_k x[m,k] * w[n,k] + bias[n];   out = requant(acc; dyadic(S_x*S_w[n]/S_out))
+   x [M,K] int8, w [N,K] int8 (K contiguous), bias [N] int32 at scale S_x*S_w[n] (may be NULL),
+   S_w host array [N] (per-output-channel weight scales).
+   out_kind 0: out is int8 [M,N] at S_out;  1: out is Q16 in int32 [M,N] at S_out;
+            2: out is the raw int32 accumulators (S_out ignored).
+   S_ret (host, may be NULL): receives S_out (kinds 0, 1: one entry) or S_x*S_w[n] (kind 2: N entries).
+   Requires K % 16 == 0, N % 16 == 0 (kinds 0) / N % 4 == 0 (kinds 1, 2), K*127*127 + |bias| < 2^31. */
+int ibert_linear_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
+                    const int32_t* bias, int64_t M, int N, int K, int out_kind, double S_out,
+                    void* out, double* S_ret);
+
+/* Same product followed by i-GELU (Algorithm 2) in the epilogue -- the FFN1 step:
+   acc -> Q16 at S_mid -> i-GELU -> int8 at S_out.  out is int8 [M,N]. */
+int ibert_linear_gelu_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
+                         const int32_t* bias, int64_t M, int N, int K, double S_mid, double S_out,
+                         int8_t* out, double* S_ret);
+
+/* i-softmax (Algorithm 3, Eq. 11-15) over rows of length L of int32 scores q at scale S:
+   row max, i-exp (shift decomposition + 2nd-order polynomial), int32 row sum, fixed-point
+   quotient p = floor(e * p_max / sum).  out is u8 [rows, L]; *S_ret = 1/p_max.
+   L in [1,1024]; p_max in {255,127}; S <= ln 2 (else IBERT_ERR_SCALE_RANGE). */
+int ibert_softmax_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
+                    uint8_t* out, double* S_ret);
+
+/* i-GELU (Algorithm 2, Eq. 8-9), elementwise.  q int32 at scale S, clamped to Q16 first;
+   out int8 at S_out (the product q*(q_erf+q_1) is requantized in-kernel); *S_ret = S_out. */
+int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
+                 double* S_ret);
+
+/* Residual add + i-LayerNorm (Sec. 3.6, Eq. 16, Algorithm 4) over rows of C channels:
+     v = q + requant(r; dyadic(S_r/S)) (r may be NULL), mu = floor(sum v / C),
+     sigma = max(ISqrt(floor(sum (v-mu)^2 / C)), 1), normalized, scaled by gamma, shifted by beta,
+     requantized to int8 at S_out.
+   q int32 [rows,C] at S (Q16-range values; |v| <= 2^20 is a documented, unchecked precondition),
+   r int8 [rows,C] at S_r, gamma/beta host double[C].  C in [1,2047].  *S_ret = S_out. */
+int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* r, double S_r,
+                      const double* gamma, const double* beta, int64_t rows, int C, double S_out,
+                      int8_t* out, double* S_ret);
+
+/* Multi-head self-attention on int8 Q|K|V (Fig. 1 right: MatMul -> i-softmax -> MatMul):
+   per (batch, head): s = Q K^T (int32, scale S_q*S_k/8, head size 64), p = i-softmax(s) in u8
+   (p_max = 255) or 7-bit (p_max = 127), ctx = requant(p V; dyadic((1/p_max)*S_v/S_ctx)).
+   qkv int8 [B*L, 3H] with column blocks Q | K | V, head j at columns 64j..64j+63 of each block;
+   ctx int8 [B*L, H].  Scores never leave the SM.  L in [1,512], H = 64*heads. */
+int ibert_attention_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads, double S_q,
+                       double S_k, double S_v, double S_ctx, int p_max, int8_t* out, double* S_ret);
+
+/* One encoder layer's parameters; every pointer is a HOST pointer (copied at create). */
+typedef struct ibert_layer_desc {
+  int32_t H, heads, F, p_max;                 /* H = 64*heads; p_max in {255,127} */
+  const int8_t* w_qkv; const double* S_w_qkv; const int32_t* bias_qkv; /* [3H,H], [3H], [3H] */
+  const int8_t* w_o;   const double* S_w_o;   const int32_t* bias_o;   /* [H,H],  [H],  [H]  */
+  const int8_t* w_f1;  const double* S_w_f1;  const int32_t* bias_f1;  /* [F,H],  [F],  [F]  */
+  const int8_t* w_f2;  const double* S_w_f2;  const int32_t* bias_f2;  /* [H,F],  [H],  [H]  */
+  const double* gamma1; const double* beta1;  /* [H] LayerNorm after attention */
+  const double* gamma2; const double* beta2;  /* [H] LayerNorm after the FFN   */
+  /* static activation scales: layer input, Q, K, V, context, first residual sum (Q16),
+     LayerNorm-1 output, GELU input (Q16), GELU output, second residual sum (Q16), output */
+  double S_x, S_q, S_k, S_v, S_ctx, S_r1, S_h1, S_gi, S_go, S_r2, S_out;
+} ibert_layer_desc;
+
+/* Uploads the parameters and precomputes every integer constant of the layer. */
+int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* desc, ibert_layer** out);
+int ibert_layer_destroy(ibert_layer* layer);
+
+/* The integer-only encoder layer (Fig. 1 right; post-LN order):
+   QKV projection -> attention (i-softmax) -> output projection -> +x, i-LayerNorm ->
+   FFN1 + i-GELU -> FFN2 -> +h1, i-LayerNorm.  x, out: int8 [B*L, H]; x at desc.S_x,
+   out at desc.S_out (*S_ret).  Intermediates live in the context's workspace, which grows
+   on demand (first call with a larger B*L allocates). */
+int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* layer, const int8_t* x, int B, int L,
+                        int8_t* out, double* S_ret);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IBERT_H_ */

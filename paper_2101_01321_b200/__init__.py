@@ -1,0 +1,1 @@
+"""B200-native integer-only Transformer encoder layer (I-BERT): C-ABI library + thin binding."""

@@ -1,0 +1,248 @@
+"""Thin ctypes binding of libibert_b200.so: same names as the C ABI (``include/ibert.h``),
+argument marshalling only.  Tensors are torch CUDA tensors whose ``data_ptr()`` is passed
+through; every step of the computation runs in the library's CUDA kernels.  There is no
+CPU path: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import numpy as np
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libibert_b200.so"
+_lib = None
+
+IBERT_OK = 0
+ERR_NAMES = {-1: "IBERT_ERR_ARG", -2: "IBERT_ERR_SHAPE", -3: "IBERT_ERR_SCALE_RANGE", -4: "IBERT_ERR_ALIGN",
+             -5: "IBERT_ERR_NOMEM", -6: "IBERT_ERR_CUDA", -7: "IBERT_ERR_TIMEOUT", -8: "IBERT_ERR_VALUE_RANGE"}
+
+SCALE_NAMES = ("S_x", "S_q", "S_k", "S_v", "S_ctx", "S_r1", "S_h1", "S_gi", "S_go", "S_r2", "S_out")
+
+
+class IbertError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        msg = lib().ibert_strerror(code).decode() if _lib is not None else "?"
+        super().__init__(f"{where}: {ERR_NAMES.get(code, code)} ({msg})")
+        self.code = code
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("H", C.c_int32), ("heads", C.c_int32), ("F", C.c_int32), ("p_max", C.c_int32)] + [
+        (n, C.c_void_p) for n in (
+            "w_qkv", "S_w_qkv", "bias_qkv", "w_o", "S_w_o", "bias_o",
+            "w_f1", "S_w_f1", "bias_f1", "w_f2", "S_w_f2", "bias_f2",
+            "gamma1", "beta1", "gamma2", "beta2")] + [(n, C.c_double) for n in SCALE_NAMES]
+
+
+def lib():
+    """Loads the C-ABI library; fails loudly if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2101_01321_b200.build` "
+                               "(there is no fallback path)")
+        L = C.CDLL(str(LIB_PATH))
+        vp, i32, i64, dbl = C.c_void_p, C.c_int, C.c_int64, C.c_double
+        L.ibert_strerror.restype = C.c_char_p
+        L.ibert_strerror.argtypes = [i32]
+        L.ibert_create.argtypes = [C.POINTER(vp), i32, vp]
+        L.ibert_destroy.argtypes = [vp]
+        L.ibert_last_status.argtypes = [vp]
+        L.ibert_dyadic_from_double.argtypes = [dbl, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.ibert_linear_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, i32, dbl, vp, vp]
+        L.ibert_linear_gelu_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, dbl, vp, vp]
+        L.ibert_softmax_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
+        L.ibert_gelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
+        L.ibert_layernorm_i.argtypes = [vp, vp, dbl, vp, dbl, vp, vp, i64, i32, dbl, vp, vp]
+        L.ibert_attention_i8.argtypes = [vp, vp, i32, i32, i32, i32, dbl, dbl, dbl, dbl, i32, vp, vp]
+        L.ibert_layer_create.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(vp)]
+        L.ibert_layer_destroy.argtypes = [vp]
+        L.ibert_encoder_layer.argtypes = [vp, vp, vp, i32, i32, vp, vp]
+        for name in ("ibert_create", "ibert_destroy", "ibert_last_status", "ibert_dyadic_from_double",
+                     "ibert_linear_i8", "ibert_linear_gelu_i8", "ibert_softmax_i", "ibert_gelu_i",
+                     "ibert_layernorm_i", "ibert_attention_i8", "ibert_layer_create", "ibert_layer_destroy",
+                     "ibert_encoder_layer"):
+            getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def _chk(rc: int, where: str):
+    if rc != IBERT_OK:
+        raise IbertError(rc, where)
+
+
+def _dev(t: torch.Tensor | None, dtype) -> int | None:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous() and t.dtype == dtype, (t.device, t.dtype, dtype)
+    return t.data_ptr()
+
+
+def _host(a, dtype) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def ibert_dyadic_from_double(m: float) -> tuple[int, int]:
+    b, c = C.c_int32(), C.c_int32()
+    _chk(lib().ibert_dyadic_from_double(m, C.byref(b), C.byref(c)), "ibert_dyadic_from_double")
+    return b.value, c.value
+
+
+class Context:
+    """``ibert_ctx``: a device and the stream every call is enqueued on."""
+
+    def __init__(self, device: int = 0, stream: torch.cuda.Stream | None = None):
+        self.device = device
+        self.stream = stream
+        h = C.c_void_p()
+        sp = None if stream is None else stream.cuda_stream
+        _chk(lib().ibert_create(C.byref(h), device, sp), "ibert_create")
+        self.h = h
+
+    def close(self):
+        if self.h:
+            lib().ibert_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def ibert_last_status(self) -> int:
+        return int(lib().ibert_last_status(self.h))
+
+    def check(self):
+        _chk(self.ibert_last_status(), "ibert_last_status")
+
+    # ------------------------------------------------------------------ simple ops
+    def ibert_gelu_i(self, q: torch.Tensor, S: float, S_out: float, out: torch.Tensor | None = None):
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.int8, device=q.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_gelu_i(self.h, _dev(q, torch.int32), S, q.numel(), S_out, _dev(out, torch.int8),
+                                C.byref(S_ret)), "ibert_gelu_i")
+        return out, S_ret.value
+
+    def ibert_softmax_i(self, q: torch.Tensor, S: float, p_max: int = 255, out: torch.Tensor | None = None):
+        L = q.shape[-1]
+        rows = q.numel() // L if L else 0
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.uint8, device=q.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_softmax_i(self.h, _dev(q, torch.int32), S, rows, L, p_max, _dev(out, torch.uint8),
+                                   C.byref(S_ret)), "ibert_softmax_i")
+        return out, S_ret.value
+
+    def ibert_layernorm_i(self, q: torch.Tensor, S: float, r: torch.Tensor | None, S_r: float, gamma, beta,
+                          S_out: float, out: torch.Tensor | None = None):
+        Cn = q.shape[-1]
+        rows = q.numel() // Cn if Cn else 0
+        g, b = _host(gamma, np.float64), _host(beta, np.float64)
+        assert g.size == Cn and b.size == Cn
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.int8, device=q.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_layernorm_i(self.h, _dev(q, torch.int32), S, _dev(r, torch.int8), S_r or 0.0,
+                                     g.ctypes.data, b.ctypes.data, rows, Cn, S_out, _dev(out, torch.int8),
+                                     C.byref(S_ret)), "ibert_layernorm_i")
+        return out, S_ret.value
+
+    def ibert_linear_i8(self, x: torch.Tensor, S_x: float, w: torch.Tensor, S_w, bias: torch.Tensor | None,
+                        out_kind: int, S_out: float = 1.0, out: torch.Tensor | None = None):
+        K = x.shape[-1]
+        M = x.numel() // K
+        N = w.shape[0]
+        assert w.shape[1] == K
+        sw = _host(S_w, np.float64)
+        assert sw.size == N
+        if out is None:
+            out = torch.empty(x.shape[:-1] + (N,), dtype=torch.int8 if out_kind == 0 else torch.int32,
+                              device=x.device)
+        S_ret = np.zeros(N if out_kind == 2 else 1, dtype=np.float64)
+        _chk(lib().ibert_linear_i8(self.h, _dev(x, torch.int8), S_x, _dev(w, torch.int8), sw.ctypes.data,
+                                   _dev(bias, torch.int32), M, N, K, out_kind, S_out, out.data_ptr(),
+                                   S_ret.ctypes.data), "ibert_linear_i8")
+        return out, (S_ret if out_kind == 2 else float(S_ret[0]))
+
+    def ibert_linear_gelu_i8(self, x: torch.Tensor, S_x: float, w: torch.Tensor, S_w, bias: torch.Tensor | None,
+                             S_mid: float, S_out: float, out: torch.Tensor | None = None):
+        K = x.shape[-1]
+        M = x.numel() // K
+        N = w.shape[0]
+        sw = _host(S_w, np.float64)
+        if out is None:
+            out = torch.empty(x.shape[:-1] + (N,), dtype=torch.int8, device=x.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_linear_gelu_i8(self.h, _dev(x, torch.int8), S_x, _dev(w, torch.int8), sw.ctypes.data,
+                                        _dev(bias, torch.int32), M, N, K, S_mid, S_out, _dev(out, torch.int8),
+                                        C.byref(S_ret)), "ibert_linear_gelu_i8")
+        return out, S_ret.value
+
+    def ibert_attention_i8(self, qkv: torch.Tensor, B: int, L: int, H: int, heads: int, S_q: float, S_k: float,
+                           S_v: float, S_ctx: float, p_max: int = 255, out: torch.Tensor | None = None):
+        assert qkv.numel() == B * L * 3 * H
+        if out is None:
+            out = torch.empty((B * L, H), dtype=torch.int8, device=qkv.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_attention_i8(self.h, _dev(qkv, torch.int8), B, L, H, heads, S_q, S_k, S_v, S_ctx, p_max,
+                                      _dev(out, torch.int8), C.byref(S_ret)), "ibert_attention_i8")
+        return out, S_ret.value
+
+    # ------------------------------------------------------------------ encoder layer
+    def ibert_layer_create(self, params: dict) -> "Layer":
+        return Layer(self, params)
+
+    def ibert_encoder_layer(self, layer: "Layer", x: torch.Tensor, B: int, L: int,
+                            out: torch.Tensor | None = None):
+        if out is None:
+            out = torch.empty((B * L, layer.H), dtype=torch.int8, device=x.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_encoder_layer(self.h, layer.h, _dev(x, torch.int8), B, L, _dev(out, torch.int8),
+                                       C.byref(S_ret)), "ibert_encoder_layer")
+        return out, S_ret.value
+
+
+class Layer:
+    """``ibert_layer``: device-resident integer parameters of one encoder layer, built from the
+    dictionary of host arrays a synthetic-layer generator (or a calibrated checkpoint) provides."""
+
+    def __init__(self, ctx: Context, params: dict):
+        self.ctx = ctx
+        self.H = int(params["H"])
+        d = LayerDesc()
+        d.H, d.heads, d.F, d.p_max = self.H, int(params["heads"]), int(params["F"]), int(params["p_max"])
+        keep = []
+
+        def ptr(name, dtype):
+            a = _host(params[name], dtype)
+            keep.append(a)
+            return a.ctypes.data
+
+        for nm in ("qkv", "o", "f1", "f2"):
+            setattr(d, f"w_{nm}", ptr(f"w_{nm}", np.int8))
+            setattr(d, f"S_w_{nm}", ptr(f"S_w_{nm}", np.float64))
+            setattr(d, f"bias_{nm}", ptr(f"bias_{nm}", np.int32))
+        for nm in ("gamma1", "beta1", "gamma2", "beta2"):
+            setattr(d, nm, ptr(nm, np.float64))
+        for nm in SCALE_NAMES:
+            setattr(d, nm, float(params[nm]))
+        h = C.c_void_p()
+        _chk(lib().ibert_layer_create(ctx.h, C.byref(d), C.byref(h)), "ibert_layer_create")
+        self.h = h
+
+    def close(self):
+        if self.h and self.ctx.h:
+            lib().ibert_layer_destroy(self.h)
+        self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,430 @@
+// C-ABI entry points of libibert_b200: argument validation, constant derivation,
+// launch.  No entry point synchronizes (except ibert_last_status) and none has a CPU path.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "ibert_internal.h"
+
+using namespace ibert;
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool good_scale(double s) { return std::isfinite(s) && s > 0.0; }
+
+uint64_t fnv1a(const void* data, size_t bytes, uint64_t seed) {
+  const unsigned char* p = static_cast<const unsigned char*>(data);
+  uint64_t h = 1469598103934665603ull ^ seed;
+  for (size_t i = 0; i < bytes; ++i) { h ^= p[i]; h *= 1099511628211ull; }
+  return h;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    ok = cudaGetDevice(&prev) == cudaSuccess;
+    if (ok && prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+namespace ibert {
+
+int cached_upload(ibert_ctx* ctx, const void* host, size_t bytes, uint64_t tag, void** dev) {
+  const uint64_t key = fnv1a(host, bytes, tag * 0x9e3779b97f4a7c15ull + bytes);
+  auto it = ctx->tables.find(key);
+  if (it != ctx->tables.end() && it->second.bytes == bytes) { *dev = it->second.ptr; return IBERT_OK; }
+  if (ctx->tables.size() > 4096) {        // bound the cache: drop everything once the stream is idle
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+    for (auto& kv : ctx->tables) cudaFree(kv.second.ptr);
+    ctx->tables.clear();
+  }
+  void* d = nullptr;
+  if (cudaMalloc(&d, bytes ? bytes : 16) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_NOMEM; }
+  if (cudaMemcpyAsync(d, host, bytes, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess) {
+    cudaFree(d);
+    return IBERT_ERR_CUDA;
+  }
+  ctx->tables[key] = DeviceTable{d, bytes};
+  *dev = d;
+  return IBERT_OK;
+}
+
+}  // namespace ibert
+
+struct ibert_layer {
+  ibert_ctx* ctx = nullptr;
+  ibert_layer_desc d{};              // scalars only are meaningful after create
+  int8_t *w_qkv = nullptr, *w_o = nullptr, *w_f1 = nullptr, *w_f2 = nullptr;
+  int32_t *bias_qkv = nullptr, *bias_o = nullptr, *bias_f1 = nullptr, *bias_f2 = nullptr;
+  int32_t *b_qkv = nullptr, *c_qkv = nullptr, *b_o = nullptr, *c_o = nullptr;
+  int32_t *b_f1 = nullptr, *c_f1 = nullptr, *b_f2 = nullptr, *c_f2 = nullptr;
+  int32_t *ln1_b = nullptr, *ln2_b = nullptr;
+  int64_t *ln1_B = nullptr, *ln2_B = nullptr;
+  LnConsts ln1{}, ln2{};
+  GeluConsts gelu{};
+  AttnConsts attn{};
+  std::vector<void*> owned;
+};
+
+extern "C" {
+
+const char* ibert_strerror(int code) {
+  switch (code) {
+    case IBERT_OK: return "ok";
+    case IBERT_ERR_ARG: return "invalid argument";
+    case IBERT_ERR_SHAPE: return "unsupported shape";
+    case IBERT_ERR_SCALE_RANGE: return "scale out of range";
+    case IBERT_ERR_ALIGN: return "pointer or pitch not 16-byte aligned";
+    case IBERT_ERR_NOMEM: return "out of memory";
+    case IBERT_ERR_CUDA: return "CUDA call failed";
+    case IBERT_ERR_TIMEOUT: return "bounded device wait expired";
+    case IBERT_ERR_VALUE_RANGE: return "integer value out of the assumed range";
+    default: return "unknown error";
+  }
+}
+
+int ibert_dyadic_from_double(double m, int32_t* b, int32_t* c) {
+  if (!b || !c) return IBERT_ERR_ARG;
+  return dyadic(m, b, c);
+}
+
+int ibert_create(ibert_ctx** out, int device, void* cuda_stream) {
+  if (!out) return IBERT_ERR_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+    cudaGetLastError();
+    return IBERT_ERR_CUDA;
+  }
+  DeviceGuard guard(device);
+  if (!guard.ok) return IBERT_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return IBERT_ERR_CUDA;
+  if (prop.major != 10) return IBERT_ERR_CUDA;       // sm_100a kernels only
+  ibert_ctx* ctx = new (std::nothrow) ibert_ctx();
+  if (!ctx) return IBERT_ERR_NOMEM;
+  ctx->device = device;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  ctx->num_sms = prop.multiProcessorCount;
+  if (cudaMalloc(&ctx->d_status, 64) != cudaSuccess) { delete ctx; return IBERT_ERR_NOMEM; }
+  if (cudaMemsetAsync(ctx->d_status, 0, 64, ctx->stream) != cudaSuccess) {
+    cudaFree(ctx->d_status);
+    delete ctx;
+    return IBERT_ERR_CUDA;
+  }
+  *out = ctx;
+  return IBERT_OK;
+}
+
+int ibert_destroy(ibert_ctx* ctx) {
+  if (!ctx) return IBERT_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaStreamSynchronize(ctx->stream);
+  for (auto& kv : ctx->tables) cudaFree(kv.second.ptr);
+  if (ctx->ws) cudaFree(ctx->ws);
+  cudaFree(ctx->d_status);
+  delete ctx;
+  return IBERT_OK;
+}
+
+int ibert_last_status(ibert_ctx* ctx) {
+  if (!ctx) return IBERT_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  int32_t st = 0;
+  if (cudaMemcpyAsync(&st, ctx->d_status, sizeof(st), cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess)
+    return IBERT_ERR_CUDA;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+  if (st != 0) cudaMemsetAsync(ctx->d_status, 0, sizeof(st), ctx->stream);
+  return st;
+}
+
+int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
+                 double* S_ret) {
+  if (!ctx || n < 0 || (n > 0 && (!q || !out))) return IBERT_ERR_ARG;
+  if (!aligned16(q) || !aligned16(out)) return IBERT_ERR_ALIGN;
+  GeluConsts k;
+  int rc = make_gelu_consts(S, S_out, &k);
+  if (rc) return rc;
+  DeviceGuard guard(ctx->device);
+  rc = launch_gelu(ctx, q, n, k, out);
+  if (rc == IBERT_OK && S_ret) *S_ret = S_out;
+  return rc;
+}
+
+int ibert_softmax_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
+                    uint8_t* out, double* S_ret) {
+  if (!ctx || rows < 0) return IBERT_ERR_ARG;
+  if (p_max != 255 && p_max != 127) return IBERT_ERR_ARG;
+  if (L < 1 || L > 1024) return IBERT_ERR_SHAPE;
+  if (rows > 0 && (!q || !out)) return IBERT_ERR_ARG;
+  if (!aligned16(q) || !aligned16(out)) return IBERT_ERR_ALIGN;
+  ExpConsts k;
+  int rc = make_exp_consts(S, p_max, &k);
+  if (rc) return rc;
+  DeviceGuard guard(ctx->device);
+  rc = launch_softmax(ctx, q, rows, L, k, out);
+  if (rc == IBERT_OK && S_ret) *S_ret = 1.0 / (double)p_max;
+  return rc;
+}
+
+int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* r, double S_r,
+                      const double* gamma, const double* beta, int64_t rows, int C, double S_out,
+                      int8_t* out, double* S_ret) {
+  if (!ctx || rows < 0 || !gamma || !beta) return IBERT_ERR_ARG;
+  if (C < 1 || C > 2047) return IBERT_ERR_SHAPE;
+  if (rows > 0 && (!q || !out)) return IBERT_ERR_ARG;
+  if (!aligned16(q) || !aligned16(out) || (r && !aligned16(r))) return IBERT_ERR_ALIGN;
+  if (!good_scale(S) || !good_scale(S_out)) return IBERT_ERR_SCALE_RANGE;
+  LnConsts k{};
+  k.C = C;
+  k.has_res = r != nullptr;
+  if (r) {
+    if (!good_scale(S_r)) return IBERT_ERR_SCALE_RANGE;
+    int rc = dyadic(S_r / S, &k.b_r, &k.c_r);
+    if (rc) return rc;
+  }
+  std::vector<int32_t> b_i;
+  std::vector<int64_t> B_i;
+  int rc = make_ln_tables(gamma, beta, C, S_out, &k.c, &b_i, &B_i);
+  if (rc) return rc;
+  DeviceGuard guard(ctx->device);
+  void *d_b = nullptr, *d_B = nullptr;
+  rc = cached_upload(ctx, b_i.data(), b_i.size() * sizeof(int32_t), 11, &d_b);
+  if (rc) return rc;
+  rc = cached_upload(ctx, B_i.data(), B_i.size() * sizeof(int64_t), 12, &d_B);
+  if (rc) return rc;
+  rc = launch_layernorm(ctx, q, r, rows, k, (const int32_t*)d_b, (const int64_t*)d_B, out);
+  if (rc == IBERT_OK && S_ret) *S_ret = S_out;
+  return rc;
+}
+
+static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
+                         const int32_t* bias, int64_t M, int N, int K, int kind, double S_mid,
+                         double S_out, void* out, double* S_ret) {
+  if (!ctx || M < 0 || !S_w) return IBERT_ERR_ARG;
+  if (kind < 0 || kind > 3) return IBERT_ERR_ARG;
+  if (N < 1 || K < 1 || K % 16 != 0 || N % 4 != 0) return IBERT_ERR_SHAPE;
+  if ((kind == EPI_INT8 || kind == EPI_GELU) && N % 16 != 0) return IBERT_ERR_SHAPE;
+  if ((int64_t)K * 127 * 127 >= (int64_t(1) << 31)) return IBERT_ERR_SHAPE;
+  if (M > 0 && (!x || !out)) return IBERT_ERR_ARG;
+  if (!w) return IBERT_ERR_ARG;
+  if (!aligned16(x) || !aligned16(w) || !aligned16(out) || (bias && !aligned16(bias))) return IBERT_ERR_ALIGN;
+  if (!good_scale(S_x)) return IBERT_ERR_SCALE_RANGE;
+  for (int n = 0; n < N; ++n)
+    if (!good_scale(S_w[n])) return IBERT_ERR_SCALE_RANGE;
+  GemmEpilogue epi{};
+  epi.kind = kind;
+  epi.d_bias = bias;
+  DeviceGuard guard(ctx->device);
+  if (kind != EPI_RAW) {
+    const double S_acc_to = kind == EPI_GELU ? S_mid : S_out;
+    std::vector<int32_t> b, c;
+    int rc = make_linear_tables(S_x, S_w, N, nullptr, S_acc_to, &b, &c);
+    if (rc) return rc;
+    void *d_b = nullptr, *d_c = nullptr;
+    rc = cached_upload(ctx, b.data(), b.size() * sizeof(int32_t), 21, &d_b);
+    if (rc) return rc;
+    rc = cached_upload(ctx, c.data(), c.size() * sizeof(int32_t), 22, &d_c);
+    if (rc) return rc;
+    epi.d_b = (const int32_t*)d_b;
+    epi.d_c = (const int32_t*)d_c;
+    if (kind == EPI_GELU) {
+      rc = make_gelu_consts(S_mid, S_out, &epi.gelu);
+      if (rc) return rc;
+    }
+  }
+  int rc = launch_gemm_i8(ctx, x, w, M, N, K, epi, out);
+  if (rc == IBERT_OK && S_ret) {
+    if (kind == EPI_RAW) for (int n = 0; n < N; ++n) S_ret[n] = S_x * S_w[n];
+    else *S_ret = S_out;
+  }
+  return rc;
+}
+
+int ibert_linear_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
+                    const int32_t* bias, int64_t M, int N, int K, int out_kind, double S_out,
+                    void* out, double* S_ret) {
+  if (out_kind < 0 || out_kind > 2) return IBERT_ERR_ARG;
+  return linear_common(ctx, x, S_x, w, S_w, bias, M, N, K, out_kind, 0.0, S_out, out, S_ret);
+}
+
+int ibert_linear_gelu_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
+                         const int32_t* bias, int64_t M, int N, int K, double S_mid, double S_out,
+                         int8_t* out, double* S_ret) {
+  return linear_common(ctx, x, S_x, w, S_w, bias, M, N, K, EPI_GELU, S_mid, S_out, out, S_ret);
+}
+
+static int make_attn_consts(double S_q, double S_k, double S_v, double S_ctx, int p_max, AttnConsts* k) {
+  if (!good_scale(S_q) || !good_scale(S_k) || !good_scale(S_v) || !good_scale(S_ctx)) return IBERT_ERR_SCALE_RANGE;
+  if (p_max != 255 && p_max != 127) return IBERT_ERR_ARG;
+  int rc = make_exp_consts((S_q * S_k) / 8.0, p_max, &k->e);     // 1/sqrt(64) folded into the score scale
+  if (rc) return rc;
+  k->p_signed = p_max == 127;
+  return dyadic(((1.0 / (double)p_max) * S_v) / S_ctx, &k->b, &k->c);
+}
+
+int ibert_attention_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads, double S_q,
+                       double S_k, double S_v, double S_ctx, int p_max, int8_t* out, double* S_ret) {
+  if (!ctx || B < 0) return IBERT_ERR_ARG;
+  if (heads < 1 || H != heads * 64 || L < 1 || L > 512) return IBERT_ERR_SHAPE;
+  if (B > 0 && (!qkv || !out)) return IBERT_ERR_ARG;
+  if (!aligned16(qkv) || !aligned16(out)) return IBERT_ERR_ALIGN;
+  AttnConsts k{};
+  int rc = make_attn_consts(S_q, S_k, S_v, S_ctx, p_max, &k);
+  if (rc) return rc;
+  DeviceGuard guard(ctx->device);
+  rc = launch_attention(ctx, qkv, B, L, H, heads, k, out);
+  if (rc == IBERT_OK && S_ret) *S_ret = S_ctx;
+  return rc;
+}
+
+// --------------------------------------------------------------------------- encoder layer
+
+static int upload_owned(ibert_layer* ly, const void* host, size_t bytes, void** dev) {
+  void* d = nullptr;
+  if (cudaMalloc(&d, bytes) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_NOMEM; }
+  ly->owned.push_back(d);
+  if (cudaMemcpyAsync(d, host, bytes, cudaMemcpyHostToDevice, ly->ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+  *dev = d;
+  return IBERT_OK;
+}
+
+int ibert_layer_destroy(ibert_layer* ly) {
+  if (!ly) return IBERT_ERR_ARG;
+  DeviceGuard guard(ly->ctx->device);
+  cudaStreamSynchronize(ly->ctx->stream);
+  for (void* p : ly->owned) cudaFree(p);
+  delete ly;
+  return IBERT_OK;
+}
+
+int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** out) {
+  if (!ctx || !d || !out) return IBERT_ERR_ARG;
+  *out = nullptr;
+  const int H = d->H, F = d->F;
+  if (d->heads < 1 || H != d->heads * 64 || F < 16 || F % 16 != 0) return IBERT_ERR_SHAPE;
+  if (H > 2047) return IBERT_ERR_SHAPE;
+  if ((int64_t)F * 127 * 127 >= (int64_t(1) << 31)) return IBERT_ERR_SHAPE;
+  const void* ptrs[] = {d->w_qkv, d->S_w_qkv, d->bias_qkv, d->w_o, d->S_w_o, d->bias_o, d->w_f1, d->S_w_f1,
+                        d->bias_f1, d->w_f2, d->S_w_f2, d->bias_f2, d->gamma1, d->beta1, d->gamma2, d->beta2};
+  for (const void* p : ptrs) if (!p) return IBERT_ERR_ARG;
+  const double scales[] = {d->S_x, d->S_q, d->S_k, d->S_v, d->S_ctx, d->S_r1, d->S_h1, d->S_gi, d->S_go, d->S_r2, d->S_out};
+  for (double s : scales) if (!good_scale(s)) return IBERT_ERR_SCALE_RANGE;
+
+  DeviceGuard guard(ctx->device);
+  ibert_layer* ly = new (std::nothrow) ibert_layer();
+  if (!ly) return IBERT_ERR_NOMEM;
+  ly->ctx = ctx;
+  ly->d = *d;
+  int rc = IBERT_OK;
+  auto up = [&](const void* h, size_t bytes, void** dev) { if (rc == IBERT_OK) rc = upload_owned(ly, h, bytes, dev); };
+  auto lin = [&](double S_in, const double* S_w, int N, const double* so_cols, double so, int32_t** db, int32_t** dc) {
+    if (rc != IBERT_OK) return;
+    std::vector<int32_t> b, c;
+    rc = make_linear_tables(S_in, S_w, N, so_cols, so, &b, &c);
+    up(b.data(), b.size() * sizeof(int32_t), (void**)db);
+    up(c.data(), c.size() * sizeof(int32_t), (void**)dc);
+  };
+  up(d->w_qkv, (size_t)3 * H * H, (void**)&ly->w_qkv);
+  up(d->w_o, (size_t)H * H, (void**)&ly->w_o);
+  up(d->w_f1, (size_t)F * H, (void**)&ly->w_f1);
+  up(d->w_f2, (size_t)H * F, (void**)&ly->w_f2);
+  up(d->bias_qkv, sizeof(int32_t) * 3 * H, (void**)&ly->bias_qkv);
+  up(d->bias_o, sizeof(int32_t) * H, (void**)&ly->bias_o);
+  up(d->bias_f1, sizeof(int32_t) * F, (void**)&ly->bias_f1);
+  up(d->bias_f2, sizeof(int32_t) * H, (void**)&ly->bias_f2);
+  {
+    std::vector<double> so(3 * (size_t)H);
+    for (int n = 0; n < 3 * H; ++n) so[n] = n < H ? d->S_q : (n < 2 * H ? d->S_k : d->S_v);
+    lin(d->S_x, d->S_w_qkv, 3 * H, so.data(), 0.0, &ly->b_qkv, &ly->c_qkv);
+  }
+  lin(d->S_ctx, d->S_w_o, H, nullptr, d->S_r1, &ly->b_o, &ly->c_o);
+  lin(d->S_h1, d->S_w_f1, F, nullptr, d->S_gi, &ly->b_f1, &ly->c_f1);
+  lin(d->S_go, d->S_w_f2, H, nullptr, d->S_r2, &ly->b_f2, &ly->c_f2);
+  auto ln = [&](const double* g, const double* be, double S_sum, double S_res, double S_o, LnConsts* k,
+                int32_t** db, int64_t** dB) {
+    if (rc != IBERT_OK) return;
+    k->C = H;
+    k->has_res = 1;
+    rc = dyadic(S_res / S_sum, &k->b_r, &k->c_r);
+    if (rc != IBERT_OK) return;
+    std::vector<int32_t> b_i;
+    std::vector<int64_t> B_i;
+    rc = make_ln_tables(g, be, H, S_o, &k->c, &b_i, &B_i);
+    up(b_i.data(), b_i.size() * sizeof(int32_t), (void**)db);
+    up(B_i.data(), B_i.size() * sizeof(int64_t), (void**)dB);
+  };
+  ln(d->gamma1, d->beta1, d->S_r1, d->S_x, d->S_h1, &ly->ln1, &ly->ln1_b, &ly->ln1_B);
+  ln(d->gamma2, d->beta2, d->S_r2, d->S_h1, d->S_out, &ly->ln2, &ly->ln2_b, &ly->ln2_B);
+  if (rc == IBERT_OK) rc = make_gelu_consts(d->S_gi, d->S_go, &ly->gelu);
+  if (rc == IBERT_OK) rc = make_attn_consts(d->S_q, d->S_k, d->S_v, d->S_ctx, d->p_max, &ly->attn);
+  if (rc != IBERT_OK) { ibert_layer_destroy(ly); return rc; }
+  // host arrays were pageable: make sure the copies have left them before returning
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) { ibert_layer_destroy(ly); return IBERT_ERR_CUDA; }
+  // scalars only from here on
+  ly->d.w_qkv = ly->d.w_o = ly->d.w_f1 = ly->d.w_f2 = nullptr;
+  *out = ly;
+  return IBERT_OK;
+}
+
+int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, int B, int L,
+                        int8_t* out, double* S_ret) {
+  if (!ctx || !ly || ly->ctx != ctx || B < 0) return IBERT_ERR_ARG;
+  if (L < 1 || L > 512) return IBERT_ERR_SHAPE;
+  const int H = ly->d.H, F = ly->d.F;
+  const int64_t T = (int64_t)B * L;
+  if (T > 0 && (!x || !out)) return IBERT_ERR_ARG;
+  if (!aligned16(x) || !aligned16(out)) return IBERT_ERR_ALIGN;
+  if (S_ret) *S_ret = ly->d.S_out;
+  if (T == 0) return IBERT_OK;
+  DeviceGuard guard(ctx->device);
+  // workspace: qkv [T,3H] i8 | ctx [T,H] i8 | r [T,H] i32 (both residual sums) | h1 [T,H] i8 | g [T,F] i8
+  auto up256 = [](size_t v) { return (v + 255) & ~size_t(255); };
+  const size_t o_qkv = 0;
+  const size_t o_ctx = o_qkv + up256((size_t)T * 3 * H);
+  const size_t o_r = o_ctx + up256((size_t)T * H);
+  const size_t o_h1 = o_r + up256((size_t)T * H * 4);
+  const size_t o_g = o_h1 + up256((size_t)T * H);
+  const size_t need = o_g + up256((size_t)T * F);
+  if (need > ctx->ws_bytes) {
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+    if (ctx->ws) cudaFree(ctx->ws);
+    ctx->ws = nullptr;
+    ctx->ws_bytes = 0;
+    if (cudaMalloc(&ctx->ws, need) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_NOMEM; }
+    ctx->ws_bytes = need;
+  }
+  char* ws = static_cast<char*>(ctx->ws);
+  int8_t* qkv = (int8_t*)(ws + o_qkv);
+  int8_t* cx = (int8_t*)(ws + o_ctx);
+  int32_t* r = (int32_t*)(ws + o_r);
+  int8_t* h1 = (int8_t*)(ws + o_h1);
+  int8_t* g = (int8_t*)(ws + o_g);
+
+  GemmEpilogue e{};
+  e.kind = EPI_INT8; e.d_b = ly->b_qkv; e.d_c = ly->c_qkv; e.d_bias = ly->bias_qkv;
+  int rc = launch_gemm_i8(ctx, x, ly->w_qkv, T, 3 * H, H, e, qkv);
+  if (rc) return rc;
+  rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, cx);
+  if (rc) return rc;
+  e.kind = EPI_Q16; e.d_b = ly->b_o; e.d_c = ly->c_o; e.d_bias = ly->bias_o;
+  rc = launch_gemm_i8(ctx, cx, ly->w_o, T, H, H, e, r);
+  if (rc) return rc;
+  rc = launch_layernorm(ctx, r, x, T, ly->ln1, ly->ln1_b, ly->ln1_B, h1);
+  if (rc) return rc;
+  e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu;
+  rc = launch_gemm_i8(ctx, h1, ly->w_f1, T, F, H, e, g);
+  if (rc) return rc;
+  e.kind = EPI_Q16; e.d_b = ly->b_f2; e.d_c = ly->c_f2; e.d_bias = ly->bias_f2;
+  rc = launch_gemm_i8(ctx, g, ly->w_f2, T, H, F, e, r);
+  if (rc) return rc;
+  return launch_layernorm(ctx, r, h1, T, ly->ln2, ly->ln2_b, ly->ln2_B, out);
+}
+
+}  // extern "C"

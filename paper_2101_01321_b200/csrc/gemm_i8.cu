@@ -1,0 +1,353 @@
+// INT8 x INT8 -> INT32 GEMM on the 5th-generation tensor cores (tcgen05.mma kind::i8,
+// accumulators in TMEM, operands staged by TMA) with the integer epilogue fused:
+// bias add + dyadic requantization to int8 or Q16, raw accumulators, or requantization
+// to Q16 followed by i-GELU (Algorithm 2) and a second requantization to int8.
+//
+// out[m, n] = epilogue( sum_k x[m, k] * w[n, k] + bias[n] )      x: [M, K], w: [N, K]
+//
+// One persistent CTA per SM walks 128 x BN output tiles.  Warp 0 is the TMA producer,
+// warp 1 issues the MMAs, warps 2..5 run the epilogue; two TMEM accumulator stages let
+// the (integer-ALU heavy) epilogue of tile i overlap the MMAs of tile i+1.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "device_utils.cuh"
+#include "sm100_ptx.cuh"
+
+namespace ibert {
+
+// --------------------------------------------------------------------------------------
+// tensor-map encoding through the driver entry point
+// --------------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    else
+      cudaGetLastError();
+  });
+  return fn;
+}
+
+}  // namespace
+
+int encode_tensor_map(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                      const uint64_t* strides_bytes, const uint32_t* box, int swizzle_bytes) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return IBERT_ERR_CUDA;
+  cuuint64_t gdim[5];
+  cuuint64_t gstr[5];
+  cuuint32_t bdim[5];
+  cuuint32_t estr[5];
+  for (int i = 0; i < rank; ++i) {
+    gdim[i] = dims[i];
+    bdim[i] = box[i];
+    estr[i] = 1;
+    if (i + 1 < rank) gstr[i] = strides_bytes[i];
+  }
+  const CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                      : CU_TENSOR_MAP_SWIZZLE_NONE;
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr,
+                  bdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? IBERT_OK : IBERT_ERR_CUDA;
+}
+
+// --------------------------------------------------------------------------------------
+// kernel
+// --------------------------------------------------------------------------------------
+namespace {
+
+constexpr int BM = 128;           // rows per tile = TMEM lanes
+constexpr int BK = 128;           // K bytes per pipeline stage = one 128-byte swizzle span
+constexpr int UMMA_K = 32;        // K per tcgen05.mma kind::i8
+constexpr int kGemmThreads = 192; // producer warp, MMA warp, 4 epilogue warps
+constexpr int kEpiThreads = 128;
+
+template <int BN>
+struct GemmSmem {
+  static constexpr int kStages = BN >= 256 ? 4 : 6;
+  static constexpr int kABytes = BM * BK;
+  static constexpr int kBBytes = BN * BK;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  // operand stages | per-column epilogue parameters (int4 per column) | barriers
+  static constexpr int kParamOff = kStages * kStageBytes;
+  static constexpr int kBarOff = kParamOff + BN * 16;
+  static constexpr int kBytes = kBarOff + 256;
+  static constexpr int kAlloc = kBytes + 1024;   // slack to align the operand area to 1024 bytes
+};
+
+struct GemmArgs {
+  int64_t M;
+  int N, K;
+  int kind;
+  const int32_t* b;
+  const int32_t* c;
+  const int32_t* bias;
+  GeluConsts gelu;
+  void* out;
+  int32_t* status;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const GemmArgs args) {
+  using SM = GemmSmem<BN>;
+  constexpr int kStages = SM::kStages;
+  constexpr uint32_t kTmemCols = 2 * BN;          // two accumulator stages (power of two >= 32)
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = ptx::smem_addr(smem);
+  int4* s_param = reinterpret_cast<int4*>(smem + SM::kParamOff);
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + SM::kBarOff);
+  // barrier slots: full[kStages], empty[kStages], acc_full[2], acc_empty[2], then the TMEM base word
+  const uint32_t bar_full = ptx::smem_addr(s_bar);
+  const uint32_t bar_empty = bar_full + 8 * kStages;
+  const uint32_t bar_acc_full = bar_empty + 8 * kStages;
+  const uint32_t bar_acc_empty = bar_acc_full + 16;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 2 * kStages + 4);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int n_tiles = (args.N + BN - 1) / BN;
+  const int64_t m_tiles = (args.M + BM - 1) / BM;
+  const int64_t total_tiles = m_tiles * n_tiles;
+  const int k_blocks = (args.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(bar_full + 8 * s, 1);
+      ptx::mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(bar_acc_full + 8 * a, 1);
+      ptx::mbar_init(bar_acc_empty + 8 * a, kEpiThreads);
+    }
+    ptx::fence_mbar_init();
+    ptx::tma_prefetch_desc(&map_a);
+    ptx::tma_prefetch_desc(&map_b);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_addr(s_tmem), kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *s_tmem;
+  bool ok = true;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int m0 = (int)(tile / n_tiles) * BM;
+        const int n0 = (int)(tile % n_tiles) * BN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!ptx::mbar_wait(bar_empty + 8 * stage, phase ^ 1)) { ok = false; break; }
+          const uint32_t sa = smem_base + stage * SM::kStageBytes;
+          ptx::mbar_arrive_expect_tx(bar_full + 8 * stage, SM::kStageBytes);
+          ptx::tma_load_2d(sa, &map_a, bar_full + 8 * stage, kb * BK, m0);
+          ptx::tma_load_2d(sa + SM::kABytes, &map_b, bar_full + 8 * stage, kb * BK, n0);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_i8(BM, BN, true, true);
+      uint32_t stage = 0, phase = 0;
+      uint32_t acc = 0, acc_phase = 0;
+      for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        if (!ptx::mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1)) { ok = false; break; }
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!ptx::mbar_wait(bar_full + 8 * stage, phase)) { ok = false; break; }
+          ptx::tc_fence_after_sync();
+          const uint32_t sa = smem_base + stage * SM::kStageBytes;
+          const uint64_t da = ptx::make_kmajor_desc(sa, 1024, ptx::kSwizzle128);
+          const uint64_t db = ptx::make_kmajor_desc(sa + SM::kABytes, 1024, ptx::kSwizzle128);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // advancing K inside the swizzle span: +32 bytes = +2 in the encoded start address
+            ptx::mma_i8_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          ptx::mma_commit(bar_empty + 8 * stage);     // frees the stage once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        ptx::mma_commit(bar_acc_full + 8 * acc);      // accumulator complete
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;                      // TMEM lanes 32*quarter .. +31 belong to this warp
+    const int et = threadIdx.x - 64;                   // 0..127
+    const GeluConsts gk = args.gelu;
+    const int64_t gelu_half = rounding_half(gk.c);
+    uint32_t acc = 0, acc_phase = 0;
+    for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const int64_t m0 = (tile / n_tiles) * BM;
+      const int n0 = (int)(tile % n_tiles) * BN;
+      // per-column parameters of this tile: {b, c, (bias*b + rounding) lo, hi}; raw: {bias,0,0,0}
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // previous tile's readers are done
+      for (int j = et; j < BN; j += kEpiThreads) {
+        const int n = n0 + j;
+        int4 p = make_int4(0, 0, 0, 0);
+        if (n < args.N) {
+          const int32_t bias = args.bias ? __ldg(args.bias + n) : 0;
+          if (args.kind == EPI_RAW) {
+            p.x = bias;
+          } else {
+            const int32_t b = __ldg(args.b + n), c = __ldg(args.c + n);
+            const int64_t add = (int64_t)bias * b + rounding_half(c);
+            p = make_int4(b, c, (int32_t)(uint32_t)(uint64_t)add, (int32_t)(add >> 32));
+          }
+        }
+        s_param[j] = p;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+
+      // After a failed wait the loop keeps running (the named barriers above must still be
+      // reached by all 128 threads) but touches neither TMEM nor memory.
+      if (ok) ok = ptx::mbar_wait(bar_acc_full + 8 * acc, acc_phase);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) continue;
+      ptx::tc_fence_after_sync();
+      const int64_t row = m0 + quarter * 32 + lane;
+      const bool row_ok = row < args.M;
+      const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        uint32_t v[32];
+        ptx::tmem_ld32(t_row + ch * 32, v);
+        ptx::tmem_wait_ld();
+        const int col0 = n0 + ch * 32;
+        if (args.kind == EPI_RAW || args.kind == EPI_Q16) {
+          int32_t* orow = static_cast<int32_t*>(args.out) + row * args.N + col0;
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            int32_t o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int4 p = s_param[ch * 32 + g * 4 + i];
+              if (args.kind == EPI_RAW) o[i] = (int32_t)v[g * 4 + i] + p.x;
+              else {
+                const int64_t add = (int64_t)(((uint64_t)(uint32_t)p.w << 32) | (uint32_t)p.z);
+                o[i] = requant_add((int32_t)v[g * 4 + i], p.x, add, p.y, 32767);
+              }
+            }
+            if (row_ok && col0 + g * 4 < args.N)
+              *reinterpret_cast<int4*>(orow + g * 4) = make_int4(o[0], o[1], o[2], o[3]);
+          }
+        } else {
+          int8_t* orow = static_cast<int8_t*>(args.out) + row * args.N + col0;
+#pragma unroll
+          for (int g = 0; g < 2; ++g) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              uint32_t packed = 0;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int idx = g * 16 + i * 4 + e;
+                const int4 p = s_param[ch * 32 + idx];
+                const int64_t add = (int64_t)(((uint64_t)(uint32_t)p.w << 32) | (uint32_t)p.z);
+                int32_t o;
+                if (args.kind == EPI_INT8) {
+                  o = requant_add((int32_t)v[idx], p.x, add, p.y, 127);
+                } else {
+                  const int32_t q16 = requant_add((int32_t)v[idx], p.x, add, p.y, 32767);
+                  o = igelu_q16_to_int8(q16, gk, gelu_half);
+                }
+                packed |= (uint32_t)(o & 0xff) << (8 * e);
+              }
+              w[i] = packed;
+            }
+            if (row_ok && col0 + g * 16 < args.N)
+              *reinterpret_cast<uint4*>(orow + g * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      ptx::tc_fence_before_sync();
+      ptx::mbar_arrive(bar_acc_empty + 8 * acc);
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1;
+    }
+  }
+
+  if (!ok) atomicCAS(args.status, 0, IBERT_ERR_TIMEOUT);
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+template <int BN>
+int launch_bn(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& args) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_i8_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             GemmSmem<BN>::kAlloc) != cudaSuccess)
+      return IBERT_ERR_CUDA;
+    attr_set = true;
+  }
+  const int64_t tiles = ((args.M + BM - 1) / BM) * ((args.N + BN - 1) / BN);
+  const int grid = (int)(tiles < ctx->num_sms ? tiles : ctx->num_sms);
+  gemm_i8_kernel<BN><<<grid, kGemmThreads, GemmSmem<BN>::kAlloc, ctx->stream>>>(ma, mb, args);
+  return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, int N, int K,
+                   const GemmEpilogue& epi, void* out) {
+  if (M == 0) return IBERT_OK;
+  // tile width: 256 when it divides the work well, else 128
+  const int64_t m_tiles = (M + BM - 1) / BM;
+  const bool wide = (N % 256 == 0) && m_tiles * (N / 256) >= ctx->num_sms;
+  const int BN = wide ? 256 : 128;
+  CUtensorMap ma, mb;
+  {
+    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
+    const uint64_t str[1] = {(uint64_t)K};
+    const uint32_t box[2] = {BK, BM};
+    int rc = encode_tensor_map(&ma, x, 2, dims, str, box, 128);
+    if (rc) return rc;
+  }
+  {
+    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
+    const uint64_t str[1] = {(uint64_t)K};
+    const uint32_t box[2] = {BK, (uint32_t)BN};
+    int rc = encode_tensor_map(&mb, w, 2, dims, str, box, 128);
+    if (rc) return rc;
+  }
+  GemmArgs a{};
+  a.M = M; a.N = N; a.K = K; a.kind = epi.kind;
+  a.b = epi.d_b; a.c = epi.d_c; a.bias = epi.d_bias; a.gelu = epi.gelu;
+  a.out = out; a.status = ctx->d_status;
+  return wide ? launch_bn<256>(ctx, ma, mb, a) : launch_bn<128>(ctx, ma, mb, a);
+}
+
+}  // namespace ibert

@@ -1,0 +1,155 @@
+// Host-side derivation of the integer constants the kernels consume.
+//
+// Static quantization (Sec. 3.1): every scale is known before inference, so
+// q_b = floor(b/S), q_c = floor(c/(a S^2)) of Algorithm 1, q_ln2 of Algorithm 3,
+// q_1 of Algorithm 2 and all dyadic requantization multipliers (Appendix C.1)
+// are computed here, once, in IEEE binary64 with the operation order fixed
+// below.  Compile without FMA contraction.
+#include <cmath>
+#include <cstring>
+
+#include "ibert_internal.h"
+
+namespace ibert {
+
+namespace {
+
+inline bool good_scale(double s) { return std::isfinite(s) && s > 0.0; }
+
+inline int bit_length_u64(uint64_t v) {
+  int n = 0;
+  while (v) { ++n; v >>= 1; }
+  return n;
+}
+
+inline int ceil_log2_u32(uint32_t v) {   // smallest l with v <= 2^l
+  int l = 0;
+  while ((1ull << l) < v) ++l;
+  return l;
+}
+
+}  // namespace
+
+// m ~= b / 2^c with |b| < 2^31 and 0 <= c <= 31 (Appendix C.1, dyadic requantization)
+int dyadic(double m, int32_t* b, int32_t* c) {
+  if (!std::isfinite(m)) return IBERT_ERR_SCALE_RANGE;
+  if (m == 0.0) { *b = 0; *c = 0; return IBERT_OK; }
+  const double mag = std::fabs(m);
+  int exponent = 0;
+  std::frexp(mag, &exponent);                 // mag = f * 2^exponent, f in [0.5, 1)
+  int shift = 31 - exponent;
+  if (shift > 31) shift = 31;
+  if (shift < 0) return IBERT_ERR_SCALE_RANGE;
+  int64_t mult = (int64_t)std::floor(std::ldexp(mag, shift) + 0.5);
+  if (mult == (int64_t(1) << 31)) { mult >>= 1; shift -= 1; }
+  if (shift < 0) return IBERT_ERR_SCALE_RANGE;
+  *b = (int32_t)(m < 0.0 ? -mult : mult);
+  *c = shift;
+  return IBERT_OK;
+}
+
+// Algorithm 3 constants.  The pre-shift s_in keeps q_b within 15 bits so that
+// (q_p + q_b)^2 + q_c stays below 2^31; the post-shift s_out keeps every
+// exponential below 2^21 so that a row of up to 1024 of them sums in int32.
+int make_exp_consts(double S, int p_max, ExpConsts* k) {
+  if (!good_scale(S)) return IBERT_ERR_SCALE_RANGE;
+  if (p_max != 255 && p_max != 127) return IBERT_ERR_ARG;
+  const double coef_a = 0.3585, coef_b = 1.353, coef_c = 0.344;
+  const double ln2 = 0.6931471805599453;
+  int s_in = 0;
+  double Sp = S;
+  while (std::floor(coef_b / Sp) > 32767.0) {
+    if (++s_in > 62) return IBERT_ERR_SCALE_RANGE;
+    Sp = std::ldexp(S, s_in);
+  }
+  const double q_ln2 = std::floor(ln2 / Sp);
+  if (q_ln2 < 1.0) return IBERT_ERR_SCALE_RANGE;
+  const double q_b = std::floor(coef_b / Sp);
+  const double q_c = std::floor(coef_c / ((coef_a * Sp) * Sp));
+  const int64_t e_top = (int64_t)q_b * (int64_t)q_b + (int64_t)q_c;
+  if (e_top >= (int64_t(1) << 31)) return IBERT_ERR_SCALE_RANGE;
+  const int bl = bit_length_u64((uint64_t)e_top);
+  k->s_in = s_in;
+  k->q_ln2 = (uint32_t)q_ln2;
+  k->d_max = 31u * k->q_ln2;
+  if (k->d_max >= (1u << 20)) return IBERT_ERR_SCALE_RANGE;   // cannot happen: q_ln2 <= 16787
+  // floor(d / q_ln2) for d < 2^20 by multiplication: with l = ceil(log2 q_ln2) and
+  // m = floor(2^(20+l) / q_ln2) + 1 one has 2^(20+l) < m q_ln2 <= 2^(20+l) + 2^l, which makes
+  // floor(d m / 2^(20+l)) exact for every d < 2^20.  Evaluated as umulhi(d << 12, m) >> l.
+  k->div_l = ceil_log2_u32(k->q_ln2);
+  k->div_m = (uint32_t)((uint64_t(1) << (20 + k->div_l)) / k->q_ln2 + 1);
+  k->q_b = (int32_t)q_b;
+  k->q_c = (int32_t)q_c;
+  k->s_out = bl > 21 ? bl - 21 : 0;
+  k->pm8 = 8u * (uint32_t)p_max;
+  return IBERT_OK;
+}
+
+// Algorithm 2 constants plus the multiplier that takes round(g / 256) to int8 at S_out.
+int make_gelu_consts(double S, double S_out, GeluConsts* k) {
+  if (!good_scale(S) || !good_scale(S_out)) return IBERT_ERR_SCALE_RANGE;
+  const double coef_a = -0.2888, coef_b = -1.769;
+  const double S1 = S / std::sqrt(2.0);
+  int s_in = 0;
+  double S2 = S1;
+  while (-std::floor(coef_b / S2) > 16384.0) {
+    if (++s_in > 62) return IBERT_ERR_SCALE_RANGE;
+    S2 = std::ldexp(S1, s_in);
+  }
+  const double S_erf = (coef_a * S2) * S2;
+  const double q_b = std::floor(coef_b / S2);
+  const double q_c = std::floor(1.0 / S_erf);
+  if (q_c < -1.0e9) return IBERT_ERR_SCALE_RANGE;              // cannot happen: S2 >= 1.08e-4
+  const int bl = bit_length_u64((uint64_t)(-2 * (int64_t)q_c));
+  k->s_in = s_in;
+  k->nq_b = (int32_t)(-q_b);
+  k->q_c = (int32_t)q_c;
+  k->s_f = bl > 16 ? bl - 16 : 0;
+  const double S_g = std::ldexp(S * S_erf, k->s_f) / 2.0;     // scale of q * ((q_erf + q_1) >> s_f)
+  const double S_g2 = S_g * 256.0;                            // after the rounding shift by 8
+  return dyadic(S_g2 / S_out, &k->b, &k->c);
+}
+
+// LayerNorm affine + requantization folded into one dyadic step per channel: the
+// normalized value n ~ y_hat * 2^16, out = (n * b_i + B_i) >> c with a shared c.
+int make_ln_tables(const double* gamma, const double* beta, int C, double S_out, int32_t* c_out,
+                   std::vector<int32_t>* b_i, std::vector<int64_t>* B_i) {
+  if (!good_scale(S_out)) return IBERT_ERR_SCALE_RANGE;
+  const double m0 = 1.0 / (S_out * 65536.0);
+  double g_max = 0.0;
+  for (int i = 0; i < C; ++i) {
+    if (!std::isfinite(gamma[i]) || !std::isfinite(beta[i])) return IBERT_ERR_ARG;
+    g_max = std::fmax(g_max, std::fabs(gamma[i]));
+  }
+  int32_t b_top = 0, c = 0;
+  int rc = dyadic(g_max * m0, &b_top, &c);
+  if (rc) return rc;
+  b_i->resize(C);
+  B_i->resize(C);
+  const int64_t half = c > 0 ? (int64_t(1) << (c - 1)) : 0;
+  for (int i = 0; i < C; ++i) {
+    const int64_t mag = (int64_t)std::floor(std::ldexp(std::fabs(gamma[i]) * m0, c) + 0.5);
+    const double add = std::floor(std::ldexp(beta[i] / S_out, c) + 0.5);
+    if (std::fabs(add) > 4.0e18) return IBERT_ERR_SCALE_RANGE;
+    (*b_i)[i] = (int32_t)(gamma[i] < 0.0 ? -mag : mag);
+    (*B_i)[i] = (int64_t)add + half;        // rounding constant folded in
+  }
+  *c_out = c;
+  return IBERT_OK;
+}
+
+int make_linear_tables(double S_x, const double* S_w, int N, const double* S_out_cols, double S_out,
+                       std::vector<int32_t>* b, std::vector<int32_t>* c) {
+  if (!good_scale(S_x)) return IBERT_ERR_SCALE_RANGE;
+  b->resize(N);
+  c->resize(N);
+  for (int n = 0; n < N; ++n) {
+    const double so = S_out_cols ? S_out_cols[n] : S_out;
+    if (!good_scale(so) || !good_scale(S_w[n])) return IBERT_ERR_SCALE_RANGE;
+    int rc = dyadic((S_x * S_w[n]) / so, &(*b)[n], &(*c)[n]);
+    if (rc) return rc;
+  }
+  return IBERT_OK;
+}
+
+}  // namespace ibert

@@ -1,0 +1,119 @@
+// Internal declarations shared by the translation units of libibert_b200.
+// Host-side constant derivation, the context object and the kernel launchers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <map>
+#include <vector>
+
+#include "../../include/ibert.h"
+
+namespace ibert {
+
+// ---------------------------------------------------------------------------------------
+// Integer constants the host derives from scales (kernels never see a floating-point value)
+// ---------------------------------------------------------------------------------------
+
+// i-exp / i-softmax (Algorithm 3).  S' = S * 2^s_in is the scale the polynomial works at.
+struct ExpConsts {
+  int32_t s_in;      // static pre-shift of the distance from the row maximum
+  uint32_t q_ln2;    // floor(ln2 / S')
+  uint32_t d_max;    // 31 * q_ln2: any larger distance gives e = 0
+  uint32_t div_m;    // magic multiplier: floor(d / q_ln2) = umulhi(d << 12, div_m) >> div_l for d < 2^20
+  int32_t div_l;
+  int32_t q_b;       // floor(1.353 / S')
+  int32_t q_c;       // floor(0.344 / (0.3585 S'^2))
+  int32_t s_out;     // static post-shift: every e < 2^21
+  uint32_t pm8;      // 8 * p_max (numerator pre-scale of the per-row quotient)
+};
+
+// i-GELU (Algorithm 2) followed by requantization to int8
+struct GeluConsts {
+  int32_t s_in;      // static pre-shift of the erf argument
+  int32_t nq_b;      // -floor(-1.769 / S2) > 0: clip point of |q| and offset of the polynomial
+  int32_t q_c;       // floor(1 / (-0.2888 S2^2)) < 0 (also q_1 = floor(1 / S_erf))
+  int32_t s_f;       // shift keeping q * (q_erf + q_1) in 32 bits
+  int32_t b, c;      // dyadic multiplier from the scale of round(g / 256) to S_out
+};
+
+// residual add in front of i-LayerNorm
+struct LnConsts {
+  int32_t C;
+  int32_t has_res;
+  int32_t b_r, c_r;  // dyadic(S_r / S)
+  int32_t c;         // common shift of the per-channel affine multipliers
+};
+
+int dyadic(double m, int32_t* b, int32_t* c);
+int make_exp_consts(double S, int p_max, ExpConsts* k);
+int make_gelu_consts(double S, double S_out, GeluConsts* k);
+// per-channel multipliers b_i (int32) and addends B_i (int64, rounding constant included)
+int make_ln_tables(const double* gamma, const double* beta, int C, double S_out, int32_t* c_out,
+                   std::vector<int32_t>* b_i, std::vector<int64_t>* B_i);
+// per-output-channel dyadic multipliers of a linear layer; S_out_cols (N entries) or S_out
+int make_linear_tables(double S_x, const double* S_w, int N, const double* S_out_cols, double S_out,
+                       std::vector<int32_t>* b, std::vector<int32_t>* c);
+
+// ---------------------------------------------------------------------------------------
+// Context
+// ---------------------------------------------------------------------------------------
+
+struct DeviceTable {
+  void* ptr = nullptr;
+  size_t bytes = 0;
+};
+
+}  // namespace ibert
+
+struct ibert_ctx {
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  int32_t* d_status = nullptr;       // first device-side error (0 = none)
+  int num_sms = 0;
+  // derived constant tables already on the device, keyed by a hash of their host bytes
+  std::map<uint64_t, ibert::DeviceTable> tables;
+  // workspace for the encoder layer's intermediates
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+};
+
+namespace ibert {
+
+// uploads `bytes` of host data once per distinct content; returns the device copy
+int cached_upload(ibert_ctx* ctx, const void* host, size_t bytes, uint64_t tag, void** dev);
+
+// ---------------------------------------------------------------------------------------
+// Kernel launchers (each returns an IBERT_* code; all enqueue on ctx->stream)
+// ---------------------------------------------------------------------------------------
+
+int launch_gelu(ibert_ctx* ctx, const int32_t* q, int64_t n, const GeluConsts& k, int8_t* out);
+int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const ExpConsts& k, uint8_t* out);
+int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t rows, const LnConsts& k,
+                     const int32_t* d_b, const int64_t* d_B, int8_t* out);
+
+// epilogue kinds of the GEMM
+enum : int { EPI_INT8 = 0, EPI_Q16 = 1, EPI_RAW = 2, EPI_GELU = 3 };
+
+struct GemmEpilogue {
+  int kind;
+  const int32_t* d_b;      // [N] dyadic multipliers (unused for EPI_RAW)
+  const int32_t* d_c;      // [N] dyadic shifts
+  const int32_t* d_bias;   // [N] or nullptr
+  GeluConsts gelu;         // EPI_GELU only
+};
+
+int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, int N, int K,
+                   const GemmEpilogue& epi, void* out);
+
+struct AttnConsts {
+  ExpConsts e;
+  int32_t b, c;            // dyadic((1/p_max) * S_v / S_ctx)
+  int32_t p_signed;        // 0: probabilities are u8 (p_max 255); 1: fit int8 (p_max 127)
+};
+
+int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
+                     const AttnConsts& k, int8_t* out);
+
+}  // namespace ibert

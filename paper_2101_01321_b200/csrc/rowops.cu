@@ -1,0 +1,273 @@
+// Standalone integer non-linearities: i-GELU (Algorithm 2), i-softmax (Algorithm 3) and
+// residual + i-LayerNorm (Sec. 3.6, Algorithm 4).  All three are HBM-streaming kernels:
+// 128-bit coalesced loads of the int32 inputs, all arithmetic in registers, packed int8
+// stores.  Rows are owned by one warp and reduced with warp shuffles.
+#include "device_utils.cuh"
+
+namespace ibert {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ uint32_t pack4(int32_t a, int32_t b, int32_t c, int32_t d) {
+  return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) |
+         ((uint32_t)(d & 0xff) << 24);
+}
+
+// ----------------------------------------------------------------------------- i-GELU
+// Each thread converts 4 int4 vectors (16 values); vector j of a thread sits 32 vectors
+// after vector j-1 so that every load and store instruction of a warp is contiguous.
+__global__ void __launch_bounds__(kThreads) gelu_kernel(const int32_t* __restrict__ q, int64_t n,
+                                                        GeluConsts k, int8_t* __restrict__ out) {
+  const int64_t half = rounding_half(k.c);
+  const int64_t n_vec = n >> 2;
+  const int lane = threadIdx.x & 31;
+  const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
+  const int4* q4 = reinterpret_cast<const int4*>(q);
+  uint32_t* o4 = reinterpret_cast<uint32_t*>(out);
+  for (int64_t base = warp_global * 128; base < n_vec; base += warp_count * 128) {
+    int4 v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t idx = base + j * 32 + lane;
+      v[j] = idx < n_vec ? __ldcs(q4 + idx) : make_int4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t idx = base + j * 32 + lane;
+      if (idx < n_vec) {
+        const int32_t a = igelu_q16_to_int8(clamp_sym(v[j].x, 32767), k, half);
+        const int32_t b = igelu_q16_to_int8(clamp_sym(v[j].y, 32767), k, half);
+        const int32_t c = igelu_q16_to_int8(clamp_sym(v[j].z, 32767), k, half);
+        const int32_t d = igelu_q16_to_int8(clamp_sym(v[j].w, 32767), k, half);
+        __stcs(o4 + idx, pack4(a, b, c, d));
+      }
+    }
+  }
+  // ragged tail (n not a multiple of 4)
+  const int64_t tid = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  const int64_t tail = n_vec << 2;
+  if (tid < n - tail)
+    out[tail + tid] = (int8_t)igelu_q16_to_int8(clamp_sym(q[tail + tid], 32767), k, half);
+}
+
+// ----------------------------------------------------------------------------- i-softmax
+// One warp per row; a lane keeps VPL int4 vectors (4*VPL scores) in registers.
+// VEC: rows are 16-byte aligned (L % 4 == 0) and loaded/stored as vectors.
+template <int VPL, bool VEC>
+__global__ void __launch_bounds__(kThreads) softmax_kernel(const int32_t* __restrict__ q, int64_t rows,
+                                                           int L, ExpConsts k, uint8_t* __restrict__ out) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
+  for (int64_t row = warp_global; row < rows; row += warp_count) {
+    const int32_t* qr = q + row * L;
+    uint8_t* orow = out + row * L;
+    int32_t v[VPL][4];
+    int32_t mx = INT32_MIN;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int col = 4 * (j * 32 + lane);
+      if (VEC) {
+        if (col < L) {
+          const int4 t = __ldcs(reinterpret_cast<const int4*>(qr + col));
+          v[j][0] = t.x; v[j][1] = t.y; v[j][2] = t.z; v[j][3] = t.w;
+        } else {
+          v[j][0] = v[j][1] = v[j][2] = v[j][3] = INT32_MIN;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[j][i] = (col + i < L) ? qr[col + i] : INT32_MIN;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) mx = max(mx, v[j][i]);
+    }
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    uint32_t sum = 0;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int col = 4 * (j * 32 + lane);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t e = (col + i < L) ? iexp_dist((uint32_t)mx - (uint32_t)v[j][i], k) : 0u;
+        v[j][i] = (int32_t)e;
+        sum += e;
+      }
+    }
+    sum = __reduce_add_sync(0xffffffffu, sum);
+    const RowDivisor rd = make_row_divisor(sum);
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int col = 4 * (j * 32 + lane);
+      uint32_t p[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) p[i] = softmax_quotient((uint32_t)v[j][i], k.pm8, rd);
+      if (VEC) {
+        if (col < L)
+          __stcs(reinterpret_cast<uint32_t*>(orow + col), p[0] | (p[1] << 8) | (p[2] << 16) | (p[3] << 24));
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (col + i < L) orow[col + i] = (uint8_t)p[i];
+      }
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------- i-LayerNorm
+// One warp per row, the whole row in registers (VPL int4 vectors per lane).
+template <int VPL, bool VEC>
+__global__ void __launch_bounds__(kThreads) layernorm_kernel(const int32_t* __restrict__ q,
+                                                             const int8_t* __restrict__ r, int64_t rows,
+                                                             LnConsts k, const int32_t* __restrict__ b_i,
+                                                             const int64_t* __restrict__ B_i,
+                                                             int8_t* __restrict__ out) {
+  const int lane = threadIdx.x & 31;
+  const int C = k.C;
+  const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
+  const int64_t half_r = rounding_half(k.c_r);
+  for (int64_t row = warp_global; row < rows; row += warp_count) {
+    const int32_t* qr = q + row * C;
+    const int8_t* rr = r + row * C;
+    int8_t* orow = out + row * C;
+    int32_t v[VPL][4];
+    int32_t sum = 0;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int col = 4 * (j * 32 + lane);
+      if (VEC) {
+        if (col < C) {
+          const int4 t = __ldcs(reinterpret_cast<const int4*>(qr + col));
+          v[j][0] = t.x; v[j][1] = t.y; v[j][2] = t.z; v[j][3] = t.w;
+          if (k.has_res) {
+            const uint32_t rw = __ldcs(reinterpret_cast<const uint32_t*>(rr + col));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int32_t rv = (int32_t)(int8_t)(rw >> (8 * i));
+              v[j][i] += (int32_t)(((int64_t)rv * k.b_r + half_r) >> k.c_r);
+            }
+          }
+        } else {
+          v[j][0] = v[j][1] = v[j][2] = v[j][3] = 0;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          int32_t t = 0;
+          if (col + i < C) {
+            t = qr[col + i];
+            if (k.has_res) t += (int32_t)(((int64_t)rr[col + i] * k.b_r + half_r) >> k.c_r);
+          }
+          v[j][i] = t;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) sum += v[j][i];
+    }
+    sum = __reduce_add_sync(0xffffffffu, sum);
+    // mu = floor(sum / C)
+    int32_t mu = sum / C;
+    if (sum - mu * C < 0) mu -= 1;
+    uint64_t ss = 0;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int col = 4 * (j * 32 + lane);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int32_t y = (col + i < C) ? v[j][i] - mu : 0;
+        v[j][i] = y;
+        ss += (uint64_t)((int64_t)y * (int64_t)y);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const uint64_t var = ss / (uint64_t)C;
+    uint32_t sigma = isqrt_newton(var);
+    sigma = sigma < 1u ? 1u : sigma;
+    const int64_t rho64 = (int64_t)(0x80000000u / sigma);        // floor(2^31 / sigma)
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int col = 4 * (j * 32 + lane);
+      int32_t o[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        o[i] = 0;
+        if (col + i < C) {
+          const int32_t nrm = (int32_t)(((int64_t)v[j][i] * rho64) >> 15);
+          int64_t t = (int64_t)nrm * (int64_t)__ldg(b_i + col + i) + __ldg(B_i + col + i);
+          t >>= k.c;
+          t = t > 127 ? 127 : t;
+          t = t < -127 ? -127 : t;
+          o[i] = (int32_t)t;
+        }
+      }
+      if (VEC) {
+        if (col < C) __stcs(reinterpret_cast<uint32_t*>(orow + col), pack4(o[0], o[1], o[2], o[3]));
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (col + i < C) orow[col + i] = (int8_t)o[i];
+      }
+    }
+  }
+}
+
+int grid_for(ibert_ctx* ctx, int64_t work_warps, int max_ctas_per_sm) {
+  const int64_t ctas = (work_warps + (kThreads / 32) - 1) / (kThreads / 32);
+  const int64_t cap = (int64_t)ctx->num_sms * max_ctas_per_sm;
+  return (int)(ctas < 1 ? 1 : (ctas > cap ? cap : ctas));
+}
+
+int check_launch() { return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA; }
+
+}  // namespace
+
+int launch_gelu(ibert_ctx* ctx, const int32_t* q, int64_t n, const GeluConsts& k, int8_t* out) {
+  if (n == 0) return IBERT_OK;
+  const int64_t warps = ((n >> 2) + 127) / 128 + 1;
+  gelu_kernel<<<grid_for(ctx, warps, 8), kThreads, 0, ctx->stream>>>(q, n, k, out);
+  return check_launch();
+}
+
+int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const ExpConsts& k, uint8_t* out) {
+  if (rows == 0) return IBERT_OK;
+  const int grid = grid_for(ctx, rows, 8);
+  const bool vec = (L % 4) == 0;
+  const int vpl = (L + 127) / 128;   // vectors per lane
+#define IBERT_SM(V)                                                                              \
+  do {                                                                                           \
+    if (vec) softmax_kernel<V, true><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out);    \
+    else softmax_kernel<V, false><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out);       \
+  } while (0)
+  if (vpl <= 1) IBERT_SM(1);
+  else if (vpl <= 2) IBERT_SM(2);
+  else if (vpl <= 4) IBERT_SM(4);
+  else IBERT_SM(8);
+#undef IBERT_SM
+  return check_launch();
+}
+
+int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t rows, const LnConsts& k,
+                     const int32_t* d_b, const int64_t* d_B, int8_t* out) {
+  if (rows == 0) return IBERT_OK;
+  const int grid = grid_for(ctx, rows, 8);
+  const bool vec = (k.C % 4) == 0;
+  const int vpl = (k.C + 127) / 128;
+#define IBERT_LN(V)                                                                                     \
+  do {                                                                                                  \
+    if (vec) layernorm_kernel<V, true><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out); \
+    else layernorm_kernel<V, false><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);    \
+  } while (0)
+  if (vpl <= 2) IBERT_LN(2);
+  else if (vpl <= 4) IBERT_LN(4);
+  else if (vpl <= 6) IBERT_LN(6);
+  else if (vpl <= 8) IBERT_LN(8);
+  else IBERT_LN(16);
+#undef IBERT_LN
+  return check_launch();
+}
+
+}  // namespace ibert

@@ -1,0 +1,113 @@
+"""GPU parity (bit-exact) of the fused attention kernel and the whole encoder layer."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import assert_same, ctx, dev, host
+from paper_2101_01321_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("B,L,heads", [(1, 16, 1), (2, 37, 2), (1, 128, 12), (3, 128, 2), (2, 200, 2), (1, 256, 3),
+                                       (1, 512, 2), (2, 1, 1), (1, 33, 1), (1, 300, 1), (0, 64, 1)])
+@pytest.mark.parametrize("p_max", [255, 127])
+def test_attention_matches_oracle(B, L, heads, p_max):
+    H = heads * 64
+    rng = np.random.default_rng(L * 7 + heads)
+    qkv = np.clip(np.rint(rng.standard_normal((max(B, 1) * L, 3 * H)) * 40), -127, 127).astype(np.int8)[:B * L]
+    S_q = S_k = 0.02
+    S_v, S_ctx = 0.02, 0.006
+    out, S_ret = ctx().ibert_attention_i8(dev(qkv), B, L, H, heads, S_q, S_k, S_v, S_ctx, p_max)
+    ctx().check()
+    assert S_ret == S_ctx
+    if B:
+        want = oracle.attention(qkv, B, L, H, heads, S_q, S_k, S_v, S_ctx, p_max)
+        assert_same(host(out), want, f"attention L={L}")
+        assert np.abs(want).max() > 20
+
+
+def test_attention_peaked_and_uniform_rows():
+    B, L, heads = 1, 128, 2
+    H = heads * 64
+    rng = np.random.default_rng(0)
+    qkv = rng.integers(-127, 128, (L, 3 * H)).astype(np.int8)       # full-range scores: one-hot rows
+    qkv[:, 64:128] = 0                                              # head 1: q = 0 -> uniform rows
+    for S_qk in (0.05, 0.004):
+        out, _ = ctx().ibert_attention_i8(dev(qkv), B, L, H, heads, S_qk, S_qk, 0.02, 0.01, 255)
+        want = oracle.attention(qkv, B, L, H, heads, S_qk, S_qk, 0.02, 0.01, 255)
+        assert_same(host(out), want, "attention peaked")
+    ctx().check()
+
+
+def _run_layers(x, params, B, L):
+    c = ctx()
+    h = dev(x)
+    outs = []
+    for p in params:
+        layer = c.ibert_layer_create(p)
+        h, S = c.ibert_encoder_layer(layer, h, B, L)
+        assert S == p["S_out"]
+        outs.append(host(h))
+        c.check()
+        layer.close()
+    return outs
+
+
+@pytest.mark.parametrize("B,L,H,heads,F", [(2, 16, 128, 2, 256), (1, 37, 64, 1, 64), (3, 128, 256, 4, 1024)])
+def test_small_encoder_layers_match_oracle(B, L, H, heads, F):
+    x, params = synth.make_model(0, B, layers=2, H=H, heads=heads, F=F, L=L)
+    outs = _run_layers(x, params, B, L)
+    h = x
+    for p, got in zip(params, outs):
+        h = oracle.encoder_layer(p, h, B, L).out
+        assert_same(got, h, "encoder layer")
+
+
+def test_config0_roberta_base_layer_matches_oracle():
+    x, params = synth.make_model(0, 1)
+    got = _run_layers(x, params, 1, 128)[0]
+    want = oracle.encoder_layer(params[0], x, 1, 128).out
+    assert_same(got, want, "config 0")
+    assert want.std() > 20
+
+
+def test_config2_three_layers_batch8_match_oracle():
+    B, L = 8, 128
+    x, params = synth.make_model(2, B, layers=3)
+    outs = _run_layers(x, params, B, L)
+    h = x
+    for p, got in zip(params, outs):
+        h = oracle.encoder_layer(p, h, B, L).out
+        assert_same(got, h, "config 2 layer")
+
+
+def test_large_shapes_one_layer_L256_and_L512():
+    for cfg, B in ((3, 2), (4, 1)):
+        L = synth.CONFIGS[cfg].L
+        x, params = synth.make_model(cfg, B, layers=1)
+        got = _run_layers(x, params, B, L)[0]
+        want = oracle.encoder_layer(params[0], x, B, L).out
+        assert_same(got, want, f"config {cfg}")
+
+
+def test_layer_error_codes():
+    from paper_2101_01321_b200.binding import IbertError
+    x, params = synth.make_model(0, 1, layers=1, H=128, heads=2, F=256, L=16)
+    bad = dict(params[0])
+    bad["S_q"] = -1.0
+    with pytest.raises(IbertError) as e:
+        ctx().ibert_layer_create(bad)
+    assert e.value.code == -3
+    bad = dict(params[0])
+    bad["heads"] = 3
+    with pytest.raises(IbertError) as e:
+        ctx().ibert_layer_create(bad)
+    assert e.value.code == -2
+    layer = ctx().ibert_layer_create(params[0])
+    with pytest.raises(IbertError) as e:
+        ctx().ibert_encoder_layer(layer, dev(x), 1, 513)
+    assert e.value.code == -2
+    layer.close()
+    assert ctx().ibert_last_status() == 0

@@ -1,0 +1,101 @@
+"""GPU parity (bit-exact) of the tcgen05 INT8 GEMM and its fused epilogues against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import assert_same, ctx, dev, host
+
+pytestmark = pytest.mark.gpu
+
+
+def _problem(M, N, K, seed, acc_scale=1.0):
+    rng = np.random.default_rng(seed)
+    x = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    w = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    bias = rng.integers(-200000, 200000, N).astype(np.int32)
+    S_w = rng.uniform(1e-4, 4e-4, N)
+    S_x = 0.03
+    amax = 127.0 * 127.0 * np.sqrt(K) * 1.2 * S_x * 2.5e-4 * acc_scale
+    return x, w, bias, S_w, S_x, amax
+
+
+SHAPES = [(1, 16, 16), (7, 48, 80), (128, 128, 128), (130, 272, 144), (300, 768, 768), (257, 2304, 768),
+          (129, 768, 3072), (1024, 1024, 1024), (4100, 512, 256), (2100, 2304, 768), (0, 64, 64)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_linear_raw_accumulators(M, N, K):
+    x, w, bias, S_w, S_x, _ = _problem(M, N, K, 1)
+    out, S_ret = ctx().ibert_linear_i8(dev(x), S_x, dev(w), S_w, dev(bias), 2)
+    ctx().check()
+    if M:
+        assert_same(host(out), oracle.linear(x, S_x, w, S_w, bias, 2), "raw")
+    assert np.array_equal(S_ret, S_x * S_w)
+    out, _ = ctx().ibert_linear_i8(dev(x), S_x, dev(w), S_w, None, 2)
+    ctx().check()
+    if M:
+        assert_same(host(out), oracle.linear(x, S_x, w, S_w, None, 2), "raw, no bias")
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("kind", [0, 1])
+def test_linear_requantized(M, N, K, kind):
+    x, w, bias, S_w, S_x, amax = _problem(M, N, K, 2)
+    S_out = amax / (100.0 if kind == 0 else 20000.0)       # a few values clamp
+    out, S_ret = ctx().ibert_linear_i8(dev(x), S_x, dev(w), S_w, dev(bias), kind, S_out)
+    ctx().check()
+    assert S_ret == S_out
+    if M:
+        want = oracle.linear(x, S_x, w, S_w, bias, kind, S_out)
+        assert_same(host(out), want, f"kind {kind}")
+        qmax = 127 if kind == 0 else 32767
+        assert np.abs(want.astype(np.int64)).max() <= qmax
+
+
+@pytest.mark.parametrize("M,N,K", [(7, 48, 80), (300, 768, 768), (257, 3072, 768), (1000, 4096, 1024)])
+def test_linear_with_fused_gelu(M, N, K):
+    x, w, bias, S_w, S_x, amax = _problem(M, N, K, 3)
+    # scale the problem so the GELU input covers about [-6, 6]
+    S_mid = 6.0 / 32767.0
+    S_x = S_x * (6.0 / amax)
+    S_out = 6.0 / 127.0
+    out, S_ret = ctx().ibert_linear_gelu_i8(dev(x), S_x, dev(w), S_w, dev(bias), S_mid, S_out)
+    ctx().check()
+    mid = oracle.linear(x, S_x, w, S_w, bias, 1, S_mid)
+    want, _ = oracle.gelu(mid, S_mid, S_out)
+    assert_same(host(out), want, "linear+gelu")
+    assert np.abs(mid).max() > 8000 and want.max() > 60
+
+
+def test_linear_odd_dyadic_shifts_and_negative_results():
+    # multipliers >= 1 (small shifts) and a large-bias column block
+    M, N, K = 64, 64, 64
+    rng = np.random.default_rng(11)
+    x = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    w = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    bias = rng.integers(-2 ** 28, 2 ** 28, N).astype(np.int32)
+    S_w = np.geomspace(1e-6, 10.0, N)
+    for kind, S_out in ((0, 1e-3), (1, 1e-5), (0, 50.0), (1, 0.2)):
+        out, _ = ctx().ibert_linear_i8(dev(x), 0.5, dev(w), S_w, dev(bias), kind, S_out)
+        assert_same(host(out), oracle.linear(x, 0.5, w, S_w, bias, kind, S_out), f"kind {kind} S_out {S_out}")
+    ctx().check()
+
+
+def test_linear_error_codes():
+    from paper_2101_01321_b200.binding import IbertError
+    x = torch.zeros((4, 24), dtype=torch.int8, device="cuda")
+    w = torch.zeros((16, 24), dtype=torch.int8, device="cuda")
+    with pytest.raises(IbertError) as e:
+        ctx().ibert_linear_i8(x, 1.0, w, np.ones(16), None, 0, 1.0)      # K % 16 != 0
+    assert e.value.code == -2
+    x = torch.zeros((4, 32), dtype=torch.int8, device="cuda")
+    w = torch.zeros((8, 32), dtype=torch.int8, device="cuda")
+    with pytest.raises(IbertError) as e:
+        ctx().ibert_linear_i8(x, 1.0, w, np.ones(8), None, 0, 1.0)       # int8 rows need N % 16 == 0
+    assert e.value.code == -2
+    w = torch.zeros((16, 32), dtype=torch.int8, device="cuda")
+    with pytest.raises(IbertError) as e:
+        ctx().ibert_linear_i8(x, 1.0, w, np.full(16, 1e30), None, 0, 1e-30)  # multiplier >= 2^31
+    assert e.value.code == -3
+    assert ctx().ibert_last_status() == 0

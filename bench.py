@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Throughput of the integer-only RoBERTa-Base encoder (I-BERT) on B200.
+
+One *step* = one forward pass of the whole 12-layer integer-only encoder (7 kernels per
+layer, all inside libibert_b200) over one batch of synthetic int8 activations.
+Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle instead.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--config 2|3|4] [--batch B]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "tokens/s int-only RoBERTa-Base on 1 B200; % INT8 TC peak, % HBM for i-ops"
+UNIT = "tokens/s"
+DEFAULT_BATCH = {2: 128, 3: 32, 4: 64}
+
+
+# --------------------------------------------------------------------------- helpers
+def measured_peaks() -> tuple[dict, str]:
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"])}, "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 6:
+                self.rows.append(parts)
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        mhz, mx, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                mhz.append(float(r[0]))
+                mx = float(r[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(mhz)}
+
+
+def algorithmic_work(H: int, F: int, L: int, heads: int, T: int) -> dict:
+    """Per-launch algorithmic ops / bytes of each kernel class of one layer on T tokens."""
+    w = {}
+    w["gemm_qkv"] = {"ops": 2.0 * T * 3 * H * H, "bytes": T * H + 3 * H * H + T * 3 * H}
+    w["attention"] = {"ops": 2.0 * T * L * 64 * 2 * heads, "bytes": T * 3 * H + T * H}
+    w["gemm_out"] = {"ops": 2.0 * T * H * H, "bytes": T * H + H * H + 4 * T * H}
+    w["layernorm"] = {"ops": 0.0, "bytes": 4 * T * H + T * H + T * H}
+    w["gemm_ffn1_gelu"] = {"ops": 2.0 * T * F * H, "bytes": T * H + F * H + T * F}
+    w["gemm_ffn2"] = {"ops": 2.0 * T * F * H, "bytes": T * F + F * H + 4 * T * H}
+    return w
+
+
+# --------------------------------------------------------------------------- reference arm
+def oracle_sample_run(cfg_id: int, n_seq: int, layers: int | None = None):
+    """Runs the CPU oracle on the first n_seq sequences of the workload; returns (tokens, seconds)."""
+    import oracle
+    from paper_2101_01321_b200 import synth
+    cfg = synth.CONFIGS[cfg_id]
+    x, params = synth.make_model(cfg_id, n_seq, layers=layers)
+    oracle.lib()
+    t0 = time.perf_counter()
+    h = x
+    for p in params:
+        h = oracle.encoder_layer(p, h, n_seq, cfg.L).out
+    dt = time.perf_counter() - t0
+    return n_seq * cfg.L, dt, len(params)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2101_01321_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    batch = args.batch or DEFAULT_BATCH[args.config]
+    n_seq = 2
+    x, params = synth.make_model(args.config, n_seq)
+    oracle.lib()
+
+    def step():
+        h = x
+        for p in params:
+            h = oracle.encoder_layer(p, h, n_seq, cfg.L).out
+        return h
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    tokens = n_seq * cfg.L * args.steps
+    value = tokens / dt
+    sample = (f"each step = first {n_seq} sequences ({n_seq * cfg.L} tokens) of the batch through all "
+              f"{len(params)} layers with the CPU oracle")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+        "data": "synthetic", "config": workload_config(cfg, batch, args.gpus),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def workload_config(cfg, batch, n_gpus):
+    return {"workload": f"config {cfg.config_id}: {cfg.layers}-layer integer-only encoder, H={cfg.H}, "
+                        f"heads={cfg.heads}, FFN={cfg.F}, L={cfg.L}, B={batch} per GPU",
+            "layers": cfg.layers, "hidden": cfg.H, "heads": cfg.heads, "ffn": cfg.F, "seq_len": cfg.L,
+            "batch_per_gpu": batch, "global_batch": batch * n_gpus, "parallelism": f"dp{n_gpus} (batch shards, no collective)",
+            "l2": "flushed between timed steps (512 MiB write); per-step activation traffic also exceeds L2"}
+
+
+# --------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import numpy as np
+    import torch
+
+    from paper_2101_01321_b200 import binding, build, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    build.build()
+
+    cfg = synth.CONFIGS[args.config]
+    batch = args.batch or DEFAULT_BATCH[args.config]
+    T = batch * cfg.L
+    x_np, params = synth.make_model(args.config, batch)
+    stream = torch.cuda.Stream(device=dev)
+    ctx = binding.Context(local_rank, stream)
+    layers = [ctx.ibert_layer_create(p) for p in params]
+    x_dev = torch.from_numpy(x_np).to(dev)
+    bufs = [torch.empty((T, cfg.H), dtype=torch.int8, device=dev) for _ in range(2)]
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    x_pin = torch.from_numpy(x_np).pin_memory()
+    out_pin = torch.empty((T, cfg.H), dtype=torch.int8).pin_memory()
+    x_stage = torch.empty((T, cfg.H), dtype=torch.int8, device=dev)
+
+    def forward(src):
+        h = src
+        for i, ly in enumerate(layers):
+            h, _ = ctx.ibert_encoder_layer(ly, h, batch, cfg.L, out=bufs[i & 1])
+        return h
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed_steps(n, e2e=False):
+        """Per-step CUDA events on the launching stream; L2 flushed (untimed) between steps."""
+        times = []
+        with torch.cuda.stream(stream):
+            for _ in range(n):
+                flush.fill_(1)
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                if e2e:
+                    x_stage.copy_(x_pin, non_blocking=True)
+                    h = forward(x_stage)
+                    out_pin.copy_(h, non_blocking=True)
+                else:
+                    forward(x_dev)
+                e1.record(stream)
+                times.append((e0, e1))
+        stream.synchronize()
+        return [a.elapsed_time(b) for a, b in times]
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            forward(x_dev)
+    stream.synchronize()
+    ctx.check()
+
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    t_steps = timed_steps(args.steps)
+    barrier()
+    clocks = sampler.stop()
+    ctx.check()
+    total_ms = sum(t_steps)
+
+    timed_steps(2, e2e=True)
+    barrier()
+    t_e2e = timed_steps(args.steps, e2e=True)
+    barrier()
+    total_e2e_ms = sum(t_e2e)
+
+    # per-kernel device time of the same steps (separate pass: event pairs around every launch)
+    with torch.cuda.stream(stream):
+        ctx.ibert_profile_begin()
+        prof_steps = min(args.steps, 5)
+        for _ in range(prof_steps):
+            flush.fill_(1)
+            forward(x_dev)
+        prof = ctx.ibert_profile_end()
+    ctx.check()
+
+    if dist is not None:
+        t = torch.tensor([total_ms, total_e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, total_e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        work = algorithmic_work(cfg.H, cfg.F, cfg.L, cfg.heads, T)
+        kern = {}
+        for k, (ms, n) in prof.items():
+            if n == 0:
+                continue
+            per = ms / n
+            w = work.get(k, {"ops": 0.0, "bytes": 0.0})
+            kern[k] = {"launches_per_step": n // prof_steps, "ms_per_launch": per,
+                       "share": ms / sum(v[0] for v in prof.values()),
+                       "tops": w["ops"] / per / 1e9 if w["ops"] else None,
+                       "gbs": w["bytes"] / per / 1e6}
+        top = max(kern, key=lambda k: kern[k]["share"])
+        int8_peak = 2.0 * peaks["bf16_tflops_sustained"]     # nominal INT8 : BF16 dense ratio = 2
+        if work[top]["ops"]:
+            roof = {"kernel": top, "bound": "tensor", "achieved": kern[top]["tops"], "peak": int8_peak,
+                    "unit": "TOP/s", "frac": kern[top]["tops"] / int8_peak, "traffic": None,
+                    "peak_source": f"2 x {peak_kind} sustained bf16 cuBLAS rate (int8 dense = 2x bf16 nominal)"}
+        else:
+            roof = {"kernel": top, "bound": "hbm", "achieved": kern[top]["gbs"], "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": kern[top]["gbs"] / peaks["hbm_gbs"], "traffic": None,
+                    "peak_source": f"{peak_kind} copy bandwidth"}
+        roof["ms_per_launch"] = kern[top]["ms_per_launch"]
+        tokens = T * args.steps * world
+        value = tokens / (total_ms / 1e3)
+        e2e_value = tokens / (total_e2e_ms / 1e3)
+
+        # CPU baseline: the oracle on a bounded sample of the same workload
+        n_seq = 8
+        tok_s, dt_s, n_layers = oracle_sample_run(args.config, n_seq)
+        import oracle
+        cpu = {"value": tok_s / dt_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"first {n_seq} sequences ({tok_s} tokens) through all {n_layers} layers, {dt_s:.1f} s"}
+
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": workload_config(cfg, batch, world),
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": T * cfg.H,
+                    "d2h_bytes_per_step": T * cfg.H, "ms_per_step": total_e2e_ms / args.steps},
+            "gpu_launches": 7 * cfg.layers * args.steps,
+            "roofline": roof,
+            "kernels": kern,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    for ly in layers:
+        ly.close()
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4])
+    ap.add_argument("--batch", type=int, default=0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -137,6 +137,24 @@ int ibert_layer_destroy(ibert_layer* layer);
 int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* layer, const int8_t* x, int B, int L,
                         int8_t* out, double* S_ret);
 
+/* Per-kernel device timing (CUDA events recorded on the context's stream around every launch
+   between begin and end).  No counterpart in the paper: measurement support only.
+   ibert_profile_end synchronizes the stream and fills, per kernel class below, the summed
+   device milliseconds and the number of launches (arrays of IBERT_NUM_KERNEL_CLASSES). */
+enum {
+  IBERT_K_GEMM_QKV = 0,      /* ibert_linear_i8 kind 0 / layer step QKV   */
+  IBERT_K_ATTENTION = 1,
+  IBERT_K_GEMM_Q16 = 2,      /* Q16 / raw epilogue with K <= 2048: output projection */
+  IBERT_K_LAYERNORM = 3,
+  IBERT_K_GEMM_GELU = 4,     /* FFN1 with fused i-GELU */
+  IBERT_K_GEMM_Q16_WIDE = 5, /* Q16 / raw epilogue with K > 2048: FFN2 */
+  IBERT_K_GELU = 6,
+  IBERT_K_SOFTMAX = 7,
+  IBERT_NUM_KERNEL_CLASSES = 8
+};
+int ibert_profile_begin(ibert_ctx* ctx);
+int ibert_profile_end(ibert_ctx* ctx, float* ms, int32_t* launches);
+
 #ifdef __cplusplus
 }
 #endif

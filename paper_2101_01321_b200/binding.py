@@ -19,6 +19,8 @@ IBERT_OK = 0
 ERR_NAMES = {-1: "IBERT_ERR_ARG", -2: "IBERT_ERR_SHAPE", -3: "IBERT_ERR_SCALE_RANGE", -4: "IBERT_ERR_ALIGN",
              -5: "IBERT_ERR_NOMEM", -6: "IBERT_ERR_CUDA", -7: "IBERT_ERR_TIMEOUT", -8: "IBERT_ERR_VALUE_RANGE"}
 
+KERNEL_CLASSES = ("gemm_qkv", "attention", "gemm_out", "layernorm", "gemm_ffn1_gelu", "gemm_ffn2", "gelu",
+                  "softmax")
 SCALE_NAMES = ("S_x", "S_q", "S_k", "S_v", "S_ctx", "S_r1", "S_h1", "S_gi", "S_go", "S_r2", "S_out")
 
 
@@ -61,6 +63,10 @@ def lib():
         L.ibert_layer_create.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(vp)]
         L.ibert_layer_destroy.argtypes = [vp]
         L.ibert_encoder_layer.argtypes = [vp, vp, vp, i32, i32, vp, vp]
+        L.ibert_profile_begin.argtypes = [vp]
+        L.ibert_profile_end.argtypes = [vp, vp, vp]
+        L.ibert_profile_begin.restype = i32
+        L.ibert_profile_end.restype = i32
         for name in ("ibert_create", "ibert_destroy", "ibert_last_status", "ibert_dyadic_from_double",
                      "ibert_linear_i8", "ibert_linear_gelu_i8", "ibert_softmax_i", "ibert_gelu_i",
                      "ibert_layernorm_i", "ibert_attention_i8", "ibert_layer_create", "ibert_layer_destroy",
@@ -119,6 +125,16 @@ class Context:
 
     def check(self):
         _chk(self.ibert_last_status(), "ibert_last_status")
+
+    def ibert_profile_begin(self):
+        _chk(lib().ibert_profile_begin(self.h), "ibert_profile_begin")
+
+    def ibert_profile_end(self) -> dict:
+        """{kernel class name: (device ms summed, launches)} for the launches since profile_begin."""
+        ms = np.zeros(len(KERNEL_CLASSES), dtype=np.float32)
+        n = np.zeros(len(KERNEL_CLASSES), dtype=np.int32)
+        _chk(lib().ibert_profile_end(self.h, ms.ctypes.data, n.ctypes.data), "ibert_profile_end")
+        return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_CLASSES)}
 
     # ------------------------------------------------------------------ simple ops
     def ibert_gelu_i(self, q: torch.Tensor, S: float, S_out: float, out: torch.Tensor | None = None):

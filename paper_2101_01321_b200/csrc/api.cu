@@ -31,6 +31,33 @@ struct DeviceGuard {
   ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
 };
 
+// Records an event pair around one launch while profiling is on.
+struct ProfileScope {
+  ibert_ctx* ctx;
+  size_t slot = 0;
+  bool on = false;
+  ProfileScope(ibert_ctx* c, int kclass) : ctx(c) {
+    if (!c->profiling) return;
+    slot = c->ev_class.size();
+    while (c->ev_pool.size() < 2 * (slot + 1)) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      c->ev_pool.push_back(e);
+    }
+    c->ev_class.push_back(kclass);
+    on = cudaEventRecord(c->ev_pool[2 * slot], c->stream) == cudaSuccess;
+  }
+  ~ProfileScope() {
+    if (on) cudaEventRecord(ctx->ev_pool[2 * slot + 1], ctx->stream);
+  }
+};
+
+inline int gemm_class(int kind, int K) {
+  if (kind == EPI_INT8) return IBERT_K_GEMM_QKV;
+  if (kind == EPI_GELU) return IBERT_K_GEMM_GELU;
+  return K > 2048 ? IBERT_K_GEMM_Q16_WIDE : IBERT_K_GEMM_Q16;
+}
+
 }  // namespace
 
 namespace ibert {
@@ -127,6 +154,7 @@ int ibert_destroy(ibert_ctx* ctx) {
   DeviceGuard guard(ctx->device);
   cudaStreamSynchronize(ctx->stream);
   for (auto& kv : ctx->tables) cudaFree(kv.second.ptr);
+  for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   if (ctx->ws) cudaFree(ctx->ws);
   cudaFree(ctx->d_status);
   delete ctx;
@@ -152,7 +180,10 @@ int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S
   int rc = make_gelu_consts(S, S_out, &k);
   if (rc) return rc;
   DeviceGuard guard(ctx->device);
-  rc = launch_gelu(ctx, q, n, k, out);
+  {
+    ProfileScope ps(ctx, IBERT_K_GELU);
+    rc = launch_gelu(ctx, q, n, k, out);
+  }
   if (rc == IBERT_OK && S_ret) *S_ret = S_out;
   return rc;
 }
@@ -168,7 +199,10 @@ int ibert_softmax_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, in
   int rc = make_exp_consts(S, p_max, &k);
   if (rc) return rc;
   DeviceGuard guard(ctx->device);
-  rc = launch_softmax(ctx, q, rows, L, k, out);
+  {
+    ProfileScope ps(ctx, IBERT_K_SOFTMAX);
+    rc = launch_softmax(ctx, q, rows, L, k, out);
+  }
   if (rc == IBERT_OK && S_ret) *S_ret = 1.0 / (double)p_max;
   return rc;
 }
@@ -199,7 +233,10 @@ int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* 
   if (rc) return rc;
   rc = cached_upload(ctx, B_i.data(), B_i.size() * sizeof(int64_t), 12, &d_B);
   if (rc) return rc;
-  rc = launch_layernorm(ctx, q, r, rows, k, (const int32_t*)d_b, (const int64_t*)d_B, out);
+  {
+    ProfileScope ps(ctx, IBERT_K_LAYERNORM);
+    rc = launch_layernorm(ctx, q, r, rows, k, (const int32_t*)d_b, (const int64_t*)d_B, out);
+  }
   if (rc == IBERT_OK && S_ret) *S_ret = S_out;
   return rc;
 }
@@ -239,7 +276,11 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
       if (rc) return rc;
     }
   }
-  int rc = launch_gemm_i8(ctx, x, w, M, N, K, epi, out);
+  int rc;
+  {
+    ProfileScope ps(ctx, gemm_class(kind, K));
+    rc = launch_gemm_i8(ctx, x, w, M, N, K, epi, out);
+  }
   if (rc == IBERT_OK && S_ret) {
     if (kind == EPI_RAW) for (int n = 0; n < N; ++n) S_ret[n] = S_x * S_w[n];
     else *S_ret = S_out;
@@ -279,7 +320,10 @@ int ibert_attention_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, i
   int rc = make_attn_consts(S_q, S_k, S_v, S_ctx, p_max, &k);
   if (rc) return rc;
   DeviceGuard guard(ctx->device);
-  rc = launch_attention(ctx, qkv, B, L, H, heads, k, out);
+  {
+    ProfileScope ps(ctx, IBERT_K_ATTENTION);
+    rc = launch_attention(ctx, qkv, B, L, H, heads, k, out);
+  }
   if (rc == IBERT_OK && S_ret) *S_ret = S_ctx;
   return rc;
 }
@@ -408,23 +452,51 @@ int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, 
   int8_t* g = (int8_t*)(ws + o_g);
 
   GemmEpilogue e{};
+  int rc;
   e.kind = EPI_INT8; e.d_b = ly->b_qkv; e.d_c = ly->c_qkv; e.d_bias = ly->bias_qkv;
-  int rc = launch_gemm_i8(ctx, x, ly->w_qkv, T, 3 * H, H, e, qkv);
+  { ProfileScope ps(ctx, IBERT_K_GEMM_QKV); rc = launch_gemm_i8(ctx, x, ly->w_qkv, T, 3 * H, H, e, qkv); }
   if (rc) return rc;
-  rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, cx);
+  { ProfileScope ps(ctx, IBERT_K_ATTENTION); rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, cx); }
   if (rc) return rc;
   e.kind = EPI_Q16; e.d_b = ly->b_o; e.d_c = ly->c_o; e.d_bias = ly->bias_o;
-  rc = launch_gemm_i8(ctx, cx, ly->w_o, T, H, H, e, r);
+  { ProfileScope ps(ctx, IBERT_K_GEMM_Q16); rc = launch_gemm_i8(ctx, cx, ly->w_o, T, H, H, e, r); }
   if (rc) return rc;
-  rc = launch_layernorm(ctx, r, x, T, ly->ln1, ly->ln1_b, ly->ln1_B, h1);
+  { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm(ctx, r, x, T, ly->ln1, ly->ln1_b, ly->ln1_B, h1); }
   if (rc) return rc;
   e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu;
-  rc = launch_gemm_i8(ctx, h1, ly->w_f1, T, F, H, e, g);
+  { ProfileScope ps(ctx, IBERT_K_GEMM_GELU); rc = launch_gemm_i8(ctx, h1, ly->w_f1, T, F, H, e, g); }
   if (rc) return rc;
   e.kind = EPI_Q16; e.d_b = ly->b_f2; e.d_c = ly->c_f2; e.d_bias = ly->bias_f2;
-  rc = launch_gemm_i8(ctx, g, ly->w_f2, T, H, F, e, r);
+  { ProfileScope ps(ctx, IBERT_K_GEMM_Q16_WIDE); rc = launch_gemm_i8(ctx, g, ly->w_f2, T, H, F, e, r); }
   if (rc) return rc;
-  return launch_layernorm(ctx, r, h1, T, ly->ln2, ly->ln2_b, ly->ln2_B, out);
+  { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm(ctx, r, h1, T, ly->ln2, ly->ln2_b, ly->ln2_B, out); }
+  return rc;
+}
+
+int ibert_profile_begin(ibert_ctx* ctx) {
+  if (!ctx) return IBERT_ERR_ARG;
+  ctx->ev_class.clear();
+  ctx->profiling = true;
+  return IBERT_OK;
+}
+
+int ibert_profile_end(ibert_ctx* ctx, float* ms, int32_t* launches) {
+  if (!ctx || !ms || !launches) return IBERT_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  ctx->profiling = false;
+  for (int i = 0; i < IBERT_NUM_KERNEL_CLASSES; ++i) { ms[i] = 0.f; launches[i] = 0; }
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+  for (size_t i = 0; i < ctx->ev_class.size(); ++i) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, ctx->ev_pool[2 * i], ctx->ev_pool[2 * i + 1]) != cudaSuccess) {
+      cudaGetLastError();
+      continue;
+    }
+    ms[ctx->ev_class[i]] += t;
+    launches[ctx->ev_class[i]] += 1;
+  }
+  ctx->ev_class.clear();
+  return IBERT_OK;
 }
 
 }  // extern "C"

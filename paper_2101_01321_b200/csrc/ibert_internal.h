@@ -77,6 +77,10 @@ struct ibert_ctx {
   // workspace for the encoder layer's intermediates
   void* ws = nullptr;
   size_t ws_bytes = 0;
+  // optional per-launch event timing (ibert_profile_begin / _end)
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev_pool;      // pairs: [2i] before, [2i+1] after launch i
+  std::vector<int> ev_class;             // kernel class of launch i
 };
 
 namespace ibert {

@@ -25,7 +25,7 @@ def test_attention_matches_oracle(B, L, heads, p_max):
     if B:
         want = oracle.attention(qkv, B, L, H, heads, S_q, S_k, S_v, S_ctx, p_max)
         assert_same(host(out), want, f"attention L={L}")
-        assert np.abs(want).max() > 20
+        assert np.abs(want).max() > 5
 
 
 def test_attention_peaked_and_uniform_rows():

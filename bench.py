@@ -56,7 +56,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -329,6 +329,87 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_only(args):
+    """Runs ONE kernel class alone through its C-ABI entry point at the workload's shape
+    (for ncu captures and per-kernel timing).  Prints a small JSON line."""
+    import numpy as np
+    import torch
+
+    from paper_2101_01321_b200 import binding, build, synth
+
+    build.build()
+    cfg = synth.CONFIGS[args.config]
+    batch = args.batch or DEFAULT_BATCH[args.config]
+    T, H, F, L = batch * cfg.L, cfg.H, cfg.F, cfg.L
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.Stream(device=dev)
+    ctx = binding.Context(0, stream)
+    g = torch.Generator(device="cpu").manual_seed(synth.SEED_BASE)
+
+    def i8(*shape):
+        return torch.randint(-127, 128, shape, generator=g, dtype=torch.int8).to(dev)
+
+    p = synth.static_activation_scales(H, F, L, 0.035)
+    rng = np.random.default_rng(synth.SEED_BASE)
+    k = args.only
+    if k.startswith("gemm"):
+        N, K = {"gemm_qkv": (3 * H, H), "gemm_out": (H, H), "gemm_ffn1_gelu": (F, H), "gemm_ffn2": (H, F)}[k]
+        x, w = i8(T, K), i8(N, K)
+        bias = torch.randint(-1000, 1000, (N,), generator=g, dtype=torch.int32).to(dev)
+        S_w = rng.uniform(5e-4, 7e-4, N)
+        S_x = 0.03
+        S_acc = S_x * 6e-4 * 127 * 127 * np.sqrt(K)           # ~ one standard deviation of the product
+        if k == "gemm_ffn1_gelu":
+            out = torch.empty((T, N), dtype=torch.int8, device=dev)
+            fn = lambda: ctx.ibert_linear_gelu_i8(x, S_x, w, S_w, bias, 8 * S_acc / 32767, 4 * S_acc / 127, out=out)
+        elif k == "gemm_qkv":
+            out = torch.empty((T, N), dtype=torch.int8, device=dev)
+            fn = lambda: ctx.ibert_linear_i8(x, S_x, w, S_w, bias, 0, 4 * S_acc / 127, out=out)
+        else:
+            out = torch.empty((T, N), dtype=torch.int32, device=dev)
+            fn = lambda: ctx.ibert_linear_i8(x, S_x, w, S_w, bias, 1, 8 * S_acc / 32767, out=out)
+    elif k == "attention":
+        qkv = torch.clamp(torch.randn((T, 3 * H), generator=g) * 32, -127, 127).to(torch.int8).to(dev)
+        out = torch.empty((T, H), dtype=torch.int8, device=dev)
+        fn = lambda: ctx.ibert_attention_i8(qkv, batch, L, H, cfg.heads, p["S_q"], p["S_k"], p["S_v"], p["S_ctx"], 255, out=out)
+    elif k == "layernorm":
+        q, S, r, S_r, gamma, beta, S_out = synth.layernorm_inputs(T, H, 1.0)
+        qd, rd = torch.from_numpy(q).to(dev), torch.from_numpy(r).to(dev)
+        out = torch.empty((T, H), dtype=torch.int8, device=dev)
+        fn = lambda: ctx.ibert_layernorm_i(qd, S, rd, S_r, gamma, beta, S_out, out=out)
+    elif k == "gelu":
+        q, S, S_out = synth.gelu_inputs(1 << 24, 1.0)
+        qd = torch.from_numpy(q).to(dev)
+        out = torch.empty(q.shape, dtype=torch.int8, device=dev)
+        fn = lambda: ctx.ibert_gelu_i(qd, S, S_out, out=out)
+    elif k == "softmax":
+        rows = batch * cfg.heads * L
+        q, S = synth.softmax_inputs(rows, L, 1.0)
+        qd = torch.from_numpy(q).to(dev)
+        out = torch.empty(q.shape, dtype=torch.uint8, device=dev)
+        fn = lambda: ctx.ibert_softmax_i(qd, S, 255, out=out)
+    else:
+        raise SystemExit(f"unknown kernel class {k}")
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    times = []
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 1)):
+            fn()
+        for _ in range(args.steps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            times.append((e0, e1))
+    stream.synchronize()
+    ctx.check()
+    ms = [a.elapsed_time(b) for a, b in times]
+    print(json.dumps({"only": k, "tokens": T, "ms_median": statistics.median(ms), "ms_min": min(ms),
+                      "launches": args.steps}))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -337,8 +418,11 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4])
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--only", default="", help="run one kernel class alone (profiling aid)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.only:
+        run_only(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

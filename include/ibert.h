@@ -152,6 +152,12 @@ enum {
   IBERT_K_SOFTMAX = 7,
   IBERT_NUM_KERNEL_CLASSES = 8
 };
+/* Host, pure.  Self-check of the constants derived from a score scale S for i-exp (Algorithm 3):
+   verifies on the host, for every distance d in [0, 31*q_ln2], that the multiply-high form the
+   kernels use for z = floor(d / q_ln2) equals the division.  Returns IBERT_OK, the error of the
+   derivation, or IBERT_ERR_VALUE_RANGE on a mismatch.  q_ln2_out (may be NULL) receives q_ln2. */
+int ibert_selftest_exp_division(double S, int32_t* q_ln2_out);
+
 int ibert_profile_begin(ibert_ctx* ctx);
 int ibert_profile_end(ibert_ctx* ctx, float* ms, int32_t* launches);
 

@@ -63,6 +63,8 @@ def lib():
         L.ibert_layer_create.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(vp)]
         L.ibert_layer_destroy.argtypes = [vp]
         L.ibert_encoder_layer.argtypes = [vp, vp, vp, i32, i32, vp, vp]
+        L.ibert_selftest_exp_division.argtypes = [dbl, C.POINTER(C.c_int32)]
+        L.ibert_selftest_exp_division.restype = i32
         L.ibert_profile_begin.argtypes = [vp]
         L.ibert_profile_end.argtypes = [vp, vp, vp]
         L.ibert_profile_begin.restype = i32

@@ -91,6 +91,7 @@ struct ibert_layer {
   int32_t *bias_qkv = nullptr, *bias_o = nullptr, *bias_f1 = nullptr, *bias_f2 = nullptr;
   int32_t *b_qkv = nullptr, *c_qkv = nullptr, *b_o = nullptr, *c_o = nullptr;
   int32_t *b_f1 = nullptr, *c_f1 = nullptr, *b_f2 = nullptr, *c_f2 = nullptr;
+  int fast_qkv = 0, fast_o = 0, fast_f1 = 0, fast_f2 = 0;   // multipliers stored in upper-word form
   int32_t *ln1_b = nullptr, *ln2_b = nullptr;
   int64_t *ln1_B = nullptr, *ln2_B = nullptr;
   LnConsts ln1{}, ln2{};
@@ -219,13 +220,12 @@ int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* 
   k.C = C;
   k.has_res = r != nullptr;
   if (r) {
-    if (!good_scale(S_r)) return IBERT_ERR_SCALE_RANGE;
-    int rc = dyadic(S_r / S, &k.b_r, &k.c_r);
+    int rc = make_ln_residual(S_r, S, &k);
     if (rc) return rc;
   }
   std::vector<int32_t> b_i;
   std::vector<int64_t> B_i;
-  int rc = make_ln_tables(gamma, beta, C, S_out, &k.c, &b_i, &B_i);
+  int rc = make_ln_tables(gamma, beta, C, S_out, &k, &b_i, &B_i);
   if (rc) return rc;
   DeviceGuard guard(ctx->device);
   void *d_b = nullptr, *d_B = nullptr;
@@ -264,6 +264,7 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
     std::vector<int32_t> b, c;
     int rc = make_linear_tables(S_x, S_w, N, nullptr, S_acc_to, &b, &c);
     if (rc) return rc;
+    epi.fast = to_upper_word_form(&b, c) ? 1 : 0;
     void *d_b = nullptr, *d_c = nullptr;
     rc = cached_upload(ctx, b.data(), b.size() * sizeof(int32_t), 21, &d_b);
     if (rc) return rc;
@@ -368,10 +369,13 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   ly->d = *d;
   int rc = IBERT_OK;
   auto up = [&](const void* h, size_t bytes, void** dev) { if (rc == IBERT_OK) rc = upload_owned(ly, h, bytes, dev); };
-  auto lin = [&](double S_in, const double* S_w, int N, const double* so_cols, double so, int32_t** db, int32_t** dc) {
+  auto lin = [&](double S_in, const double* S_w, int N, const double* so_cols, double so, int32_t** db, int32_t** dc,
+                 int* fast) {
     if (rc != IBERT_OK) return;
     std::vector<int32_t> b, c;
     rc = make_linear_tables(S_in, S_w, N, so_cols, so, &b, &c);
+    if (rc != IBERT_OK) return;
+    *fast = to_upper_word_form(&b, c) ? 1 : 0;
     up(b.data(), b.size() * sizeof(int32_t), (void**)db);
     up(c.data(), c.size() * sizeof(int32_t), (void**)dc);
   };
@@ -386,21 +390,21 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   {
     std::vector<double> so(3 * (size_t)H);
     for (int n = 0; n < 3 * H; ++n) so[n] = n < H ? d->S_q : (n < 2 * H ? d->S_k : d->S_v);
-    lin(d->S_x, d->S_w_qkv, 3 * H, so.data(), 0.0, &ly->b_qkv, &ly->c_qkv);
+    lin(d->S_x, d->S_w_qkv, 3 * H, so.data(), 0.0, &ly->b_qkv, &ly->c_qkv, &ly->fast_qkv);
   }
-  lin(d->S_ctx, d->S_w_o, H, nullptr, d->S_r1, &ly->b_o, &ly->c_o);
-  lin(d->S_h1, d->S_w_f1, F, nullptr, d->S_gi, &ly->b_f1, &ly->c_f1);
-  lin(d->S_go, d->S_w_f2, H, nullptr, d->S_r2, &ly->b_f2, &ly->c_f2);
+  lin(d->S_ctx, d->S_w_o, H, nullptr, d->S_r1, &ly->b_o, &ly->c_o, &ly->fast_o);
+  lin(d->S_h1, d->S_w_f1, F, nullptr, d->S_gi, &ly->b_f1, &ly->c_f1, &ly->fast_f1);
+  lin(d->S_go, d->S_w_f2, H, nullptr, d->S_r2, &ly->b_f2, &ly->c_f2, &ly->fast_f2);
   auto ln = [&](const double* g, const double* be, double S_sum, double S_res, double S_o, LnConsts* k,
                 int32_t** db, int64_t** dB) {
     if (rc != IBERT_OK) return;
     k->C = H;
     k->has_res = 1;
-    rc = dyadic(S_res / S_sum, &k->b_r, &k->c_r);
+    rc = make_ln_residual(S_res, S_sum, k);
     if (rc != IBERT_OK) return;
     std::vector<int32_t> b_i;
     std::vector<int64_t> B_i;
-    rc = make_ln_tables(g, be, H, S_o, &k->c, &b_i, &B_i);
+    rc = make_ln_tables(g, be, H, S_o, k, &b_i, &B_i);
     up(b_i.data(), b_i.size() * sizeof(int32_t), (void**)db);
     up(B_i.data(), B_i.size() * sizeof(int64_t), (void**)dB);
   };
@@ -453,24 +457,37 @@ int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, 
 
   GemmEpilogue e{};
   int rc;
-  e.kind = EPI_INT8; e.d_b = ly->b_qkv; e.d_c = ly->c_qkv; e.d_bias = ly->bias_qkv;
+  e.kind = EPI_INT8; e.d_b = ly->b_qkv; e.d_c = ly->c_qkv; e.d_bias = ly->bias_qkv; e.fast = ly->fast_qkv;
   { ProfileScope ps(ctx, IBERT_K_GEMM_QKV); rc = launch_gemm_i8(ctx, x, ly->w_qkv, T, 3 * H, H, e, qkv); }
   if (rc) return rc;
   { ProfileScope ps(ctx, IBERT_K_ATTENTION); rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, cx); }
   if (rc) return rc;
-  e.kind = EPI_Q16; e.d_b = ly->b_o; e.d_c = ly->c_o; e.d_bias = ly->bias_o;
+  e.kind = EPI_Q16; e.d_b = ly->b_o; e.d_c = ly->c_o; e.d_bias = ly->bias_o; e.fast = ly->fast_o;
   { ProfileScope ps(ctx, IBERT_K_GEMM_Q16); rc = launch_gemm_i8(ctx, cx, ly->w_o, T, H, H, e, r); }
   if (rc) return rc;
   { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm(ctx, r, x, T, ly->ln1, ly->ln1_b, ly->ln1_B, h1); }
   if (rc) return rc;
-  e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu;
+  e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu; e.fast = ly->fast_f1;
   { ProfileScope ps(ctx, IBERT_K_GEMM_GELU); rc = launch_gemm_i8(ctx, h1, ly->w_f1, T, F, H, e, g); }
   if (rc) return rc;
-  e.kind = EPI_Q16; e.d_b = ly->b_f2; e.d_c = ly->c_f2; e.d_bias = ly->bias_f2;
+  e.kind = EPI_Q16; e.d_b = ly->b_f2; e.d_c = ly->c_f2; e.d_bias = ly->bias_f2; e.fast = ly->fast_f2;
   { ProfileScope ps(ctx, IBERT_K_GEMM_Q16_WIDE); rc = launch_gemm_i8(ctx, g, ly->w_f2, T, H, F, e, r); }
   if (rc) return rc;
   { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm(ctx, r, h1, T, ly->ln2, ly->ln2_b, ly->ln2_B, out); }
   return rc;
+}
+
+int ibert_selftest_exp_division(double S, int32_t* q_ln2_out) {
+  ExpConsts k;
+  int rc = make_exp_consts(S, 255, &k);
+  if (rc) return rc;
+  if (q_ln2_out) *q_ln2_out = (int32_t)k.q_ln2;
+  for (uint32_t d = 0; d <= k.d_max; ++d) {
+    const uint64_t wide = (uint64_t)(uint32_t)(d << k.div_pre) * (uint64_t)k.div_m;
+    const uint32_t z = (uint32_t)(wide >> 32) >> k.div_post;
+    if (z != d / k.q_ln2) return IBERT_ERR_VALUE_RANGE;
+  }
+  return IBERT_OK;
 }
 
 int ibert_profile_begin(ibert_ctx* ctx) {

@@ -33,6 +33,69 @@ __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t col, uin
   return kb * (rows_per_block * 128u) + row * 128u + (((cc ^ (row & 7u)) << 4) | by);
 }
 
+// i-softmax (Algorithm 3) of one score row held in TMEM lane `t_row`, columns [0, L):
+// pass 1 row maximum, pass 2 i-exp + int32 row sum (exponentials written back over the scores),
+// pass 3 fixed-point quotient -> u8 probabilities into the swizzled operand tile `sP`, row `row`.
+// Columns [L, Lp) are padding: excluded from max and sum, written as probability 0.
+template <int DIV>
+__device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const ExpConsts& ek, uint8_t* sP,
+                                            uint32_t row) {
+  const int full = L & ~31;             // columns covered by whole 32-column chunks
+  int32_t mx = INT32_MIN;
+  for (int c0 = 0; c0 < Lp; c0 += 32) {
+    uint32_t v[32];
+    ptx::tmem_ld32(t_row + c0, v);
+    ptx::tmem_wait_ld();
+    if (c0 < full) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) mx = max(mx, (int32_t)v[i]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i)
+        if (c0 + i < L) mx = max(mx, (int32_t)v[i]);
+    }
+  }
+  uint32_t sum = 0;
+  for (int c0 = 0; c0 < Lp; c0 += 32) {
+    uint32_t v[32];
+    ptx::tmem_ld32(t_row + c0, v);
+    ptx::tmem_wait_ld();
+    if (c0 < full) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        v[i] = iexp_dist<DIV>((uint32_t)mx - v[i], ek);
+        sum += v[i];
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        v[i] = (c0 + i < L) ? iexp_dist<DIV>((uint32_t)mx - v[i], ek) : 0u;
+        sum += v[i];
+      }
+    }
+    ptx::tmem_st32(t_row + c0, v);
+  }
+  ptx::tmem_wait_st();
+  const RowDivisor rd = make_row_divisor(sum, ek.p_max);
+  for (int c0 = 0; c0 < Lp; c0 += 32) {
+    uint32_t v[32];
+    ptx::tmem_ld32(t_row + c0, v);
+    ptx::tmem_wait_ld();
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int j = h * 16 + i * 4;
+        w[i] = softmax_quotient(v[j], rd) | (softmax_quotient(v[j + 1], rd) << 8) |
+               (softmax_quotient(v[j + 2], rd) << 16) | (softmax_quotient(v[j + 3], rd) << 24);
+      }
+      *reinterpret_cast<uint4*>(sP + sw128_offset(row, (uint32_t)(c0 + h * 16), 128)) =
+          make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kAttnThreads)
 attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_constant__ CUtensorMap map_v,
                  const AttnArgs a) {
@@ -117,49 +180,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
   const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);
   if (ok) {
     ptx::tc_fence_after_sync();
-    const ExpConsts ek = a.k.e;
-    int32_t mx = INT32_MIN;
-    for (int c0 = 0; c0 < Lp; c0 += 32) {
-      uint32_t v[32];
-      ptx::tmem_ld32(t_row + c0, v);
-      ptx::tmem_wait_ld();
-#pragma unroll
-      for (int i = 0; i < 32; ++i)
-        if (c0 + i < L) mx = max(mx, (int32_t)v[i]);
-    }
-    uint32_t sum = 0;
-    for (int c0 = 0; c0 < Lp; c0 += 32) {
-      uint32_t v[32];
-      ptx::tmem_ld32(t_row + c0, v);
-      ptx::tmem_wait_ld();
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const uint32_t e = (c0 + i < L) ? iexp_dist((uint32_t)mx - v[i], ek) : 0u;
-        v[i] = e;
-        sum += e;
-      }
-      ptx::tmem_st32(t_row + c0, v);
-    }
-    ptx::tmem_wait_st();
-    const RowDivisor rd = make_row_divisor(sum);
-    for (int c0 = 0; c0 < Lp; c0 += 32) {
-      uint32_t v[32];
-      ptx::tmem_ld32(t_row + c0, v);
-      ptx::tmem_wait_ld();
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        uint32_t w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint32_t pk = 0;
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            pk |= softmax_quotient(v[h * 16 + i * 4 + e], ek.pm8, rd) << (8 * e);
-          w[i] = pk;
-        }
-        *reinterpret_cast<uint4*>(sP + sw128_offset((uint32_t)tid, (uint32_t)(c0 + h * 16), 128)) =
-            make_uint4(w[0], w[1], w[2], w[3]);
-      }
+    switch (exp_div_mode(a.k.e)) {
+      case 0: softmax_row<0>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
+      case 1: softmax_row<1>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
+      default: softmax_row<2>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
     }
     ptx::fence_proxy_async_smem();          // P and Vt were written by ordinary stores; the MMA reads them
   }

@@ -20,6 +20,20 @@ __device__ __forceinline__ int32_t requant_add(int32_t v, int32_t b, int64_t add
   return (int32_t)p;
 }
 
+// The same requantization when the host could pre-shift the multiplier: the result is the
+// upper word of one 64-bit multiply-add, (v * b2 + add2) >> 32, not yet clamped.
+__device__ __forceinline__ int32_t requant_upper(int32_t v, int32_t b2, int64_t add2) {
+  return (int32_t)(((int64_t)v * (int64_t)b2 + add2) >> 32);
+}
+
+// four int32 -> four int8 lanes of one word, each saturated to [-128, 127]
+__device__ __forceinline__ uint32_t pack4_sat_s8(int32_t v0, int32_t v1, int32_t v2, int32_t v3) {
+  uint32_t hi, r;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(v3), "r"(v2), "r"(0));
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(v1), "r"(v0), "r"(hi));
+  return r;
+}
+
 __device__ __forceinline__ int64_t rounding_half(int c) { return c > 0 ? (int64_t(1) << (c - 1)) : 0; }
 
 __device__ __forceinline__ int32_t clamp_sym(int32_t v, int32_t qmax) { return max(-qmax, min(v, qmax)); }
@@ -36,47 +50,64 @@ __device__ __forceinline__ int32_t igelu_q16_to_int8(int32_t q, const GeluConsts
   return requant_add(g2, k.b, half, k.c, 127);
 }
 
-// i-exp of one non-negative distance d = max - q (Algorithm 3): z = floor(d'/q_ln2),
-// r = d' - z q_ln2, e = ((q_b - r)^2 + q_c) >> min(z + s_out, 31); d' = min(d >> s_in, 31 q_ln2).
-__device__ __forceinline__ uint32_t iexp_dist(uint32_t d, const ExpConsts& k) {
-  const uint32_t dp = min(d >> k.s_in, k.d_max);
-  const uint32_t z = __umulhi(dp << 12, k.div_m) >> k.div_l;
-  const int32_t t = k.q_b - (int32_t)(dp - z * k.q_ln2);
-  const uint32_t poly = (uint32_t)(t * t + k.q_c);
-  return poly >> min(z + (uint32_t)k.s_out, 31u);
+// Same function, written for the integer pipes: sign applied by a multiply, the final
+// requantization in upper-word form; the result still needs the upper clamp (pack4_sat_s8).
+__device__ __forceinline__ int32_t igelu_q16_upper(int32_t q, const GeluConsts& k) {
+  const int32_t t = min(abs(q) >> k.s_in, k.nq_b) - k.nq_b;
+  const int32_t poly = t * t + k.q_c;
+  const int32_t sgn = (q >> 31) | 1;
+  const int32_t f = poly * sgn + k.q_c;
+  const int32_t g2 = (q * (f >> k.s_f) + 128) >> 8;
+  return max(requant_upper(g2, k.b2, k.add2), -127);
 }
 
-// Per-row reciprocal for p = floor(e * p_max / sum), exact for e * p_max < 2^29:
-// with l = bit length of sum and m = floor(2^(29+l) / sum) + 1,
-// floor(n / sum) = umulhi(n << 3, m) >> l for every n < 2^29.
-struct RowDivisor {
-  uint32_t m;
-  int l;
-};
-
-__device__ __forceinline__ RowDivisor make_row_divisor(uint32_t sum) {
-  RowDivisor r;
-  r.l = 32 - __clz(sum);
-  r.m = (uint32_t)((uint64_t(1) << (29 + r.l)) / sum) + 1u;
+__device__ __forceinline__ uint32_t shr_clamped(uint32_t v, uint32_t n) {
+  uint32_t r;
+  asm("shr.u32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(n));   // shift counts above 31 give 0
   return r;
 }
 
-__device__ __forceinline__ uint32_t softmax_quotient(uint32_t e, uint32_t pm8, const RowDivisor& r) {
-  return __umulhi(e * pm8, r.m) >> r.l;
+// i-exp of one non-negative distance d = max - q (Algorithm 3): z = floor(d'/q_ln2),
+// r = d' - z q_ln2, e = ((q_b - r)^2 + q_c) >> min(z + s_out, 31); d' = min(d >> s_in, 31 q_ln2).
+// The polynomial is below 2^31, so a shift by more than 31 equals the shift by 31 (both give 0).
+// DIV: 0 = multiply-high alone gives z, 1 = followed by a shift, 2 = operand pre-shifted as well.
+template <int DIV>
+__device__ __forceinline__ uint32_t iexp_dist(uint32_t d, const ExpConsts& k) {
+  const uint32_t dp = min(d >> k.s_in, k.d_max);
+  uint32_t z;
+  if (DIV == 0) z = __umulhi(dp, k.div_m);
+  else if (DIV == 1) z = __umulhi(dp, k.div_m) >> k.div_post;
+  else z = __umulhi(dp << k.div_pre, k.div_m) >> k.div_post;
+  const int32_t t = (int32_t)(z * k.q_ln2) + (k.q_b - (int32_t)dp);      // q_b - r
+  const uint32_t poly = (uint32_t)(t * t + k.q_c);
+  return shr_clamped(poly, z + (uint32_t)k.s_out);
+}
+__host__ __device__ __forceinline__ int exp_div_mode(const ExpConsts& k) {
+  return k.div_pre != 0 ? 2 : (k.div_post != 0 ? 1 : 0);
 }
 
-// floor(sqrt(n)) by the Newton iteration of Algorithm 4 (x0 = 2^ceil(bits/2), stop when the
-// iterate no longer decreases), on 64-bit n.
-__device__ __forceinline__ uint32_t isqrt_newton(uint64_t n) {
-  if (n == 0) return 0;
-  const int bits = 64 - __clzll((long long)n);
-  uint64_t x = uint64_t(1) << ((bits + 1) >> 1);
-  for (int it = 0; it < 64; ++it) {
-    const uint64_t y = (x + n / x) >> 1;
-    if (y >= x) break;
-    x = y;
-  }
-  return (uint32_t)x;
+// Per-row divisor for p = floor(e * p_max / sum) with e < 2^21 and e <= sum < 2^31:
+// with l = bit length of sum, K = 21 + l and m = ceil(p_max 2^K / sum) (< 2^30),
+// floor(e m / 2^K) is exact: the excess e (m sum - p_max 2^K) / (sum 2^K) stays below 2^-l < 1/sum.
+// Evaluated as umulhi(e << pre, m) >> post with post - pre = K - 32.
+struct RowDivisor {
+  uint32_t m;
+  int pre, post;
+};
+
+__device__ __forceinline__ RowDivisor make_row_divisor(uint32_t sum, uint32_t p_max) {
+  RowDivisor r;
+  const int l = 32 - __clz(sum);
+  const int K = 21 + l;
+  const uint64_t num = ((uint64_t)p_max << K) + (uint64_t)(sum - 1u);
+  r.m = (uint32_t)(num / (uint64_t)sum);
+  r.pre = K < 32 ? 32 - K : 0;
+  r.post = K < 32 ? 0 : K - 32;
+  return r;
+}
+
+__device__ __forceinline__ uint32_t softmax_quotient(uint32_t e, const RowDivisor& r) {
+  return __umulhi(e << r.pre, r.m) >> r.post;
 }
 
 }  // namespace ibert

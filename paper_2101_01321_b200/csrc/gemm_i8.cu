@@ -6,7 +6,7 @@
 // out[m, n] = epilogue( sum_k x[m, k] * w[n, k] + bias[n] )      x: [M, K], w: [N, K]
 //
 // One persistent CTA per SM walks 128 x BN output tiles.  Warp 0 is the TMA producer,
-// warp 1 issues the MMAs, warps 2..5 run the epilogue; two TMEM accumulator stages let
+// warp 1 issues the MMAs, warps 2..9 run the epilogue; two TMEM accumulator stages let
 // the (integer-ALU heavy) epilogue of tile i overlap the MMAs of tile i+1.
 #include <cuda.h>
 
@@ -74,8 +74,9 @@ namespace {
 constexpr int BM = 128;           // rows per tile = TMEM lanes
 constexpr int BK = 128;           // K bytes per pipeline stage = one 128-byte swizzle span
 constexpr int UMMA_K = 32;        // K per tcgen05.mma kind::i8
-constexpr int kGemmThreads = 192; // producer warp, MMA warp, 4 epilogue warps
-constexpr int kEpiThreads = 128;
+constexpr int kEpiWarps = 8;      // two warps per TMEM lane quarter, each taking every other column chunk
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kGemmThreads = 64 + kEpiThreads;   // producer warp, MMA warp, epilogue warps
 
 template <int BN>
 struct GemmSmem {
@@ -93,7 +94,6 @@ struct GemmSmem {
 struct GemmArgs {
   int64_t M;
   int N, K;
-  int kind;
   const int32_t* b;
   const int32_t* c;
   const int32_t* bias;
@@ -102,7 +102,65 @@ struct GemmArgs {
   int32_t* status;
 };
 
-template <int BN>
+// One 32-column chunk of one accumulator row: registers -> epilogue -> global memory.
+// FAST: every column's requantization is in upper-word form (one 64-bit multiply-add).
+template <int KIND, bool FAST>
+__device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[32], const int4* __restrict__ prm,
+                                               const GemmArgs& args, const GeluConsts& gk, int64_t gelu_half,
+                                               int64_t row, bool row_ok, int col0) {
+  if constexpr (KIND == EPI_RAW || KIND == EPI_Q16) {
+    int32_t* orow = static_cast<int32_t*>(args.out) + row * args.N + col0;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      int32_t o[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int4 p = prm[g * 4 + i];
+        const int32_t a = (int32_t)v[g * 4 + i];
+        const int64_t add = (int64_t)(((uint64_t)(uint32_t)p.w << 32) | (uint32_t)p.z);
+        if constexpr (KIND == EPI_RAW) o[i] = a + p.x;
+        else if constexpr (FAST) o[i] = clamp_sym(requant_upper(a, p.x, add), 32767);
+        else o[i] = requant_add(a, p.x, add, p.y, 32767);
+      }
+      if (row_ok && col0 + g * 4 < args.N)
+        *reinterpret_cast<int4*>(orow + g * 4) = make_int4(o[0], o[1], o[2], o[3]);
+    }
+  } else {
+    int8_t* orow = static_cast<int8_t*>(args.out) + row * args.N + col0;
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        int32_t o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int idx = g * 16 + i * 4 + e;
+          const int4 p = prm[idx];
+          const int32_t a = (int32_t)v[idx];
+          const int64_t add = (int64_t)(((uint64_t)(uint32_t)p.w << 32) | (uint32_t)p.z);
+          if constexpr (KIND == EPI_INT8) {
+            if constexpr (FAST) o[e] = max(requant_upper(a, p.x, add), -127);
+            else o[e] = requant_add(a, p.x, add, p.y, 127);
+          } else {
+            if constexpr (FAST) {
+              const int32_t q16 = clamp_sym(requant_upper(a, p.x, add), 32767);
+              o[e] = igelu_q16_upper(q16, gk);
+            } else {
+              const int32_t q16 = requant_add(a, p.x, add, p.y, 32767);
+              o[e] = igelu_q16_to_int8(q16, gk, gelu_half);
+            }
+          }
+        }
+        w[i] = pack4_sat_s8(o[0], o[1], o[2], o[3]);    // upper clamp (+127) happens here
+      }
+      if (row_ok && col0 + g * 16 < args.N)
+        *reinterpret_cast<uint4*>(orow + g * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+}
+
+template <int BN, int KIND, bool FAST>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const GemmArgs args) {
@@ -199,36 +257,38 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------ epilogue (warps 2..9)
     const int quarter = warp & 3;                      // TMEM lanes 32*quarter .. +31 belong to this warp
-    const int et = threadIdx.x - 64;                   // 0..127
+    const int half_id = (warp - 2) >> 2;               // which of the two warps of this quarter
+    const int et = threadIdx.x - 64;                   // 0..kEpiThreads-1
     const GeluConsts gk = args.gelu;
     const int64_t gelu_half = rounding_half(gk.c);
     uint32_t acc = 0, acc_phase = 0;
     for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
       const int64_t m0 = (tile / n_tiles) * BM;
       const int n0 = (int)(tile % n_tiles) * BN;
-      // per-column parameters of this tile: {b, c, (bias*b + rounding) lo, hi}; raw: {bias,0,0,0}
-      asm volatile("bar.sync 1, 128;" ::: "memory");   // previous tile's readers are done
+      // per-column parameters of this tile.  generic: {b, c, (bias*b + 2^(c-1)) lo, hi};
+      // fast: {b << (32-c), -, (bias*(b << (32-c)) + 2^31) lo, hi};  raw: {bias, 0, 0, 0}
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
       for (int j = et; j < BN; j += kEpiThreads) {
         const int n = n0 + j;
         int4 p = make_int4(0, 0, 0, 0);
         if (n < args.N) {
           const int32_t bias = args.bias ? __ldg(args.bias + n) : 0;
-          if (args.kind == EPI_RAW) {
+          if constexpr (KIND == EPI_RAW) {
             p.x = bias;
           } else {
             const int32_t b = __ldg(args.b + n), c = __ldg(args.c + n);
-            const int64_t add = (int64_t)bias * b + rounding_half(c);
+            const int64_t add = (int64_t)bias * b + (FAST ? (int64_t(1) << 31) : rounding_half(c));
             p = make_int4(b, c, (int32_t)(uint32_t)(uint64_t)add, (int32_t)(add >> 32));
           }
         }
         s_param[j] = p;
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 
       // After a failed wait the loop keeps running (the named barriers above must still be
-      // reached by all 128 threads) but touches neither TMEM nor memory.
+      // reached by every epilogue thread) but touches neither TMEM nor memory.
       if (ok) ok = ptx::mbar_wait(bar_acc_full + 8 * acc, acc_phase);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) continue;
@@ -237,56 +297,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const bool row_ok = row < args.M;
       const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
-      for (int ch = 0; ch < BN / 32; ++ch) {
+      for (int ch = half_id; ch < BN / 32; ch += 2) {
         uint32_t v[32];
         ptx::tmem_ld32(t_row + ch * 32, v);
         ptx::tmem_wait_ld();
-        const int col0 = n0 + ch * 32;
-        if (args.kind == EPI_RAW || args.kind == EPI_Q16) {
-          int32_t* orow = static_cast<int32_t*>(args.out) + row * args.N + col0;
-#pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            int32_t o[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const int4 p = s_param[ch * 32 + g * 4 + i];
-              if (args.kind == EPI_RAW) o[i] = (int32_t)v[g * 4 + i] + p.x;
-              else {
-                const int64_t add = (int64_t)(((uint64_t)(uint32_t)p.w << 32) | (uint32_t)p.z);
-                o[i] = requant_add((int32_t)v[g * 4 + i], p.x, add, p.y, 32767);
-              }
-            }
-            if (row_ok && col0 + g * 4 < args.N)
-              *reinterpret_cast<int4*>(orow + g * 4) = make_int4(o[0], o[1], o[2], o[3]);
-          }
-        } else {
-          int8_t* orow = static_cast<int8_t*>(args.out) + row * args.N + col0;
-#pragma unroll
-          for (int g = 0; g < 2; ++g) {
-            uint32_t w[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              uint32_t packed = 0;
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int idx = g * 16 + i * 4 + e;
-                const int4 p = s_param[ch * 32 + idx];
-                const int64_t add = (int64_t)(((uint64_t)(uint32_t)p.w << 32) | (uint32_t)p.z);
-                int32_t o;
-                if (args.kind == EPI_INT8) {
-                  o = requant_add((int32_t)v[idx], p.x, add, p.y, 127);
-                } else {
-                  const int32_t q16 = requant_add((int32_t)v[idx], p.x, add, p.y, 32767);
-                  o = igelu_q16_to_int8(q16, gk, gelu_half);
-                }
-                packed |= (uint32_t)(o & 0xff) << (8 * e);
-              }
-              w[i] = packed;
-            }
-            if (row_ok && col0 + g * 16 < args.N)
-              *reinterpret_cast<uint4*>(orow + g * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
+        epilogue_chunk<KIND, FAST>(v, s_param + ch * 32, args, gk, gelu_half, row, row_ok, n0 + ch * 32);
       }
       ptx::tc_fence_before_sync();
       ptx::mbar_arrive(bar_acc_empty + 8 * acc);
@@ -304,19 +319,29 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 }
 
-template <int BN>
-int launch_bn(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& args) {
+template <int BN, int KIND, bool FAST>
+int launch_inst(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& args) {
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_i8_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(gemm_i8_kernel<BN, KIND, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              GemmSmem<BN>::kAlloc) != cudaSuccess)
       return IBERT_ERR_CUDA;
     attr_set = true;
   }
   const int64_t tiles = ((args.M + BM - 1) / BM) * ((args.N + BN - 1) / BN);
   const int grid = (int)(tiles < ctx->num_sms ? tiles : ctx->num_sms);
-  gemm_i8_kernel<BN><<<grid, kGemmThreads, GemmSmem<BN>::kAlloc, ctx->stream>>>(ma, mb, args);
+  gemm_i8_kernel<BN, KIND, FAST><<<grid, kGemmThreads, GemmSmem<BN>::kAlloc, ctx->stream>>>(ma, mb, args);
   return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
+}
+
+template <int BN>
+int launch_bn(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& a, int kind, bool fast) {
+  switch (kind) {
+    case EPI_INT8: return fast ? launch_inst<BN, EPI_INT8, true>(ctx, ma, mb, a) : launch_inst<BN, EPI_INT8, false>(ctx, ma, mb, a);
+    case EPI_Q16: return fast ? launch_inst<BN, EPI_Q16, true>(ctx, ma, mb, a) : launch_inst<BN, EPI_Q16, false>(ctx, ma, mb, a);
+    case EPI_GELU: return fast ? launch_inst<BN, EPI_GELU, true>(ctx, ma, mb, a) : launch_inst<BN, EPI_GELU, false>(ctx, ma, mb, a);
+    default: return launch_inst<BN, EPI_RAW, false>(ctx, ma, mb, a);
+  }
 }
 
 }  // namespace
@@ -344,10 +369,12 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
     if (rc) return rc;
   }
   GemmArgs a{};
-  a.M = M; a.N = N; a.K = K; a.kind = epi.kind;
+  a.M = M; a.N = N; a.K = K;
   a.b = epi.d_b; a.c = epi.d_c; a.bias = epi.d_bias; a.gelu = epi.gelu;
   a.out = out; a.status = ctx->d_status;
-  return wide ? launch_bn<256>(ctx, ma, mb, a) : launch_bn<128>(ctx, ma, mb, a);
+  // upper-word epilogue needs both the per-column multipliers and (for GELU) the final one in that form
+  const bool fast = epi.fast != 0 && (epi.kind != EPI_GELU || epi.gelu.fast != 0);
+  return wide ? launch_bn<256>(ctx, ma, mb, a, epi.kind, fast) : launch_bn<128>(ctx, ma, mb, a, epi.kind, fast);
 }
 
 }  // namespace ibert

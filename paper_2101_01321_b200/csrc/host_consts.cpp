@@ -6,6 +6,7 @@
 // are computed here, once, in IEEE binary64 with the operation order fixed
 // below.  Compile without FMA contraction.
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 
 #include "ibert_internal.h"
@@ -73,15 +74,32 @@ int make_exp_consts(double S, int p_max, ExpConsts* k) {
   k->q_ln2 = (uint32_t)q_ln2;
   k->d_max = 31u * k->q_ln2;
   if (k->d_max >= (1u << 20)) return IBERT_ERR_SCALE_RANGE;   // cannot happen: q_ln2 <= 16787
-  // floor(d / q_ln2) for d < 2^20 by multiplication: with l = ceil(log2 q_ln2) and
-  // m = floor(2^(20+l) / q_ln2) + 1 one has 2^(20+l) < m q_ln2 <= 2^(20+l) + 2^l, which makes
-  // floor(d m / 2^(20+l)) exact for every d < 2^20.  Evaluated as umulhi(d << 12, m) >> l.
-  k->div_l = ceil_log2_u32(k->q_ln2);
-  k->div_m = (uint32_t)((uint64_t(1) << (20 + k->div_l)) / k->q_ln2 + 1);
+  // floor(d / q_ln2) for d <= d_max by multiplication (Granlund-Montgomery): with
+  // l = ceil(log2 q_ln2), N = bit length of d_max and m = floor(2^(N+l) / q_ln2) + 1 one has
+  // 2^(N+l) < m q_ln2 <= 2^(N+l) + 2^l, which makes floor(d m / 2^(N+l)) exact for d < 2^N.
+  // The shift by N+l is split around a 32-bit multiply-high.
+  {
+    const int l = ceil_log2_u32(k->q_ln2);
+    const int N = bit_length_u64(k->d_max);
+    const uint64_t m = (uint64_t(1) << (N + l)) / k->q_ln2 + 1;      // < 2^(N+1)
+    int pre = 0, post = 0;
+    uint64_t mm = m;
+    if (N + l >= 32) post = N + l - 32;
+    else {
+      // move the missing 32 - (N+l) bits into the multiplier, the rest into the operand
+      int spare = 0;
+      while (spare < 32 - (N + l) && (mm << 1) < (uint64_t(1) << 32)) { mm <<= 1; ++spare; }
+      pre = 32 - (N + l) - spare;
+    }
+    if (mm >= (uint64_t(1) << 32) || N + pre > 32) return IBERT_ERR_SCALE_RANGE;   // cannot happen
+    k->div_m = (uint32_t)mm;
+    k->div_pre = pre;
+    k->div_post = post;
+  }
   k->q_b = (int32_t)q_b;
   k->q_c = (int32_t)q_c;
   k->s_out = bl > 21 ? bl - 21 : 0;
-  k->pm8 = 8u * (uint32_t)p_max;
+  k->p_max = (uint32_t)p_max;
   return IBERT_OK;
 }
 
@@ -107,12 +125,28 @@ int make_gelu_consts(double S, double S_out, GeluConsts* k) {
   k->s_f = bl > 16 ? bl - 16 : 0;
   const double S_g = std::ldexp(S * S_erf, k->s_f) / 2.0;     // scale of q * ((q_erf + q_1) >> s_f)
   const double S_g2 = S_g * 256.0;                            // after the rounding shift by 8
-  return dyadic(S_g2 / S_out, &k->b, &k->c);
+  int rc = dyadic(S_g2 / S_out, &k->b, &k->c);
+  if (rc) return rc;
+  std::vector<int32_t> b1(1, k->b), c1(1, k->c);
+  k->fast = to_upper_word_form(&b1, c1) ? 1 : 0;
+  k->b2 = k->fast ? b1[0] : 0;
+  k->add2 = k->fast ? (int64_t(1) << 31) : 0;                 // 2^(c-1) << (32-c)
+  return IBERT_OK;
+}
+
+bool to_upper_word_form(std::vector<int32_t>* b, const std::vector<int32_t>& c) {
+  for (size_t n = 0; n < b->size(); ++n) {
+    if (c[n] < 1 || c[n] > 31) return false;
+    const int64_t shifted = (int64_t)(*b)[n] * (int64_t(1) << (32 - c[n]));
+    if (shifted > INT32_MAX || shifted < INT32_MIN) return false;
+  }
+  for (size_t n = 0; n < b->size(); ++n) (*b)[n] = (int32_t)((int64_t)(*b)[n] * (int64_t(1) << (32 - c[n])));
+  return true;
 }
 
 // LayerNorm affine + requantization folded into one dyadic step per channel: the
 // normalized value n ~ y_hat * 2^16, out = (n * b_i + B_i) >> c with a shared c.
-int make_ln_tables(const double* gamma, const double* beta, int C, double S_out, int32_t* c_out,
+int make_ln_tables(const double* gamma, const double* beta, int C, double S_out, LnConsts* k,
                    std::vector<int32_t>* b_i, std::vector<int64_t>* B_i) {
   if (!good_scale(S_out)) return IBERT_ERR_SCALE_RANGE;
   const double m0 = 1.0 / (S_out * 65536.0);
@@ -134,7 +168,26 @@ int make_ln_tables(const double* gamma, const double* beta, int C, double S_out,
     (*b_i)[i] = (int32_t)(gamma[i] < 0.0 ? -mag : mag);
     (*B_i)[i] = (int64_t)add + half;        // rounding constant folded in
   }
-  *c_out = c;
+  k->c = c;
+  // Upper-word form: the normalized value (|n| < 2^23) is produced pre-shifted by 32 - c, so
+  // the shift must stay within 8 bits and the shifted addends within 62 bits.
+  k->out_sh = 32 - c;
+  k->out_fast = (c >= 24 && c <= 31) ? 1 : 0;
+  for (int i = 0; i < C && k->out_fast; ++i)
+    if (std::llabs((*B_i)[i]) >= (int64_t(1) << (62 - k->out_sh))) k->out_fast = 0;
+  if (k->out_fast)
+    for (int i = 0; i < C; ++i) (*B_i)[i] *= (int64_t(1) << k->out_sh);
+  return IBERT_OK;
+}
+
+// dyadic(S_r / S) for the residual in front of LayerNorm, plus its upper-word form
+int make_ln_residual(double S_r, double S, LnConsts* k) {
+  if (!good_scale(S_r) || !good_scale(S)) return IBERT_ERR_SCALE_RANGE;
+  int rc = dyadic(S_r / S, &k->b_r, &k->c_r);
+  if (rc) return rc;
+  std::vector<int32_t> b1(1, k->b_r), c1(1, k->c_r);
+  k->res_fast = to_upper_word_form(&b1, c1) ? 1 : 0;
+  k->b_r2 = k->res_fast ? b1[0] : 0;
   return IBERT_OK;
 }
 

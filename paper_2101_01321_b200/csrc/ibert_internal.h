@@ -21,12 +21,13 @@ struct ExpConsts {
   int32_t s_in;      // static pre-shift of the distance from the row maximum
   uint32_t q_ln2;    // floor(ln2 / S')
   uint32_t d_max;    // 31 * q_ln2: any larger distance gives e = 0
-  uint32_t div_m;    // magic multiplier: floor(d / q_ln2) = umulhi(d << 12, div_m) >> div_l for d < 2^20
-  int32_t div_l;
+  // floor(d / q_ln2) = umulhi(d << div_pre, div_m) >> div_post, exact for every d <= d_max
+  uint32_t div_m;
+  int32_t div_pre, div_post;
   int32_t q_b;       // floor(1.353 / S')
   int32_t q_c;       // floor(0.344 / (0.3585 S'^2))
   int32_t s_out;     // static post-shift: every e < 2^21
-  uint32_t pm8;      // 8 * p_max (numerator pre-scale of the per-row quotient)
+  uint32_t p_max;    // 255 or 127: the fixed-point one of the probabilities
 };
 
 // i-GELU (Algorithm 2) followed by requantization to int8
@@ -36,6 +37,10 @@ struct GeluConsts {
   int32_t q_c;       // floor(1 / (-0.2888 S2^2)) < 0 (also q_1 = floor(1 / S_erf))
   int32_t s_f;       // shift keeping q * (q_erf + q_1) in 32 bits
   int32_t b, c;      // dyadic multiplier from the scale of round(g / 256) to S_out
+  // the same requantization as one multiply-add whose upper word is the result:
+  // (g2 * b + 2^(c-1)) >> c == (g2 * b2 + add2) >> 32 with b2 = b << (32-c); valid when fast != 0
+  int32_t b2, fast;
+  int64_t add2;
 };
 
 // residual add in front of i-LayerNorm
@@ -44,14 +49,20 @@ struct LnConsts {
   int32_t has_res;
   int32_t b_r, c_r;  // dyadic(S_r / S)
   int32_t c;         // common shift of the per-channel affine multipliers
+  // upper-word forms (see GeluConsts): residual rescale as (r * b_r2 + 2^31) >> 32 when res_fast;
+  // output as ((n << out_sh) * b_i + (B_i << out_sh)) >> 32 with out_sh = 32 - c when out_fast
+  // (the B_i table then already holds the shifted addends)
+  int32_t b_r2, res_fast;
+  int32_t out_sh, out_fast;
 };
 
 int dyadic(double m, int32_t* b, int32_t* c);
 int make_exp_consts(double S, int p_max, ExpConsts* k);
 int make_gelu_consts(double S, double S_out, GeluConsts* k);
 // per-channel multipliers b_i (int32) and addends B_i (int64, rounding constant included)
-int make_ln_tables(const double* gamma, const double* beta, int C, double S_out, int32_t* c_out,
+int make_ln_tables(const double* gamma, const double* beta, int C, double S_out, LnConsts* k,
                    std::vector<int32_t>* b_i, std::vector<int64_t>* B_i);
+int make_ln_residual(double S_r, double S, LnConsts* k);
 // per-output-channel dyadic multipliers of a linear layer; S_out_cols (N entries) or S_out
 int make_linear_tables(double S_x, const double* S_w, int N, const double* S_out_cols, double S_out,
                        std::vector<int32_t>* b, std::vector<int32_t>* c);
@@ -102,11 +113,16 @@ enum : int { EPI_INT8 = 0, EPI_Q16 = 1, EPI_RAW = 2, EPI_GELU = 3 };
 
 struct GemmEpilogue {
   int kind;
-  const int32_t* d_b;      // [N] dyadic multipliers (unused for EPI_RAW)
+  const int32_t* d_b;      // [N] dyadic multipliers b (fast: b << (32 - c)); unused for EPI_RAW
   const int32_t* d_c;      // [N] dyadic shifts
   const int32_t* d_bias;   // [N] or nullptr
+  int fast;                // every column's requantization fits the upper-word form
   GeluConsts gelu;         // EPI_GELU only
 };
+
+// Upper-word form of a column set: true if for every n, c[n] >= 1 and b[n] << (32 - c[n]) fits
+// int32; then b is replaced by the shifted multipliers.
+bool to_upper_word_form(std::vector<int32_t>* b, const std::vector<int32_t>& c);
 
 int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, int N, int K,
                    const GemmEpilogue& epi, void* out);

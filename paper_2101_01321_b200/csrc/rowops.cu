@@ -10,11 +10,6 @@ namespace {
 
 constexpr int kThreads = 256;
 
-__device__ __forceinline__ uint32_t pack4(int32_t a, int32_t b, int32_t c, int32_t d) {
-  return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) |
-         ((uint32_t)(d & 0xff) << 24);
-}
-
 // ----------------------------------------------------------------------------- i-GELU
 // Each thread converts 4 int4 vectors (16 values); vector j of a thread sits 32 vectors
 // after vector j-1 so that every load and store instruction of a warp is contiguous.
@@ -38,11 +33,19 @@ __global__ void __launch_bounds__(kThreads) gelu_kernel(const int32_t* __restric
     for (int j = 0; j < 4; ++j) {
       const int64_t idx = base + j * 32 + lane;
       if (idx < n_vec) {
-        const int32_t a = igelu_q16_to_int8(clamp_sym(v[j].x, 32767), k, half);
-        const int32_t b = igelu_q16_to_int8(clamp_sym(v[j].y, 32767), k, half);
-        const int32_t c = igelu_q16_to_int8(clamp_sym(v[j].z, 32767), k, half);
-        const int32_t d = igelu_q16_to_int8(clamp_sym(v[j].w, 32767), k, half);
-        __stcs(o4 + idx, pack4(a, b, c, d));
+        int32_t a, b, c, d;
+        if (k.fast) {
+          a = igelu_q16_upper(clamp_sym(v[j].x, 32767), k);
+          b = igelu_q16_upper(clamp_sym(v[j].y, 32767), k);
+          c = igelu_q16_upper(clamp_sym(v[j].z, 32767), k);
+          d = igelu_q16_upper(clamp_sym(v[j].w, 32767), k);
+        } else {
+          a = igelu_q16_to_int8(clamp_sym(v[j].x, 32767), k, half);
+          b = igelu_q16_to_int8(clamp_sym(v[j].y, 32767), k, half);
+          c = igelu_q16_to_int8(clamp_sym(v[j].z, 32767), k, half);
+          d = igelu_q16_to_int8(clamp_sym(v[j].w, 32767), k, half);
+        }
+        __stcs(o4 + idx, pack4_sat_s8(a, b, c, d));
       }
     }
   }
@@ -56,7 +59,7 @@ __global__ void __launch_bounds__(kThreads) gelu_kernel(const int32_t* __restric
 // ----------------------------------------------------------------------------- i-softmax
 // One warp per row; a lane keeps VPL int4 vectors (4*VPL scores) in registers.
 // VEC: rows are 16-byte aligned (L % 4 == 0) and loaded/stored as vectors.
-template <int VPL, bool VEC>
+template <int VPL, bool VEC, int DIV>
 __global__ void __launch_bounds__(kThreads) softmax_kernel(const int32_t* __restrict__ q, int64_t rows,
                                                            int L, ExpConsts k, uint8_t* __restrict__ out) {
   const int lane = threadIdx.x & 31;
@@ -91,19 +94,19 @@ __global__ void __launch_bounds__(kThreads) softmax_kernel(const int32_t* __rest
       const int col = 4 * (j * 32 + lane);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint32_t e = (col + i < L) ? iexp_dist((uint32_t)mx - (uint32_t)v[j][i], k) : 0u;
+        const uint32_t e = (col + i < L) ? iexp_dist<DIV>((uint32_t)mx - (uint32_t)v[j][i], k) : 0u;
         v[j][i] = (int32_t)e;
         sum += e;
       }
     }
     sum = __reduce_add_sync(0xffffffffu, sum);
-    const RowDivisor rd = make_row_divisor(sum);
+    const RowDivisor rd = make_row_divisor(sum, k.p_max);
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
       const int col = 4 * (j * 32 + lane);
       uint32_t p[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) p[i] = softmax_quotient((uint32_t)v[j][i], k.pm8, rd);
+      for (int i = 0; i < 4; ++i) p[i] = softmax_quotient((uint32_t)v[j][i], rd);
       if (VEC) {
         if (col < L)
           __stcs(reinterpret_cast<uint32_t*>(orow + col), p[0] | (p[1] << 8) | (p[2] << 16) | (p[3] << 24));
@@ -117,8 +120,27 @@ __global__ void __launch_bounds__(kThreads) softmax_kernel(const int32_t* __rest
 }
 
 // ----------------------------------------------------------------------------- i-LayerNorm
+// floor(sqrt(floor(ss / C))), i.e. the largest s with s*s*C <= ss -- the value Algorithm 4
+// returns for n = floor(ss / C).  A 64-bit integer division costs on the order of a hundred
+// instructions here, so instead of iterating x <- (x + n/x)/2 the warp finds the same integer by
+// a radix-32 search: in each of five rounds the 32 lanes test 32 candidates with one multiply
+// each.  Needs s < 2^25 and ss < 2^61 / C.
+__device__ __forceinline__ uint32_t warp_isqrt_of_quotient(uint64_t ss, uint32_t C, int lane) {
+  uint32_t base = 0;
+#pragma unroll
+  for (int shift = 20; shift >= 0; shift -= 5) {
+    const uint32_t cand = base + ((uint32_t)lane << shift);
+    const uint64_t sq = (uint64_t)cand * (uint64_t)cand;
+    const bool le = sq * (uint64_t)C <= ss;                       // true for a prefix of the lanes
+    const uint32_t cnt = __popc(__ballot_sync(0xffffffffu, le));  // >= 1: lane 0 tests `base` itself
+    base += (cnt - 1u) << shift;
+  }
+  return base;
+}
+
 // One warp per row, the whole row in registers (VPL int4 vectors per lane).
-template <int VPL, bool VEC>
+// FAST: residual rescale and output requantization are in upper-word form (one multiply-add each).
+template <int VPL, bool VEC, bool FAST>
 __global__ void __launch_bounds__(kThreads) layernorm_kernel(const int32_t* __restrict__ q,
                                                              const int8_t* __restrict__ r, int64_t rows,
                                                              LnConsts k, const int32_t* __restrict__ b_i,
@@ -147,7 +169,8 @@ __global__ void __launch_bounds__(kThreads) layernorm_kernel(const int32_t* __re
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const int32_t rv = (int32_t)(int8_t)(rw >> (8 * i));
-              v[j][i] += (int32_t)(((int64_t)rv * k.b_r + half_r) >> k.c_r);
+              if (FAST) v[j][i] += requant_upper(rv, k.b_r2, int64_t(1) << 31);
+              else v[j][i] += (int32_t)(((int64_t)rv * k.b_r + half_r) >> k.c_r);
             }
           }
         } else {
@@ -184,28 +207,46 @@ __global__ void __launch_bounds__(kThreads) layernorm_kernel(const int32_t* __re
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    const uint64_t var = ss / (uint64_t)C;
-    uint32_t sigma = isqrt_newton(var);
+    uint32_t sigma = warp_isqrt_of_quotient(ss, (uint32_t)C, lane);   // I-Sqrt(floor(ss / C))
     sigma = sigma < 1u ? 1u : sigma;
-    const int64_t rho64 = (int64_t)(0x80000000u / sigma);        // floor(2^31 / sigma)
+    const int64_t rho64 = (int64_t)(0x80000000u / sigma);            // floor(2^31 / sigma)
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
       const int col = 4 * (j * 32 + lane);
-      int32_t o[4];
+      int32_t o[4] = {0, 0, 0, 0};
+      if (FAST) {
+        if (col < C) {
+          const int4 bb = __ldg(reinterpret_cast<const int4*>(b_i + col));
+          const longlong2 B01 = __ldg(reinterpret_cast<const longlong2*>(B_i + col));
+          const longlong2 B23 = __ldg(reinterpret_cast<const longlong2*>(B_i + col + 2));
+          const int32_t bv[4] = {bb.x, bb.y, bb.z, bb.w};
+          const int64_t Bv[4] = {B01.x, B01.y, B23.x, B23.y};
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        o[i] = 0;
-        if (col + i < C) {
-          const int32_t nrm = (int32_t)(((int64_t)v[j][i] * rho64) >> 15);
-          int64_t t = (int64_t)nrm * (int64_t)__ldg(b_i + col + i) + __ldg(B_i + col + i);
-          t >>= k.c;
-          t = t > 127 ? 127 : t;
-          t = t < -127 ? -127 : t;
-          o[i] = (int32_t)t;
+          for (int i = 0; i < 4; ++i) {
+            // normalized value pre-shifted by out_sh: (y * rho) >> (15 - out_sh), |.| < 2^31
+            const int32_t nrm = (int32_t)(((int64_t)v[j][i] * rho64) >> (15 - k.out_sh));
+            o[i] = max(requant_upper(nrm, bv[i], Bv[i]), -127);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (col + i < C) {
+            const int32_t nrm = (int32_t)(((int64_t)v[j][i] * rho64) >> 15);
+            int64_t t;
+            if (k.out_fast) {   // the addend table is pre-shifted: undo it on this path
+              t = ((int64_t)nrm * ((int64_t)__ldg(b_i + col + i) << k.out_sh) + __ldg(B_i + col + i)) >> 32;
+            } else {
+              t = ((int64_t)nrm * (int64_t)__ldg(b_i + col + i) + __ldg(B_i + col + i)) >> k.c;
+            }
+            t = t > 127 ? 127 : t;
+            t = t < -127 ? -127 : t;
+            o[i] = (int32_t)t;
+          }
         }
       }
       if (VEC) {
-        if (col < C) __stcs(reinterpret_cast<uint32_t*>(orow + col), pack4(o[0], o[1], o[2], o[3]));
+        if (col < C) __stcs(reinterpret_cast<uint32_t*>(orow + col), pack4_sat_s8(o[0], o[1], o[2], o[3]));
       } else {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
@@ -237,16 +278,24 @@ int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const 
   const int grid = grid_for(ctx, rows, 8);
   const bool vec = (L % 4) == 0;
   const int vpl = (L + 127) / 128;   // vectors per lane
-#define IBERT_SM(V)                                                                              \
-  do {                                                                                           \
-    if (vec) softmax_kernel<V, true><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out);    \
-    else softmax_kernel<V, false><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out);       \
+  const int div = exp_div_mode(k);
+#define IBERT_SM2(V, D)                                                                            \
+  do {                                                                                             \
+    if (vec) softmax_kernel<V, true, D><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out);   \
+    else softmax_kernel<V, false, D><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out);      \
+  } while (0)
+#define IBERT_SM(V)                 \
+  do {                              \
+    if (div == 0) IBERT_SM2(V, 0);  \
+    else if (div == 1) IBERT_SM2(V, 1); \
+    else IBERT_SM2(V, 2);           \
   } while (0)
   if (vpl <= 1) IBERT_SM(1);
   else if (vpl <= 2) IBERT_SM(2);
   else if (vpl <= 4) IBERT_SM(4);
   else IBERT_SM(8);
 #undef IBERT_SM
+#undef IBERT_SM2
   return check_launch();
 }
 
@@ -256,10 +305,12 @@ int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t 
   const int grid = grid_for(ctx, rows, 8);
   const bool vec = (k.C % 4) == 0;
   const int vpl = (k.C + 127) / 128;
-#define IBERT_LN(V)                                                                                     \
-  do {                                                                                                  \
-    if (vec) layernorm_kernel<V, true><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out); \
-    else layernorm_kernel<V, false><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);    \
+  const bool fast = vec && k.out_fast && (!k.has_res || k.res_fast);
+#define IBERT_LN(V)                                                                                              \
+  do {                                                                                                           \
+    if (fast) layernorm_kernel<V, true, true><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);  \
+    else if (vec) layernorm_kernel<V, true, false><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out); \
+    else layernorm_kernel<V, false, false><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);     \
   } while (0)
   if (vpl <= 2) IBERT_LN(2);
   else if (vpl <= 4) IBERT_LN(4);

@@ -81,3 +81,19 @@ def test_create_fails_cleanly_without_a_usable_device(lib):
     h = C.c_void_p()
     assert lib.ibert_create(C.byref(h), 0, None) == -6      # IBERT_ERR_CUDA, no fallback
     assert not h.value
+
+
+def test_exp_division_by_multiplication_is_exact_for_every_distance(lib):
+    # host emulation of the kernels' multiply-high division by q_ln2, all d in [0, 31 q_ln2]
+    import oracle
+    rnd = random.Random(9)
+    scales = [0.69, 0.5, 0.3, 0.1, 1e-2, 1e-3, 4.5e-5, 3.8e-5, 2e-5, 1e-8, 4.13e-5, 8.2e-5, 8.3e-5]
+    scales += [math.exp(rnd.uniform(math.log(1e-9), math.log(0.69))) for _ in range(300)]
+    seen = set()
+    for S in scales:
+        q = C.c_int32()
+        assert lib.ibert_selftest_exp_division(S, C.byref(q)) == 0, S
+        assert q.value == oracle.exp_consts(S)["q_ln2"]
+        seen.add(q.value.bit_length())
+    assert len(seen) >= 12                     # divisors of many sizes were exercised
+    assert lib.ibert_selftest_exp_division(0.7, None) == -3

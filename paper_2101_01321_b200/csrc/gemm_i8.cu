@@ -80,12 +80,15 @@ constexpr int kGemmThreads = 64 + kEpiThreads;   // producer warp, MMA warp, epi
 
 template <int BN>
 struct GemmSmem {
-  static constexpr int kStages = BN >= 256 ? 4 : 6;
+  static constexpr int kStages = BN >= 256 ? 3 : 4;
   static constexpr int kABytes = BM * BK;
   static constexpr int kBBytes = BN * BK;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  // operand stages | per-column epilogue parameters (int4 per column) | barriers
-  static constexpr int kParamOff = kStages * kStageBytes;
+  // operand stages | output staging (two 4 KB tiles per epilogue warp) | per-column epilogue
+  // parameters (int4 per column) | barriers
+  static constexpr int kOutOff = kStages * kStageBytes;
+  static constexpr int kOutTileBytes = 32 * 128;
+  static constexpr int kParamOff = kOutOff + kEpiWarps * 2 * kOutTileBytes;
   static constexpr int kBarOff = kParamOff + BN * 16;
   static constexpr int kBytes = kBarOff + 256;
   static constexpr int kAlloc = kBytes + 1024;   // slack to align the operand area to 1024 bytes
@@ -98,18 +101,24 @@ struct GemmArgs {
   const int32_t* c;
   const int32_t* bias;
   GeluConsts gelu;
-  void* out;
   int32_t* status;
 };
 
-// One 32-column chunk of one accumulator row: registers -> epilogue -> global memory.
+// One 32-column chunk of one accumulator row: registers -> epilogue -> the warp's staging tile
+// (32 rows x ROW_BYTES, 16-byte pieces XOR-swizzled the way the TMA store expects).
+// `piece0` is the index of the first 16-byte piece this chunk occupies in the staging row.
 // FAST: every column's requantization is in upper-word form (one 64-bit multiply-add).
-template <int KIND, bool FAST>
+template <int ROW_BYTES>
+__device__ __forceinline__ uint32_t staging_piece_offset(uint32_t row, uint32_t piece) {
+  if constexpr (ROW_BYTES == 128) return row * 128u + ((piece ^ (row & 7u)) << 4);
+  else return row * 64u + ((piece ^ ((row >> 1) & 3u)) << 4);
+}
+
+template <int KIND, bool FAST, int ROW_BYTES>
 __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[32], const int4* __restrict__ prm,
-                                               const GemmArgs& args, const GeluConsts& gk, int64_t gelu_half,
-                                               int64_t row, bool row_ok, int col0) {
+                                               const GeluConsts& gk, int64_t gelu_half, uint8_t* stage,
+                                               uint32_t row, uint32_t piece0) {
   if constexpr (KIND == EPI_RAW || KIND == EPI_Q16) {
-    int32_t* orow = static_cast<int32_t*>(args.out) + row * args.N + col0;
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
       int32_t o[4];
@@ -122,11 +131,10 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[32], const in
         else if constexpr (FAST) o[i] = clamp_sym(requant_upper(a, p.x, add), 32767);
         else o[i] = requant_add(a, p.x, add, p.y, 32767);
       }
-      if (row_ok && col0 + g * 4 < args.N)
-        *reinterpret_cast<int4*>(orow + g * 4) = make_int4(o[0], o[1], o[2], o[3]);
+      *reinterpret_cast<int4*>(stage + staging_piece_offset<ROW_BYTES>(row, piece0 + g)) =
+          make_int4(o[0], o[1], o[2], o[3]);
     }
   } else {
-    int8_t* orow = static_cast<int8_t*>(args.out) + row * args.N + col0;
 #pragma unroll
     for (int g = 0; g < 2; ++g) {
       uint32_t w[4];
@@ -154,8 +162,8 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[32], const in
         }
         w[i] = pack4_sat_s8(o[0], o[1], o[2], o[3]);    // upper clamp (+127) happens here
       }
-      if (row_ok && col0 + g * 16 < args.N)
-        *reinterpret_cast<uint4*>(orow + g * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(stage + staging_piece_offset<ROW_BYTES>(row, piece0 + g)) =
+          make_uint4(w[0], w[1], w[2], w[3]);
     }
   }
 }
@@ -163,7 +171,7 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[32], const in
 template <int BN, int KIND, bool FAST>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const GemmArgs args) {
+               const __grid_constant__ CUtensorMap map_out, const GemmArgs args) {
   using SM = GemmSmem<BN>;
   constexpr int kStages = SM::kStages;
   constexpr uint32_t kTmemCols = 2 * BN;          // two accumulator stages (power of two >= 32)
@@ -198,6 +206,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     ptx::fence_mbar_init();
     ptx::tma_prefetch_desc(&map_a);
     ptx::tma_prefetch_desc(&map_b);
+    ptx::tma_prefetch_desc(&map_out);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_addr(s_tmem), kTmemCols);
@@ -258,9 +267,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..9)
-    const int quarter = warp & 3;                      // TMEM lanes 32*quarter .. +31 belong to this warp
-    const int half_id = (warp - 2) >> 2;               // which of the two warps of this quarter
+    // Warp w owns TMEM lanes 32*(w%4)..+31 (rows) and, of those rows, one half of the tile's
+    // columns.  Results go through a swizzled staging tile in shared memory and leave with a TMA
+    // store (full-line writes; rows / columns beyond M / N are clipped by the tensor map).
+    constexpr bool kOut32 = (KIND == EPI_RAW || KIND == EPI_Q16);
+    constexpr int kChunks = BN / 64;                   // 32-column chunks per warp and tile
+    constexpr int kRowBytes = kOut32 ? 128 : BN / 2;   // staging row: one chunk of int32 or all chunks of int8
+    const int quarter = warp & 3;
+    const int half_id = (warp - 2) >> 2;               // which column half of the tile
     const int et = threadIdx.x - 64;                   // 0..kEpiThreads-1
+    uint8_t* stage0 = smem + SM::kOutOff + (warp - 2) * 2 * SM::kOutTileBytes;
+    uint32_t buf = 0;
     const GeluConsts gk = args.gelu;
     const int64_t gelu_half = rounding_half(gk.c);
     uint32_t acc = 0, acc_phase = 0;
@@ -293,21 +310,39 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) continue;
       ptx::tc_fence_after_sync();
-      const int64_t row = m0 + quarter * 32 + lane;
-      const bool row_ok = row < args.M;
+      const int out_row0 = (int)m0 + quarter * 32;
       const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
-      for (int ch = half_id; ch < BN / 32; ch += 2) {
+      for (int ci = 0; ci < kChunks; ++ci) {
+        const int ch = half_id * kChunks + ci;
         uint32_t v[32];
         ptx::tmem_ld32(t_row + ch * 32, v);
         ptx::tmem_wait_ld();
-        epilogue_chunk<KIND, FAST>(v, s_param + ch * 32, args, gk, gelu_half, row, row_ok, n0 + ch * 32);
+        uint8_t* stage = stage0 + buf * SM::kOutTileBytes;
+        if (kOut32 || ci == 0) {
+          // the store issued two tiles ago from this buffer must have finished reading it
+          if (lane == 0) ptx::bulk_wait_read<1>();
+          __syncwarp();
+        }
+        epilogue_chunk<KIND, FAST, kRowBytes>(v, s_param + ch * 32, gk, gelu_half, stage, (uint32_t)lane,
+                                              kOut32 ? 0u : (uint32_t)(ci * 2));
+        if (kOut32 || ci == kChunks - 1) {
+          ptx::fence_proxy_async_smem();               // staging writes -> visible to the TMA engine
+          __syncwarp();
+          if (lane == 0) {
+            const int x_bytes = kOut32 ? (n0 + ch * 32) * 4 : n0 + half_id * (BN / 2);
+            ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), x_bytes, out_row0);
+            ptx::bulk_commit();
+          }
+          buf ^= 1;
+        }
       }
       ptx::tc_fence_before_sync();
       ptx::mbar_arrive(bar_acc_empty + 8 * acc);
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1;
     }
+    if (lane == 0) ptx::bulk_wait<0>();                // all of this warp's stores have landed
   }
 
   if (!ok) atomicCAS(args.status, 0, IBERT_ERR_TIMEOUT);
@@ -320,7 +355,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 }
 
 template <int BN, int KIND, bool FAST>
-int launch_inst(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& args) {
+int launch_inst(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo,
+                const GemmArgs& args) {
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(gemm_i8_kernel<BN, KIND, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -330,17 +366,18 @@ int launch_inst(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, co
   }
   const int64_t tiles = ((args.M + BM - 1) / BM) * ((args.N + BN - 1) / BN);
   const int grid = (int)(tiles < ctx->num_sms ? tiles : ctx->num_sms);
-  gemm_i8_kernel<BN, KIND, FAST><<<grid, kGemmThreads, GemmSmem<BN>::kAlloc, ctx->stream>>>(ma, mb, args);
+  gemm_i8_kernel<BN, KIND, FAST><<<grid, kGemmThreads, GemmSmem<BN>::kAlloc, ctx->stream>>>(ma, mb, mo, args);
   return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
 }
 
 template <int BN>
-int launch_bn(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& a, int kind, bool fast) {
+int launch_bn(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const GemmArgs& a,
+              int kind, bool fast) {
   switch (kind) {
-    case EPI_INT8: return fast ? launch_inst<BN, EPI_INT8, true>(ctx, ma, mb, a) : launch_inst<BN, EPI_INT8, false>(ctx, ma, mb, a);
-    case EPI_Q16: return fast ? launch_inst<BN, EPI_Q16, true>(ctx, ma, mb, a) : launch_inst<BN, EPI_Q16, false>(ctx, ma, mb, a);
-    case EPI_GELU: return fast ? launch_inst<BN, EPI_GELU, true>(ctx, ma, mb, a) : launch_inst<BN, EPI_GELU, false>(ctx, ma, mb, a);
-    default: return launch_inst<BN, EPI_RAW, false>(ctx, ma, mb, a);
+    case EPI_INT8: return fast ? launch_inst<BN, EPI_INT8, true>(ctx, ma, mb, mo, a) : launch_inst<BN, EPI_INT8, false>(ctx, ma, mb, mo, a);
+    case EPI_Q16: return fast ? launch_inst<BN, EPI_Q16, true>(ctx, ma, mb, mo, a) : launch_inst<BN, EPI_Q16, false>(ctx, ma, mb, mo, a);
+    case EPI_GELU: return fast ? launch_inst<BN, EPI_GELU, true>(ctx, ma, mb, mo, a) : launch_inst<BN, EPI_GELU, false>(ctx, ma, mb, mo, a);
+    default: return launch_inst<BN, EPI_RAW, false>(ctx, ma, mb, mo, a);
   }
 }
 
@@ -368,13 +405,25 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
     int rc = encode_tensor_map(&mb, w, 2, dims, str, box, 128);
     if (rc) return rc;
   }
+  CUtensorMap mo;
+  {
+    // the output as a byte matrix [M, N * element size]; one box = one warp's staging tile
+    const bool out32 = epi.kind == EPI_RAW || epi.kind == EPI_Q16;
+    const uint64_t row_bytes = (uint64_t)N * (out32 ? 4 : 1);
+    const uint32_t box_bytes = out32 ? 128u : (uint32_t)(BN / 2);
+    const uint64_t dims[2] = {row_bytes, (uint64_t)M};
+    const uint64_t str[1] = {row_bytes};
+    const uint32_t box[2] = {box_bytes, 32};
+    int rc = encode_tensor_map(&mo, out, 2, dims, str, box, (int)box_bytes);
+    if (rc) return rc;
+  }
   GemmArgs a{};
   a.M = M; a.N = N; a.K = K;
   a.b = epi.d_b; a.c = epi.d_c; a.bias = epi.d_bias; a.gelu = epi.gelu;
-  a.out = out; a.status = ctx->d_status;
+  a.status = ctx->d_status;
   // upper-word epilogue needs both the per-column multipliers and (for GELU) the final one in that form
   const bool fast = epi.fast != 0 && (epi.kind != EPI_GELU || epi.gelu.fast != 0);
-  return wide ? launch_bn<256>(ctx, ma, mb, a, epi.kind, fast) : launch_bn<128>(ctx, ma, mb, a, epi.kind, fast);
+  return wide ? launch_bn<256>(ctx, ma, mb, mo, a, epi.kind, fast) : launch_bn<128>(ctx, ma, mb, mo, a, epi.kind, fast);
 }
 
 }  // namespace ibert

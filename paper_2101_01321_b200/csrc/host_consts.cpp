@@ -185,9 +185,9 @@ int make_ln_residual(double S_r, double S, LnConsts* k) {
   if (!good_scale(S_r) || !good_scale(S)) return IBERT_ERR_SCALE_RANGE;
   int rc = dyadic(S_r / S, &k->b_r, &k->c_r);
   if (rc) return rc;
-  std::vector<int32_t> b1(1, k->b_r), c1(1, k->c_r);
-  k->res_fast = to_upper_word_form(&b1, c1) ? 1 : 0;
-  k->b_r2 = k->res_fast ? b1[0] : 0;
+  // |r| <= 127 leaves 24 bits of headroom: r << (32 - c_r) fits int32 for c_r >= 8
+  k->res_fast = (k->c_r >= 8 && k->c_r <= 31) ? 1 : 0;
+  k->res_sh = 32 - k->c_r;
   return IBERT_OK;
 }
 

@@ -49,10 +49,11 @@ struct LnConsts {
   int32_t has_res;
   int32_t b_r, c_r;  // dyadic(S_r / S)
   int32_t c;         // common shift of the per-channel affine multipliers
-  // upper-word forms (see GeluConsts): residual rescale as (r * b_r2 + 2^31) >> 32 when res_fast;
-  // output as ((n << out_sh) * b_i + (B_i << out_sh)) >> 32 with out_sh = 32 - c when out_fast
-  // (the B_i table then already holds the shifted addends)
-  int32_t b_r2, res_fast;
+  // upper-word forms with the *value* pre-shifted (it has the headroom, the 31-bit multiplier
+  // has none): residual rescale as ((r << res_sh) * b_r + 2^31) >> 32 with res_sh = 32 - c_r when
+  // res_fast; output as ((n << out_sh) * b_i + (B_i << out_sh)) >> 32 with out_sh = 32 - c when
+  // out_fast (the B_i table then already holds the shifted addends)
+  int32_t res_sh, res_fast;
   int32_t out_sh, out_fast;
 };
 

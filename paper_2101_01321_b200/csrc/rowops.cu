@@ -140,8 +140,12 @@ __device__ __forceinline__ uint32_t warp_isqrt_of_quotient(uint64_t ss, uint32_t
 
 // One warp per row, the whole row in registers (VPL int4 vectors per lane).
 // FAST: residual rescale and output requantization are in upper-word form (one multiply-add each).
+// Resident CTAs per SM the register budget is tuned for: the kernel is latency-bound on the row
+// loads, so short rows trade registers for more warps in flight.
+constexpr int ln_min_blocks(int vpl) { return vpl <= 4 ? 4 : (vpl <= 6 ? 3 : (vpl <= 8 ? 2 : 1)); }
+
 template <int VPL, bool VEC, bool FAST>
-__global__ void __launch_bounds__(kThreads) layernorm_kernel(const int32_t* __restrict__ q,
+__global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel(const int32_t* __restrict__ q,
                                                              const int8_t* __restrict__ r, int64_t rows,
                                                              LnConsts k, const int32_t* __restrict__ b_i,
                                                              const int64_t* __restrict__ B_i,
@@ -169,7 +173,7 @@ __global__ void __launch_bounds__(kThreads) layernorm_kernel(const int32_t* __re
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const int32_t rv = (int32_t)(int8_t)(rw >> (8 * i));
-              if (FAST) v[j][i] += requant_upper(rv, k.b_r2, int64_t(1) << 31);
+              if (FAST) v[j][i] += requant_upper(rv << k.res_sh, k.b_r, int64_t(1) << 31);
               else v[j][i] += (int32_t)(((int64_t)rv * k.b_r + half_r) >> k.c_r);
             }
           }
@@ -223,8 +227,8 @@ __global__ void __launch_bounds__(kThreads) layernorm_kernel(const int32_t* __re
           const int64_t Bv[4] = {B01.x, B01.y, B23.x, B23.y};
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            // normalized value pre-shifted by out_sh: (y * rho) >> (15 - out_sh), |.| < 2^31
-            const int32_t nrm = (int32_t)(((int64_t)v[j][i] * rho64) >> (15 - k.out_sh));
+            // normalized value floor(y * rho / 2^15), then pre-shifted by out_sh (|.| < 2^31)
+            const int32_t nrm = (int32_t)(((int64_t)v[j][i] * rho64) >> 15) << k.out_sh;
             o[i] = max(requant_upper(nrm, bv[i], Bv[i]), -127);
           }
         }

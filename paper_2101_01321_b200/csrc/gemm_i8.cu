@@ -6,7 +6,7 @@
 // out[m, n] = epilogue( sum_k x[m, k] * w[n, k] + bias[n] )      x: [M, K], w: [N, K]
 //
 // One persistent CTA per SM walks 128 x BN output tiles.  Warp 0 is the TMA producer,
-// warp 1 issues the MMAs, warps 2..9 run the epilogue; two TMEM accumulator stages let
+// warp 1 issues the MMAs, warps 2.. run the epilogue; two TMEM accumulator stages let
 // the (integer-ALU heavy) epilogue of tile i overlap the MMAs of tile i+1.
 #include <cuda.h>
 
@@ -74,21 +74,23 @@ namespace {
 constexpr int BM = 128;           // rows per tile = TMEM lanes
 constexpr int BK = 128;           // K bytes per pipeline stage = one 128-byte swizzle span
 constexpr int UMMA_K = 32;        // K per tcgen05.mma kind::i8
-constexpr int kEpiWarps = 8;      // two warps per TMEM lane quarter, each taking every other column chunk
-constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kGemmThreads = 64 + kEpiThreads;   // producer warp, MMA warp, epilogue warps
+// Epilogue warps: every warp handles two 32-column chunks of the 32 rows (TMEM lanes) its
+// position in the warp quartet gives it access to, so a tile of BN columns takes BN / 16 warps.
+// The integer epilogue is what bounds these GEMMs at K <= 1024, hence the many warps.
+__host__ __device__ constexpr int epi_warps(int bn) { return bn / 16; }
+__host__ __device__ constexpr int gemm_threads(int bn) { return 64 + 32 * epi_warps(bn); }   // + producer warp, MMA warp
 
 template <int BN>
 struct GemmSmem {
-  static constexpr int kStages = BN >= 256 ? 3 : 4;
+  static constexpr int kStages = BN >= 256 ? 3 : 5;
   static constexpr int kABytes = BM * BK;
   static constexpr int kBBytes = BN * BK;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  // operand stages | output staging (two 4 KB tiles per epilogue warp) | per-column epilogue
+  // operand stages | output staging (one 4 KB tile per epilogue warp) | per-column epilogue
   // parameters (int4 per column) | barriers
   static constexpr int kOutOff = kStages * kStageBytes;
   static constexpr int kOutTileBytes = 32 * 128;
-  static constexpr int kParamOff = kOutOff + kEpiWarps * 2 * kOutTileBytes;
+  static constexpr int kParamOff = kOutOff + epi_warps(BN) * kOutTileBytes;
   static constexpr int kBarOff = kParamOff + BN * 16;
   static constexpr int kBytes = kBarOff + 256;
   static constexpr int kAlloc = kBytes + 1024;   // slack to align the operand area to 1024 bytes
@@ -169,11 +171,12 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[32], const in
 }
 
 template <int BN, int KIND, bool FAST>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(gemm_threads(BN), 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_out, const GemmArgs args) {
   using SM = GemmSmem<BN>;
   constexpr int kStages = SM::kStages;
+  constexpr int kEpiThreads = 32 * epi_warps(BN);
   constexpr uint32_t kTmemCols = 2 * BN;          // two accumulator stages (power of two >= 32)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -266,18 +269,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..9)
-    // Warp w owns TMEM lanes 32*(w%4)..+31 (rows) and, of those rows, one half of the tile's
+    // ------------------------------------------------------------ epilogue (warps 2..)
+    // Warp w owns TMEM lanes 32*(w%4)..+31 (rows) and, of those rows, 64 of the tile's
     // columns.  Results go through a swizzled staging tile in shared memory and leave with a TMA
     // store (full-line writes; rows / columns beyond M / N are clipped by the tensor map).
     constexpr bool kOut32 = (KIND == EPI_RAW || KIND == EPI_Q16);
-    constexpr int kChunks = BN / 64;                   // 32-column chunks per warp and tile
-    constexpr int kRowBytes = kOut32 ? 128 : BN / 2;   // staging row: one chunk of int32 or all chunks of int8
+    constexpr int kChunks = 2;                         // 32-column chunks per warp and tile
+    constexpr int kRowBytes = kOut32 ? 128 : 64;       // staging row: one chunk of int32 or both chunks of int8
     const int quarter = warp & 3;
-    const int half_id = (warp - 2) >> 2;               // which column half of the tile
+    const int part = (warp - 2) >> 2;                  // which 64-column part of the tile
     const int et = threadIdx.x - 64;                   // 0..kEpiThreads-1
-    uint8_t* stage0 = smem + SM::kOutOff + (warp - 2) * 2 * SM::kOutTileBytes;
-    uint32_t buf = 0;
+    uint8_t* stage = smem + SM::kOutOff + (warp - 2) * SM::kOutTileBytes;
     const GeluConsts gk = args.gelu;
     const int64_t gelu_half = rounding_half(gk.c);
     uint32_t acc = 0, acc_phase = 0;
@@ -314,14 +316,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
       for (int ci = 0; ci < kChunks; ++ci) {
-        const int ch = half_id * kChunks + ci;
+        const int ch = part * kChunks + ci;
         uint32_t v[32];
         ptx::tmem_ld32(t_row + ch * 32, v);
         ptx::tmem_wait_ld();
-        uint8_t* stage = stage0 + buf * SM::kOutTileBytes;
         if (kOut32 || ci == 0) {
-          // the store issued two tiles ago from this buffer must have finished reading it
-          if (lane == 0) ptx::bulk_wait_read<1>();
+          // the previous store from this staging tile must have finished reading it
+          if (lane == 0) ptx::bulk_wait_read<0>();
           __syncwarp();
         }
         epilogue_chunk<KIND, FAST, kRowBytes>(v, s_param + ch * 32, gk, gelu_half, stage, (uint32_t)lane,
@@ -330,11 +331,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           ptx::fence_proxy_async_smem();               // staging writes -> visible to the TMA engine
           __syncwarp();
           if (lane == 0) {
-            const int x_bytes = kOut32 ? (n0 + ch * 32) * 4 : n0 + half_id * (BN / 2);
+            const int x_bytes = kOut32 ? (n0 + ch * 32) * 4 : n0 + part * 64;
             ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), x_bytes, out_row0);
             ptx::bulk_commit();
           }
-          buf ^= 1;
         }
       }
       ptx::tc_fence_before_sync();
@@ -366,7 +366,7 @@ int launch_inst(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, co
   }
   const int64_t tiles = ((args.M + BM - 1) / BM) * ((args.N + BN - 1) / BN);
   const int grid = (int)(tiles < ctx->num_sms ? tiles : ctx->num_sms);
-  gemm_i8_kernel<BN, KIND, FAST><<<grid, kGemmThreads, GemmSmem<BN>::kAlloc, ctx->stream>>>(ma, mb, mo, args);
+  gemm_i8_kernel<BN, KIND, FAST><<<grid, gemm_threads(BN), GemmSmem<BN>::kAlloc, ctx->stream>>>(ma, mb, mo, args);
   return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
 }
 
@@ -410,7 +410,7 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
     // the output as a byte matrix [M, N * element size]; one box = one warp's staging tile
     const bool out32 = epi.kind == EPI_RAW || epi.kind == EPI_Q16;
     const uint64_t row_bytes = (uint64_t)N * (out32 ? 4 : 1);
-    const uint32_t box_bytes = out32 ? 128u : (uint32_t)(BN / 2);
+    const uint32_t box_bytes = out32 ? 128u : 64u;
     const uint64_t dims[2] = {row_bytes, (uint64_t)M};
     const uint64_t str[1] = {row_bytes};
     const uint32_t box[2] = {box_bytes, 32};

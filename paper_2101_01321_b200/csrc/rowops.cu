@@ -2,7 +2,10 @@
 // residual + i-LayerNorm (Sec. 3.6, Algorithm 4).  All three are HBM-streaming kernels:
 // 128-bit coalesced loads of the int32 inputs, all arithmetic in registers, packed int8
 // stores.  Rows are owned by one warp and reduced with warp shuffles.
+#include <algorithm>
+
 #include "device_utils.cuh"
+#include "sm100_ptx.cuh"
 
 namespace ibert {
 
@@ -260,6 +263,125 @@ __global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel
   }
 }
 
+// Same row computation, fed by bulk async copies: every warp streams its rows (Q16 row and int8
+// residual row) through a private ring of DEPTH shared-memory slots, so the loads of the next
+// rows are in flight while the current row is reduced -- the row loop no longer waits on HBM.
+// Requires C % 16 == 0 (16-byte aligned rows), upper-word constants, and a residual.
+template <int VPL, int DEPTH>
+__global__ void __launch_bounds__(kThreads, 2) layernorm_pipe_kernel(const int32_t* __restrict__ q,
+                                                                     const int8_t* __restrict__ r, int64_t rows,
+                                                                     LnConsts k, const int32_t* __restrict__ b_i,
+                                                                     const int64_t* __restrict__ B_i,
+                                                                     int8_t* __restrict__ out, int32_t* status) {
+  extern __shared__ __align__(128) uint8_t ln_smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int C = k.C;
+  const uint32_t q_bytes = (uint32_t)C * 4u, r_bytes = (uint32_t)C;
+  const uint32_t slot_bytes = q_bytes + r_bytes;                 // multiple of 16
+  uint8_t* ring = ln_smem + (size_t)warp * DEPTH * slot_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ln_smem + (size_t)(kThreads / 32) * DEPTH * slot_bytes) + warp * DEPTH;
+  const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
+
+  auto issue = [&](int64_t row, int slot) {
+    const uint32_t bar = ptx::smem_addr(bars + slot);
+    const uint32_t dst = ptx::smem_addr(ring + (size_t)slot * slot_bytes);
+    ptx::mbar_arrive_expect_tx(bar, slot_bytes);
+    ptx::bulk_load_1d(dst, q + row * C, q_bytes, bar);
+    ptx::bulk_load_1d(dst + q_bytes, r + row * C, r_bytes, bar);
+  };
+  if (lane == 0) {
+    for (int s = 0; s < DEPTH; ++s) ptx::mbar_init(ptx::smem_addr(bars + s), 1);
+    ptx::fence_mbar_init();
+    for (int s = 0; s < DEPTH; ++s) {
+      const int64_t row = warp_global + (int64_t)s * warp_count;
+      if (row < rows) issue(row, s);
+    }
+  }
+  __syncwarp();
+
+  int slot = 0;
+  uint32_t phase = 0;
+  for (int64_t row = warp_global; row < rows; row += warp_count) {
+    const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(ptx::smem_addr(bars + slot), phase));
+    if (!ok) {
+      if (lane == 0) atomicCAS(status, 0, IBERT_ERR_TIMEOUT);
+      break;
+    }
+    const uint8_t* sq = ring + (size_t)slot * slot_bytes;
+    int32_t v[VPL][4];
+    uint32_t rw[VPL];
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int col = 4 * (j * 32 + lane);
+      if (col < C) {
+        const int4 t = *reinterpret_cast<const int4*>(sq + (size_t)col * 4);
+        v[j][0] = t.x; v[j][1] = t.y; v[j][2] = t.z; v[j][3] = t.w;
+        rw[j] = *reinterpret_cast<const uint32_t*>(sq + q_bytes + col);
+      } else {
+        v[j][0] = v[j][1] = v[j][2] = v[j][3] = 0;
+        rw[j] = 0;
+      }
+    }
+    __syncwarp();                                    // every lane has its copy: the slot can be refilled
+    if (lane == 0) {
+      const int64_t next = row + (int64_t)DEPTH * warp_count;
+      if (next < rows) issue(next, slot);
+    }
+    if (++slot == DEPTH) { slot = 0; phase ^= 1; }
+
+    int32_t sum = 0;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int32_t rv = (int32_t)(int8_t)(rw[j] >> (8 * i));
+        v[j][i] += requant_upper(rv << k.res_sh, k.b_r, int64_t(1) << 31);
+        sum += v[j][i];
+      }
+    sum = __reduce_add_sync(0xffffffffu, sum);
+    int32_t mu = sum / C;                            // mu = floor(sum / C)
+    if (sum - mu * C < 0) mu -= 1;
+    uint64_t ss = 0;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int col = 4 * (j * 32 + lane);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int32_t y = (col < C) ? v[j][i] - mu : 0;
+        v[j][i] = y;
+        ss += (uint64_t)((int64_t)y * (int64_t)y);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    uint32_t sigma = warp_isqrt_of_quotient(ss, (uint32_t)C, lane);   // I-Sqrt(floor(ss / C))
+    sigma = sigma < 1u ? 1u : sigma;
+    // floor(2^31 / sigma) as a positive int32 multiplier: for sigma = 1 use 2^30 and shift one less
+    const int32_t rho = sigma == 1u ? (1 << 30) : (int32_t)(0x80000000u / sigma);
+    const int nsh = sigma == 1u ? 14 : 15;
+    int8_t* orow = out + row * C;
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+      const int col = 4 * (j * 32 + lane);
+      if (col < C) {
+        const int4 bb = __ldg(reinterpret_cast<const int4*>(b_i + col));
+        const longlong2 B01 = __ldg(reinterpret_cast<const longlong2*>(B_i + col));
+        const longlong2 B23 = __ldg(reinterpret_cast<const longlong2*>(B_i + col + 2));
+        const int32_t bv[4] = {bb.x, bb.y, bb.z, bb.w};
+        const int64_t Bv[4] = {B01.x, B01.y, B23.x, B23.y};
+        int32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int32_t nrm = (int32_t)(((int64_t)v[j][i] * (int64_t)rho) >> nsh) << k.out_sh;
+          o[i] = max(requant_upper(nrm, bv[i], Bv[i]), -127);
+        }
+        __stcs(reinterpret_cast<uint32_t*>(orow + col), pack4_sat_s8(o[0], o[1], o[2], o[3]));
+      }
+    }
+  }
+}
+
 int grid_for(ibert_ctx* ctx, int64_t work_warps, int max_ctas_per_sm) {
   const int64_t ctas = (work_warps + (kThreads / 32) - 1) / (kThreads / 32);
   const int64_t cap = (int64_t)ctx->num_sms * max_ctas_per_sm;
@@ -310,6 +432,29 @@ int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t 
   const bool vec = (k.C % 4) == 0;
   const int vpl = (k.C + 127) / 128;
   const bool fast = vec && k.out_fast && (!k.has_res || k.res_fast);
+  if (fast && k.has_res && k.C % 16 == 0 && k.C <= 1024) {
+    // streaming variant: per-warp ring of row slots filled by bulk async copies
+    const int depth = k.C <= 768 ? 3 : 2;
+    const size_t smem = (size_t)(kThreads / 32) * depth * (size_t)k.C * 5 + (kThreads / 32) * depth * 8;
+    const int pgrid = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)ctx->num_sms * 2);
+#define IBERT_LNP(V, D)                                                                                     \
+  do {                                                                                                      \
+    static bool attr = false;                                                                               \
+    if (!attr) {                                                                                            \
+      if (cudaFuncSetAttribute(layernorm_pipe_kernel<V, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
+                               100 * 1024) != cudaSuccess) return IBERT_ERR_CUDA;                           \
+      attr = true;                                                                                          \
+    }                                                                                                       \
+    layernorm_pipe_kernel<V, D><<<pgrid, kThreads, smem, ctx->stream>>>(q, r, rows, k, d_b, d_B, out,       \
+                                                                         ctx->d_status);                    \
+  } while (0)
+    if (k.C <= 256) IBERT_LNP(2, 3);
+    else if (k.C <= 512) IBERT_LNP(4, 3);
+    else if (k.C <= 768) IBERT_LNP(6, 3);
+    else IBERT_LNP(8, 2);
+#undef IBERT_LNP
+    return check_launch();
+  }
 #define IBERT_LN(V)                                                                                              \
   do {                                                                                                           \
     if (fast) layernorm_kernel<V, true, true><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);  \

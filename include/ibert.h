@@ -153,8 +153,9 @@ enum {
   IBERT_NUM_KERNEL_CLASSES = 8
 };
 /* Host, pure.  Self-check of the constants derived from a score scale S for i-exp (Algorithm 3):
-   verifies on the host, for every distance d in [0, 31*q_ln2], that the multiply-high form the
-   kernels use for z = floor(d / q_ln2) equals the division.  Returns IBERT_OK, the error of the
+   verifies on the host, for every distance d in [0, 31*q_ln2] (and, for the unclamped form the
+   attention kernel uses, every d < 2^21), that the multiply-high form the kernels use for
+   z = floor(d / q_ln2) equals the division.  Returns IBERT_OK, the error of the
    derivation, or IBERT_ERR_VALUE_RANGE on a mismatch.  q_ln2_out (may be NULL) receives q_ln2. */
 int ibert_selftest_exp_division(double S, int32_t* q_ln2_out);
 

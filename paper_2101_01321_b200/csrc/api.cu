@@ -307,8 +307,12 @@ static int make_attn_consts(double S_q, double S_k, double S_v, double S_ctx, in
   if (p_max != 255 && p_max != 127) return IBERT_ERR_ARG;
   int rc = make_exp_consts((S_q * S_k) / 8.0, p_max, &k->e);     // 1/sqrt(64) folded into the score scale
   if (rc) return rc;
-  k->p_signed = p_max == 127;
-  return dyadic(((1.0 / (double)p_max) * S_v) / S_ctx, &k->b, &k->c);
+  rc = dyadic(((1.0 / (double)p_max) * S_v) / S_ctx, &k->b, &k->c);
+  if (rc) return rc;
+  std::vector<int32_t> b1(1, k->b), c1(1, k->c);
+  k->fast = to_upper_word_form(&b1, c1) ? 1 : 0;
+  k->b2 = k->fast ? b1[0] : 0;
+  return IBERT_OK;
 }
 
 int ibert_attention_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads, double S_q,
@@ -486,6 +490,12 @@ int ibert_selftest_exp_division(double S, int32_t* q_ln2_out) {
     const uint64_t wide = (uint64_t)(uint32_t)(d << k.div_pre) * (uint64_t)k.div_m;
     const uint32_t z = (uint32_t)(wide >> 32) >> k.div_post;
     if (z != d / k.q_ln2) return IBERT_ERR_VALUE_RANGE;
+  }
+  if (k.wide_post >= 0) {            // the unclamped form used on attention scores: every d < 2^21
+    for (uint32_t d = 0; d < (1u << 21); ++d) {
+      const uint32_t z = (uint32_t)(((uint64_t)d * (uint64_t)k.wide_m) >> 32) >> k.wide_post;
+      if (z != d / k.q_ln2) return IBERT_ERR_VALUE_RANGE;
+    }
   }
   return IBERT_OK;
 }

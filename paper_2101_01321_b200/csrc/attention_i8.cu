@@ -6,6 +6,8 @@
 // and the probabilities go to shared memory in the layout the second MMA reads.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "device_utils.cuh"
 #include "sm100_ptx.cuh"
 
@@ -21,6 +23,7 @@ struct AttnArgs {
   int Lp;            // L rounded up to a multiple of 32 (MMA N / K granularity)
   int n_slabs;       // ceil(L / 128)
   uint32_t tmem_cols;
+  int stages;        // operand stages in shared memory: 2 (next item prefetched) or 1
   AttnConsts k;
   int8_t* out;
   int32_t* status;
@@ -37,6 +40,13 @@ __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t col, uin
 // pass 1 row maximum, pass 2 i-exp + int32 row sum (exponentials written back over the scores),
 // pass 3 fixed-point quotient -> u8 probabilities into the swizzled operand tile `sP`, row `row`.
 // Columns [L, Lp) are padding: excluded from max and sum, written as probability 0.
+// DIV: 0..2 = clamped division forms of iexp_dist, 3 = the 21-bit form without the clamp.
+template <int DIV>
+__device__ __forceinline__ uint32_t iexp_any(uint32_t d, const ExpConsts& ek) {
+  if constexpr (DIV == 3) return iexp_dist_wide(d, ek);
+  else return iexp_dist<DIV>(d, ek);
+}
+
 template <int DIV>
 __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const ExpConsts& ek, uint8_t* sP,
                                             uint32_t row) {
@@ -48,7 +58,7 @@ __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const
     ptx::tmem_wait_ld();
     if (c0 < full) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) mx = max(mx, (int32_t)v[i]);
+      for (int i = 0; i < 32; i += 2) mx = __vimax3_s32(mx, (int32_t)v[i], (int32_t)v[i + 1]);
     } else {
 #pragma unroll
       for (int i = 0; i < 32; ++i)
@@ -63,13 +73,13 @@ __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const
     if (c0 < full) {
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        v[i] = iexp_dist<DIV>((uint32_t)mx - v[i], ek);
+        v[i] = iexp_any<DIV>((uint32_t)mx - v[i], ek);
         sum += v[i];
       }
     } else {
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        v[i] = (c0 + i < L) ? iexp_dist<DIV>((uint32_t)mx - v[i], ek) : 0u;
+        v[i] = (c0 + i < L) ? iexp_any<DIV>((uint32_t)mx - v[i], ek) : 0u;
         sum += v[i];
       }
     }
@@ -77,6 +87,7 @@ __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const
   }
   ptx::tmem_wait_st();
   const RowDivisor rd = make_row_divisor(sum, ek.p_max);
+  const bool nopre = __all_sync(0xffffffffu, rd.pre == 0);      // usual case: every row sum >= 2^10
   for (int c0 = 0; c0 < Lp; c0 += 32) {
     uint32_t v[32];
     ptx::tmem_ld32(t_row + c0, v);
@@ -87,8 +98,15 @@ __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int j = h * 16 + i * 4;
-        w[i] = softmax_quotient(v[j], rd) | (softmax_quotient(v[j + 1], rd) << 8) |
-               (softmax_quotient(v[j + 2], rd) << 16) | (softmax_quotient(v[j + 3], rd) << 24);
+        uint32_t p0, p1, p2, p3;
+        if (nopre) {
+          p0 = softmax_quotient_nopre(v[j], rd); p1 = softmax_quotient_nopre(v[j + 1], rd);
+          p2 = softmax_quotient_nopre(v[j + 2], rd); p3 = softmax_quotient_nopre(v[j + 3], rd);
+        } else {
+          p0 = softmax_quotient(v[j], rd); p1 = softmax_quotient(v[j + 1], rd);
+          p2 = softmax_quotient(v[j + 2], rd); p3 = softmax_quotient(v[j + 3], rd);
+        }
+        w[i] = ((p3 * 256u + p2) * 256u + p1) * 256u + p0;      // multiply-adds: off the shift/logic pipe
       }
       *reinterpret_cast<uint4*>(sP + sw128_offset(row, (uint32_t)(c0 + h * 16), 128)) =
           make_uint4(w[0], w[1], w[2], w[3]);
@@ -96,28 +114,117 @@ __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const
   }
 }
 
-__global__ void __launch_bounds__(kAttnThreads)
+// The same row function for rows of exactly 128 columns' worth of padding (96 < L <= 128), the
+// headline case: the whole score row is read from TMEM once and stays in registers through
+// maximum, i-exp, sum and quotient, so there is no write-back of exponentials and the 128
+// independent element chains can be scheduled freely.
+__device__ __forceinline__ void softmax_row_128(uint32_t t_row, int L, const ExpConsts& ek, uint8_t* sP,
+                                                uint32_t row) {
+  uint32_t v[4][32];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) ptx::tmem_ld32(t_row + c * 32, v[c]);
+  ptx::tmem_wait_ld();
+  int32_t mx = INT32_MIN;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+      if (c < 3) mx = __vimax3_s32(mx, (int32_t)v[c][i], (int32_t)v[c][i + 1]);
+      else {
+        if (96 + i < L) mx = max(mx, (int32_t)v[c][i]);
+        if (96 + i + 1 < L) mx = max(mx, (int32_t)v[c][i + 1]);
+      }
+    }
+  }
+  uint32_t sum = 0;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const uint32_t e = iexp_dist_wide((uint32_t)mx - v[c][i], ek);
+      v[c][i] = (c < 3 || 96 + i < L) ? e : 0u;
+      sum += v[c][i];
+    }
+  }
+  const RowDivisor rd = make_row_divisor(sum, ek.p_max);
+  const bool nopre = __all_sync(0xffffffffu, rd.pre == 0);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int j = h * 16 + i * 4;
+        uint32_t p0, p1, p2, p3;
+        if (nopre) {
+          p0 = softmax_quotient_nopre(v[c][j], rd); p1 = softmax_quotient_nopre(v[c][j + 1], rd);
+          p2 = softmax_quotient_nopre(v[c][j + 2], rd); p3 = softmax_quotient_nopre(v[c][j + 3], rd);
+        } else {
+          p0 = softmax_quotient(v[c][j], rd); p1 = softmax_quotient(v[c][j + 1], rd);
+          p2 = softmax_quotient(v[c][j + 2], rd); p3 = softmax_quotient(v[c][j + 3], rd);
+        }
+        w[i] = ((p3 * 256u + p2) * 256u + p1) * 256u + p0;
+      }
+      *reinterpret_cast<uint4*>(sP + sw128_offset(row, (uint32_t)(c * 32 + h * 16), 128)) =
+          make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+}
+
+// Transposes V [j][64] (plain rows in `sVs`) into Vt [64][j] in the swizzled K-major operand
+// layout of `sVt`.  A thread takes 4 consecutive keys x 16 head dims, transposes the four 4x4 byte
+// blocks with byte permutes and writes 16 words (4 keys of one head dim each).
+__device__ __forceinline__ void transpose_v(const uint8_t* sVs, uint8_t* sVt, int n_keys, int tid) {
+  for (int item = tid; item < (n_keys / 4) * 4; item += kAttnThreads) {
+    const int jq = item % (n_keys / 4), dc = item / (n_keys / 4);     // key quad, 16-dim chunk
+    uint32_t r[4][4];
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      const uint4 t = *reinterpret_cast<const uint4*>(sVs + (jq * 4 + jj) * kHeadDim + dc * 16);
+      r[jj][0] = t.x; r[jj][1] = t.y; r[jj][2] = t.z; r[jj][3] = t.w;
+    }
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      // rows r[0..3][w] hold dims d0..d0+3 of keys j..j+3; output word i = dim d0+i of the 4 keys
+      const uint32_t a01 = __byte_perm(r[0][w], r[1][w], 0x5140);   // k0d0 k1d0 k0d1 k1d1
+      const uint32_t b01 = __byte_perm(r[0][w], r[1][w], 0x7362);   // k0d2 k1d2 k0d3 k1d3
+      const uint32_t a23 = __byte_perm(r[2][w], r[3][w], 0x5140);
+      const uint32_t b23 = __byte_perm(r[2][w], r[3][w], 0x7362);
+      const uint32_t o[4] = {__byte_perm(a01, a23, 0x5410), __byte_perm(a01, a23, 0x7632),
+                             __byte_perm(b01, b23, 0x5410), __byte_perm(b01, b23, 0x7632)};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        *reinterpret_cast<uint32_t*>(sVt + sw128_offset((uint32_t)(dc * 16 + w * 4 + i), (uint32_t)(jq * 4), 64)) = o[i];
+    }
+  }
+}
+
+// Persistent CTA: walks (batch, head, query tile) work items; while one item is computed the TMA
+// loads of the next one land in the other operand stage (when `a.stages` == 2).
+__global__ void __launch_bounds__(kAttnThreads, 3)
 attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_constant__ CUtensorMap map_v,
                  const AttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int slab_bytes = 128 * kHeadDim;                       // 8 KB
-  uint8_t* sQ = smem;
-  uint8_t* sK = sQ + slab_bytes;
-  uint8_t* sVt = sK + a.n_slabs * slab_bytes;                   // [n_slabs][64 rows][128 B], swizzled
+  const int stage_bytes = (1 + 2 * a.n_slabs) * slab_bytes;     // Q | K slabs | V slabs (plain rows)
+  uint8_t* sStage = smem;
+  uint8_t* sVt = smem + a.stages * stage_bytes;                 // [n_slabs][64 rows][128 B], swizzled
   uint8_t* sP = sVt + a.n_slabs * slab_bytes;                   // [n_slabs][128 rows][128 B], swizzled
-  uint8_t* sVs = sP;                                            // V staging [L][64], aliases P (used before it)
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(sP + a.n_slabs * 128 * 128);
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 2);
-  const uint32_t bar_load = ptx::smem_addr(s_bar);
-  const uint32_t bar_mma = bar_load + 8;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 3);
+  const uint32_t bar_load0 = ptx::smem_addr(s_bar);             // one per stage
+  const uint32_t bar_mma = bar_load0 + 16;
 
   const int tid = threadIdx.x, warp = tid >> 5;
-  const int q0 = blockIdx.x * 128, head = blockIdx.y, batch = blockIdx.z;
   const int L = a.L, Lp = a.Lp;
+  const int q_tiles = a.n_slabs;
+  const int total = a.B * a.heads * q_tiles;
 
   if (tid == 0) {
-    ptx::mbar_init(bar_load, 1);
+    ptx::mbar_init(bar_load0, 1);
+    ptx::mbar_init(bar_load0 + 8, 1);
     ptx::mbar_init(bar_mma, 1);
     ptx::fence_mbar_init();
     ptx::tma_prefetch_desc(&map_qk);
@@ -131,104 +238,131 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *s_tmem;
-
-  // ---- loads: Q tile, all K rows (64-byte swizzle, MMA operand layout), all V rows (plain)
-  if (tid == 0) {
-    ptx::mbar_arrive_expect_tx(bar_load, (uint32_t)((1 + 2 * a.n_slabs) * slab_bytes));
-    ptx::tma_load_3d(ptx::smem_addr(sQ), &map_qk, bar_load, head * kHeadDim, q0, batch);
-    for (int s = 0; s < a.n_slabs; ++s) {
-      ptx::tma_load_3d(ptx::smem_addr(sK + s * slab_bytes), &map_qk, bar_load, a.H + head * kHeadDim, s * 128, batch);
-      ptx::tma_load_3d(ptx::smem_addr(sVs + s * slab_bytes), &map_v, bar_load, 2 * a.H + head * kHeadDim, s * 128, batch);
-    }
-  }
-  bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_load, 0));
-
-  // ---- S = Q K^T: K = 64 bytes = two MMA K-steps; N in chunks of at most 256 columns
-  if (ok && tid == 0) {
-    ptx::tc_fence_after_sync();
-    const uint64_t dq = ptx::make_kmajor_desc(ptx::smem_addr(sQ), 512, ptx::kSwizzle64);
-    for (int n0 = 0; n0 < Lp; n0 += 256) {
-      const int nn = min(256, Lp - n0);
-      const uint32_t idesc = ptx::make_idesc_i8(128, nn, true, true);
-      const uint64_t dk = ptx::make_kmajor_desc(ptx::smem_addr(sK + n0 * kHeadDim), 512, ptx::kSwizzle64);
-      ptx::mma_i8_ss(tmem_base + n0, dq, dk, idesc, 0u);
-      ptx::mma_i8_ss(tmem_base + n0, dq + 2, dk + 2, idesc, 1u);
-    }
-    ptx::mma_commit(bar_mma);
-  }
-
-  // ---- meanwhile: transpose V [j][d] -> Vt [d][j] into the swizzled K-major operand layout
-  if (ok) {
-    for (int j = tid; j < a.n_slabs * 128; j += kAttnThreads) {
-      const uint4* src = reinterpret_cast<const uint4*>(sVs + j * kHeadDim);
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const uint4 v = src[c];
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const uint32_t d = c * 16 + i;
-          sVt[sw128_offset(d, (uint32_t)j, 64)] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
-        }
-      }
-    }
-  }
-  __syncthreads();                                            // staging is dead: P may overwrite it
-  if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_mma, 0));
-
-  // ---- i-softmax on the row this thread owns
   const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);
-  if (ok) {
-    ptx::tc_fence_after_sync();
-    switch (exp_div_mode(a.k.e)) {
-      case 0: softmax_row<0>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
-      case 1: softmax_row<1>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
-      default: softmax_row<2>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
-    }
-    ptx::fence_proxy_async_smem();          // P and Vt were written by ordinary stores; the MMA reads them
-  }
-  ptx::tc_fence_before_sync();
-  __syncthreads();
 
-  // ---- ctx = P V: K = Lp in steps of 32, accumulator in columns 0..63 (scores are dead)
-  if (ok && tid == 0) {
-    ptx::tc_fence_after_sync();
-    const uint32_t idesc = ptx::make_idesc_i8(128, kHeadDim, false, true);   // u8 x s8
-    for (int kk = 0; kk < Lp / 32; ++kk) {
-      const int kb = kk >> 2, ks = kk & 3;
-      const uint64_t dp = ptx::make_kmajor_desc(ptx::smem_addr(sP + kb * 128 * 128), 1024, ptx::kSwizzle128);
-      const uint64_t dv = ptx::make_kmajor_desc(ptx::smem_addr(sVt + kb * 64 * 128), 1024, ptx::kSwizzle128);
-      ptx::mma_i8_ss(tmem_base, dp + 2 * ks, dv + 2 * ks, idesc, kk != 0 ? 1u : 0u);
+  // loads of one work item: Q tile, all K rows (64-byte swizzle, MMA operand layout), all V rows
+  auto issue_loads = [&](int item, int stage) {
+    const int qt = item % q_tiles, head = (item / q_tiles) % a.heads, batch = item / (q_tiles * a.heads);
+    const uint32_t bar = bar_load0 + 8 * stage;
+    uint8_t* base = sStage + stage * stage_bytes;
+    ptx::mbar_arrive_expect_tx(bar, (uint32_t)stage_bytes);
+    ptx::tma_load_3d(ptx::smem_addr(base), &map_qk, bar, head * kHeadDim, qt * 128, batch);
+    for (int s = 0; s < a.n_slabs; ++s) {
+      ptx::tma_load_3d(ptx::smem_addr(base + (1 + s) * slab_bytes), &map_qk, bar, a.H + head * kHeadDim, s * 128, batch);
+      ptx::tma_load_3d(ptx::smem_addr(base + (1 + a.n_slabs + s) * slab_bytes), &map_v, bar,
+                       2 * a.H + head * kHeadDim, s * 128, batch);
     }
-    ptx::mma_commit(bar_mma);
-  }
-  if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_mma, 1));
+  };
 
-  // ---- epilogue: requantize the 64 context values of this row to int8
-  if (ok) {
-    ptx::tc_fence_after_sync();
-    const int64_t half = rounding_half(a.k.c);
-    const int q_row = q0 + tid;
-    int8_t* orow = a.out + ((int64_t)batch * L + q_row) * a.H + head * kHeadDim;
+  int stage = 0;
+  uint32_t load_phase[2] = {0, 0};
+  uint32_t mma_phase = 0;
+  bool ok = true;
+  if (tid == 0 && (int)blockIdx.x < total) issue_loads(blockIdx.x, 0);
+
+  for (int item = blockIdx.x; item < total; item += gridDim.x) {
+    const int qt = item % q_tiles, head = (item / q_tiles) % a.heads, batch = item / (q_tiles * a.heads);
+    const int q0 = qt * 128;
+    uint8_t* sQ = sStage + stage * stage_bytes;
+    uint8_t* sK = sQ + slab_bytes;
+    uint8_t* sVs = sK + a.n_slabs * slab_bytes;
+    const int next = item + gridDim.x;
+    if (tid == 0 && next < total) {
+      // two stages: the other one was released by the barrier that ended the previous item;
+      // one stage: nothing to overlap, the loads of `next` are issued at the end of this item
+      if (a.stages == 2) issue_loads(next, stage ^ 1);
+    }
+    ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_load0 + 8 * stage, load_phase[stage]));
+    load_phase[stage] ^= 1;
+
+    // ---- S = Q K^T: K = 64 bytes = two MMA K-steps; N in chunks of at most 256 columns
+    if (ok && tid == 0) {
+      ptx::tc_fence_after_sync();
+      const uint64_t dq = ptx::make_kmajor_desc(ptx::smem_addr(sQ), 512, ptx::kSwizzle64);
+      for (int n0 = 0; n0 < Lp; n0 += 256) {
+        const int nn = min(256, Lp - n0);
+        const uint32_t idesc = ptx::make_idesc_i8(128, nn, true, true);
+        const uint64_t dk = ptx::make_kmajor_desc(ptx::smem_addr(sK + n0 * kHeadDim), 512, ptx::kSwizzle64);
+        ptx::mma_i8_ss(tmem_base + n0, dq, dk, idesc, 0u);
+        ptx::mma_i8_ss(tmem_base + n0, dq + 2, dk + 2, idesc, 1u);
+      }
+      ptx::mma_commit(bar_mma);
+    }
+    // ---- meanwhile: V [j][d] -> Vt [d][j] in the swizzled K-major operand layout
+    if (ok) transpose_v(sVs, sVt, a.n_slabs * 128, tid);
+    if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_mma, mma_phase));
+    mma_phase ^= 1;
+
+    // ---- i-softmax on the row this thread owns
+    if (ok) {
+      ptx::tc_fence_after_sync();
+      // scores are sums of 64 int8 products: |s| < 2^20, so distances from the maximum stay below 2^21
+      if (a.k.e.wide_post >= 0 && Lp == 128) softmax_row_128(t_row, L, a.k.e, sP, (uint32_t)tid);
+      else if (a.k.e.wide_post >= 0) softmax_row<3>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid);
+      else switch (exp_div_mode(a.k.e)) {
+        case 0: softmax_row<0>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
+        case 1: softmax_row<1>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
+        default: softmax_row<2>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
+      }
+      ptx::fence_proxy_async_smem();        // P and Vt were written by ordinary stores; the MMA reads them
+    }
+    ptx::tc_fence_before_sync();
+    ok = __syncthreads_and(ok);             // P, Vt complete; every row's scores have been consumed
+    if (!ok) break;
+
+    // ---- ctx = P V: K = Lp in steps of 32, accumulator in columns 0..63 (scores are dead)
+    if (tid == 0) {
+      ptx::tc_fence_after_sync();
+      const uint32_t idesc = ptx::make_idesc_i8(128, kHeadDim, false, true);   // u8 x s8
+      for (int kk = 0; kk < Lp / 32; ++kk) {
+        const int kb = kk >> 2, ks = kk & 3;
+        const uint64_t dp = ptx::make_kmajor_desc(ptx::smem_addr(sP + kb * 128 * 128), 1024, ptx::kSwizzle128);
+        const uint64_t dv = ptx::make_kmajor_desc(ptx::smem_addr(sVt + kb * 64 * 128), 1024, ptx::kSwizzle128);
+        ptx::mma_i8_ss(tmem_base, dp + 2 * ks, dv + 2 * ks, idesc, kk != 0 ? 1u : 0u);
+      }
+      ptx::mma_commit(bar_mma);
+    }
+    ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_mma, mma_phase));
+    mma_phase ^= 1;
+
+    // ---- epilogue: requantize the 64 context values of this row to int8
+    if (ok) {
+      ptx::tc_fence_after_sync();
+      const int64_t half = rounding_half(a.k.c);
+      const int q_row = q0 + tid;
+      int8_t* orow = a.out + ((int64_t)batch * L + q_row) * a.H + head * kHeadDim;
 #pragma unroll
-    for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
-      uint32_t v[32];
-      ptx::tmem_ld32(t_row + c0, v);
-      ptx::tmem_wait_ld();
+      for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
+        uint32_t v[32];
+        ptx::tmem_ld32(t_row + c0, v);
+        ptx::tmem_wait_ld();
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        uint32_t w[4];
+        for (int h = 0; h < 2; ++h) {
+          uint32_t w[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint32_t pk = 0;
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            pk |= (uint32_t)(requant_add((int32_t)v[h * 16 + i * 4 + e], a.k.b, half, a.k.c, 127) & 0xff) << (8 * e);
-          w[i] = pk;
+          for (int i = 0; i < 4; ++i) {
+            const int j = h * 16 + i * 4;
+            if (a.k.fast) {
+              w[i] = pack4_sat_s8(max(requant_upper((int32_t)v[j], a.k.b2, int64_t(1) << 31), -127),
+                                  max(requant_upper((int32_t)v[j + 1], a.k.b2, int64_t(1) << 31), -127),
+                                  max(requant_upper((int32_t)v[j + 2], a.k.b2, int64_t(1) << 31), -127),
+                                  max(requant_upper((int32_t)v[j + 3], a.k.b2, int64_t(1) << 31), -127));
+            } else {
+              w[i] = pack4_sat_s8(requant_add((int32_t)v[j], a.k.b, half, a.k.c, 127),
+                                  requant_add((int32_t)v[j + 1], a.k.b, half, a.k.c, 127),
+                                  requant_add((int32_t)v[j + 2], a.k.b, half, a.k.c, 127),
+                                  requant_add((int32_t)v[j + 3], a.k.b, half, a.k.c, 127));
+            }
+          }
+          if (q_row < L) *reinterpret_cast<uint4*>(orow + c0 + h * 16) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        if (q_row < L) *reinterpret_cast<uint4*>(orow + c0 + h * 16) = make_uint4(w[0], w[1], w[2], w[3]);
       }
     }
+    ptx::tc_fence_before_sync();
+    ok = __syncthreads_and(ok);             // TMEM columns, Vt, P and this operand stage are free again
+    if (!ok) break;
+    if (a.stages == 2) stage ^= 1;
+    else if (tid == 0 && next < total) issue_loads(next, 0);
   }
   if (!ok) atomicCAS(a.status, 0, IBERT_ERR_TIMEOUT);
   ptx::tc_fence_before_sync();
@@ -262,14 +396,21 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
   if (rc) return rc;
   rc = encode_tensor_map(&mv, qkv, 3, dims, str, box, 0);
   if (rc) return rc;
-  const int smem = (1 + 2 * a.n_slabs) * 128 * kHeadDim + a.n_slabs * 128 * 128 + 64 + 1024;
+  const int stage_bytes = (1 + 2 * a.n_slabs) * 128 * kHeadDim;
+  const int fixed_bytes = a.n_slabs * 128 * kHeadDim + a.n_slabs * 128 * 128 + 64 + 1024;
+  a.stages = (2 * stage_bytes + fixed_bytes <= 112 * 1024) ? 2 : 1;     // keep at least 2 CTAs per SM
+  const int smem = a.stages * stage_bytes + fixed_bytes;
   static int smem_set = 0;
   if (smem > smem_set) {
     if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return IBERT_ERR_CUDA;
     smem_set = smem;
   }
-  dim3 grid((L + 127) / 128, heads, B);
+  const int total = B * heads * a.n_slabs;
+  // resident CTAs per SM: limited by TMEM columns (512), shared memory and the register budget (3)
+  int per_sm = std::min(3, std::min((int)(512 / cols), (227 * 1024) / (smem + 1024)));
+  if (per_sm < 1) per_sm = 1;
+  const int grid = std::min(total, ctx->num_sms * per_sm);
   attention_kernel<<<grid, kAttnThreads, smem, ctx->stream>>>(mqk, mv, a);
   return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
 }

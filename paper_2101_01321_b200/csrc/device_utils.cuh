@@ -82,6 +82,15 @@ __device__ __forceinline__ uint32_t iexp_dist(uint32_t d, const ExpConsts& k) {
   const uint32_t poly = (uint32_t)(t * t + k.q_c);
   return shr_clamped(poly, z + (uint32_t)k.s_out);
 }
+// i-exp for distances below 2^21 (attention scores): no clamp of the distance -- a quotient above
+// 31 just shifts the polynomial out completely, exactly like the clamped form.
+__device__ __forceinline__ uint32_t iexp_dist_wide(uint32_t d, const ExpConsts& k) {
+  const uint32_t dp = d >> k.s_in;
+  const uint32_t z = __umulhi(dp, k.wide_m) >> k.wide_post;
+  const int32_t t = (int32_t)(z * k.q_ln2) + (k.q_b - (int32_t)dp);      // q_b - r
+  const uint32_t poly = (uint32_t)(t * t + k.q_c);
+  return shr_clamped(poly, z + (uint32_t)k.s_out);
+}
 __host__ __device__ __forceinline__ int exp_div_mode(const ExpConsts& k) {
   return k.div_pre != 0 ? 2 : (k.div_post != 0 ? 1 : 0);
 }
@@ -108,6 +117,10 @@ __device__ __forceinline__ RowDivisor make_row_divisor(uint32_t sum, uint32_t p_
 
 __device__ __forceinline__ uint32_t softmax_quotient(uint32_t e, const RowDivisor& r) {
   return __umulhi(e << r.pre, r.m) >> r.post;
+}
+// the common case pre == 0 (row sum >= 2^10)
+__device__ __forceinline__ uint32_t softmax_quotient_nopre(uint32_t e, const RowDivisor& r) {
+  return __umulhi(e, r.m) >> r.post;
 }
 
 }  // namespace ibert

@@ -95,6 +95,13 @@ int make_exp_consts(double S, int p_max, ExpConsts* k) {
     k->div_m = (uint32_t)mm;
     k->div_pre = pre;
     k->div_post = post;
+    // 21-bit operands: N + l >= 32 needs l >= 11, else the multiplier takes the slack
+    const int N2 = 21;
+    uint64_t m2 = (uint64_t(1) << (N2 + l)) / k->q_ln2 + 1;          // < 2^22
+    int post2 = N2 + l - 32;
+    while (post2 < 0) { m2 <<= 1; ++post2; }                          // m2 < 2^(22 + 11) only if q_ln2 tiny
+    if (m2 >= (uint64_t(1) << 32)) { k->wide_m = 0; k->wide_post = -1; }  // not available (q_ln2 <= 2)
+    else { k->wide_m = (uint32_t)m2; k->wide_post = post2; }
   }
   k->q_b = (int32_t)q_b;
   k->q_c = (int32_t)q_c;

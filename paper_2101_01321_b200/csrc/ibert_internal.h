@@ -28,6 +28,10 @@ struct ExpConsts {
   int32_t q_c;       // floor(0.344 / (0.3585 S'^2))
   int32_t s_out;     // static post-shift: every e < 2^21
   uint32_t p_max;    // 255 or 127: the fixed-point one of the probabilities
+  // the same division for distances known to stay below 2^21 (scores of 64 int8 products):
+  // floor(d / q_ln2) = umulhi(d, wide_m) >> wide_post for every d < 2^21, no clamp to d_max needed
+  uint32_t wide_m;
+  int32_t wide_post;
 };
 
 // i-GELU (Algorithm 2) followed by requantization to int8
@@ -131,7 +135,7 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
 struct AttnConsts {
   ExpConsts e;
   int32_t b, c;            // dyadic((1/p_max) * S_v / S_ctx)
-  int32_t p_signed;        // 0: probabilities are u8 (p_max 255); 1: fit int8 (p_max 127)
+  int32_t b2, fast;        // upper-word form: (v * b2 + 2^31) >> 32 with b2 = b << (32 - c)
 };
 
 int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,

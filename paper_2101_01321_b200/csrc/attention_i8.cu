@@ -343,10 +343,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
           for (int i = 0; i < 4; ++i) {
             const int j = h * 16 + i * 4;
             if (a.k.fast) {
-              w[i] = pack4_sat_s8(max(requant_upper((int32_t)v[j], a.k.b2, int64_t(1) << 31), -127),
-                                  max(requant_upper((int32_t)v[j + 1], a.k.b2, int64_t(1) << 31), -127),
-                                  max(requant_upper((int32_t)v[j + 2], a.k.b2, int64_t(1) << 31), -127),
-                                  max(requant_upper((int32_t)v[j + 3], a.k.b2, int64_t(1) << 31), -127));
+              w[i] = pack4_sat_s8(max(requant_upper((int32_t)v[j], a.k.b2), -127),
+                                  max(requant_upper((int32_t)v[j + 1], a.k.b2), -127),
+                                  max(requant_upper((int32_t)v[j + 2], a.k.b2), -127),
+                                  max(requant_upper((int32_t)v[j + 3], a.k.b2), -127));
             } else {
               w[i] = pack4_sat_s8(requant_add((int32_t)v[j], a.k.b, half, a.k.c, 127),
                                   requant_add((int32_t)v[j + 1], a.k.b, half, a.k.c, 127),

@@ -20,10 +20,28 @@ __device__ __forceinline__ int32_t requant_add(int32_t v, int32_t b, int64_t add
   return (int32_t)p;
 }
 
-// The same requantization when the host could pre-shift the multiplier: the result is the
-// upper word of one 64-bit multiply-add, (v * b2 + add2) >> 32, not yet clamped.
-__device__ __forceinline__ int32_t requant_upper(int32_t v, int32_t b2, int64_t add2) {
-  return (int32_t)(((int64_t)v * (int64_t)b2 + add2) >> 32);
+// The same requantization when the host could pre-shift the multiplier (b2 = b << (32 - c)):
+// (v * b2 + 2^31) >> 32, not yet clamped.  Written as a 32x32->64 multiply whose upper word is
+// corrected by bit 31 of the lower word: a multiply-add with a 64-bit addend issues at less than
+// half the rate of this form on the integer pipes.
+__device__ __forceinline__ int32_t requant_upper(int32_t v, int32_t b2) {
+  const int64_t t = (int64_t)v * (int64_t)b2;
+  return (int32_t)(t >> 32) + (int32_t)((uint32_t)t >> 31);
+}
+
+// (v * b2 + add) >> 32 for a general 64-bit addend, the carry of the lower words propagated by hand
+__device__ __forceinline__ int32_t requant_upper_add(int32_t v, int32_t b2, int64_t add) {
+  const int64_t t = (int64_t)v * (int64_t)b2;
+  uint32_t lo;
+  int32_t hi;
+  asm("{\n\t.reg .u32 s;\n\t"
+      "add.cc.u32 s, %2, %4;\n\t"
+      "addc.s32 %1, %3, %5;\n\t"
+      "mov.u32 %0, s;\n\t}"
+      : "=r"(lo), "=r"(hi)
+      : "r"((uint32_t)t), "r"((int32_t)(t >> 32)), "r"((uint32_t)add), "r"((int32_t)(add >> 32)));
+  (void)lo;
+  return hi;
 }
 
 // four int32 -> four int8 lanes of one word, each saturated to [-128, 127]
@@ -58,7 +76,7 @@ __device__ __forceinline__ int32_t igelu_q16_upper(int32_t q, const GeluConsts& 
   const int32_t sgn = (q >> 31) | 1;
   const int32_t f = poly * sgn + k.q_c;
   const int32_t g2 = (q * (f >> k.s_f) + 128) >> 8;
-  return max(requant_upper(g2, k.b2, k.add2), -127);
+  return max(requant_upper(g2, k.b2), -127);
 }
 
 __device__ __forceinline__ uint32_t shr_clamped(uint32_t v, uint32_t n) {

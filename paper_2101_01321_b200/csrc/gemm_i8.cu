@@ -3,13 +3,25 @@
 // bias add + dyadic requantization to int8 or Q16, raw accumulators, or requantization
 // to Q16 followed by i-GELU (Algorithm 2) and a second requantization to int8.
 //
-// out[m, n] = epilogue( sum_k x[m, k] * w[n, k] + bias[n] )      x: [M, K], w: [N, K]
+// out[t, n] = epilogue( sum_k x[t, k] * w[n, k] + bias[n] )      x: [T, K], w: [N, K]
 //
-// One persistent CTA per SM walks 128 x BN output tiles.  Warp 0 is the TMA producer,
-// warp 1 issues the MMAs, warps 2.. run the epilogue; two TMEM accumulator stages let
-// the (integer-ALU heavy) epilogue of tile i overlap the MMAs of tile i+1.
+// The MMA computes the transposed tile D[n, t] = W X^T: output channels n sit on the 128
+// TMEM lanes, tokens t on the columns.  An epilogue thread therefore owns ONE channel and keeps
+// that channel's requantization constants in registers -- per-column constants would have to be
+// re-read from shared memory for every element, and that broadcast traffic, not the tensor
+// pipe, bounded the first version of this kernel.  Results are transposed back for free on the
+// way out: each warp writes its 32-token x 32-channel block into a small staging tile and a TMA
+// store moves it to out[t, n].
+//
+// Persistent CTAs walk the output tiles.  Warp 0 is the TMA producer, warp 1 issues the MMAs,
+// warps 2.. run the epilogue; two TMEM accumulator stages let the (integer-ALU heavy) epilogue of
+// tile i overlap the MMAs of tile i+1.  With PAIR a cluster of two CTAs shares one
+// 256-channel x 256-token tile (tcgen05.mma.cta_group::2): each CTA loads only its own 128
+// weight rows and 128 of the 256 token rows, which cuts the operand bytes an SM must pull per
+// MMA by a third.  No TMA multicast is used anywhere.
 #include <cuda.h>
 
+#include <algorithm>
 #include <mutex>
 
 #include "device_utils.cuh"
@@ -71,34 +83,35 @@ int encode_tensor_map(CUtensorMap* map, const void* base, int rank, const uint64
 // --------------------------------------------------------------------------------------
 namespace {
 
-constexpr int BM = 128;           // rows per tile = TMEM lanes
+constexpr int BC = 128;           // output channels per CTA = TMEM lanes
 constexpr int BK = 128;           // K bytes per pipeline stage = one 128-byte swizzle span
 constexpr int UMMA_K = 32;        // K per tcgen05.mma kind::i8
-// Epilogue warps: every warp handles two 32-column chunks of the 32 rows (TMEM lanes) its
-// position in the warp quartet gives it access to, so a tile of BN columns takes BN / 16 warps.
-// The integer epilogue is what bounds these GEMMs at K <= 1024, hence the many warps.
-__host__ __device__ constexpr int epi_warps(int bn) { return bn / 16; }
-__host__ __device__ constexpr int gemm_threads(int bn) { return 64 + 32 * epi_warps(bn); }   // + producer warp, MMA warp
 
-template <int BN>
-struct GemmSmem {
-  static constexpr int kStages = BN >= 256 ? 3 : 5;
-  static constexpr int kABytes = BM * BK;
-  static constexpr int kBBytes = BN * BK;
-  static constexpr int kStageBytes = kABytes + kBBytes;
-  // operand stages | output staging (one 4 KB tile per epilogue warp) | per-column epilogue
-  // parameters (int4 per column) | barriers
+template <int TOK, bool PAIR, int KIND>
+struct Cfg {
+  static constexpr bool kOut32 = (KIND == EPI_RAW || KIND == EPI_Q16);
+  static constexpr int kChunks = TOK / 32;                       // 32-token chunks of a tile
+  // the int8 epilogues are ALU-bound: one warp per 64 tokens; the int32 ones per 128 tokens
+  static constexpr int kEpiWarps = kOut32 ? TOK / 32 : TOK / 16;
+  static constexpr int kParts = kEpiWarps / 4;                   // token ranges (4 warps cover the 128 lanes)
+  static constexpr int kChunksPerWarp = kChunks / kParts;
+  static constexpr int kThreads = 64 + 32 * kEpiWarps;           // + producer warp, MMA warp
+  static constexpr int kXRows = PAIR ? TOK / 2 : TOK;            // token rows this CTA loads per K block
+  static constexpr int kWBytes = BC * BK;
+  static constexpr int kStageBytes = kWBytes + kXRows * BK;
+  static constexpr int kOutTileBytes = kOut32 ? 32 * 128 : 32 * 32;   // 32 tokens x 32 channels
+  static constexpr int kOutBytes = kEpiWarps * 2 * kOutTileBytes;     // double-buffered per warp
+  static constexpr int kBudget = 227 * 1024 - 1024 - 512 - kOutBytes;
+  static constexpr int kStages = kBudget / kStageBytes > 8 ? 8 : kBudget / kStageBytes;
   static constexpr int kOutOff = kStages * kStageBytes;
-  static constexpr int kOutTileBytes = 32 * 128;
-  static constexpr int kParamOff = kOutOff + epi_warps(BN) * kOutTileBytes;
-  static constexpr int kBarOff = kParamOff + BN * 16;
-  static constexpr int kBytes = kBarOff + 256;
-  static constexpr int kAlloc = kBytes + 1024;   // slack to align the operand area to 1024 bytes
+  static constexpr int kBarOff = kOutOff + kOutBytes;
+  static constexpr int kAlloc = kBarOff + 512 + 1024;            // + slack to align to 1024 bytes
+  static_assert(kEpiWarps % 4 == 0 && kChunks % kParts == 0 && kStages >= 3, "tile configuration");
 };
 
 struct GemmArgs {
-  int64_t M;
-  int N, K;
+  int64_t T;       // tokens (rows of x and of out)
+  int N, K;        // output channels, reduction length
   const int32_t* b;
   const int32_t* c;
   const int32_t* bias;
@@ -106,84 +119,19 @@ struct GemmArgs {
   int32_t* status;
 };
 
-// One 32-column chunk of one accumulator row: registers -> epilogue -> the warp's staging tile
-// (32 rows x ROW_BYTES, 16-byte pieces XOR-swizzled the way the TMA store expects).
-// `piece0` is the index of the first 16-byte piece this chunk occupies in the staging row.
-// FAST: every column's requantization is in upper-word form (one 64-bit multiply-add).
-template <int ROW_BYTES>
-__device__ __forceinline__ uint32_t staging_piece_offset(uint32_t row, uint32_t piece) {
-  if constexpr (ROW_BYTES == 128) return row * 128u + ((piece ^ (row & 7u)) << 4);
-  else return row * 64u + ((piece ^ ((row >> 1) & 3u)) << 4);
-}
-
-template <int KIND, bool FAST, int ROW_BYTES>
-__device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[32], const int4* __restrict__ prm,
-                                               const GeluConsts& gk, int64_t gelu_half, uint8_t* stage,
-                                               uint32_t row, uint32_t piece0) {
-  if constexpr (KIND == EPI_RAW || KIND == EPI_Q16) {
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      int32_t o[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int4 p = prm[g * 4 + i];
-        const int32_t a = (int32_t)v[g * 4 + i];
-        const int64_t add = (int64_t)(((uint64_t)(uint32_t)p.w << 32) | (uint32_t)p.z);
-        if constexpr (KIND == EPI_RAW) o[i] = a + p.x;
-        else if constexpr (FAST) o[i] = clamp_sym(requant_upper(a, p.x, add), 32767);
-        else o[i] = requant_add(a, p.x, add, p.y, 32767);
-      }
-      *reinterpret_cast<int4*>(stage + staging_piece_offset<ROW_BYTES>(row, piece0 + g)) =
-          make_int4(o[0], o[1], o[2], o[3]);
-    }
-  } else {
-#pragma unroll
-    for (int g = 0; g < 2; ++g) {
-      uint32_t w[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        int32_t o[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int idx = g * 16 + i * 4 + e;
-          const int4 p = prm[idx];
-          const int32_t a = (int32_t)v[idx];
-          const int64_t add = (int64_t)(((uint64_t)(uint32_t)p.w << 32) | (uint32_t)p.z);
-          if constexpr (KIND == EPI_INT8) {
-            if constexpr (FAST) o[e] = max(requant_upper(a, p.x, add), -127);
-            else o[e] = requant_add(a, p.x, add, p.y, 127);
-          } else {
-            if constexpr (FAST) {
-              const int32_t q16 = clamp_sym(requant_upper(a, p.x, add), 32767);
-              o[e] = igelu_q16_upper(q16, gk);
-            } else {
-              const int32_t q16 = requant_add(a, p.x, add, p.y, 32767);
-              o[e] = igelu_q16_to_int8(q16, gk, gelu_half);
-            }
-          }
-        }
-        w[i] = pack4_sat_s8(o[0], o[1], o[2], o[3]);    // upper clamp (+127) happens here
-      }
-      *reinterpret_cast<uint4*>(stage + staging_piece_offset<ROW_BYTES>(row, piece0 + g)) =
-          make_uint4(w[0], w[1], w[2], w[3]);
-    }
-  }
-}
-
-template <int BN, int KIND, bool FAST>
-__global__ void __launch_bounds__(gemm_threads(BN), 1)
-gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+template <int TOK, bool PAIR, int KIND, bool FAST>
+__global__ void __launch_bounds__(Cfg<TOK, PAIR, KIND>::kThreads, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __grid_constant__ CUtensorMap map_out, const GemmArgs args) {
-  using SM = GemmSmem<BN>;
-  constexpr int kStages = SM::kStages;
-  constexpr int kEpiThreads = 32 * epi_warps(BN);
-  constexpr uint32_t kTmemCols = 2 * BN;          // two accumulator stages (power of two >= 32)
+  using C = Cfg<TOK, PAIR, KIND>;
+  constexpr int kStages = C::kStages;
+  constexpr uint32_t kTmemCols = 2 * TOK;          // two accumulator stages
+  constexpr int kTileChannels = PAIR ? 2 * BC : BC;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = ptx::smem_addr(smem);
-  int4* s_param = reinterpret_cast<int4*>(smem + SM::kParamOff);
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + SM::kBarOff);
-  // barrier slots: full[kStages], empty[kStages], acc_full[2], acc_empty[2], then the TMEM base word
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + C::kBarOff);
+  // full[kStages] (PAIR: the leader's only), empty[kStages], acc_full[2], acc_empty[2] (leader's), TMEM base
   const uint32_t bar_full = ptx::smem_addr(s_bar);
   const uint32_t bar_empty = bar_full + 8 * kStages;
   const uint32_t bar_acc_full = bar_empty + 8 * kStages;
@@ -192,9 +140,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int n_tiles = (args.N + BN - 1) / BN;
-  const int64_t m_tiles = (args.M + BM - 1) / BM;
-  const int64_t total_tiles = m_tiles * n_tiles;
+  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;   // 0 = leader: issues the MMAs
+  const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int num_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int c_tiles = (args.N + kTileChannels - 1) / kTileChannels;
+  const int64_t t_tiles = (args.T + TOK - 1) / TOK;
+  const int64_t total_tiles = t_tiles * c_tiles;
   const int k_blocks = (args.K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
@@ -204,19 +155,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(bar_acc_full + 8 * a, 1);
-      ptx::mbar_init(bar_acc_empty + 8 * a, kEpiThreads);
+      ptx::mbar_init(bar_acc_empty + 8 * a, (PAIR ? 2 : 1) * C::kEpiWarps);   // one lane per epilogue warp
     }
     ptx::fence_mbar_init();
-    ptx::tma_prefetch_desc(&map_a);
-    ptx::tma_prefetch_desc(&map_b);
+    ptx::tma_prefetch_desc(&map_w);
+    ptx::tma_prefetch_desc(&map_x);
     ptx::tma_prefetch_desc(&map_out);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_addr(s_tmem), kTmemCols);
-    ptx::tmem_relinquish();
+    if constexpr (PAIR) { ptx::tmem_alloc_pair(ptx::smem_addr(s_tmem), kTmemCols); ptx::tmem_relinquish_pair(); }
+    else { ptx::tmem_alloc(ptx::smem_addr(s_tmem), kTmemCols); ptx::tmem_relinquish(); }
   }
   ptx::tc_fence_before_sync();
-  __syncthreads();
+  if constexpr (PAIR) ptx::cluster_sync(); else __syncthreads();   // barriers (of both CTAs) are initialised
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *s_tmem;
   bool ok = true;
@@ -225,120 +176,136 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
-      for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m0 = (int)(tile / n_tiles) * BM;
-        const int n0 = (int)(tile % n_tiles) * BN;
+      for (int64_t tile = worker; tile < total_tiles && ok; tile += num_workers) {
+        const int c0 = (int)(tile % c_tiles) * kTileChannels + (int)rank * BC;
+        const int t0 = (int)(tile / c_tiles) * TOK + (int)rank * C::kXRows;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!ptx::mbar_wait(bar_empty + 8 * stage, phase ^ 1)) { ok = false; break; }
-          const uint32_t sa = smem_base + stage * SM::kStageBytes;
-          ptx::mbar_arrive_expect_tx(bar_full + 8 * stage, SM::kStageBytes);
-          ptx::tma_load_2d(sa, &map_a, bar_full + 8 * stage, kb * BK, m0);
-          ptx::tma_load_2d(sa + SM::kABytes, &map_b, bar_full + 8 * stage, kb * BK, n0);
+          const uint32_t sw = smem_base + stage * C::kStageBytes;
+          if constexpr (PAIR) {
+            // both CTAs' copies complete on the leader's barrier, which expects the bytes of both
+            const uint32_t full_leader = ptx::map_to_cta(bar_full + 8 * stage, 0);
+            if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * C::kStageBytes);
+            ptx::tma_load_2d_pair(sw, &map_w, full_leader, kb * BK, c0);
+            ptx::tma_load_2d_pair(sw + C::kWBytes, &map_x, full_leader, kb * BK, t0);
+          } else {
+            ptx::mbar_arrive_expect_tx(bar_full + 8 * stage, C::kStageBytes);
+            ptx::tma_load_2d(sw, &map_w, bar_full + 8 * stage, kb * BK, c0);
+            ptx::tma_load_2d(sw + C::kWBytes, &map_x, bar_full + 8 * stage, kb * BK, t0);
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = ptx::make_idesc_i8(BM, BN, true, true);
+    // ------------------------------------------------------------ MMA issuer (PAIR: leader CTA only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_i8(kTileChannels, TOK, true, true);
       uint32_t stage = 0, phase = 0;
       uint32_t acc = 0, acc_phase = 0;
-      for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int64_t tile = worker; tile < total_tiles && ok; tile += num_workers) {
         if (!ptx::mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1)) { ok = false; break; }
         ptx::tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + acc * BN;
+        const uint32_t d_tmem = tmem_base + acc * TOK;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!ptx::mbar_wait(bar_full + 8 * stage, phase)) { ok = false; break; }
           ptx::tc_fence_after_sync();
-          const uint32_t sa = smem_base + stage * SM::kStageBytes;
-          const uint64_t da = ptx::make_kmajor_desc(sa, 1024, ptx::kSwizzle128);
-          const uint64_t db = ptx::make_kmajor_desc(sa + SM::kABytes, 1024, ptx::kSwizzle128);
+          const uint32_t sw = smem_base + stage * C::kStageBytes;
+          const uint64_t dw = ptx::make_kmajor_desc(sw, 1024, ptx::kSwizzle128);
+          const uint64_t dx = ptx::make_kmajor_desc(sw + C::kWBytes, 1024, ptx::kSwizzle128);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing K inside the swizzle span: +32 bytes = +2 in the encoded start address
-            ptx::mma_i8_ss(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            if constexpr (PAIR) ptx::mma_i8_ss_pair(d_tmem, dw + 2 * k, dx + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            else ptx::mma_i8_ss(d_tmem, dw + 2 * k, dx + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          ptx::mma_commit(bar_empty + 8 * stage);     // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs) once these MMAs have read it
+          if constexpr (PAIR) ptx::mma_commit_pair(bar_empty + 8 * stage, 3); else ptx::mma_commit(bar_empty + 8 * stage);
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        ptx::mma_commit(bar_acc_full + 8 * acc);      // accumulator complete
+        if constexpr (PAIR) ptx::mma_commit_pair(bar_acc_full + 8 * acc, 3); else ptx::mma_commit(bar_acc_full + 8 * acc);
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1;
       }
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..)
-    // Warp w owns TMEM lanes 32*(w%4)..+31 (rows) and, of those rows, 64 of the tile's
-    // columns.  Results go through a swizzled staging tile in shared memory and leave with a TMA
-    // store (full-line writes; rows / columns beyond M / N are clipped by the tensor map).
-    constexpr bool kOut32 = (KIND == EPI_RAW || KIND == EPI_Q16);
-    constexpr int kChunks = 2;                         // 32-column chunks per warp and tile
-    constexpr int kRowBytes = kOut32 ? 128 : 64;       // staging row: one chunk of int32 or both chunks of int8
+    // Warp w reads TMEM lanes 32*(w%4)..+31: thread = one output channel, registers = 32 tokens.
+    constexpr bool kOut32 = C::kOut32;
     const int quarter = warp & 3;
-    const int part = (warp - 2) >> 2;                  // which 64-column part of the tile
-    const int et = threadIdx.x - 64;                   // 0..kEpiThreads-1
-    uint8_t* stage = smem + SM::kOutOff + (warp - 2) * SM::kOutTileBytes;
+    const int part = (warp - 2) >> 2;                  // which token range of the tile
+    uint8_t* stage0 = smem + C::kOutOff + (warp - 2) * 2 * C::kOutTileBytes;
+    uint32_t buf = 0;
     const GeluConsts gk = args.gelu;
     const int64_t gelu_half = rounding_half(gk.c);
+    uint32_t acc_empty_addr = bar_acc_empty;
+    if constexpr (PAIR) acc_empty_addr = ptx::map_to_cta(bar_acc_empty, 0);
     uint32_t acc = 0, acc_phase = 0;
-    for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const int64_t m0 = (tile / n_tiles) * BM;
-      const int n0 = (int)(tile % n_tiles) * BN;
-      // per-column parameters of this tile.  generic: {b, c, (bias*b + 2^(c-1)) lo, hi};
-      // fast: {b << (32-c), -, (bias*(b << (32-c)) + 2^31) lo, hi};  raw: {bias, 0, 0, 0}
-      asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // previous tile's readers are done
-      for (int j = et; j < BN; j += kEpiThreads) {
-        const int n = n0 + j;
-        int4 p = make_int4(0, 0, 0, 0);
-        if (n < args.N) {
-          const int32_t bias = args.bias ? __ldg(args.bias + n) : 0;
-          if constexpr (KIND == EPI_RAW) {
-            p.x = bias;
-          } else {
-            const int32_t b = __ldg(args.b + n), c = __ldg(args.c + n);
-            const int64_t add = (int64_t)bias * b + (FAST ? (int64_t(1) << 31) : rounding_half(c));
-            p = make_int4(b, c, (int32_t)(uint32_t)(uint64_t)add, (int32_t)(add >> 32));
-          }
+    for (int64_t tile = worker; tile < total_tiles; tile += num_workers) {
+      const int ch0 = (int)(tile % c_tiles) * kTileChannels + (int)rank * BC + quarter * 32;   // this warp's channels
+      const int t0 = (int)(tile / c_tiles) * TOK + part * (C::kChunksPerWarp * 32);
+      // this thread's channel constants.  generic: b, c, bias*b + 2^(c-1);
+      // fast: b << (32-c) (the bias is added to the accumulator first);  raw: bias
+      const int n = ch0 + lane;
+      int32_t pb = 0, pc = 0, bias = 0;
+      int64_t padd = 0;
+      if (n < args.N) {
+        bias = args.bias ? __ldg(args.bias + n) : 0;
+        if constexpr (KIND != EPI_RAW) {
+          pb = __ldg(args.b + n);
+          pc = __ldg(args.c + n);
+          padd = (int64_t)bias * pb + rounding_half(pc);
         }
-        s_param[j] = p;
       }
-      asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-
-      // After a failed wait the loop keeps running (the named barriers above must still be
-      // reached by every epilogue thread) but touches neither TMEM nor memory.
       if (ok) ok = ptx::mbar_wait(bar_acc_full + 8 * acc, acc_phase);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) continue;
+      if (!ok) continue;                               // keep walking the tiles, touch nothing
       ptx::tc_fence_after_sync();
-      const int out_row0 = (int)m0 + quarter * 32;
-      const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
+      const uint32_t t_row = tmem_base + acc * TOK + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
-      for (int ci = 0; ci < kChunks; ++ci) {
-        const int ch = part * kChunks + ci;
+      for (int ci = 0; ci < C::kChunksPerWarp; ++ci) {
+        const int col = (part * C::kChunksPerWarp + ci) * 32;
         uint32_t v[32];
-        ptx::tmem_ld32(t_row + ch * 32, v);
+        ptx::tmem_ld32(t_row + col, v);
         ptx::tmem_wait_ld();
-        if (kOut32 || ci == 0) {
-          // the previous store from this staging tile must have finished reading it
-          if (lane == 0) ptx::bulk_wait_read<0>();
-          __syncwarp();
-        }
-        epilogue_chunk<KIND, FAST, kRowBytes>(v, s_param + ch * 32, gk, gelu_half, stage, (uint32_t)lane,
-                                              kOut32 ? 0u : (uint32_t)(ci * 2));
-        if (kOut32 || ci == kChunks - 1) {
-          ptx::fence_proxy_async_smem();               // staging writes -> visible to the TMA engine
-          __syncwarp();
-          if (lane == 0) {
-            const int x_bytes = kOut32 ? (n0 + ch * 32) * 4 : n0 + part * 64;
-            ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), x_bytes, out_row0);
-            ptx::bulk_commit();
+        // the store issued two chunks ago from this staging tile must have finished reading it
+        if (lane == 0) ptx::bulk_wait_read<1>();
+        __syncwarp();
+        uint8_t* stage = stage0 + buf * C::kOutTileBytes;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int32_t a = (int32_t)v[i];
+          int32_t o;
+          if constexpr (KIND == EPI_RAW) o = a + bias;
+          else if constexpr (KIND == EPI_Q16) {
+            if constexpr (FAST) o = clamp_sym(requant_upper(a + bias, pb), 32767);
+            else o = requant_add(a, pb, padd, pc, 32767);
+          } else if constexpr (KIND == EPI_INT8) {
+            if constexpr (FAST) o = clamp_sym(requant_upper(a + bias, pb), 127);
+            else o = requant_add(a, pb, padd, pc, 127);
+          } else {
+            if constexpr (FAST) o = min(igelu_q16_upper(clamp_sym(requant_upper(a + bias, pb), 32767), gk), 127);
+            else o = igelu_q16_to_int8(requant_add(a, pb, padd, pc, 32767), gk, gelu_half);
           }
+          // staging tile: row = token i, column = this lane's channel
+          if constexpr (kOut32) reinterpret_cast<int32_t*>(stage)[i * 32 + lane] = o;
+          else reinterpret_cast<int8_t*>(stage)[i * 32 + lane] = (int8_t)o;
         }
+        ptx::fence_proxy_async_smem();                 // staging writes -> visible to the TMA engine
+        __syncwarp();
+        if (lane == 0) {
+          ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), ch0 * (kOut32 ? 4 : 1), t0 + ci * 32);
+          ptx::bulk_commit();
+        }
+        buf ^= 1;
       }
       ptx::tc_fence_before_sync();
-      ptx::mbar_arrive(bar_acc_empty + 8 * acc);
+      __syncwarp();
+      if (lane == 0) {                                 // this warp is done with the accumulator stage
+        if (PAIR && rank != 0) ptx::mbar_arrive_remote(acc_empty_addr + 8 * acc);
+        else ptx::mbar_arrive(bar_acc_empty + 8 * acc);
+      }
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1;
     }
@@ -347,37 +314,53 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (!ok) atomicCAS(args.status, 0, IBERT_ERR_TIMEOUT);
   ptx::tc_fence_before_sync();
-  __syncthreads();
+  if constexpr (PAIR) ptx::cluster_sync(); else __syncthreads();   // nobody leaves while a peer may use its memory
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, kTmemCols);
+    if constexpr (PAIR) ptx::tmem_dealloc_pair(tmem_base, kTmemCols); else ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
-template <int BN, int KIND, bool FAST>
-int launch_inst(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo,
+template <int TOK, bool PAIR, int KIND, bool FAST>
+int launch_inst(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& mo,
                 const GemmArgs& args) {
+  using C = Cfg<TOK, PAIR, KIND>;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_i8_kernel<BN, KIND, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             GemmSmem<BN>::kAlloc) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_i8_kernel<TOK, PAIR, KIND, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             C::kAlloc) != cudaSuccess)
       return IBERT_ERR_CUDA;
     attr_set = true;
   }
-  const int64_t tiles = ((args.M + BM - 1) / BM) * ((args.N + BN - 1) / BN);
-  const int grid = (int)(tiles < ctx->num_sms ? tiles : ctx->num_sms);
-  gemm_i8_kernel<BN, KIND, FAST><<<grid, gemm_threads(BN), GemmSmem<BN>::kAlloc, ctx->stream>>>(ma, mb, mo, args);
-  return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
+  const int64_t tiles = ((args.T + TOK - 1) / TOK) * ((args.N + (PAIR ? 255 : 127)) / (PAIR ? 256 : 128));
+  const int workers = (int)std::min<int64_t>(tiles, PAIR ? ctx->num_sms / 2 : ctx->num_sms);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(PAIR ? 2 * workers : workers);
+  cfg.blockDim = dim3(C::kThreads);
+  cfg.dynamicSmemBytes = C::kAlloc;
+  cfg.stream = ctx->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, gemm_i8_kernel<TOK, PAIR, KIND, FAST>, mw, mx, mo, args) != cudaSuccess) {
+    cudaGetLastError();
+    return IBERT_ERR_CUDA;
+  }
+  return IBERT_OK;
 }
 
-template <int BN>
-int launch_bn(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const GemmArgs& a,
-              int kind, bool fast) {
+template <int TOK, bool PAIR>
+int launch_shape(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& mo, const GemmArgs& a,
+                 int kind, bool fast) {
   switch (kind) {
-    case EPI_INT8: return fast ? launch_inst<BN, EPI_INT8, true>(ctx, ma, mb, mo, a) : launch_inst<BN, EPI_INT8, false>(ctx, ma, mb, mo, a);
-    case EPI_Q16: return fast ? launch_inst<BN, EPI_Q16, true>(ctx, ma, mb, mo, a) : launch_inst<BN, EPI_Q16, false>(ctx, ma, mb, mo, a);
-    case EPI_GELU: return fast ? launch_inst<BN, EPI_GELU, true>(ctx, ma, mb, mo, a) : launch_inst<BN, EPI_GELU, false>(ctx, ma, mb, mo, a);
-    default: return launch_inst<BN, EPI_RAW, false>(ctx, ma, mb, mo, a);
+    case EPI_INT8: return fast ? launch_inst<TOK, PAIR, EPI_INT8, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_INT8, false>(ctx, mw, mx, mo, a);
+    case EPI_Q16: return fast ? launch_inst<TOK, PAIR, EPI_Q16, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_Q16, false>(ctx, mw, mx, mo, a);
+    case EPI_GELU: return fast ? launch_inst<TOK, PAIR, EPI_GELU, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_GELU, false>(ctx, mw, mx, mo, a);
+    default: return launch_inst<TOK, PAIR, EPI_RAW, false>(ctx, mw, mx, mo, a);
   }
 }
 
@@ -386,44 +369,46 @@ int launch_bn(ibert_ctx* ctx, const CUtensorMap& ma, const CUtensorMap& mb, cons
 int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, int N, int K,
                    const GemmEpilogue& epi, void* out) {
   if (M == 0) return IBERT_OK;
-  // tile width: 256 when it divides the work well, else 128
-  const int64_t m_tiles = (M + BM - 1) / BM;
-  const bool wide = (N % 256 == 0) && m_tiles * (N / 256) >= ctx->num_sms;
-  const int BN = wide ? 256 : 128;
-  CUtensorMap ma, mb;
-  {
-    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
-    const uint64_t str[1] = {(uint64_t)K};
-    const uint32_t box[2] = {BK, BM};
-    int rc = encode_tensor_map(&ma, x, 2, dims, str, box, 128);
-    if (rc) return rc;
-  }
+  // tile shape: 256 channels x 256 tokens on a CTA pair when that fills every pair, else one CTA
+  // per 128 channels x 256 (or 128) tokens
+  const int64_t t256 = (M + 255) / 256;
+  const bool pair = ctx->num_sms >= 2 && t256 * ((N + 255) / 256) >= ctx->num_sms / 2;
+  const bool wide = pair || t256 * ((N + 127) / 128) >= ctx->num_sms;
+  const int TOK = wide ? 256 : 128;
+  const bool out32 = epi.kind == EPI_RAW || epi.kind == EPI_Q16;
+  CUtensorMap mw, mx, mo;
   {
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
     const uint64_t str[1] = {(uint64_t)K};
-    const uint32_t box[2] = {BK, (uint32_t)BN};
-    int rc = encode_tensor_map(&mb, w, 2, dims, str, box, 128);
+    const uint32_t box[2] = {BK, BC};
+    int rc = encode_tensor_map(&mw, w, 2, dims, str, box, 128);
     if (rc) return rc;
   }
-  CUtensorMap mo;
   {
-    // the output as a byte matrix [M, N * element size]; one box = one warp's staging tile
-    const bool out32 = epi.kind == EPI_RAW || epi.kind == EPI_Q16;
+    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
+    const uint64_t str[1] = {(uint64_t)K};
+    const uint32_t box[2] = {BK, (uint32_t)(pair ? TOK / 2 : TOK)};   // a pair's CTA loads half of the token rows
+    int rc = encode_tensor_map(&mx, x, 2, dims, str, box, 128);
+    if (rc) return rc;
+  }
+  {
+    // the output as a byte matrix [T, N * element size]; one box = one warp's 32-token x 32-channel block
     const uint64_t row_bytes = (uint64_t)N * (out32 ? 4 : 1);
-    const uint32_t box_bytes = out32 ? 128u : 64u;
     const uint64_t dims[2] = {row_bytes, (uint64_t)M};
     const uint64_t str[1] = {row_bytes};
-    const uint32_t box[2] = {box_bytes, 32};
-    int rc = encode_tensor_map(&mo, out, 2, dims, str, box, (int)box_bytes);
+    const uint32_t box[2] = {out32 ? 128u : 32u, 32};
+    int rc = encode_tensor_map(&mo, out, 2, dims, str, box, 0);
     if (rc) return rc;
   }
   GemmArgs a{};
-  a.M = M; a.N = N; a.K = K;
+  a.T = M; a.N = N; a.K = K;
   a.b = epi.d_b; a.c = epi.d_c; a.bias = epi.d_bias; a.gelu = epi.gelu;
   a.status = ctx->d_status;
-  // upper-word epilogue needs both the per-column multipliers and (for GELU) the final one in that form
+  // upper-word epilogue needs both the per-channel multipliers and (for GELU) the final one in that form
   const bool fast = epi.fast != 0 && (epi.kind != EPI_GELU || epi.gelu.fast != 0);
-  return wide ? launch_bn<256>(ctx, ma, mb, mo, a, epi.kind, fast) : launch_bn<128>(ctx, ma, mb, mo, a, epi.kind, fast);
+  if (pair) return launch_shape<256, true>(ctx, mw, mx, mo, a, epi.kind, fast);
+  return wide ? launch_shape<256, false>(ctx, mw, mx, mo, a, epi.kind, fast)
+              : launch_shape<128, false>(ctx, mw, mx, mo, a, epi.kind, fast);
 }
 
 }  // namespace ibert

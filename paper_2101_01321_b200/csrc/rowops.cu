@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const int32_t rv = (int32_t)(int8_t)(rw >> (8 * i));
-              if (FAST) v[j][i] += requant_upper(rv << k.res_sh, k.b_r, int64_t(1) << 31);
+              if (FAST) v[j][i] += requant_upper(rv << k.res_sh, k.b_r);
               else v[j][i] += (int32_t)(((int64_t)rv * k.b_r + half_r) >> k.c_r);
             }
           }
@@ -232,7 +232,7 @@ __global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel
           for (int i = 0; i < 4; ++i) {
             // normalized value floor(y * rho / 2^15), then pre-shifted by out_sh (|.| < 2^31)
             const int32_t nrm = (int32_t)(((int64_t)v[j][i] * rho64) >> 15) << k.out_sh;
-            o[i] = max(requant_upper(nrm, bv[i], Bv[i]), -127);
+            o[i] = max(requant_upper_add(nrm, bv[i], Bv[i]), -127);
           }
         }
       } else {
@@ -336,7 +336,7 @@ __global__ void __launch_bounds__(kThreads, 2) layernorm_pipe_kernel(const int32
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int32_t rv = (int32_t)(int8_t)(rw[j] >> (8 * i));
-        v[j][i] += requant_upper(rv << k.res_sh, k.b_r, int64_t(1) << 31);
+        v[j][i] += requant_upper(rv << k.res_sh, k.b_r);
         sum += v[j][i];
       }
     sum = __reduce_add_sync(0xffffffffu, sum);
@@ -374,7 +374,7 @@ __global__ void __launch_bounds__(kThreads, 2) layernorm_pipe_kernel(const int32
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int32_t nrm = (int32_t)(((int64_t)v[j][i] * (int64_t)rho) >> nsh) << k.out_sh;
-          o[i] = max(requant_upper(nrm, bv[i], Bv[i]), -127);
+          o[i] = max(requant_upper_add(nrm, bv[i], Bv[i]), -127);
         }
         __stcs(reinterpret_cast<uint32_t*>(orow + col), pack4_sat_s8(o[0], o[1], o[2], o[3]));
       }

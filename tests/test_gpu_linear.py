@@ -21,7 +21,7 @@ def _problem(M, N, K, seed, acc_scale=1.0):
 
 
 SHAPES = [(1, 16, 16), (7, 48, 80), (128, 128, 128), (130, 272, 144), (300, 768, 768), (257, 2304, 768),
-          (129, 768, 3072), (1024, 1024, 1024), (4100, 512, 256), (2100, 2304, 768), (0, 64, 64)]
+          (129, 768, 3072), (1024, 1024, 1024), (4100, 512, 256), (2100, 2304, 768), (4800, 1024, 512), (19000, 256, 64), (0, 64, 64)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
@@ -53,7 +53,7 @@ def test_linear_requantized(M, N, K, kind):
         assert np.abs(want.astype(np.int64)).max() <= qmax
 
 
-@pytest.mark.parametrize("M,N,K", [(7, 48, 80), (300, 768, 768), (257, 3072, 768), (1000, 4096, 1024)])
+@pytest.mark.parametrize("M,N,K", [(7, 48, 80), (300, 768, 768), (257, 3072, 768), (1000, 4096, 1024), (2500, 3072, 768)])
 def test_linear_with_fused_gelu(M, N, K):
     x, w, bias, S_w, S_x, amax = _problem(M, N, K, 3)
     # scale the problem so the GELU input covers about [-6, 6]

@@ -175,7 +175,7 @@ def run_ours(args):
     import numpy as np
     import torch
 
-    from paper_2101_01321_b200 import binding, build, synth
+    from paper_2101_01321_b200 import binding, build, dp, synth
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -195,7 +195,10 @@ def run_ours(args):
     cfg = synth.CONFIGS[args.config]
     batch = args.batch or DEFAULT_BATCH[args.config]
     T = batch * cfg.L
-    x_np, params = synth.make_model(args.config, batch)
+    # weak scaling: rank r owns sequences [r*batch, (r+1)*batch) of the global batch
+    first, last = dp.shard_range(batch * world, world, rank)
+    assert last - first == batch
+    x_np, params = synth.make_model(args.config, batch, shard=rank)
     stream = torch.cuda.Stream(device=dev)
     ctx = binding.Context(local_rank, stream)
     layers = [ctx.ibert_layer_create(p) for p in params]
@@ -268,10 +271,7 @@ def run_ours(args):
         prof = ctx.ibert_profile_end()
     ctx.check()
 
-    if dist is not None:
-        t = torch.tensor([total_ms, total_e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, total_e2e_ms = float(t[0]), float(t[1])
+    total_ms, total_e2e_ms = dp.max_over_ranks([total_ms, total_e2e_ms], device=dev)
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()

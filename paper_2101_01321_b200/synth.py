@@ -107,11 +107,18 @@ def static_activation_scales(H: int, F: int, L: int, S_x: float, w_std: float = 
     return s
 
 
-def make_input(config_id: int, B: int, L: int, H: int):
-    """x ~ N(0,1) as int8 with S_x = max|x| / 127.  Returns (x_q [B*L, H], S_x)."""
-    rng = rng_for(config_id, 0, _T_X)
-    x = rng.standard_normal((B * L, H), dtype=np.float32).astype(np.float64)
-    S_x = float(np.abs(x).max() / 127.0)
+def make_input(config_id: int, B: int, L: int, H: int, shard: int = 0):
+    """x ~ N(0,1) as int8 with S_x = max|x| / 127.  Returns (x_q [B*L, H], S_x).
+
+    `shard` selects the slice of a data-parallel global batch (one seeded stream per shard,
+    tensor id 100*shard).  The static scale S_x is always the one of shard 0, so every rank
+    quantizes with the same scale (later shards clip the few values beyond it)."""
+    x0 = rng_for(config_id, 0, _T_X).standard_normal((B * L, H), dtype=np.float32).astype(np.float64)
+    S_x = float(np.abs(x0).max() / 127.0)
+    if shard == 0:
+        x = x0
+    else:
+        x = rng_for(config_id, 0, _T_X + 100 * shard).standard_normal((B * L, H), dtype=np.float32).astype(np.float64)
     return quantize_sym(x, S_x, 127).astype(np.int8), S_x
 
 
@@ -138,7 +145,7 @@ def make_layer(config_id: int, layer: int, H: int, heads: int, F: int, L: int, S
 
 
 def make_model(config_id: int, B: int, layers: int | None = None, H: int | None = None,
-               heads: int | None = None, F: int | None = None, L: int | None = None):
+               heads: int | None = None, F: int | None = None, L: int | None = None, shard: int = 0):
     """Input and per-layer parameters of one of the encoder configs (0, 2, 3, 4).
     Layer l+1 consumes layer l's int8 output, so its S_x is layer l's S_out."""
     cfg = CONFIGS[config_id]
@@ -147,7 +154,7 @@ def make_model(config_id: int, B: int, layers: int | None = None, H: int | None 
     F = F or cfg.F
     L = L or cfg.L
     layers = layers or cfg.layers
-    x, S_x = make_input(config_id, B, L, H)
+    x, S_x = make_input(config_id, B, L, H, shard)
     params = []
     s_in = S_x
     for l in range(layers):

@@ -103,6 +103,25 @@ int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* 
                       const double* gamma, const double* beta, int64_t rows, int C, double S_out,
                       int8_t* out, double* S_ret);
 
+/* The same operation for callers that cannot allocate device memory (no counterpart in the
+   paper: a deployment convenience).  ibert_layernorm_i keeps its per-channel constant tables in
+   memory it obtains with cudaMalloc; code that runs where allocation is forbidden -- inside a
+   region that must not touch the allocator, under a memory budget owned by another component,
+   or in a host thread that may not block on the driver's allocation lock -- can call this
+   variant instead.  It needs no ibert_ctx: work is enqueued on `cuda_stream` (a cudaStream_t,
+   NULL = legacy default stream) of the CURRENT device, and the tables plus a status word live in
+   a fixed device array of 24,832 bytes that every GPU loading the library holds until exit.
+   It calls no cudaMalloc / cudaFree nor any other routine that allocates device memory.
+   Limits and caveats: C <= IBERT_STATIC_LN_MAX_C (larger C -> IBERT_ERR_SHAPE); all calls on a
+   device share the one array, so two calls whose GPU work may overlap (different streams without
+   ordering) race on it -- serialize them; the first call on each device looks up the array's
+   device address, so make that first call outside any stream capture.
+   Arguments and results are exactly those of ibert_layernorm_i. */
+#define IBERT_STATIC_LN_MAX_C 2047
+int ibert_layernorm_i_static(void* cuda_stream, const int32_t* q, double S, const int8_t* r, double S_r,
+                             const double* gamma, const double* beta, int64_t rows, int C, double S_out,
+                             int8_t* out, double* S_ret);
+
 /* Multi-head self-attention on int8 Q|K|V (Fig. 1 right: MatMul -> i-softmax -> MatMul):
    per (batch, head): s = Q K^T (int32, scale S_q*S_k/8, head size 64), p = i-softmax(s) in u8
    (p_max = 255) or 7-bit (p_max = 127), ctx = requant(p V; dyadic((1/p_max)*S_v/S_ctx)).

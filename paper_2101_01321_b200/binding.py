@@ -63,6 +63,8 @@ def lib():
         L.ibert_layer_create.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(vp)]
         L.ibert_layer_destroy.argtypes = [vp]
         L.ibert_encoder_layer.argtypes = [vp, vp, vp, i32, i32, vp, vp]
+        L.ibert_layernorm_i_static.argtypes = [vp, vp, dbl, vp, dbl, vp, vp, i64, i32, dbl, vp, vp]
+        L.ibert_layernorm_i_static.restype = i32
         L.ibert_selftest_exp_division.argtypes = [dbl, C.POINTER(C.c_int32)]
         L.ibert_selftest_exp_division.restype = i32
         L.ibert_profile_begin.argtypes = [vp]
@@ -98,6 +100,23 @@ def ibert_dyadic_from_double(m: float) -> tuple[int, int]:
     b, c = C.c_int32(), C.c_int32()
     _chk(lib().ibert_dyadic_from_double(m, C.byref(b), C.byref(c)), "ibert_dyadic_from_double")
     return b.value, c.value
+
+
+def ibert_layernorm_i_static(q: torch.Tensor, S: float, r: torch.Tensor | None, S_r: float, gamma, beta,
+                             S_out: float, out: torch.Tensor | None = None, stream: torch.cuda.Stream | None = None):
+    """Residual + i-LayerNorm through the entry point that allocates nothing inside the library
+    (no context needed; runs on `stream` of the current device)."""
+    Cn = q.shape[-1]
+    rows = q.numel() // Cn if Cn else 0
+    g, b = _host(gamma, np.float64), _host(beta, np.float64)
+    if out is None:
+        out = torch.empty(q.shape, dtype=torch.int8, device=q.device)
+    S_ret = C.c_double()
+    sp = None if stream is None else stream.cuda_stream
+    _chk(lib().ibert_layernorm_i_static(sp, _dev(q, torch.int32), S, _dev(r, torch.int8), S_r or 0.0,
+                                        g.ctypes.data, b.ctypes.data, rows, Cn, S_out, _dev(out, torch.int8),
+                                        C.byref(S_ret)), "ibert_layernorm_i_static")
+    return out, S_ret.value
 
 
 class Context:

@@ -29,6 +29,12 @@ UNIT = "tokens/s"
 DEFAULT_BATCH = {2: 128, 3: 32, 4: 64}
 
 
+# DRAM bytes (read + write) per launch from one ncu capture of each kernel class at the default
+# workload (config 2, B=128; cold L2; summaries under profiles/).  Other workloads report null.
+NCU_DRAM_TRAFFIC_BYTES = {(2, 128): {"gemm_qkv": 14.5e6, "attention": 37.8e6, "gemm_out": 14.2e6, "layernorm": 64.7e6,
+                                     "gemm_ffn1_gelu": 17.1e6, "gemm_ffn2": 61.3e6}}
+
+
 # --------------------------------------------------------------------------- helpers
 def measured_peaks() -> tuple[dict, str]:
     p = ROOT / "MEASURED_PEAKS.json"
@@ -297,6 +303,9 @@ def run_ours(args):
                     "unit": "GB/s", "frac": kern[top]["gbs"] / peaks["hbm_gbs"], "traffic": None,
                     "peak_source": f"{peak_kind} copy bandwidth"}
         roof["ms_per_launch"] = kern[top]["ms_per_launch"]
+        roof["traffic"] = NCU_DRAM_TRAFFIC_BYTES.get((args.config, batch), {}).get(top)
+        roof["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)"
+        roof["algorithmic"] = work[top]["ops"] if work[top]["ops"] else work[top]["bytes"]
         tokens = T * args.steps * world
         value = tokens / (total_ms / 1e3)
         e2e_value = tokens / (total_e2e_ms / 1e3)

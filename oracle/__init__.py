@@ -29,12 +29,17 @@ class OracleError(RuntimeError):
 
 def build(force: bool = False) -> Path:
     """Compile the oracle (gcc -O2, OpenMP, no FMA contraction)."""
-    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+    import hashlib
+    digest = hashlib.sha256(_SRC.read_bytes()).hexdigest()
+    stamp = _LIB.with_suffix(".so.srchash")
+    # (file times do not survive a copy of the tree: compare a hash of the source instead)
+    if force or not _LIB.exists() or not stamp.exists() or stamp.read_text().strip() != digest:
         tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
         subprocess.check_call(
             ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
              "-fPIC", "-shared", "-Wall", "-Wno-maybe-uninitialized", "-o", str(tmp), str(_SRC), "-lm"])
         os.replace(tmp, _LIB)
+        stamp.write_text(digest + "\n")
     return _LIB
 
 

@@ -16,13 +16,25 @@ def _sources():
     return [CSRC / s for s in SOURCES if (CSRC / s).exists()]
 
 
+def _source_hash() -> str:
+    """Hash of every source the library is built from (file times do not survive a copy of the tree)."""
+    import hashlib
+    h = hashlib.sha256()
+    deps = sorted(list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + list(CSRC.glob("*.h")) +
+                  list(CSRC.glob("*.cpp")) + [PKG.parent / "include" / "ibert.h", Path(__file__)])
+    for d in deps:
+        h.update(d.name.encode())
+        h.update(d.read_bytes())
+    return h.hexdigest()
+
+
+HASH_FILE = PKG / "libibert_b200.so.srchash"
+
+
 def _stale() -> bool:
-    if not LIB.exists():
+    if not LIB.exists() or not HASH_FILE.exists():
         return True
-    t = LIB.stat().st_mtime
-    deps = list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + list(CSRC.glob("*.h")) + \
-        list(CSRC.glob("*.cpp")) + [PKG.parent / "include" / "ibert.h"]
-    return any(d.stat().st_mtime > t for d in deps)
+    return HASH_FILE.read_text().strip() != _source_hash()
 
 
 def build(force: bool = False, verbose: bool = False) -> Path:
@@ -38,6 +50,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     cmd += [str(s) for s in _sources()]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
+    HASH_FILE.write_text(_source_hash() + "\n")
     return LIB
 
 

@@ -32,15 +32,12 @@ __device__ __forceinline__ int32_t requant_upper(int32_t v, int32_t b2) {
 // (v * b2 + add) >> 32 for a general 64-bit addend, the carry of the lower words propagated by hand
 __device__ __forceinline__ int32_t requant_upper_add(int32_t v, int32_t b2, int64_t add) {
   const int64_t t = (int64_t)v * (int64_t)b2;
-  uint32_t lo;
   int32_t hi;
   asm("{\n\t.reg .u32 s;\n\t"
-      "add.cc.u32 s, %2, %4;\n\t"
-      "addc.s32 %1, %3, %5;\n\t"
-      "mov.u32 %0, s;\n\t}"
-      : "=r"(lo), "=r"(hi)
+      "add.cc.u32 s, %1, %3;\n\t"
+      "addc.s32 %0, %2, %4;\n\t}"
+      : "=r"(hi)
       : "r"((uint32_t)t), "r"((int32_t)(t >> 32)), "r"((uint32_t)add), "r"((int32_t)(add >> 32)));
-  (void)lo;
   return hi;
 }
 

@@ -1,0 +1,79 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times.
+
+The encoder never mixes sequences, so the oracle recomputes a sample of whole sequences through
+every layer and the GPU rows of those sequences (taken from the full-batch run) must match bit
+for bit.  The standalone sweeps of config 1 are compared in full."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import assert_same, ctx, dev, host
+from paper_2101_01321_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _full_model_check(config_id, B, sample):
+    cfg = synth.CONFIGS[config_id]
+    L = cfg.L
+    x, params = synth.make_model(config_id, B)
+    c = ctx()
+    layers = [c.ibert_layer_create(p) for p in params]
+    h = dev(x)
+    bufs = [torch.empty_like(h), torch.empty_like(h)]
+    for i, ly in enumerate(layers):
+        h, _ = c.ibert_encoder_layer(ly, h, B, L, out=bufs[i & 1])
+    c.check()
+    got = host(h).reshape(B, L, cfg.H)
+    for ly in layers:
+        ly.close()
+    for s in sample:
+        ref = x.reshape(B, L, cfg.H)[s].reshape(L, cfg.H)
+        for p in params:
+            ref = oracle.encoder_layer(p, ref, 1, L).out
+        assert_same(got[s], ref, f"config {config_id}, sequence {s}")
+    assert got.std() > 20                      # the stack stays well scaled through all layers
+
+
+def test_config2_twelve_layers_batch128_sampled_sequences():
+    _full_model_check(2, 128, sample=(0, 77, 127))
+
+
+def test_config2_small_batches():
+    for B in (1, 8, 32):
+        _full_model_check(2, B, sample=(0, B - 1))
+
+
+def test_config3_large_24_layers_L256_batch32_sampled_sequence():
+    _full_model_check(3, 32, sample=(5,))
+
+
+def test_config4_large_24_layers_L512_batch64_sampled_sequence():
+    _full_model_check(4, 64, sample=(63,))
+
+
+@pytest.mark.parametrize("sigma", [1.0, 4.0])
+def test_config1_gelu_16m_elements(sigma):
+    q, S, S_out = synth.gelu_inputs(1 << 24, sigma)
+    out, _ = ctx().ibert_gelu_i(dev(q), S, S_out)
+    ctx().check()
+    assert_same(host(out), oracle.gelu(q, S, S_out)[0], "gelu 16M")
+
+
+@pytest.mark.parametrize("rows,L", [(96 * 128, 128), (384 * 512, 512)])
+def test_config1_softmax_score_tensors(rows, L):
+    for sigma in (1.0, 4.0):
+        q, S = synth.softmax_inputs(rows, L, sigma)
+        out, _ = ctx().ibert_softmax_i(dev(q), S, 255)
+        ctx().check()
+        assert_same(host(out), oracle.softmax(q, S, 255)[0], f"softmax [{rows},{L}]")
+
+
+@pytest.mark.parametrize("rows,C", [(4096, 768), (16384, 1024)])
+def test_config1_layernorm_rows(rows, C):
+    for sigma in (1.0, 4.0):
+        q, S, r, S_r, gamma, beta, S_out = synth.layernorm_inputs(rows, C, sigma)
+        out, _ = ctx().ibert_layernorm_i(dev(q), S, dev(r), S_r, gamma, beta, S_out)
+        ctx().check()
+        assert_same(host(out), oracle.layernorm(q, S, r, S_r, gamma, beta, S_out)[0], f"layernorm [{rows},{C}]")

@@ -239,6 +239,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *s_tmem;
   const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();              // the kernel that wrote qkv has completed
 
   // loads of one work item: Q tile, all K rows (64-byte swizzle, MMA operand layout), all V rows
   auto issue_loads = [&](int item, int stage) {
@@ -411,7 +413,8 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
   int per_sm = std::min(3, std::min((int)(512 / cols), (227 * 1024) / (smem + 1024)));
   if (per_sm < 1) per_sm = 1;
   const int grid = std::min(total, ctx->num_sms * per_sm);
-  attention_kernel<<<grid, kAttnThreads, smem, ctx->stream>>>(mqk, mv, a);
+  if (int rc = launch_pdl(attention_kernel, dim3(grid), dim3(kAttnThreads), (size_t)smem, ctx->stream, 1, mqk, mv, a))
+    return rc;
   return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
 }
 

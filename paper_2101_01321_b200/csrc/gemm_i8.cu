@@ -171,6 +171,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *s_tmem;
   bool ok = true;
+  // set-up done: the next kernel may be scheduled; the previous one must be complete before
+  // any operand is read or any output written
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -334,23 +338,8 @@ int launch_inst(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, co
   }
   const int64_t tiles = ((args.T + TOK - 1) / TOK) * ((args.N + (PAIR ? 255 : 127)) / (PAIR ? 256 : 128));
   const int workers = (int)std::min<int64_t>(tiles, PAIR ? ctx->num_sms / 2 : ctx->num_sms);
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(PAIR ? 2 * workers : workers);
-  cfg.blockDim = dim3(C::kThreads);
-  cfg.dynamicSmemBytes = C::kAlloc;
-  cfg.stream = ctx->stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, gemm_i8_kernel<TOK, PAIR, KIND, FAST>, mw, mx, mo, args) != cudaSuccess) {
-    cudaGetLastError();
-    return IBERT_ERR_CUDA;
-  }
-  return IBERT_OK;
+  return launch_pdl(gemm_i8_kernel<TOK, PAIR, KIND, FAST>, dim3(PAIR ? 2 * workers : workers), dim3(C::kThreads),
+                    (size_t)C::kAlloc, ctx->stream, PAIR ? 2 : 1, mw, mx, mo, args);
 }
 
 template <int TOK, bool PAIR>

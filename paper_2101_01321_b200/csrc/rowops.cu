@@ -283,6 +283,8 @@ __global__ void __launch_bounds__(kThreads, 2) layernorm_pipe_kernel(const int32
   const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
   const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
 
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();              // the kernel that produced q (and r) has completed
   auto issue = [&](int64_t row, int slot) {
     const uint32_t bar = ptx::smem_addr(bars + slot);
     const uint32_t dst = ptx::smem_addr(ring + (size_t)slot * slot_bytes);
@@ -445,8 +447,9 @@ int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t 
                                100 * 1024) != cudaSuccess) return IBERT_ERR_CUDA;                           \
       attr = true;                                                                                          \
     }                                                                                                       \
-    layernorm_pipe_kernel<V, D><<<pgrid, kThreads, smem, ctx->stream>>>(q, r, rows, k, d_b, d_B, out,       \
-                                                                         ctx->d_status);                    \
+    if (int rc_ = launch_pdl(layernorm_pipe_kernel<V, D>, dim3(pgrid), dim3(kThreads), smem, ctx->stream, 1, q, r, \
+                             rows, k, d_b, d_B, out, ctx->d_status))                                        \
+      return rc_;                                                                                           \
   } while (0)
     if (k.C <= 256) IBERT_LNP(2, 3);
     else if (k.C <= 512) IBERT_LNP(4, 3);

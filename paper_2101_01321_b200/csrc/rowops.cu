@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel
 // rows are in flight while the current row is reduced -- the row loop no longer waits on HBM.
 // Requires C % 16 == 0 (16-byte aligned rows), upper-word constants, and a residual.
 template <int VPL, int DEPTH>
-__global__ void __launch_bounds__(kThreads, 2) layernorm_pipe_kernel(const int32_t* __restrict__ q,
+__global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_kernel(const int32_t* __restrict__ q,
                                                                      const int8_t* __restrict__ r, int64_t rows,
                                                                      LnConsts k, const int32_t* __restrict__ b_i,
                                                                      const int64_t* __restrict__ B_i,
@@ -436,9 +436,9 @@ int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t 
   const bool fast = vec && k.out_fast && (!k.has_res || k.res_fast);
   if (fast && k.has_res && k.C % 16 == 0 && k.C <= 1024) {
     // streaming variant: per-warp ring of row slots filled by bulk async copies
-    const int depth = k.C <= 768 ? 3 : 2;
+    const int depth = 2;
     const size_t smem = (size_t)(kThreads / 32) * depth * (size_t)k.C * 5 + (kThreads / 32) * depth * 8;
-    const int pgrid = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)ctx->num_sms * 2);
+    const int pgrid = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)ctx->num_sms * 3);
 #define IBERT_LNP(V, D)                                                                                     \
   do {                                                                                                      \
     static bool attr = false;                                                                               \
@@ -451,9 +451,9 @@ int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t 
                              rows, k, d_b, d_B, out, ctx->d_status))                                        \
       return rc_;                                                                                           \
   } while (0)
-    if (k.C <= 256) IBERT_LNP(2, 3);
-    else if (k.C <= 512) IBERT_LNP(4, 3);
-    else if (k.C <= 768) IBERT_LNP(6, 3);
+    if (k.C <= 256) IBERT_LNP(2, 2);
+    else if (k.C <= 512) IBERT_LNP(4, 2);
+    else if (k.C <= 768) IBERT_LNP(6, 2);
     else IBERT_LNP(8, 2);
 #undef IBERT_LNP
     return check_launch();

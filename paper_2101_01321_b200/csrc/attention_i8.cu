@@ -269,11 +269,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
     uint8_t* sK = sQ + slab_bytes;
     uint8_t* sVs = sK + a.n_slabs * slab_bytes;
     const int next = item + gridDim.x;
-    if (tid == 0 && next < total) {
-      // two stages: the other one was released by the barrier that ended the previous item;
-      // one stage: nothing to overlap, the loads of `next` are issued at the end of this item
-      if (a.stages == 2) issue_loads(next, stage ^ 1);
-    }
     ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_load0 + 8 * stage, load_phase[stage]));
     load_phase[stage] ^= 1;
 
@@ -290,6 +285,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
       }
       ptx::mma_commit(bar_mma);
     }
+    // two stages: the other one was released by the barrier that ended the previous item, so the
+    // next item's loads go out now, behind the MMAs and off this item's critical path
+    // (one stage: nothing to overlap, they are issued at the end of this item)
+    if (tid == 0 && next < total && a.stages == 2) issue_loads(next, stage ^ 1);
     // ---- meanwhile: V [j][d] -> Vt [d][j] in the swizzled K-major operand layout
     if (ok) transpose_v(sVs, sVt, a.n_slabs * 128, tid);
     if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_mma, mma_phase));

@@ -65,13 +65,13 @@ __device__ __forceinline__ int32_t igelu_q16_to_int8(int32_t q, const GeluConsts
   return requant_add(g2, k.b, half, k.c, 127);
 }
 
-// Same function, written for the integer pipes: sign applied by a multiply, the final
+// Same function, written for the integer pipes: sign applied by a select, the final
 // requantization in upper-word form; the result still needs the upper clamp (pack4_sat_s8).
 __device__ __forceinline__ int32_t igelu_q16_upper(int32_t q, const GeluConsts& k) {
   const int32_t t = min(abs(q) >> k.s_in, k.nq_b) - k.nq_b;
-  const int32_t poly = t * t + k.q_c;
-  const int32_t sgn = (q >> 31) | 1;
-  const int32_t f = poly * sgn + k.q_c;
+  const int32_t tt = t * t;
+  // q_erf + q_1 = sgn(q) (t^2 + q_c) + q_c: -t^2 for q < 0, t^2 + 2 q_c otherwise (unused for q = 0)
+  const int32_t f = q < 0 ? -tt : tt + 2 * k.q_c;
   const int32_t g2 = (q * (f >> k.s_f) + 128) >> 8;
   return max(requant_upper(g2, k.b2), -127);
 }

@@ -246,15 +246,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     uint32_t acc_empty_addr = bar_acc_empty;
     if constexpr (PAIR) acc_empty_addr = ptx::map_to_cta(bar_acc_empty, 0);
     uint32_t acc = 0, acc_phase = 0;
-    for (int64_t tile = worker; tile < total_tiles; tile += num_workers) {
-      const int ch0 = (int)(tile % c_tiles) * kTileChannels + (int)rank * BC + quarter * 32;   // this warp's channels
-      const int t0 = (int)(tile / c_tiles) * TOK + part * (C::kChunksPerWarp * 32);
-      // this thread's channel constants.  generic: b, c, bias*b + 2^(c-1);
-      // fast: b << (32-c) (the bias is added to the accumulator first);  raw: bias
-      const int n = ch0 + lane;
-      int32_t pb = 0, pc = 0, bias = 0;
-      int64_t padd = 0;
-      if (n < args.N) {
+    // this thread's channel constants for a tile.  generic: b, c, bias*b + 2^(c-1);
+    // fast: b << (32-c) (the bias is added to the accumulator first);  raw: bias
+    int32_t pb = 0, pc = 0, bias = 0;
+    int64_t padd = 0;
+    auto load_constants = [&](int64_t tile) {
+      const int n = (int)(tile % c_tiles) * kTileChannels + (int)rank * BC + quarter * 32 + lane;
+      pb = 0; pc = 0; bias = 0; padd = 0;
+      if (tile < total_tiles && n < args.N) {
         bias = args.bias ? __ldg(args.bias + n) : 0;
         if constexpr (KIND != EPI_RAW) {
           pb = __ldg(args.b + n);
@@ -262,6 +261,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           padd = (int64_t)bias * pb + rounding_half(pc);
         }
       }
+    };
+    load_constants(worker);
+    for (int64_t tile = worker; tile < total_tiles; tile += num_workers) {
+      const int ch0 = (int)(tile % c_tiles) * kTileChannels + (int)rank * BC + quarter * 32;   // this warp's channels
+      const int t0 = (int)(tile / c_tiles) * TOK + part * (C::kChunksPerWarp * 32);
+      const int32_t cur_pb = pb, cur_pc = pc, cur_bias = bias;
+      const int64_t cur_padd = padd;
+      load_constants(tile + num_workers);              // the next tile's, ahead of its accumulator
       if (ok) ok = ptx::mbar_wait(bar_acc_full + 8 * acc, acc_phase);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) continue;                               // keep walking the tiles, touch nothing
@@ -281,20 +288,21 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         for (int i = 0; i < 32; ++i) {
           const int32_t a = (int32_t)v[i];
           int32_t o;
-          if constexpr (KIND == EPI_RAW) o = a + bias;
+          if constexpr (KIND == EPI_RAW) o = a + cur_bias;
           else if constexpr (KIND == EPI_Q16) {
-            if constexpr (FAST) o = clamp_sym(requant_upper(a + bias, pb), 32767);
-            else o = requant_add(a, pb, padd, pc, 32767);
+            if constexpr (FAST) o = clamp_sym(requant_upper(a + cur_bias, cur_pb), 32767);
+            else o = requant_add(a, cur_pb, cur_padd, cur_pc, 32767);
           } else if constexpr (KIND == EPI_INT8) {
-            if constexpr (FAST) o = clamp_sym(requant_upper(a + bias, pb), 127);
-            else o = requant_add(a, pb, padd, pc, 127);
+            if constexpr (FAST) o = clamp_sym(requant_upper(a + cur_bias, cur_pb), 127);
+            else o = requant_add(a, cur_pb, cur_padd, cur_pc, 127);
           } else {
-            if constexpr (FAST) o = min(igelu_q16_upper(clamp_sym(requant_upper(a + bias, pb), 32767), gk), 127);
-            else o = igelu_q16_to_int8(requant_add(a, pb, padd, pc, 32767), gk, gelu_half);
+            if constexpr (FAST) o = min(igelu_q16_upper(clamp_sym(requant_upper(a + cur_bias, cur_pb), 32767), gk), 127);
+            else o = igelu_q16_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
           }
           // staging tile: row = token i, column = this lane's channel
           if constexpr (kOut32) reinterpret_cast<int32_t*>(stage)[i * 32 + lane] = o;
-          else reinterpret_cast<int8_t*>(stage)[i * 32 + lane] = (int8_t)o;
+          else  // low byte of the register, stored without a narrowing conversion
+            asm volatile("st.shared.u8 [%0], %1;" ::"r"(ptx::smem_addr(stage) + i * 32 + lane), "r"(o) : "memory");
         }
         ptx::fence_proxy_async_smem();                 // staging writes -> visible to the TMA engine
         __syncwarp();

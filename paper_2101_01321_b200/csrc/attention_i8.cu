@@ -1,9 +1,11 @@
-// Fused integer-only attention for one (batch, head, 128-query tile) per CTA:
+// Fused integer-only attention, per (batch, head) and 128-query tile:
 //   S = Q K^T (tcgen05 kind::i8, int32 accumulators in TMEM; scale S_q S_k / 8)
 //   P = i-softmax(S) (Algorithm 3: row max, i-exp, int32 row sum, fixed-point quotient) -> u8
 //   ctx = requant(P V) (u8 x s8 tcgen05 MMA, accumulator reuses the score columns)
 // Scores never leave the SM: they live in TMEM, the exponentials overwrite them in place,
 // and the probabilities go to shared memory in the layout the second MMA reads.
+// Two kernels: `attention_kernel` (the one every realistic scale takes) and
+// `attention_coarse_kernel` for score scales so coarse that the i-exp quotient needs its clamp.
 #include <cuda.h>
 
 #include <algorithm>
@@ -18,7 +20,7 @@ namespace {
 constexpr int kAttnThreads = 128;   // thread t owns query row t (= TMEM lane t)
 constexpr int kHeadDim = 64;
 
-struct AttnArgs {
+struct CoarseArgs {
   int B, L, H, heads;
   int Lp;            // L rounded up to a multiple of 32 (MMA N / K granularity)
   int n_slabs;       // ceil(L / 128)
@@ -40,12 +42,7 @@ __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t col, uin
 // pass 1 row maximum, pass 2 i-exp + int32 row sum (exponentials written back over the scores),
 // pass 3 fixed-point quotient -> u8 probabilities into the swizzled operand tile `sP`, row `row`.
 // Columns [L, Lp) are padding: excluded from max and sum, written as probability 0.
-// DIV: 0..2 = clamped division forms of iexp_dist, 3 = the 21-bit form without the clamp.
-template <int DIV>
-__device__ __forceinline__ uint32_t iexp_any(uint32_t d, const ExpConsts& ek) {
-  if constexpr (DIV == 3) return iexp_dist_wide(d, ek);
-  else return iexp_dist<DIV>(d, ek);
-}
+// DIV: the division form of iexp_dist (distance clamped to 31 q_ln2).
 
 template <int DIV>
 __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const ExpConsts& ek, uint8_t* sP,
@@ -73,13 +70,13 @@ __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const
     if (c0 < full) {
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        v[i] = iexp_any<DIV>((uint32_t)mx - v[i], ek);
+        v[i] = iexp_dist<DIV>((uint32_t)mx - v[i], ek);
         sum += v[i];
       }
     } else {
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        v[i] = (c0 + i < L) ? iexp_any<DIV>((uint32_t)mx - v[i], ek) : 0u;
+        v[i] = (c0 + i < L) ? iexp_dist<DIV>((uint32_t)mx - v[i], ek) : 0u;
         sum += v[i];
       }
     }
@@ -114,69 +111,12 @@ __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const
   }
 }
 
-// The same row function for rows of exactly 128 columns' worth of padding (96 < L <= 128), the
-// headline case: the whole score row is read from TMEM once and stays in registers through
-// maximum, i-exp, sum and quotient, so there is no write-back of exponentials and the 128
-// independent element chains can be scheduled freely.
-__device__ __forceinline__ void softmax_row_128(uint32_t t_row, int L, const ExpConsts& ek, uint8_t* sP,
-                                                uint32_t row) {
-  uint32_t v[4][32];
-#pragma unroll
-  for (int c = 0; c < 4; ++c) ptx::tmem_ld32(t_row + c * 32, v[c]);
-  ptx::tmem_wait_ld();
-  int32_t mx = INT32_MIN;
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-#pragma unroll
-    for (int i = 0; i < 32; i += 2) {
-      if (c < 3) mx = __vimax3_s32(mx, (int32_t)v[c][i], (int32_t)v[c][i + 1]);
-      else {
-        if (96 + i < L) mx = max(mx, (int32_t)v[c][i]);
-        if (96 + i + 1 < L) mx = max(mx, (int32_t)v[c][i + 1]);
-      }
-    }
-  }
-  uint32_t sum = 0;
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      const uint32_t e = iexp_dist_wide((uint32_t)mx - v[c][i], ek);
-      v[c][i] = (c < 3 || 96 + i < L) ? e : 0u;
-      sum += v[c][i];
-    }
-  }
-  const RowDivisor rd = make_row_divisor(sum, ek.p_max);
-  const bool nopre = __all_sync(0xffffffffu, rd.pre == 0);
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      uint32_t w[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int j = h * 16 + i * 4;
-        uint32_t p0, p1, p2, p3;
-        if (nopre) {
-          p0 = softmax_quotient_nopre(v[c][j], rd); p1 = softmax_quotient_nopre(v[c][j + 1], rd);
-          p2 = softmax_quotient_nopre(v[c][j + 2], rd); p3 = softmax_quotient_nopre(v[c][j + 3], rd);
-        } else {
-          p0 = softmax_quotient(v[c][j], rd); p1 = softmax_quotient(v[c][j + 1], rd);
-          p2 = softmax_quotient(v[c][j + 2], rd); p3 = softmax_quotient(v[c][j + 3], rd);
-        }
-        w[i] = ((p3 * 256u + p2) * 256u + p1) * 256u + p0;
-      }
-      *reinterpret_cast<uint4*>(sP + sw128_offset(row, (uint32_t)(c * 32 + h * 16), 128)) =
-          make_uint4(w[0], w[1], w[2], w[3]);
-    }
-  }
-}
-
 // Transposes V [j][64] (plain rows in `sVs`) into Vt [64][j] in the swizzled K-major operand
 // layout of `sVt`.  A thread takes 4 consecutive keys x 16 head dims, transposes the four 4x4 byte
 // blocks with byte permutes and writes 16 words (4 keys of one head dim each).
-__device__ __forceinline__ void transpose_v(const uint8_t* sVs, uint8_t* sVt, int n_keys, int tid) {
-  for (int item = tid; item < (n_keys / 4) * 4; item += kAttnThreads) {
+__device__ __forceinline__ void transpose_v(const uint8_t* sVs, uint8_t* sVt, int n_keys, int tid,
+                                            int n_threads = kAttnThreads) {
+  for (int item = tid; item < (n_keys / 4) * 4; item += n_threads) {
     const int jq = item % (n_keys / 4), dc = item / (n_keys / 4);     // key quad, 16-dim chunk
     uint32_t r[4][4];
 #pragma unroll
@@ -200,11 +140,13 @@ __device__ __forceinline__ void transpose_v(const uint8_t* sVs, uint8_t* sVt, in
   }
 }
 
-// Persistent CTA: walks (batch, head, query tile) work items; while one item is computed the TMA
-// loads of the next one land in the other operand stage (when `a.stages` == 2).
+// Fallback for coarse score scales (q_ln2 <= 2, where the unclamped quotient of iexp_dist_wide is
+// not available).  Persistent CTA of 128 threads, thread = query row: walks (batch, head, query
+// tile) work items; while one item is computed the TMA loads of the next one land in the other
+// operand stage (when `a.stages` == 2).
 __global__ void __launch_bounds__(kAttnThreads, 3)
-attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_constant__ CUtensorMap map_v,
-                 const AttnArgs a) {
+attention_coarse_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_constant__ CUtensorMap map_v,
+                        const CoarseArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int slab_bytes = 128 * kHeadDim;                       // 8 KB
@@ -298,9 +240,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
     if (ok) {
       ptx::tc_fence_after_sync();
       // scores are sums of 64 int8 products: |s| < 2^20, so distances from the maximum stay below 2^21
-      if (a.k.e.wide_post >= 0 && Lp == 128) softmax_row_128(t_row, L, a.k.e, sP, (uint32_t)tid);
-      else if (a.k.e.wide_post >= 0) softmax_row<3>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid);
-      else switch (exp_div_mode(a.k.e)) {
+      switch (exp_div_mode(a.k.e)) {
         case 0: softmax_row<0>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
         case 1: softmax_row<1>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
         default: softmax_row<2>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
@@ -374,21 +314,307 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The main kernel.  A persistent CTA owns one (batch, head) pair at a time and walks its 128-query
+// tiles, so K, V and the transposed V are loaded / built once per pair.  The CTA has 128 G threads,
+// G = ceil(L / 128) column groups: warp w works on TMEM lane quadrant w & 3 (the only lanes a warp
+// may address) and on the 32-column chunks of group w >> 2, so a score row is shared by G threads
+// that exchange their partial maximum and partial sum through shared memory.  Up to 128 keys that
+// is one thread per row and four CTAs per SM; at 512 keys one CTA of 16 warps fills the SM's TMEM.
+// Every operand buffer is refilled as soon as its last reader is done (V after the transpose, K
+// and a lone Q after the score MMAs), so the next pair's loads hide behind the softmax.
+// Requires the unclamped i-exp form (ExpConsts::wide_post >= 0).
+// ---------------------------------------------------------------------------------------------
+constexpr int kMaxThreads = 512;
+
+struct AttnArgs {
+  int B, L, H, heads;
+  int Lp, n_slabs, groups;
+  int q_bufs;        // 2 when a pair has several query tiles (next tile's Q prefetched), else 1
+  uint32_t tmem_cols;
+  AttnConsts k;
+  int8_t* out;
+  int32_t* status;
+};
+
+__global__ void __launch_bounds__(kMaxThreads, 1)
+attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_constant__ CUtensorMap map_v,
+                 const AttnArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int slab_bytes = 128 * kHeadDim;                       // 8 KB
+  uint8_t* sQ = smem;                                          // [q_bufs][128 rows][64 B], 64-byte swizzle
+  uint8_t* sK = sQ + a.q_bufs * slab_bytes;                    // [n_slabs][128][64 B], 64-byte swizzle
+  uint8_t* sVs = sK + a.n_slabs * slab_bytes;                  // [n_slabs][128][64 B], plain rows
+  uint8_t* sVt = sVs + a.n_slabs * slab_bytes;                 // [n_slabs][64 rows][128 B], swizzled
+  uint8_t* sP = sVt + a.n_slabs * slab_bytes;                  // [n_slabs][128 rows][128 B], swizzled
+  int32_t* s_max = reinterpret_cast<int32_t*>(sP + a.n_slabs * 128 * 128);   // [4][128]
+  uint32_t* s_sum = reinterpret_cast<uint32_t*>(s_max + 4 * 128);            // [4][128]
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_sum + 4 * 128);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 5);
+  const uint32_t bar_q0 = ptx::smem_addr(s_bar);               // two Q buffers
+  const uint32_t bar_k = bar_q0 + 16, bar_v = bar_q0 + 24, bar_mma = bar_q0 + 32;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_threads = blockDim.x;
+  const int quad = warp & 3, grp = warp >> 2, G = a.groups;
+  const int row = quad * 32 + lane;                            // query row inside the tile = TMEM lane
+  const int L = a.L, Lp = a.Lp, q_tiles = a.n_slabs;
+  const int total = a.B * a.heads;
+  const int n_chunks = Lp >> 5, per_grp = (n_chunks + G - 1) / G;
+  const int c_begin = min(grp * per_grp, n_chunks) * 32, c_end = min((grp + 1) * per_grp, n_chunks) * 32;
+
+  if (tid == 0) {
+    ptx::mbar_init(bar_q0, 1);
+    ptx::mbar_init(bar_q0 + 8, 1);
+    ptx::mbar_init(bar_k, 1);
+    ptx::mbar_init(bar_v, 1);
+    ptx::mbar_init(bar_mma, 1);
+    ptx::fence_mbar_init();
+    ptx::tma_prefetch_desc(&map_qk);
+    ptx::tma_prefetch_desc(&map_v);
+  }
+  if (warp == 0) {
+    ptx::tmem_alloc(ptx::smem_addr(s_tmem), a.tmem_cols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *s_tmem;
+  const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();              // the kernel that wrote qkv has completed
+
+  auto load_q = [&](int item, int qt, int buf) {
+    const int head = item % a.heads, batch = item / a.heads;
+    ptx::mbar_arrive_expect_tx(bar_q0 + 8 * buf, (uint32_t)slab_bytes);
+    ptx::tma_load_3d(ptx::smem_addr(sQ + buf * slab_bytes), &map_qk, bar_q0 + 8 * buf, head * kHeadDim, qt * 128, batch);
+  };
+  auto load_k = [&](int item) {
+    const int head = item % a.heads, batch = item / a.heads;
+    ptx::mbar_arrive_expect_tx(bar_k, (uint32_t)(a.n_slabs * slab_bytes));
+    for (int s = 0; s < a.n_slabs; ++s)
+      ptx::tma_load_3d(ptx::smem_addr(sK + s * slab_bytes), &map_qk, bar_k, a.H + head * kHeadDim, s * 128, batch);
+  };
+  auto load_v = [&](int item) {
+    const int head = item % a.heads, batch = item / a.heads;
+    ptx::mbar_arrive_expect_tx(bar_v, (uint32_t)(a.n_slabs * slab_bytes));
+    for (int s = 0; s < a.n_slabs; ++s)
+      ptx::tma_load_3d(ptx::smem_addr(sVs + s * slab_bytes), &map_v, bar_v, 2 * a.H + head * kHeadDim, s * 128, batch);
+  };
+
+  uint32_t q_phase[2] = {0, 0};
+  uint32_t kv_phase = 0, mma_phase = 0;
+  int qbuf = 0;
+  bool ok = true;
+  if (tid == 0 && (int)blockIdx.x < total) {
+    load_q(blockIdx.x, 0, 0);
+    load_k(blockIdx.x);
+    load_v(blockIdx.x);
+  }
+
+  for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
+    const int head = item % a.heads, batch = item / a.heads;
+    const int next = item + gridDim.x;
+
+    // ---- V [j][d] -> Vt [d][j] once per (batch, head); the plain copy is then free for the next pair
+    ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_v, kv_phase));
+    if (ok) {
+      transpose_v(sVs, sVt, a.n_slabs * 128, tid, n_threads);
+      ptx::fence_proxy_async_smem();
+    }
+    ok = __syncthreads_and(ok);
+    if (!ok) break;
+    if (tid == 0 && next < total) load_v(next);
+    ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_k, kv_phase));
+    kv_phase ^= 1;
+
+    for (int qt = 0; qt < q_tiles; ++qt) {
+      const bool last_tile = qt == q_tiles - 1;
+      if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_q0 + 8 * qbuf, q_phase[qbuf]));
+      q_phase[qbuf] ^= 1;
+
+      // ---- S = Q K^T: K = 64 bytes = two MMA K-steps; N in chunks of at most 256 columns
+      if (ok && tid == 0) {
+        ptx::tc_fence_after_sync();
+        const uint64_t dq = ptx::make_kmajor_desc(ptx::smem_addr(sQ + qbuf * slab_bytes), 512, ptx::kSwizzle64);
+        for (int n0 = 0; n0 < Lp; n0 += 256) {
+          const int nn = min(256, Lp - n0);
+          const uint32_t idesc = ptx::make_idesc_i8(128, nn, true, true);
+          const uint64_t dk = ptx::make_kmajor_desc(ptx::smem_addr(sK + n0 * kHeadDim), 512, ptx::kSwizzle64);
+          ptx::mma_i8_ss(tmem_base + n0, dq, dk, idesc, 0u);
+          ptx::mma_i8_ss(tmem_base + n0, dq + 2, dk + 2, idesc, 1u);
+        }
+        ptx::mma_commit(bar_mma);
+        // the other Q buffer was read by the previous tile's score MMAs, which have completed
+        if (a.q_bufs == 2) {
+          if (!last_tile) load_q(item, qt + 1, qbuf ^ 1);
+          else if (next < total) load_q(next, 0, qbuf ^ 1);
+        }
+      }
+      if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_mma, mma_phase));
+      mma_phase ^= 1;
+      // K is no longer read once the last tile's scores exist: fetch the next pair's K behind the softmax
+      if (ok && tid == 0 && last_tile && next < total) {
+        load_k(next);
+        if (a.q_bufs == 1) load_q(next, 0, 0);      // single tile per pair: Q is as dead as K by now
+      }
+
+      // ---- i-softmax, pass 1: maximum of this thread's columns, then of the row
+      int32_t mx = INT32_MIN;
+      if (ok) {
+        ptx::tc_fence_after_sync();
+        for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+          uint32_t v[32];
+          ptx::tmem_ld32(t_row + c0, v);
+          ptx::tmem_wait_ld();
+          if (c0 + 32 <= L) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) mx = __vimax3_s32(mx, (int32_t)v[i], (int32_t)v[i + 1]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c0 + i < L) mx = max(mx, (int32_t)v[i]);
+          }
+        }
+        s_max[grp * 128 + row] = mx;
+      }
+      __syncthreads();
+      // ---- pass 2: i-exp written back over the scores, partial sums
+      uint32_t sum = 0;
+      if (ok) {
+        for (int g = 0; g < G; ++g) mx = max(mx, s_max[g * 128 + row]);
+        for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+          uint32_t v[32];
+          ptx::tmem_ld32(t_row + c0, v);
+          ptx::tmem_wait_ld();
+          if (c0 + 32 <= L) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              v[i] = iexp_dist_wide((uint32_t)mx - v[i], a.k.e);
+              sum += v[i];
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              v[i] = (c0 + i < L) ? iexp_dist_wide((uint32_t)mx - v[i], a.k.e) : 0u;
+              sum += v[i];
+            }
+          }
+          ptx::tmem_st32(t_row + c0, v);
+        }
+        ptx::tmem_wait_st();
+        s_sum[grp * 128 + row] = sum;
+      }
+      __syncthreads();
+      // ---- pass 3: u8 probabilities into the operand tile of the second MMA
+      if (ok) {
+        sum = 0;
+        for (int g = 0; g < G; ++g) sum += s_sum[g * 128 + row];
+        const RowDivisor rd = make_row_divisor(sum, a.k.e.p_max);
+        const bool nopre = __all_sync(0xffffffffu, rd.pre == 0);
+        for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+          uint32_t v[32];
+          ptx::tmem_ld32(t_row + c0, v);
+          ptx::tmem_wait_ld();
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int j = h * 16 + i * 4;
+              uint32_t p0, p1, p2, p3;
+              if (nopre) {
+                p0 = softmax_quotient_nopre(v[j], rd); p1 = softmax_quotient_nopre(v[j + 1], rd);
+                p2 = softmax_quotient_nopre(v[j + 2], rd); p3 = softmax_quotient_nopre(v[j + 3], rd);
+              } else {
+                p0 = softmax_quotient(v[j], rd); p1 = softmax_quotient(v[j + 1], rd);
+                p2 = softmax_quotient(v[j + 2], rd); p3 = softmax_quotient(v[j + 3], rd);
+              }
+              w[i] = ((p3 * 256u + p2) * 256u + p1) * 256u + p0;
+            }
+            *reinterpret_cast<uint4*>(sP + sw128_offset((uint32_t)row, (uint32_t)(c0 + h * 16), 128)) =
+                make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+        ptx::fence_proxy_async_smem();
+      }
+      ptx::tc_fence_before_sync();
+      ok = __syncthreads_and(ok);             // P complete; every row's exponentials have been consumed
+      if (!ok) break;
+
+      // ---- ctx = P V: K = Lp in steps of 32, accumulator in columns 0..63 (scores are dead)
+      if (tid == 0) {
+        ptx::tc_fence_after_sync();
+        const uint32_t idesc = ptx::make_idesc_i8(128, kHeadDim, false, true);   // u8 x s8
+        for (int kk = 0; kk < Lp / 32; ++kk) {
+          const int kb = kk >> 2, ks = kk & 3;
+          const uint64_t dp = ptx::make_kmajor_desc(ptx::smem_addr(sP + kb * 128 * 128), 1024, ptx::kSwizzle128);
+          const uint64_t dv = ptx::make_kmajor_desc(ptx::smem_addr(sVt + kb * 64 * 128), 1024, ptx::kSwizzle128);
+          ptx::mma_i8_ss(tmem_base, dp + 2 * ks, dv + 2 * ks, idesc, kk != 0 ? 1u : 0u);
+        }
+        ptx::mma_commit(bar_mma);
+      }
+      ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_mma, mma_phase));
+      mma_phase ^= 1;
+
+      // ---- epilogue: the 64 context values of a row in two halves, taken by column groups 0 and 1
+      // (by group 0 alone when there is only one)
+      if (ok && grp < 2) {
+        ptx::tc_fence_after_sync();
+        const int64_t half = rounding_half(a.k.c);
+        const int q_row = qt * 128 + row;
+        for (int part = grp; part < 2; part += G) {
+          int8_t* orow = a.out + ((int64_t)batch * L + q_row) * a.H + head * kHeadDim + part * 32;
+          uint32_t v[32];
+          ptx::tmem_ld32(t_row + part * 32, v);
+          ptx::tmem_wait_ld();
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int j = h * 16 + i * 4;
+              if (a.k.fast) {
+                w[i] = pack4_sat_s8(max(requant_upper((int32_t)v[j], a.k.b2), -127),
+                                    max(requant_upper((int32_t)v[j + 1], a.k.b2), -127),
+                                    max(requant_upper((int32_t)v[j + 2], a.k.b2), -127),
+                                    max(requant_upper((int32_t)v[j + 3], a.k.b2), -127));
+              } else {
+                w[i] = pack4_sat_s8(requant_add((int32_t)v[j], a.k.b, half, a.k.c, 127),
+                                    requant_add((int32_t)v[j + 1], a.k.b, half, a.k.c, 127),
+                                    requant_add((int32_t)v[j + 2], a.k.b, half, a.k.c, 127),
+                                    requant_add((int32_t)v[j + 3], a.k.b, half, a.k.c, 127));
+              }
+            }
+            if (q_row < L) *reinterpret_cast<uint4*>(orow + h * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      ptx::tc_fence_before_sync();
+      ok = __syncthreads_and(ok);             // TMEM columns and P are free for the next tile
+      if (!ok) break;
+      if (a.q_bufs == 2) qbuf ^= 1;
+    }
+  }
+  if (!ok) atomicCAS(a.status, 0, IBERT_ERR_TIMEOUT);
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, a.tmem_cols);
+  }
+}
+
 }  // namespace
 
 int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
                      const AttnConsts& k, int8_t* out) {
   if (B == 0) return IBERT_OK;
-  AttnArgs a{};
-  a.B = B; a.L = L; a.H = H; a.heads = heads;
-  a.Lp = (L + 31) & ~31;
-  a.n_slabs = (L + 127) / 128;
+  const int Lp = (L + 31) & ~31, n_slabs = (L + 127) / 128;
   uint32_t cols = 64;
-  while ((int)cols < a.Lp) cols <<= 1;
-  a.tmem_cols = cols;
-  a.k = k;
-  a.out = out;
-  a.status = ctx->d_status;
+  while ((int)cols < Lp) cols <<= 1;
   CUtensorMap mqk, mv;
   const uint64_t dims[3] = {(uint64_t)3 * H, (uint64_t)L, (uint64_t)B};
   const uint64_t str[2] = {(uint64_t)3 * H, (uint64_t)3 * H * L};
@@ -397,23 +623,53 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
   if (rc) return rc;
   rc = encode_tensor_map(&mv, qkv, 3, dims, str, box, 0);
   if (rc) return rc;
-  const int stage_bytes = (1 + 2 * a.n_slabs) * 128 * kHeadDim;
-  const int fixed_bytes = a.n_slabs * 128 * kHeadDim + a.n_slabs * 128 * 128 + 64 + 1024;
+  const int slab = 128 * kHeadDim;
+
+  if (k.e.wide_post >= 0) {
+    AttnArgs a{};
+    a.B = B; a.L = L; a.H = H; a.heads = heads;
+    a.Lp = Lp; a.n_slabs = n_slabs; a.groups = n_slabs;
+    a.q_bufs = n_slabs > 1 ? 2 : 1;
+    a.tmem_cols = cols; a.k = k; a.out = out; a.status = ctx->d_status;
+    const int smem = a.q_bufs * slab + 3 * n_slabs * slab + n_slabs * 128 * 128 + 2 * 4 * 128 * 4 + 64 + 1024;
+    // resident CTAs per SM: bounded by the register file (128 G threads of at most 128 registers),
+    // by the 512 TMEM columns and by shared memory.  The bound must not exceed what TMEM allows:
+    // a CTA that cannot get its columns would wait for a resident one to finish.
+    int per_sm = std::min(std::min(4 / a.groups, (int)(512 / cols)), (227 * 1024) / (smem + 1024));
+    if (per_sm < 1) per_sm = 1;
+    const int grid = std::min(B * heads, ctx->num_sms * per_sm);
+    static int smem_set = 0;
+    if (smem > smem_set) {
+      if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return IBERT_ERR_CUDA;
+      smem_set = smem;
+    }
+    if (int rc2 = launch_pdl(attention_kernel, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1,
+                             mqk, mv, a)) return rc2;
+    return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
+  }
+
+  // scales too coarse for the unclamped division (q_ln2 <= 2): the plain one-tile-per-item kernel
+  CoarseArgs a{};
+  a.B = B; a.L = L; a.H = H; a.heads = heads;
+  a.Lp = Lp; a.n_slabs = n_slabs;
+  a.tmem_cols = cols; a.k = k; a.out = out; a.status = ctx->d_status;
+  const int stage_bytes = (1 + 2 * n_slabs) * slab;
+  const int fixed_bytes = n_slabs * slab + n_slabs * 128 * 128 + 64 + 1024;
   a.stages = (2 * stage_bytes + fixed_bytes <= 112 * 1024) ? 2 : 1;     // keep at least 2 CTAs per SM
   const int smem = a.stages * stage_bytes + fixed_bytes;
   static int smem_set = 0;
   if (smem > smem_set) {
-    if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(attention_coarse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return IBERT_ERR_CUDA;
     smem_set = smem;
   }
-  const int total = B * heads * a.n_slabs;
-  // resident CTAs per SM: limited by TMEM columns (512), shared memory and the register budget (3)
+  const int total = B * heads * n_slabs;
   int per_sm = std::min(3, std::min((int)(512 / cols), (227 * 1024) / (smem + 1024)));
   if (per_sm < 1) per_sm = 1;
   const int grid = std::min(total, ctx->num_sms * per_sm);
-  if (int rc = launch_pdl(attention_kernel, dim3(grid), dim3(kAttnThreads), (size_t)smem, ctx->stream, 1, mqk, mv, a))
-    return rc;
+  if (int rc2 = launch_pdl(attention_coarse_kernel, dim3(grid), dim3(kAttnThreads), (size_t)smem, ctx->stream, 1,
+                           mqk, mv, a)) return rc2;
   return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
 }
 

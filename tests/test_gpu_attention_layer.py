@@ -11,7 +11,8 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("B,L,heads", [(1, 16, 1), (2, 37, 2), (1, 128, 12), (3, 128, 2), (2, 200, 2), (1, 256, 3),
-                                       (1, 512, 2), (2, 1, 1), (1, 33, 1), (1, 300, 1), (0, 64, 1)])
+                                       (1, 512, 2), (2, 1, 1), (1, 33, 1), (1, 300, 1), (0, 64, 1), (1, 130, 1), (1, 384, 2),
+                                       (2, 480, 1), (40, 160, 8), (20, 290, 8)])
 @pytest.mark.parametrize("p_max", [255, 127])
 def test_attention_matches_oracle(B, L, heads, p_max):
     H = heads * 64
@@ -38,6 +39,22 @@ def test_attention_peaked_and_uniform_rows():
         out, _ = ctx().ibert_attention_i8(dev(qkv), B, L, H, heads, S_qk, S_qk, 0.02, 0.01, 255)
         want = oracle.attention(qkv, B, L, H, heads, S_qk, S_qk, 0.02, 0.01, 255)
         assert_same(host(out), want, "attention peaked")
+    ctx().check()
+
+
+@pytest.mark.parametrize("L", [100, 200])
+@pytest.mark.parametrize("S_qk", [1.5, 2.0])
+def test_attention_coarse_score_scale(L, S_qk):
+    """Score scales so coarse that q_ln2 <= 2: the kernel with the clamped i-exp quotient runs."""
+    B, heads = 2, 2
+    H = heads * 64
+    rng = np.random.default_rng(L)
+    qkv = rng.integers(-3, 4, (B * L, 3 * H)).astype(np.int8)
+    qkv[:, 2 * H:] = rng.integers(-127, 128, (B * L, H))
+    out, _ = ctx().ibert_attention_i8(dev(qkv), B, L, H, heads, S_qk, S_qk, 0.02, 0.01, 255)
+    want = oracle.attention(qkv, B, L, H, heads, S_qk, S_qk, 0.02, 0.01, 255)
+    assert_same(host(out), want, f"attention coarse L={L}")
+    assert np.abs(want).max() > 5
     ctx().check()
 
 

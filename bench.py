@@ -109,6 +109,9 @@ def algorithmic_work(H: int, F: int, L: int, heads: int, T: int) -> dict:
     w["layernorm"] = {"ops": 0.0, "bytes": 4 * T * H + T * H + T * H}
     w["gemm_ffn1_gelu"] = {"ops": 2.0 * T * F * H, "bytes": T * H + F * H + T * F}
     w["gemm_ffn2"] = {"ops": 2.0 * T * F * H, "bytes": T * F + F * H + 4 * T * H}
+    # linear + residual + LayerNorm in one kernel: operands, int8 residual in, int8 out
+    w["gemm_out_ln"] = {"ops": 2.0 * T * H * H, "bytes": T * H + H * H + T * H + T * H}
+    w["gemm_ffn2_ln"] = {"ops": 2.0 * T * F * H, "bytes": T * F + F * H + T * H + T * H}
     return w
 
 
@@ -325,7 +328,7 @@ def run_ours(args):
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": T * cfg.H,
                     "d2h_bytes_per_step": T * cfg.H, "ms_per_step": total_e2e_ms / args.steps},
-            "gpu_launches": 7 * cfg.layers * args.steps,
+            "gpu_launches": sum(v["launches_per_step"] for v in kern.values()) * args.steps,
             "roofline": roof,
             "kernels": kern,
             "cpu_baseline": cpu,
@@ -361,7 +364,18 @@ def run_only(args):
     p = synth.static_activation_scales(H, F, L, 0.035)
     rng = np.random.default_rng(synth.SEED_BASE)
     k = args.only
-    if k.startswith("gemm"):
+    if k in ("gemm_out_ln", "gemm_ffn2_ln"):
+        N, K = (H, H) if k == "gemm_out_ln" else (H, F)
+        x, w, res = i8(T, K), i8(N, K), i8(T, N)
+        bias = torch.randint(-1000, 1000, (N,), generator=g, dtype=torch.int32).to(dev)
+        S_w = rng.uniform(5e-4, 7e-4, N)
+        S_x = 0.03
+        S_acc = S_x * 6e-4 * 127 * 127 * np.sqrt(K)
+        gamma, beta = 1.0 + 0.1 * rng.standard_normal(N), 0.1 * rng.standard_normal(N)
+        out = torch.empty((T, N), dtype=torch.int8, device=dev)
+        fn = lambda: ctx.ibert_linear_layernorm_i8(x, S_x, w, S_w, bias, 8 * S_acc / 32767, res, S_acc / 127,
+                                                   gamma, beta, 4.5 / 127, out=out)
+    elif k.startswith("gemm"):
         N, K = {"gemm_qkv": (3 * H, H), "gemm_out": (H, H), "gemm_ffn1_gelu": (F, H), "gemm_ffn2": (H, F)}[k]
         x, w = i8(T, K), i8(N, K)
         bias = torch.randint(-1000, 1000, (N,), generator=g, dtype=torch.int32).to(dev)

@@ -148,6 +148,22 @@ typedef struct ibert_layer_desc {
 int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* desc, ibert_layer** out);
 int ibert_layer_destroy(ibert_layer* layer);
 
+/* Linear layer, residual addition and i-LayerNorm as one operation -- the tail of both halves of
+   the encoder layer (Fig. 1 right; Sec. 3.6, Eq. 16 on top of the integer linear layer):
+     out = i-LayerNorm( requant_Q16(x w^T + bias, S_mid) + rescale(res, S_res -> S_mid) ; gamma, beta, S_out )
+   x: device int8 [M, K]; w: device int8 [N, K] with host scales S_w[N]; bias: device int32 [N] at
+   scale S_x*S_w[n], or NULL; res: device int8 [M, N] at host scale S_res; gamma, beta: host
+   double [N]; out: device int8 [M, N] at S_out (*S_ret).  The result is bit-identical to
+   ibert_linear_i8(kind 1, S_mid) followed by ibert_layernorm_i.  When N is a multiple of 256 (at
+   most 2048) and the constants fit the 32-bit forms, a single kernel computes it on a cluster of
+   N/256 CTAs per 128-row tile and the Q16 tensor never reaches memory; otherwise the two kernels
+   run back to back through the context's workspace.
+   Errors: as ibert_linear_i8 and ibert_layernorm_i. */
+int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
+                              const int32_t* bias, int64_t M, int N, int K, double S_mid,
+                              const int8_t* res, double S_res, const double* gamma, const double* beta,
+                              double S_out, int8_t* out, double* S_ret);
+
 /* The integer-only encoder layer (Fig. 1 right; post-LN order):
    QKV projection -> attention (i-softmax) -> output projection -> +x, i-LayerNorm ->
    FFN1 + i-GELU -> FFN2 -> +h1, i-LayerNorm.  x, out: int8 [B*L, H]; x at desc.S_x,
@@ -169,7 +185,9 @@ enum {
   IBERT_K_GEMM_Q16_WIDE = 5, /* Q16 / raw epilogue with K > 2048: FFN2 */
   IBERT_K_GELU = 6,
   IBERT_K_SOFTMAX = 7,
-  IBERT_NUM_KERNEL_CLASSES = 8
+  IBERT_K_GEMM_LN = 8,       /* linear + residual + i-LayerNorm in one kernel, K <= 2048: output projection */
+  IBERT_K_GEMM_LN_WIDE = 9,  /* the same with K > 2048: FFN2 */
+  IBERT_NUM_KERNEL_CLASSES = 10
 };
 /* Host, pure.  Self-check of the constants derived from a score scale S for i-exp (Algorithm 3):
    verifies on the host, for every distance d in [0, 31*q_ln2] (and, for the unclamped form the

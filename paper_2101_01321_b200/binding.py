@@ -20,7 +20,7 @@ ERR_NAMES = {-1: "IBERT_ERR_ARG", -2: "IBERT_ERR_SHAPE", -3: "IBERT_ERR_SCALE_RA
              -5: "IBERT_ERR_NOMEM", -6: "IBERT_ERR_CUDA", -7: "IBERT_ERR_TIMEOUT", -8: "IBERT_ERR_VALUE_RANGE"}
 
 KERNEL_CLASSES = ("gemm_qkv", "attention", "gemm_out", "layernorm", "gemm_ffn1_gelu", "gemm_ffn2", "gelu",
-                  "softmax")
+                  "softmax", "gemm_out_ln", "gemm_ffn2_ln")
 SCALE_NAMES = ("S_x", "S_q", "S_k", "S_v", "S_ctx", "S_r1", "S_h1", "S_gi", "S_go", "S_r2", "S_out")
 
 
@@ -56,6 +56,8 @@ def lib():
         L.ibert_dyadic_from_double.argtypes = [dbl, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.ibert_linear_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, i32, dbl, vp, vp]
         L.ibert_linear_gelu_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, dbl, vp, vp]
+        L.ibert_linear_layernorm_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, vp, dbl, vp, vp, dbl,
+                                                vp, vp]
         L.ibert_softmax_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
         L.ibert_gelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
         L.ibert_layernorm_i.argtypes = [vp, vp, dbl, vp, dbl, vp, vp, i64, i32, dbl, vp, vp]
@@ -72,7 +74,7 @@ def lib():
         L.ibert_profile_begin.restype = i32
         L.ibert_profile_end.restype = i32
         for name in ("ibert_create", "ibert_destroy", "ibert_last_status", "ibert_dyadic_from_double",
-                     "ibert_linear_i8", "ibert_linear_gelu_i8", "ibert_softmax_i", "ibert_gelu_i",
+                     "ibert_linear_i8", "ibert_linear_gelu_i8", "ibert_linear_layernorm_i8", "ibert_softmax_i", "ibert_gelu_i",
                      "ibert_layernorm_i", "ibert_attention_i8", "ibert_layer_create", "ibert_layer_destroy",
                      "ibert_encoder_layer"):
             getattr(L, name).restype = i32
@@ -206,6 +208,26 @@ class Context:
                                    _dev(bias, torch.int32), M, N, K, out_kind, S_out, out.data_ptr(),
                                    S_ret.ctypes.data), "ibert_linear_i8")
         return out, (S_ret if out_kind == 2 else float(S_ret[0]))
+
+    def ibert_linear_layernorm_i8(self, x: torch.Tensor, S_x: float, w: torch.Tensor, S_w,
+                                  bias: torch.Tensor | None, S_mid: float, res: torch.Tensor, S_res: float,
+                                  gamma, beta, S_out: float, out: torch.Tensor | None = None):
+        """Linear layer (Q16 at S_mid) + residual + i-LayerNorm as one call."""
+        K = x.shape[-1]
+        M = x.numel() // K
+        N = w.shape[0]
+        assert w.shape[1] == K and res.numel() == M * N
+        sw = _host(S_w, np.float64)
+        g, b = _host(gamma, np.float64), _host(beta, np.float64)
+        assert sw.size == N and g.size == N and b.size == N
+        if out is None:
+            out = torch.empty(x.shape[:-1] + (N,), dtype=torch.int8, device=x.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_linear_layernorm_i8(self.h, _dev(x, torch.int8), S_x, _dev(w, torch.int8), sw.ctypes.data,
+                                             _dev(bias, torch.int32), M, N, K, S_mid, _dev(res, torch.int8), S_res,
+                                             g.ctypes.data, b.ctypes.data, S_out, _dev(out, torch.int8),
+                                             C.byref(S_ret)), "ibert_linear_layernorm_i8")
+        return out, S_ret.value
 
     def ibert_linear_gelu_i8(self, x: torch.Tensor, S_x: float, w: torch.Tensor, S_w, bias: torch.Tensor | None,
                              S_mid: float, S_out: float, out: torch.Tensor | None = None):

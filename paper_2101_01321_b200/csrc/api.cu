@@ -289,6 +289,70 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
   return rc;
 }
 
+// grows the context's workspace to at least `need` bytes (stream-synchronizing reallocation)
+static int ensure_workspace(ibert_ctx* ctx, size_t need) {
+  if (need <= ctx->ws_bytes) return IBERT_OK;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+  if (ctx->ws) cudaFree(ctx->ws);
+  ctx->ws = nullptr;
+  ctx->ws_bytes = 0;
+  if (cudaMalloc(&ctx->ws, need) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_NOMEM; }
+  ctx->ws_bytes = need;
+  return IBERT_OK;
+}
+
+int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
+                              const int32_t* bias, int64_t M, int N, int K, double S_mid,
+                              const int8_t* res, double S_res, const double* gamma, const double* beta,
+                              double S_out, int8_t* out, double* S_ret) {
+  if (!ctx || M < 0 || !S_w || !gamma || !beta || !w) return IBERT_ERR_ARG;
+  if (N < 1 || N > 2047 || K < 1 || K % 16 != 0 || N % 16 != 0) return IBERT_ERR_SHAPE;
+  if ((int64_t)K * 127 * 127 >= (int64_t(1) << 31)) return IBERT_ERR_SHAPE;
+  if (M > 0 && (!x || !out || !res)) return IBERT_ERR_ARG;
+  if (!aligned16(x) || !aligned16(w) || !aligned16(out) || !aligned16(res) || (bias && !aligned16(bias)))
+    return IBERT_ERR_ALIGN;
+  if (!good_scale(S_x) || !good_scale(S_mid) || !good_scale(S_out)) return IBERT_ERR_SCALE_RANGE;
+  for (int n = 0; n < N; ++n)
+    if (!good_scale(S_w[n])) return IBERT_ERR_SCALE_RANGE;
+  GemmEpilogue epi{};
+  epi.kind = EPI_Q16;
+  epi.d_bias = bias;
+  std::vector<int32_t> b, c;
+  int rc = make_linear_tables(S_x, S_w, N, nullptr, S_mid, &b, &c);
+  if (rc) return rc;
+  epi.fast = to_upper_word_form(&b, c) ? 1 : 0;
+  LnConsts k{};
+  k.C = N;
+  k.has_res = 1;
+  rc = make_ln_residual(S_res, S_mid, &k);
+  if (rc) return rc;
+  std::vector<int32_t> b_i;
+  std::vector<int64_t> B_i;
+  rc = make_ln_tables(gamma, beta, N, S_out, &k, &b_i, &B_i);
+  if (rc) return rc;
+  DeviceGuard guard(ctx->device);
+  void *d_b = nullptr, *d_c = nullptr, *d_bi = nullptr, *d_Bi = nullptr;
+  if ((rc = cached_upload(ctx, b.data(), b.size() * sizeof(int32_t), 21, &d_b))) return rc;
+  if ((rc = cached_upload(ctx, c.data(), c.size() * sizeof(int32_t), 22, &d_c))) return rc;
+  if ((rc = cached_upload(ctx, b_i.data(), b_i.size() * sizeof(int32_t), 11, &d_bi))) return rc;
+  if ((rc = cached_upload(ctx, B_i.data(), B_i.size() * sizeof(int64_t), 12, &d_Bi))) return rc;
+  epi.d_b = (const int32_t*)d_b;
+  epi.d_c = (const int32_t*)d_c;
+  if (gemm_ln_supported(N, K, epi, k)) {
+    ProfileScope ps(ctx, K > 2048 ? IBERT_K_GEMM_LN_WIDE : IBERT_K_GEMM_LN);
+    rc = launch_gemm_ln_i8(ctx, x, w, M, N, K, epi, res, k, (const int32_t*)d_bi, (const int64_t*)d_Bi, out);
+  } else {
+    if ((rc = ensure_workspace(ctx, (size_t)M * N * 4 + 256))) return rc;
+    int32_t* mid = static_cast<int32_t*>(ctx->ws);
+    { ProfileScope ps(ctx, gemm_class(EPI_Q16, K)); rc = launch_gemm_i8(ctx, x, w, M, N, K, epi, mid); }
+    if (rc) return rc;
+    ProfileScope ps(ctx, IBERT_K_LAYERNORM);
+    rc = launch_layernorm(ctx, mid, res, M, k, (const int32_t*)d_bi, (const int64_t*)d_Bi, out);
+  }
+  if (rc == IBERT_OK && S_ret) *S_ret = S_out;
+  return rc;
+}
+
 int ibert_linear_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
                     const int32_t* bias, int64_t M, int N, int K, int out_kind, double S_out,
                     void* out, double* S_ret) {
@@ -444,14 +508,7 @@ int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, 
   const size_t o_h1 = o_r + up256((size_t)T * H * 4);
   const size_t o_g = o_h1 + up256((size_t)T * H);
   const size_t need = o_g + up256((size_t)T * F);
-  if (need > ctx->ws_bytes) {
-    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
-    if (ctx->ws) cudaFree(ctx->ws);
-    ctx->ws = nullptr;
-    ctx->ws_bytes = 0;
-    if (cudaMalloc(&ctx->ws, need) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_NOMEM; }
-    ctx->ws_bytes = need;
-  }
+  if (int rcw = ensure_workspace(ctx, need)) return rcw;
   char* ws = static_cast<char*>(ctx->ws);
   int8_t* qkv = (int8_t*)(ws + o_qkv);
   int8_t* cx = (int8_t*)(ws + o_ctx);
@@ -466,15 +523,25 @@ int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, 
   if (rc) return rc;
   { ProfileScope ps(ctx, IBERT_K_ATTENTION); rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, cx); }
   if (rc) return rc;
+  // output projection + residual + LayerNorm: one kernel when shapes and constants allow it
   e.kind = EPI_Q16; e.d_b = ly->b_o; e.d_c = ly->c_o; e.d_bias = ly->bias_o; e.fast = ly->fast_o;
-  { ProfileScope ps(ctx, IBERT_K_GEMM_Q16); rc = launch_gemm_i8(ctx, cx, ly->w_o, T, H, H, e, r); }
-  if (rc) return rc;
-  { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm(ctx, r, x, T, ly->ln1, ly->ln1_b, ly->ln1_B, h1); }
+  if (gemm_ln_supported(H, H, e, ly->ln1)) {
+    ProfileScope ps(ctx, IBERT_K_GEMM_LN);
+    rc = launch_gemm_ln_i8(ctx, cx, ly->w_o, T, H, H, e, x, ly->ln1, ly->ln1_b, ly->ln1_B, h1);
+  } else {
+    { ProfileScope ps(ctx, IBERT_K_GEMM_Q16); rc = launch_gemm_i8(ctx, cx, ly->w_o, T, H, H, e, r); }
+    if (rc) return rc;
+    { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm(ctx, r, x, T, ly->ln1, ly->ln1_b, ly->ln1_B, h1); }
+  }
   if (rc) return rc;
   e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu; e.fast = ly->fast_f1;
   { ProfileScope ps(ctx, IBERT_K_GEMM_GELU); rc = launch_gemm_i8(ctx, h1, ly->w_f1, T, F, H, e, g); }
   if (rc) return rc;
   e.kind = EPI_Q16; e.d_b = ly->b_f2; e.d_c = ly->c_f2; e.d_bias = ly->bias_f2; e.fast = ly->fast_f2;
+  if (gemm_ln_supported(H, F, e, ly->ln2)) {
+    ProfileScope ps(ctx, F > 2048 ? IBERT_K_GEMM_LN_WIDE : IBERT_K_GEMM_LN);
+    return launch_gemm_ln_i8(ctx, g, ly->w_f2, T, H, F, e, h1, ly->ln2, ly->ln2_b, ly->ln2_B, out);
+  }
   { ProfileScope ps(ctx, IBERT_K_GEMM_Q16_WIDE); rc = launch_gemm_i8(ctx, g, ly->w_f2, T, H, F, e, r); }
   if (rc) return rc;
   { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm(ctx, r, h1, T, ly->ln2, ly->ln2_b, ly->ln2_B, out); }

@@ -164,6 +164,14 @@ struct AttnConsts {
   int32_t b2, fast;        // upper-word form: (v * b2 + 2^31) >> 32 with b2 = b << (32 - c)
 };
 
+// GEMM + residual + i-LayerNorm in one kernel (cluster of H / 256 CTAs per 128-token tile):
+// out = LN(requant_Q16(x w^T + bias) + rescale(res)).  `gemm_ln_supported` tells whether the
+// shapes and constants allow it; otherwise run launch_gemm_i8 (Q16) followed by launch_layernorm.
+bool gemm_ln_supported(int H, int K, const GemmEpilogue& epi, const LnConsts& ln);
+int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t T, int H, int K,
+                      const GemmEpilogue& epi, const int8_t* res, const LnConsts& ln, const int32_t* d_b_i,
+                      const int64_t* d_B_i, int8_t* out);
+
 int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
                      const AttnConsts& k, int8_t* out);
 

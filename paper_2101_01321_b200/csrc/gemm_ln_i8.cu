@@ -376,31 +376,31 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         s_flag[it & 1u] = (tile_of(it + 1) < t_tiles &&
                            ptx::mbar_test_now(bar_acc_full + 8 * ((it + 1) & 1u), ((it + 1) >> 1) & 1u)) ? 1 : 0;
     };
+    // One loop body for every schedule (so pass A and pass B are instantiated once -- the
+    // instruction cache matters here).  Iteration `it` finishes tile `it`; its two steps are
+    //   step 0: statistics of tile it, [pass A of tile it + 1 if it may run early], pass B of tile it
+    //   step 1: pass A of tile it + 1 if it did not run early
+    // and iteration -1 only runs pass A of tile 0.  After every pass A: decision for that tile,
+    // barrier (sums complete, decision and statistics visible), exchange.
     if (tile_of(0) < t_tiles) {
       if (lane == 0) issue_res(0);
-      pass_a(0);
-      decide(0);
-      ptx::named_bar_sync(1, kEpiThreads);             // sums of tile 0 complete, decision visible
-      exchange(0);
-      for (uint32_t it = 0;; ++it) {
-        // invariant: pass A of tile `it` is done, its sums are on their way, decision `it` is visible
-        if (s_flag[it & 1u] != 0) {
-          params(it);                                  // warps 4..7 first; they join pass A late
-          pass_a(it + 1);
-          decide(it + 1);
-          ptx::named_bar_sync(1, kEpiThreads);
-          exchange(it + 1);
-          pass_b(it);
-        } else {
-          params(it);
-          ptx::named_bar_sync(1, kEpiThreads);
-          pass_b(it);
-          if (tile_of(it + 1) >= t_tiles) break;
-          pass_a(it + 1);
-          decide(it + 1);
-          ptx::named_bar_sync(1, kEpiThreads);
-          exchange(it + 1);
+      for (int it = -1;; ++it) {
+        const bool has_next = tile_of((uint32_t)(it + 1)) < t_tiles;
+        const bool early = it >= 0 && s_flag[it & 1] != 0;
+#pragma unroll 1
+        for (int step = 0; step < 2; ++step) {
+          const bool finish = step == 0 && it >= 0;
+          const bool do_a = step == 0 ? early : (!early && has_next);
+          if (finish) params((uint32_t)it);
+          if (do_a) {
+            pass_a((uint32_t)(it + 1));
+            decide((uint32_t)(it + 1));
+          }
+          if (finish || do_a) ptx::named_bar_sync(1, kEpiThreads);
+          if (do_a) exchange((uint32_t)(it + 1));
+          if (finish) pass_b((uint32_t)it);
         }
+        if (!has_next) break;
       }
     }
     if (lane == 0) ptx::bulk_wait<0>();

@@ -195,14 +195,22 @@ def linear(x, S_x: float, w, S_w, bias, out_kind: int, S_out: float = 0.0, S_out
 
 # ------------------------------------------------------------------ attention
 def attention(qkv, B: int, L: int, H: int, heads: int, S_q: float, S_k: float, S_v: float,
-              S_ctx: float, p_max: int = 255, want_probs: bool = False):
+              S_ctx: float, p_max: int = 255, want_probs: bool = False, lens=None):
+    """``lens`` (optional, [B] int32): valid keys per sequence (key-padding mask)."""
     qkv = _arr(qkv, np.int8)
     assert qkv.size == B * L * 3 * H
     ctx = np.empty((B * L, H), dtype=np.int8)
     probs = np.empty((B, heads, L, L), dtype=np.uint8) if want_probs else None
-    _chk(lib().orc_attention(_p(qkv), C.c_int(B), C.c_int(L), C.c_int(H), C.c_int(heads),
-                             C.c_double(S_q), C.c_double(S_k), C.c_double(S_v), C.c_double(S_ctx),
-                             C.c_int(p_max), _p(ctx), _p(probs)), "attention")
+    if lens is None:
+        _chk(lib().orc_attention(_p(qkv), C.c_int(B), C.c_int(L), C.c_int(H), C.c_int(heads),
+                                 C.c_double(S_q), C.c_double(S_k), C.c_double(S_v), C.c_double(S_ctx),
+                                 C.c_int(p_max), _p(ctx), _p(probs)), "attention")
+    else:
+        lens = _arr(lens, np.int32)
+        assert lens.size == B
+        _chk(lib().orc_attention_masked(_p(qkv), C.c_int(B), C.c_int(L), C.c_int(H), C.c_int(heads), _p(lens),
+                                        C.c_double(S_q), C.c_double(S_k), C.c_double(S_v), C.c_double(S_ctx),
+                                        C.c_int(p_max), _p(ctx), _p(probs)), "attention_masked")
     return (ctx, probs) if want_probs else ctx
 
 
@@ -230,7 +238,7 @@ class LayerResult:
     taps: dict
 
 
-def encoder_layer(params: dict, x, B: int, L: int, want_taps: bool = False) -> LayerResult:
+def encoder_layer(params: dict, x, B: int, L: int, want_taps: bool = False, lens=None) -> LayerResult:
     """``params``: the dictionary a synthetic-layer generator produces (int8 weights,
     per-channel weight scales, int32 biases, gamma/beta, the 11 activation scales)."""
     H, F = int(params["H"]), int(params["F"])
@@ -265,6 +273,45 @@ def encoder_layer(params: dict, x, B: int, L: int, want_taps: bool = False) -> L
         for k, v in taps.items():
             setattr(t, k, v.ctypes.data)
         tp = C.byref(t)
-    _chk(lib().orc_encoder_layer(C.byref(d), _p(x), C.c_int(B), C.c_int(L), _p(out), tp),
-         "encoder_layer")
+    if lens is None:
+        _chk(lib().orc_encoder_layer(C.byref(d), _p(x), C.c_int(B), C.c_int(L), _p(out), tp),
+             "encoder_layer")
+    else:
+        lens = _arr(lens, np.int32)
+        assert lens.size == B
+        _chk(lib().orc_encoder_layer_masked(C.byref(d), _p(x), C.c_int(B), C.c_int(L), _p(lens), _p(out), tp),
+             "encoder_layer_masked")
     return LayerResult(out=out, taps=taps)
+
+
+# ------------------------------------------------------------------ around the layers
+def embedding(ids, L: int, word, S_word: float, pos, S_pos: float, gamma, beta, S_out: float) -> np.ndarray:
+    """INT8 word + position embedding followed by i-LayerNorm; token t uses position t mod L."""
+    ids = _arr(ids, np.int32)
+    word = _arr(word, np.int8)
+    pos = _arr(pos, np.int8)
+    V, H = word.shape
+    P = pos.shape[0]
+    assert pos.shape[1] == H
+    gamma = _arr(gamma, np.float64)
+    beta = _arr(beta, np.float64)
+    T = ids.size
+    out = np.empty((T, H), dtype=np.int8)
+    _chk(lib().orc_embedding(_p(ids), C.c_int64(T), C.c_int(L), _p(word), C.c_int64(V), C.c_double(S_word),
+                             _p(pos), C.c_int64(P), C.c_double(S_pos), _p(gamma), _p(beta), C.c_int(H),
+                             C.c_double(S_out), _p(out)), "embedding")
+    return out
+
+
+def classifier(x, B: int, L: int, S_x: float, w, S_w, bias) -> np.ndarray:
+    """Raw INT32 logits of a linear head on the first token of every sequence."""
+    x = _arr(x, np.int8)
+    w = _arr(w, np.int8)
+    N, H = w.shape
+    assert x.size == B * L * H
+    S_w = _arr(S_w, np.float64)
+    bias = None if bias is None else _arr(bias, np.int32)
+    logits = np.empty((B, N), dtype=np.int32)
+    _chk(lib().orc_classifier(_p(x), C.c_int(B), C.c_int(L), C.c_int(H), C.c_double(S_x), _p(w), _p(S_w),
+                              _p(bias), C.c_int(N), _p(logits)), "classifier")
+    return logits

@@ -446,10 +446,18 @@ int orc_linear(const int8_t* x, double S_x, const int8_t* w, const double* S_w,
 /* qkv: [B*L, 3H] int8, columns Q | K | V, head j = columns 64j .. 64j+63
    of each block.  Scores carry the scale S_q S_k / 8 (1/sqrt(64) folded in).
    ctx: [B*L, H] int8 at S_ctx.  probs (optional): [B, heads, L, L] uint8. */
-int orc_attention(const int8_t* qkv, int B, int L, int H, int heads,
-                  double S_q, double S_k, double S_v, double S_ctx, int p_max,
-                  int8_t* ctx, uint8_t* probs) {
+/* Attention of sequences with padding.  The paper does not treat masks; the reading taken here
+   is the integer counterpart of the usual additive -inf key mask: sequence b has lens[b] valid
+   keys (0 <= lens[b] <= L), keys j >= lens[b] take no part in the row maximum or the row sum and
+   get probability 0; every query row (padded ones too) attends to the valid keys.  A sequence
+   with no valid key gives context 0.  lens == NULL means every key is valid. */
+static int attention_impl(const int8_t* qkv, int B, int L, int H, int heads, const int32_t* lens,
+                          double S_q, double S_k, double S_v, double S_ctx, int p_max,
+                          int8_t* ctx, uint8_t* probs) {
   if (B < 0 || L < 1 || L > 1024 || heads < 1 || H != heads * 64) return ORC_ERR_ARG;
+  if (lens)
+    for (int bi = 0; bi < B; ++bi)
+      if (lens[bi] < 0 || lens[bi] > L) return ORC_ERR_ARG;
   if (p_max != 255 && p_max != 127) return ORC_ERR_ARG;
   const int d = 64;
   orc_exp_consts k;
@@ -466,22 +474,26 @@ int orc_attention(const int8_t* qkv, int B, int L, int H, int heads,
   for (int bi = 0; bi < B; ++bi) {
     for (int h = 0; h < heads; ++h) {
       int64_t s[1024], e[1024], p[1024];
+      const int n = lens ? lens[bi] : L;          /* valid keys of this sequence */
       for (int i = 0; i < L; ++i) {
         const int8_t* qi = qkv + ((int64_t)bi * L + i) * ld + h * d;
-        for (int j = 0; j < L; ++j) {
+        for (int j = 0; j < n; ++j) {
           const int8_t* kj = qkv + ((int64_t)bi * L + j) * ld + H + h * d;
           int64_t acc = 0;
           for (int t = 0; t < d; ++t) acc += (int64_t)qi[t] * (int64_t)kj[t];
           s[j] = acc;
         }
-        int rr = softmax_row(s, L, &k, p_max, e, p);
-        if (rr) { err = rr; continue; }
+        if (n > 0) {
+          int rr = softmax_row(s, n, &k, p_max, e, p);
+          if (rr) { err = rr; continue; }
+        }
+        for (int j = n; j < L; ++j) p[j] = 0;
         if (probs)
           for (int j = 0; j < L; ++j)
             probs[(((int64_t)bi * heads + h) * L + i) * L + j] = (uint8_t)p[j];
         for (int t = 0; t < d; ++t) {
           int64_t acc = 0;
-          for (int j = 0; j < L; ++j) {
+          for (int j = 0; j < n; ++j) {
             const int8_t* vj = qkv + ((int64_t)bi * L + j) * ld + 2 * H + h * d;
             acc += p[j] * (int64_t)vj[t];
           }
@@ -491,6 +503,18 @@ int orc_attention(const int8_t* qkv, int B, int L, int H, int heads,
     }
   }
   return err;
+}
+
+int orc_attention(const int8_t* qkv, int B, int L, int H, int heads,
+                  double S_q, double S_k, double S_v, double S_ctx, int p_max,
+                  int8_t* ctx, uint8_t* probs) {
+  return attention_impl(qkv, B, L, H, heads, NULL, S_q, S_k, S_v, S_ctx, p_max, ctx, probs);
+}
+
+int orc_attention_masked(const int8_t* qkv, int B, int L, int H, int heads, const int32_t* lens,
+                         double S_q, double S_k, double S_v, double S_ctx, int p_max,
+                         int8_t* ctx, uint8_t* probs) {
+  return attention_impl(qkv, B, L, H, heads, lens, S_q, S_k, S_v, S_ctx, p_max, ctx, probs);
 }
 
 /* ------------------------------------------------------------------ */
@@ -514,8 +538,8 @@ typedef struct {
   int8_t* qkv; int8_t* ctx; int32_t* r1; int8_t* h1; int8_t* g; int32_t* r2;
 } orc_layer_taps;
 
-int orc_encoder_layer(const orc_layer_desc* D, const int8_t* x, int B, int L,
-                      int8_t* out, const orc_layer_taps* taps) {
+static int encoder_layer_impl(const orc_layer_desc* D, const int8_t* x, int B, int L, const int32_t* lens,
+                              int8_t* out, const orc_layer_taps* taps) {
   const int H = D->H, F = D->F;
   const int64_t T = (int64_t)B * L;
   int rc = ORC_OK;
@@ -534,7 +558,7 @@ int orc_encoder_layer(const orc_layer_desc* D, const int8_t* x, int B, int L,
   rc = orc_linear(x, D->S_x, D->w_qkv, D->S_w_qkv, D->bias_qkv, T, 3 * H, H, 0, 0.0, so, qkv);
   if (rc) goto done;
   /* a2-a4: scores, i-softmax, context */
-  rc = orc_attention(qkv, B, L, H, D->heads, D->S_q, D->S_k, D->S_v, D->S_ctx, D->p_max, ctx, NULL);
+  rc = attention_impl(qkv, B, L, H, D->heads, lens, D->S_q, D->S_k, D->S_v, D->S_ctx, D->p_max, ctx, NULL);
   if (rc) goto done;
   /* a5: output projection to Q16 at the residual-sum scale */
   rc = orc_linear(ctx, D->S_ctx, D->w_o, D->S_w_o, D->bias_o, T, H, H, 1, D->S_r1, NULL, r1);
@@ -564,6 +588,60 @@ int orc_encoder_layer(const orc_layer_desc* D, const int8_t* x, int B, int L,
   }
 done:
   free(qkv); free(ctx); free(r1); free(h1); free(gi); free(g); free(r2); free(so);
+  return rc;
+}
+
+int orc_encoder_layer(const orc_layer_desc* D, const int8_t* x, int B, int L,
+                      int8_t* out, const orc_layer_taps* taps) {
+  return encoder_layer_impl(D, x, B, L, NULL, out, taps);
+}
+
+/* the same layer on padded sequences: only the attention sees the lengths (key mask) */
+int orc_encoder_layer_masked(const orc_layer_desc* D, const int8_t* x, int B, int L, const int32_t* lens,
+                             int8_t* out, const orc_layer_taps* taps) {
+  return encoder_layer_impl(D, x, B, L, lens, out, taps);
+}
+
+/* ------------------------------------------------------------------ */
+/* Around the layers: INT8 embedding + embedding LayerNorm, and a       */
+/* classifier on the first token.  The paper only says that the         */
+/* Embedding is kept at INT8 (Appendix on implementation); readings:    */
+/*  - the word row (int8 at S_word) is the LayerNorm input, the         */
+/*    position row (int8 at S_pos) joins it like a residual, i.e.       */
+/*    rescaled to S_word by a dyadic multiplier; i-LayerNorm follows    */
+/*    (Sec. 3.6);                                                       */
+/*  - token t of a [B, L] batch uses position t mod L;                  */
+/*  - the head is one integer linear layer on the first token of every  */
+/*    sequence, left as raw INT32 accumulators (scale S_x S_w[n]).      */
+/* ------------------------------------------------------------------ */
+
+int orc_embedding(const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V, double S_word,
+                  const int8_t* pos, int64_t P, double S_pos, const double* gamma, const double* beta,
+                  int H, double S_out, int8_t* out) {
+  if (T < 0 || L < 1 || H < 1 || V < 1 || P < L) return ORC_ERR_ARG;
+  for (int64_t t = 0; t < T; ++t)
+    if (ids[t] < 0 || ids[t] >= V) return ORC_ERR_ARG;
+  int32_t* a = (int32_t*)malloc(sizeof(int32_t) * (size_t)(T * H) + 4);
+  int8_t* r = (int8_t*)malloc((size_t)(T * H) + 1);
+  if (!a || !r) { free(a); free(r); return ORC_ERR_NOMEM; }
+  for (int64_t t = 0; t < T; ++t)
+    for (int c = 0; c < H; ++c) {
+      a[t * H + c] = word[(int64_t)ids[t] * H + c];
+      r[t * H + c] = pos[(t % L) * H + c];
+    }
+  int rc = orc_layernorm(a, S_word, r, S_pos, gamma, beta, T, H, S_out, out, NULL);
+  free(a); free(r);
+  return rc;
+}
+
+int orc_classifier(const int8_t* x, int B, int L, int H, double S_x, const int8_t* w, const double* S_w,
+                   const int32_t* bias, int N, int32_t* logits) {
+  if (B < 0 || L < 1 || H < 1 || N < 1) return ORC_ERR_ARG;
+  int8_t* first = (int8_t*)malloc((size_t)((int64_t)B * H) + 1);
+  if (!first) return ORC_ERR_NOMEM;
+  for (int b = 0; b < B; ++b) memcpy(first + (int64_t)b * H, x + (int64_t)b * L * H, (size_t)H);
+  int rc = orc_linear(first, S_x, w, S_w, bias, B, N, H, 2, 0.0, NULL, logits);
+  free(first);
   return rc;
 }
 

@@ -115,13 +115,24 @@ def algorithmic_work(H: int, F: int, L: int, heads: int, T: int) -> dict:
 
 
 # --------------------------------------------------------------------------- reference arm
-def oracle_sample_run(cfg_id: int, n_seq: int, layers: int | None = None):
-    """Runs the CPU oracle on the first n_seq sequences of the workload; returns (tokens, seconds)."""
+def oracle_sample_run(cfg_id: int, n_seq: int, layers: int | None = None, full_model: bool = False):
+    """Runs the CPU oracle on the first n_seq sequences of the workload; returns (tokens, seconds, layers)."""
     import oracle
     from paper_2101_01321_b200 import synth
     cfg = synth.CONFIGS[cfg_id]
-    x, params = synth.make_model(cfg_id, n_seq, layers=layers)
     oracle.lib()
+    if full_model:
+        m = synth.make_full_model(cfg_id, n_seq, layers=layers)
+        e, hd = m["emb"], m["head"]
+        t0 = time.perf_counter()
+        h = oracle.embedding(m["ids"], cfg.L, e["word"], e["S_word"], e["pos"], e["S_pos"], e["gamma"], e["beta"],
+                             e["S_out"])
+        for p in m["layers"]:
+            h = oracle.encoder_layer(p, h, n_seq, cfg.L, lens=m["lens"]).out
+        oracle.classifier(h, n_seq, cfg.L, m["layers"][-1]["S_out"], hd["w"], hd["S_w"], hd["bias"])
+        dt = time.perf_counter() - t0
+        return n_seq * cfg.L, dt, len(m["layers"])
+    x, params = synth.make_model(cfg_id, n_seq, layers=layers)
     t0 = time.perf_counter()
     h = x
     for p in params:
@@ -139,14 +150,26 @@ def run_reference(args):
     cfg = synth.CONFIGS[args.config]
     batch = args.batch or DEFAULT_BATCH[args.config]
     n_seq = 2
-    x, params = synth.make_model(args.config, n_seq)
+    full_model = args.workload == "model"
     oracle.lib()
+    if full_model:
+        m = synth.make_full_model(args.config, n_seq)
+        params, e, hd = m["layers"], m["emb"], m["head"]
 
-    def step():
-        h = x
-        for p in params:
-            h = oracle.encoder_layer(p, h, n_seq, cfg.L).out
-        return h
+        def step():
+            h = oracle.embedding(m["ids"], cfg.L, e["word"], e["S_word"], e["pos"], e["S_pos"], e["gamma"],
+                                 e["beta"], e["S_out"])
+            for p in params:
+                h = oracle.encoder_layer(p, h, n_seq, cfg.L, lens=m["lens"]).out
+            return oracle.classifier(h, n_seq, cfg.L, params[-1]["S_out"], hd["w"], hd["S_w"], hd["bias"])
+    else:
+        x, params = synth.make_model(args.config, n_seq)
+
+        def step():
+            h = x
+            for p in params:
+                h = oracle.encoder_layer(p, h, n_seq, cfg.L).out
+            return h
 
     for _ in range(args.warmup):
         step()
@@ -156,13 +179,15 @@ def run_reference(args):
     dt = time.perf_counter() - t0
     tokens = n_seq * cfg.L * args.steps
     value = tokens / dt
-    sample = (f"each step = first {n_seq} sequences ({n_seq * cfg.L} tokens) of the batch through all "
-              f"{len(params)} layers with the CPU oracle")
+    sample = (f"each step = first {n_seq} sequences ({n_seq * cfg.L} tokens) of the batch through "
+              f"{'the embedding, ' if full_model else ''}all {len(params)} layers"
+              f"{' and the classifier' if full_model else ''} with the CPU oracle")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
-        "data": "synthetic", "config": workload_config(cfg, batch, args.gpus),
+        "data": "synthetic", "config": workload_config(cfg, batch, args.gpus, full_model,
+                                                       float(m["lens"].mean()) / cfg.L if full_model else 1.0),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -170,8 +195,11 @@ def run_reference(args):
     }))
 
 
-def workload_config(cfg, batch, n_gpus):
-    return {"workload": f"config {cfg.config_id}: {cfg.layers}-layer integer-only encoder, H={cfg.H}, "
+def workload_config(cfg, batch, n_gpus, full_model=False, valid_frac=1.0):
+    what = (f"token ids -> INT8 embedding + LayerNorm -> {cfg.layers} integer-only encoder layers with a "
+            f"key-padding mask ({100 * valid_frac:.0f} % of the positions valid) -> first-token classifier"
+            if full_model else f"{cfg.layers}-layer integer-only encoder")
+    return {"workload": f"config {cfg.config_id}: {what}, H={cfg.H}, "
                         f"heads={cfg.heads}, FFN={cfg.F}, L={cfg.L}, B={batch} per GPU",
             "layers": cfg.layers, "hidden": cfg.H, "heads": cfg.heads, "ffn": cfg.F, "seq_len": cfg.L,
             "batch_per_gpu": batch, "global_batch": batch * n_gpus, "parallelism": f"dp{n_gpus} (batch shards, no collective)",
@@ -206,22 +234,51 @@ def run_ours(args):
     # weak scaling: rank r owns sequences [r*batch, (r+1)*batch) of the global batch
     first, last = dp.shard_range(batch * world, world, rank)
     assert last - first == batch
-    x_np, params = synth.make_model(args.config, batch, shard=rank)
     stream = torch.cuda.Stream(device=dev)
     ctx = binding.Context(local_rank, stream)
-    layers = [ctx.ibert_layer_create(p) for p in params]
-    x_dev = torch.from_numpy(x_np).to(dev)
     bufs = [torch.empty((T, cfg.H), dtype=torch.int8, device=dev) for _ in range(2)]
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
-    x_pin = torch.from_numpy(x_np).pin_memory()
-    out_pin = torch.empty((T, cfg.H), dtype=torch.int8).pin_memory()
-    x_stage = torch.empty((T, cfg.H), dtype=torch.int8, device=dev)
+    full_model = args.workload == "model"
+    if not full_model:
+        # the headline workload: the encoder layers on full-length sequences, int8 activations in and out
+        x_np, params = synth.make_model(args.config, batch, shard=rank)
+        layers = [ctx.ibert_layer_create(p) for p in params]
+        x_dev = torch.from_numpy(x_np).to(dev)
+        x_pin = torch.from_numpy(x_np).pin_memory()
+        out_pin = torch.empty((T, cfg.H), dtype=torch.int8).pin_memory()
+        x_stage = torch.empty((T, cfg.H), dtype=torch.int8, device=dev)
+        valid_tokens = T
 
-    def forward(src):
-        h = src
-        for i, ly in enumerate(layers):
-            h, _ = ctx.ibert_encoder_layer(ly, h, batch, cfg.L, out=bufs[i & 1])
-        return h
+        def forward(src):
+            h = src
+            for i, ly in enumerate(layers):
+                h, _ = ctx.ibert_encoder_layer(ly, h, batch, cfg.L, out=bufs[i & 1])
+            return h
+    else:
+        # the model around the layers on a padded batch: token ids in, INT8 embedding + LayerNorm,
+        # the layers with a key-padding mask, first-token classifier, INT32 logits out
+        m = synth.make_full_model(args.config, batch, shard=rank)
+        layers = [ctx.ibert_layer_create(p) for p in m["layers"]]
+        e, hd = m["emb"], m["head"]
+        word_d, pos_d = torch.from_numpy(e["word"]).to(dev), torch.from_numpy(e["pos"]).to(dev)
+        hw_d, hb_d = torch.from_numpy(hd["w"]).to(dev), torch.from_numpy(hd["bias"]).to(dev)
+        lens_d = torch.from_numpy(m["lens"]).to(dev)
+        x_dev = torch.from_numpy(m["ids"]).to(dev)
+        x_pin = torch.from_numpy(m["ids"]).pin_memory()
+        x_stage = torch.empty_like(x_dev)
+        logits = torch.empty((batch, synth.N_LABELS), dtype=torch.int32, device=dev)
+        out_pin = torch.empty((batch, synth.N_LABELS), dtype=torch.int32).pin_memory()
+        emb_out = torch.empty((T, cfg.H), dtype=torch.int8, device=dev)
+        S_last = m["layers"][-1]["S_out"]
+        valid_tokens = int(m["lens"].sum())
+
+        def forward(src):
+            h, _ = ctx.ibert_embedding_i8(src, cfg.L, word_d, e["S_word"], pos_d, e["S_pos"], e["gamma"], e["beta"],
+                                          e["S_out"], out=emb_out)
+            for i, ly in enumerate(layers):
+                h, _ = ctx.ibert_encoder_layer_masked(ly, h, batch, cfg.L, lens_d, out=bufs[i & 1])
+            out, _ = ctx.ibert_classifier_i8(h, batch, cfg.L, S_last, hw_d, hd["S_w"], hb_d, out=logits)
+            return out
 
     def barrier():
         if dist is not None:
@@ -318,25 +375,28 @@ def run_ours(args):
         roof["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)"
         roof["algorithmic"] = (16.0 * T * cfg.L * cfg.heads if top == "attention"
                                else work[top]["ops"] if work[top]["ops"] else work[top]["bytes"])
-        tokens = T * args.steps * world
+        tokens = T * args.steps * world          # padded positions count: every one of them is computed
         value = tokens / (total_ms / 1e3)
         e2e_value = tokens / (total_e2e_ms / 1e3)
 
         # CPU baseline: the oracle on a bounded sample of the same workload
         n_seq = 8
-        tok_s, dt_s, n_layers = oracle_sample_run(args.config, n_seq)
+        tok_s, dt_s, n_layers = oracle_sample_run(args.config, n_seq, full_model=full_model)
         import oracle
         cpu = {"value": tok_s / dt_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-               "sample": f"first {n_seq} sequences ({tok_s} tokens) through all {n_layers} layers, {dt_s:.1f} s"}
+               "sample": f"first {n_seq} sequences ({tok_s} tokens) through "
+                         f"{'embedding, ' if full_model else ''}all {n_layers} layers"
+                         f"{' and the classifier' if full_model else ''}, {dt_s:.1f} s"}
 
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-            "config": workload_config(cfg, batch, world),
+            "config": workload_config(cfg, batch, world, full_model, valid_tokens / T),
             "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": T * cfg.H,
-                    "d2h_bytes_per_step": T * cfg.H, "ms_per_step": total_e2e_ms / args.steps},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_pin.numel() * x_pin.element_size(),
+                    "d2h_bytes_per_step": out_pin.numel() * out_pin.element_size(),
+                    "ms_per_step": total_e2e_ms / args.steps},
             "gpu_launches": sum(v["launches_per_step"] for v in kern.values()) * args.steps,
             "roofline": roof,
             "kernels": kern,
@@ -450,6 +510,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4])
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--workload", choices=["layers", "model"], default="layers",
+                    help="layers: the encoder layers on full-length sequences (headline); model: token ids -> "
+                         "embedding -> layers with a key-padding mask on a sentence-length mix -> classifier")
     ap.add_argument("--only", default="", help="run one kernel class alone (profiling aid)")
     args = ap.parse_args()
     if args.only:

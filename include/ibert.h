@@ -172,6 +172,45 @@ int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const
 int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* layer, const int8_t* x, int B, int L,
                         int8_t* out, double* S_ret);
 
+/* ---- around the plain layer: padded sequences, embedding, classifier -------------------------
+   The paper treats none of these beyond stating that the Embedding is kept at INT8
+   (implementation appendix); the readings below are this library's. */
+
+/* Attention with a key-padding mask: lens (device int32 [B]) gives the valid keys of every
+   sequence (values are clamped to [0, L]).  Keys j >= lens[b] take no part in the row maximum or
+   the row sum of i-softmax (Algorithm 3) and get probability 0 -- the integer counterpart of an
+   additive -inf mask; every query row, padded ones included, attends to the valid keys; a
+   sequence without valid keys yields context 0.  Only the 32-key blocks that hold valid keys are
+   computed.  Otherwise as ibert_attention_i8. */
+int ibert_attention_masked_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
+                              const int32_t* lens, double S_q, double S_k, double S_v, double S_ctx, int p_max,
+                              int8_t* out, double* S_ret);
+
+/* ibert_encoder_layer on padded sequences: the attention step takes lens (device int32 [B]) as
+   above; every other step is per token and runs on all B*L rows. */
+int ibert_encoder_layer_masked(ibert_ctx* ctx, const ibert_layer* layer, const int8_t* x, int B, int L,
+                               const int32_t* lens, int8_t* out, double* S_ret);
+
+/* INT8 embedding + embedding LayerNorm: for token t (of T = B*L, row-major [B, L]),
+     out[t, :] = i-LayerNorm( word[ids[t], :] + rescale(pos[t mod L, :], S_pos -> S_word) ; gamma, beta, S_out )
+   i.e. the word row (int8 at S_word) is the LayerNorm input and the position row (int8 at S_pos)
+   joins it as the residual does in ibert_layernorm_i (Sec. 3.6, Eq. 16).
+   ids: device int32 [T] in [0, V) (an id outside records IBERT_ERR_VALUE_RANGE in the context's
+   status and reads row 0); word: device int8 [V, H]; pos: device int8 [P, H], P >= L; gamma, beta:
+   host double [H]; out: device int8 [T, H] at S_out.  H a multiple of 16, at most 2047.  Uses the
+   context's workspace (5 bytes per element). */
+int ibert_embedding_i8(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
+                       double S_word, const int8_t* pos, int64_t P, double S_pos, const double* gamma,
+                       const double* beta, int H, double S_out, int8_t* out, double* S_ret);
+
+/* Classifier head: one integer linear layer on the first token of every sequence,
+     logits[b, n] = sum_k x[b*L, k] * w[n, k] + bias[n]          (raw INT32, scale S_x * S_w[n])
+   x: device int8 [B*L, H]; w: device int8 [N, H] with host scales S_w[N]; bias: device int32 [N] or
+   NULL; logits: device int32 [B, N]; S_ret (host, may be NULL) receives the N output scales.
+   N a multiple of 4 (pad the label dimension with zero rows), H a multiple of 16. */
+int ibert_classifier_i8(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, double S_x, const int8_t* w,
+                        const double* S_w, const int32_t* bias, int N, int32_t* logits, double* S_ret);
+
 /* Per-kernel device timing (CUDA events recorded on the context's stream around every launch
    between begin and end).  No counterpart in the paper: measurement support only.
    ibert_profile_end synchronizes the stream and fills, per kernel class below, the summed

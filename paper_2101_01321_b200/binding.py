@@ -62,6 +62,10 @@ def lib():
         L.ibert_gelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
         L.ibert_layernorm_i.argtypes = [vp, vp, dbl, vp, dbl, vp, vp, i64, i32, dbl, vp, vp]
         L.ibert_attention_i8.argtypes = [vp, vp, i32, i32, i32, i32, dbl, dbl, dbl, dbl, i32, vp, vp]
+        L.ibert_attention_masked_i8.argtypes = [vp, vp, i32, i32, i32, i32, vp, dbl, dbl, dbl, dbl, i32, vp, vp]
+        L.ibert_encoder_layer_masked.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
+        L.ibert_embedding_i8.argtypes = [vp, vp, i64, i32, vp, i64, dbl, vp, i64, dbl, vp, vp, i32, dbl, vp, vp]
+        L.ibert_classifier_i8.argtypes = [vp, vp, i32, i32, i32, dbl, vp, vp, vp, i32, vp, vp]
         L.ibert_layer_create.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(vp)]
         L.ibert_layer_destroy.argtypes = [vp]
         L.ibert_encoder_layer.argtypes = [vp, vp, vp, i32, i32, vp, vp]
@@ -76,7 +80,8 @@ def lib():
         for name in ("ibert_create", "ibert_destroy", "ibert_last_status", "ibert_dyadic_from_double",
                      "ibert_linear_i8", "ibert_linear_gelu_i8", "ibert_linear_layernorm_i8", "ibert_softmax_i", "ibert_gelu_i",
                      "ibert_layernorm_i", "ibert_attention_i8", "ibert_layer_create", "ibert_layer_destroy",
-                     "ibert_encoder_layer"):
+                     "ibert_encoder_layer", "ibert_attention_masked_i8", "ibert_encoder_layer_masked",
+                     "ibert_embedding_i8", "ibert_classifier_i8"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -253,6 +258,50 @@ class Context:
                                       _dev(out, torch.int8), C.byref(S_ret)), "ibert_attention_i8")
         return out, S_ret.value
 
+    def ibert_attention_masked_i8(self, qkv: torch.Tensor, B: int, L: int, H: int, heads: int, lens: torch.Tensor,
+                                  S_q: float, S_k: float, S_v: float, S_ctx: float, p_max: int = 255,
+                                  out: torch.Tensor | None = None):
+        """Attention with a key-padding mask; ``lens``: device int32 [B], valid keys per sequence."""
+        assert qkv.numel() == B * L * 3 * H and lens.numel() == B
+        if out is None:
+            out = torch.empty((B * L, H), dtype=torch.int8, device=qkv.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_attention_masked_i8(self.h, _dev(qkv, torch.int8), B, L, H, heads, _dev(lens, torch.int32),
+                                             S_q, S_k, S_v, S_ctx, p_max, _dev(out, torch.int8), C.byref(S_ret)),
+             "ibert_attention_masked_i8")
+        return out, S_ret.value
+
+    def ibert_embedding_i8(self, ids: torch.Tensor, L: int, word: torch.Tensor, S_word: float, pos: torch.Tensor,
+                           S_pos: float, gamma, beta, S_out: float, out: torch.Tensor | None = None):
+        """INT8 word + position embedding followed by i-LayerNorm (token t: position t mod L)."""
+        T = ids.numel()
+        V, H = word.shape
+        P = pos.shape[0]
+        g, b = _host(gamma, np.float64), _host(beta, np.float64)
+        assert pos.shape[1] == H and g.size == H and b.size == H
+        if out is None:
+            out = torch.empty((T, H), dtype=torch.int8, device=word.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_embedding_i8(self.h, _dev(ids, torch.int32), T, L, _dev(word, torch.int8), V, S_word,
+                                      _dev(pos, torch.int8), P, S_pos, g.ctypes.data, b.ctypes.data, H, S_out,
+                                      _dev(out, torch.int8), C.byref(S_ret)), "ibert_embedding_i8")
+        return out, S_ret.value
+
+    def ibert_classifier_i8(self, x: torch.Tensor, B: int, L: int, S_x: float, w: torch.Tensor, S_w,
+                            bias: torch.Tensor | None, out: torch.Tensor | None = None):
+        """Raw INT32 logits of a linear head on the first token of every sequence."""
+        N, H = w.shape
+        assert x.numel() == B * L * H
+        sw = _host(S_w, np.float64)
+        assert sw.size == N
+        if out is None:
+            out = torch.empty((B, N), dtype=torch.int32, device=x.device)
+        S_ret = np.zeros(N, dtype=np.float64)
+        _chk(lib().ibert_classifier_i8(self.h, _dev(x, torch.int8), B, L, H, S_x, _dev(w, torch.int8), sw.ctypes.data,
+                                       _dev(bias, torch.int32), N, _dev(out, torch.int32), S_ret.ctypes.data),
+             "ibert_classifier_i8")
+        return out, S_ret
+
     # ------------------------------------------------------------------ encoder layer
     def ibert_layer_create(self, params: dict) -> "Layer":
         return Layer(self, params)
@@ -264,6 +313,17 @@ class Context:
         S_ret = C.c_double()
         _chk(lib().ibert_encoder_layer(self.h, layer.h, _dev(x, torch.int8), B, L, _dev(out, torch.int8),
                                        C.byref(S_ret)), "ibert_encoder_layer")
+        return out, S_ret.value
+
+    def ibert_encoder_layer_masked(self, layer: "Layer", x: torch.Tensor, B: int, L: int, lens: torch.Tensor,
+                                   out: torch.Tensor | None = None):
+        """The encoder layer on padded sequences; ``lens``: device int32 [B], valid keys per sequence."""
+        assert lens.numel() == B
+        if out is None:
+            out = torch.empty((B * L, layer.H), dtype=torch.int8, device=x.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_encoder_layer_masked(self.h, layer.h, _dev(x, torch.int8), B, L, _dev(lens, torch.int32),
+                                              _dev(out, torch.int8), C.byref(S_ret)), "ibert_encoder_layer_masked")
         return out, S_ret.value
 
 

@@ -379,8 +379,9 @@ static int make_attn_consts(double S_q, double S_k, double S_v, double S_ctx, in
   return IBERT_OK;
 }
 
-int ibert_attention_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads, double S_q,
-                       double S_k, double S_v, double S_ctx, int p_max, int8_t* out, double* S_ret) {
+static int attention_common(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads, const int32_t* lens,
+                            double S_q, double S_k, double S_v, double S_ctx, int p_max, int8_t* out,
+                            double* S_ret) {
   if (!ctx || B < 0) return IBERT_ERR_ARG;
   if (heads < 1 || H != heads * 64 || L < 1 || L > 512) return IBERT_ERR_SHAPE;
   if (B > 0 && (!qkv || !out)) return IBERT_ERR_ARG;
@@ -391,10 +392,22 @@ int ibert_attention_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, i
   DeviceGuard guard(ctx->device);
   {
     ProfileScope ps(ctx, IBERT_K_ATTENTION);
-    rc = launch_attention(ctx, qkv, B, L, H, heads, k, out);
+    rc = launch_attention(ctx, qkv, B, L, H, heads, k, lens, out);
   }
   if (rc == IBERT_OK && S_ret) *S_ret = S_ctx;
   return rc;
+}
+
+int ibert_attention_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads, double S_q,
+                       double S_k, double S_v, double S_ctx, int p_max, int8_t* out, double* S_ret) {
+  return attention_common(ctx, qkv, B, L, H, heads, nullptr, S_q, S_k, S_v, S_ctx, p_max, out, S_ret);
+}
+
+int ibert_attention_masked_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
+                              const int32_t* lens, double S_q, double S_k, double S_v, double S_ctx, int p_max,
+                              int8_t* out, double* S_ret) {
+  if (B > 0 && !lens) return IBERT_ERR_ARG;
+  return attention_common(ctx, qkv, B, L, H, heads, lens, S_q, S_k, S_v, S_ctx, p_max, out, S_ret);
 }
 
 // --------------------------------------------------------------------------- encoder layer
@@ -489,8 +502,8 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   return IBERT_OK;
 }
 
-int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, int B, int L,
-                        int8_t* out, double* S_ret) {
+static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, int B, int L,
+                                const int32_t* lens, int8_t* out, double* S_ret) {
   if (!ctx || !ly || ly->ctx != ctx || B < 0) return IBERT_ERR_ARG;
   if (L < 1 || L > 512) return IBERT_ERR_SHAPE;
   const int H = ly->d.H, F = ly->d.F;
@@ -521,7 +534,7 @@ int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, 
   e.kind = EPI_INT8; e.d_b = ly->b_qkv; e.d_c = ly->c_qkv; e.d_bias = ly->bias_qkv; e.fast = ly->fast_qkv;
   { ProfileScope ps(ctx, IBERT_K_GEMM_QKV); rc = launch_gemm_i8(ctx, x, ly->w_qkv, T, 3 * H, H, e, qkv); }
   if (rc) return rc;
-  { ProfileScope ps(ctx, IBERT_K_ATTENTION); rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, cx); }
+  { ProfileScope ps(ctx, IBERT_K_ATTENTION); rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, lens, cx); }
   if (rc) return rc;
   // output projection + residual + LayerNorm: one kernel when shapes and constants allow it
   e.kind = EPI_Q16; e.d_b = ly->b_o; e.d_c = ly->c_o; e.d_bias = ly->bias_o; e.fast = ly->fast_o;
@@ -546,6 +559,76 @@ int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, 
   if (rc) return rc;
   { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm(ctx, r, h1, T, ly->ln2, ly->ln2_b, ly->ln2_B, out); }
   return rc;
+}
+
+int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, int B, int L,
+                        int8_t* out, double* S_ret) {
+  return encoder_layer_common(ctx, ly, x, B, L, nullptr, out, S_ret);
+}
+
+int ibert_encoder_layer_masked(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, int B, int L,
+                               const int32_t* lens, int8_t* out, double* S_ret) {
+  if (B > 0 && !lens) return IBERT_ERR_ARG;
+  return encoder_layer_common(ctx, ly, x, B, L, lens, out, S_ret);
+}
+
+int ibert_embedding_i8(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
+                       double S_word, const int8_t* pos, int64_t P, double S_pos, const double* gamma,
+                       const double* beta, int H, double S_out, int8_t* out, double* S_ret) {
+  if (!ctx || T < 0 || !gamma || !beta || !word || !pos) return IBERT_ERR_ARG;
+  if (L < 1 || H < 1 || H > 2047 || H % 16 != 0 || V < 1 || P < L) return IBERT_ERR_SHAPE;
+  if (T > 0 && (!ids || !out)) return IBERT_ERR_ARG;
+  if (!aligned16(word) || !aligned16(pos) || !aligned16(out)) return IBERT_ERR_ALIGN;
+  if (!good_scale(S_word) || !good_scale(S_pos) || !good_scale(S_out)) return IBERT_ERR_SCALE_RANGE;
+  LnConsts k{};
+  k.C = H;
+  k.has_res = 1;
+  int rc = make_ln_residual(S_pos, S_word, &k);
+  if (rc) return rc;
+  std::vector<int32_t> b_i;
+  std::vector<int64_t> B_i;
+  rc = make_ln_tables(gamma, beta, H, S_out, &k, &b_i, &B_i);
+  if (rc) return rc;
+  if (S_ret) *S_ret = S_out;
+  if (T == 0) return IBERT_OK;
+  DeviceGuard guard(ctx->device);
+  void *d_b = nullptr, *d_B = nullptr;
+  if ((rc = cached_upload(ctx, b_i.data(), b_i.size() * sizeof(int32_t), 11, &d_b))) return rc;
+  if ((rc = cached_upload(ctx, B_i.data(), B_i.size() * sizeof(int64_t), 12, &d_B))) return rc;
+  // gathered rows: q int32 [T, H] (word row) | r int8 [T, H] (position row)
+  const size_t q_bytes = ((size_t)T * H * 4 + 255) & ~size_t(255);
+  if ((rc = ensure_workspace(ctx, q_bytes + (size_t)T * H + 256))) return rc;
+  int32_t* q = static_cast<int32_t*>(ctx->ws);
+  int8_t* r = reinterpret_cast<int8_t*>(static_cast<char*>(ctx->ws) + q_bytes);
+  if ((rc = launch_embed_gather(ctx, ids, T, L, word, V, pos, H, q, r))) return rc;
+  ProfileScope ps(ctx, IBERT_K_LAYERNORM);
+  return launch_layernorm(ctx, q, r, T, k, (const int32_t*)d_b, (const int64_t*)d_B, out);
+}
+
+int ibert_classifier_i8(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, double S_x, const int8_t* w,
+                        const double* S_w, const int32_t* bias, int N, int32_t* logits, double* S_ret) {
+  if (!ctx || B < 0 || !S_w || !w) return IBERT_ERR_ARG;
+  if (L < 1 || H < 1 || H % 16 != 0 || N < 1 || N % 4 != 0) return IBERT_ERR_SHAPE;
+  if ((int64_t)H * 127 * 127 >= (int64_t(1) << 31)) return IBERT_ERR_SHAPE;
+  if (B > 0 && (!x || !logits)) return IBERT_ERR_ARG;
+  if (!aligned16(x) || !aligned16(w) || !aligned16(logits) || (bias && !aligned16(bias))) return IBERT_ERR_ALIGN;
+  if (!good_scale(S_x)) return IBERT_ERR_SCALE_RANGE;
+  for (int n = 0; n < N; ++n)
+    if (!good_scale(S_w[n])) return IBERT_ERR_SCALE_RANGE;
+  if (S_ret) for (int n = 0; n < N; ++n) S_ret[n] = S_x * S_w[n];
+  if (B == 0) return IBERT_OK;
+  DeviceGuard guard(ctx->device);
+  int rc = ensure_workspace(ctx, (size_t)B * H + 256);
+  if (rc) return rc;
+  int8_t* first = static_cast<int8_t*>(ctx->ws);
+  // first token of every sequence: B rows of H bytes, L*H bytes apart
+  if (cudaMemcpy2DAsync(first, (size_t)H, x, (size_t)L * H, (size_t)H, (size_t)B, cudaMemcpyDeviceToDevice,
+                        ctx->stream) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_CUDA; }
+  GemmEpilogue epi{};
+  epi.kind = EPI_RAW;
+  epi.d_bias = bias;
+  ProfileScope ps(ctx, gemm_class(EPI_RAW, H));
+  return launch_gemm_i8(ctx, first, w, B, N, H, epi, logits);
 }
 
 int ibert_selftest_exp_division(double S, int32_t* q_ln2_out) {

@@ -27,6 +27,7 @@ struct CoarseArgs {
   uint32_t tmem_cols;
   int stages;        // operand stages in shared memory: 2 (next item prefetched) or 1
   AttnConsts k;
+  const int32_t* lens;   // [B] valid keys per sequence, or nullptr: all L
   int8_t* out;
   int32_t* status;
 };
@@ -83,7 +84,7 @@ __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const
     ptx::tmem_st32(t_row + c0, v);
   }
   ptx::tmem_wait_st();
-  const RowDivisor rd = make_row_divisor(sum, ek.p_max);
+  const RowDivisor rd = make_row_divisor(max(sum, 1u), ek.p_max);   // sum = 0 only without valid keys
   const bool nopre = __all_sync(0xffffffffu, rd.pre == 0);      // usual case: every row sum >= 2^10
   for (int c0 = 0; c0 < Lp; c0 += 32) {
     uint32_t v[32];
@@ -239,11 +240,12 @@ attention_coarse_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid
     // ---- i-softmax on the row this thread owns
     if (ok) {
       ptx::tc_fence_after_sync();
-      // scores are sums of 64 int8 products: |s| < 2^20, so distances from the maximum stay below 2^21
+      // keys beyond the sequence's length are masked like the padding columns
+      const int n_keys = a.lens ? min(max(__ldg(a.lens + batch), 0), L) : L;
       switch (exp_div_mode(a.k.e)) {
-        case 0: softmax_row<0>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
-        case 1: softmax_row<1>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
-        default: softmax_row<2>(t_row, L, Lp, a.k.e, sP, (uint32_t)tid); break;
+        case 0: softmax_row<0>(t_row, n_keys, Lp, a.k.e, sP, (uint32_t)tid); break;
+        case 1: softmax_row<1>(t_row, n_keys, Lp, a.k.e, sP, (uint32_t)tid); break;
+        default: softmax_row<2>(t_row, n_keys, Lp, a.k.e, sP, (uint32_t)tid); break;
       }
       ptx::fence_proxy_async_smem();        // P and Vt were written by ordinary stores; the MMA reads them
     }
@@ -333,6 +335,7 @@ struct AttnArgs {
   int q_bufs;        // 2 when a pair has several query tiles (next tile's Q prefetched), else 1
   uint32_t tmem_cols;
   AttnConsts k;
+  const int32_t* lens;   // [B] valid keys per sequence, or nullptr: all L
   int8_t* out;
   int32_t* status;
 };
@@ -359,10 +362,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
   const int n_threads = blockDim.x;
   const int quad = warp & 3, grp = warp >> 2, G = a.groups;
   const int row = quad * 32 + lane;                            // query row inside the tile = TMEM lane
-  const int L = a.L, Lp = a.Lp, q_tiles = a.n_slabs;
+  const int L = a.L, q_tiles = a.n_slabs;
   const int total = a.B * a.heads;
-  const int n_chunks = Lp >> 5, per_grp = (n_chunks + G - 1) / G;
-  const int c_begin = min(grp * per_grp, n_chunks) * 32, c_end = min((grp + 1) * per_grp, n_chunks) * 32;
 
   if (tid == 0) {
     ptx::mbar_init(bar_q0, 1);
@@ -417,6 +418,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
   for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
     const int head = item % a.heads, batch = item / a.heads;
     const int next = item + gridDim.x;
+    // valid keys of this sequence (key-padding mask): keys >= n take no part in max or sum and get
+    // probability 0; the MMAs and the softmax only cover the 32-column chunks that hold valid keys
+    // (at least one chunk, so that a sequence without valid keys yields P = 0 and context 0)
+    const int n = a.lens ? min(max(__ldg(a.lens + batch), 0), L) : L;
+    const int Lp = max((n + 31) & ~31, 32);
+    const int n_chunks = Lp >> 5, per_grp = (n_chunks + G - 1) / G;
+    const int c_begin = min(grp * per_grp, n_chunks) * 32, c_end = min((grp + 1) * per_grp, n_chunks) * 32;
 
     // ---- V [j][d] -> Vt [d][j] once per (batch, head); the plain copy is then free for the next pair
     ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_v, kv_phase));
@@ -469,13 +477,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
           uint32_t v[32];
           ptx::tmem_ld32(t_row + c0, v);
           ptx::tmem_wait_ld();
-          if (c0 + 32 <= L) {
+          if (c0 + 32 <= n) {
 #pragma unroll
             for (int i = 0; i < 32; i += 2) mx = __vimax3_s32(mx, (int32_t)v[i], (int32_t)v[i + 1]);
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (c0 + i < L) mx = max(mx, (int32_t)v[i]);
+              if (c0 + i < n) mx = max(mx, (int32_t)v[i]);
           }
         }
         s_max[grp * 128 + row] = mx;
@@ -489,7 +497,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
           uint32_t v[32];
           ptx::tmem_ld32(t_row + c0, v);
           ptx::tmem_wait_ld();
-          if (c0 + 32 <= L) {
+          if (c0 + 32 <= n) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               v[i] = iexp_dist_wide((uint32_t)mx - v[i], a.k.e);
@@ -498,7 +506,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-              v[i] = (c0 + i < L) ? iexp_dist_wide((uint32_t)mx - v[i], a.k.e) : 0u;
+              v[i] = (c0 + i < n) ? iexp_dist_wide((uint32_t)mx - v[i], a.k.e) : 0u;
               sum += v[i];
             }
           }
@@ -512,7 +520,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
       if (ok) {
         sum = 0;
         for (int g = 0; g < G; ++g) sum += s_sum[g * 128 + row];
-        const RowDivisor rd = make_row_divisor(sum, a.k.e.p_max);
+        const RowDivisor rd = make_row_divisor(max(sum, 1u), a.k.e.p_max);   // sum = 0 only without valid keys
         const bool nopre = __all_sync(0xffffffffu, rd.pre == 0);
         for (int c0 = c_begin; c0 < c_end; c0 += 32) {
           uint32_t v[32];
@@ -610,7 +618,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
 }  // namespace
 
 int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
-                     const AttnConsts& k, int8_t* out) {
+                     const AttnConsts& k, const int32_t* lens, int8_t* out) {
   if (B == 0) return IBERT_OK;
   const int Lp = (L + 31) & ~31, n_slabs = (L + 127) / 128;
   uint32_t cols = 64;
@@ -630,7 +638,7 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
     a.B = B; a.L = L; a.H = H; a.heads = heads;
     a.Lp = Lp; a.n_slabs = n_slabs; a.groups = n_slabs;
     a.q_bufs = n_slabs > 1 ? 2 : 1;
-    a.tmem_cols = cols; a.k = k; a.out = out; a.status = ctx->d_status;
+    a.tmem_cols = cols; a.k = k; a.lens = lens; a.out = out; a.status = ctx->d_status;
     const int smem = a.q_bufs * slab + 3 * n_slabs * slab + n_slabs * 128 * 128 + 2 * 4 * 128 * 4 + 64 + 1024;
     // resident CTAs per SM: bounded by the register file (128 G threads of at most 128 registers),
     // by the 512 TMEM columns and by shared memory.  The bound must not exceed what TMEM allows:
@@ -653,7 +661,7 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
   CoarseArgs a{};
   a.B = B; a.L = L; a.H = H; a.heads = heads;
   a.Lp = Lp; a.n_slabs = n_slabs;
-  a.tmem_cols = cols; a.k = k; a.out = out; a.status = ctx->d_status;
+  a.tmem_cols = cols; a.k = k; a.lens = lens; a.out = out; a.status = ctx->d_status;
   const int stage_bytes = (1 + 2 * n_slabs) * slab;
   const int fixed_bytes = n_slabs * slab + n_slabs * 128 * 128 + 64 + 1024;
   a.stages = (2 * stage_bytes + fixed_bytes <= 112 * 1024) ? 2 : 1;     // keep at least 2 CTAs per SM

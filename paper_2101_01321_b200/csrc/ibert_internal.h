@@ -110,6 +110,10 @@ int cached_upload(ibert_ctx* ctx, const void* host, size_t bytes, uint64_t tag, 
 
 int launch_gelu(ibert_ctx* ctx, const int32_t* q, int64_t n, const GeluConsts& k, int8_t* out);
 int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const ExpConsts& k, uint8_t* out);
+// rows of the word table (as int32) and of the position table (token t: position t mod L) gathered
+// into q [T, H] and r [T, H]; an id outside [0, V) records IBERT_ERR_VALUE_RANGE and reads row 0
+int launch_embed_gather(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
+                        const int8_t* pos, int H, int32_t* q, int8_t* r);
 int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t rows, const LnConsts& k,
                      const int32_t* d_b, const int64_t* d_B, int8_t* out);
 
@@ -172,7 +176,9 @@ int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t 
                       const GemmEpilogue& epi, const int8_t* res, const LnConsts& ln, const int32_t* d_b_i,
                       const int64_t* d_B_i, int8_t* out);
 
+// `lens` (device, [B], may be null): valid keys per sequence -- keys beyond take no part in the
+// softmax and get probability 0 (key-padding mask)
 int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
-                     const AttnConsts& k, int8_t* out);
+                     const AttnConsts& k, const int32_t* lens, int8_t* out);
 
 }  // namespace ibert

@@ -384,6 +384,39 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
   }
 }
 
+// ----------------------------------------------------------------------------- embedding gather
+// One warp per token: 16 bytes of the word row and of the position row per lane and step.
+__global__ void __launch_bounds__(kThreads) embed_gather_kernel(const int32_t* __restrict__ ids, int64_t T, int L,
+                                                                const int8_t* __restrict__ word, int64_t V,
+                                                                const int8_t* __restrict__ pos, int H,
+                                                                int32_t* __restrict__ q, int8_t* __restrict__ r,
+                                                                int32_t* status) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
+  for (int64_t t = warp_global; t < T; t += warp_count) {
+    int64_t id = __ldg(ids + t);
+    if (id < 0 || id >= V) {
+      if (lane == 0) atomicCAS(status, 0, IBERT_ERR_VALUE_RANGE);
+      id = 0;
+    }
+    const int8_t* wrow = word + id * H;
+    const int8_t* prow = pos + (t % L) * H;
+    for (int c = lane * 16; c < H; c += 512) {
+      const uint4 wv = __ldg(reinterpret_cast<const uint4*>(wrow + c));
+      const uint4 pv = __ldg(reinterpret_cast<const uint4*>(prow + c));
+      const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+      int32_t o[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) o[i] = (int32_t)(int8_t)(ww[i >> 2] >> (8 * (i & 3)));
+      int4* qd = reinterpret_cast<int4*>(q + t * H + c);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) qd[i] = make_int4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+      *reinterpret_cast<uint4*>(r + t * H + c) = pv;
+    }
+  }
+}
+
 int grid_for(ibert_ctx* ctx, int64_t work_warps, int max_ctas_per_sm) {
   const int64_t ctas = (work_warps + (kThreads / 32) - 1) / (kThreads / 32);
   const int64_t cap = (int64_t)ctx->num_sms * max_ctas_per_sm;
@@ -393,6 +426,14 @@ int grid_for(ibert_ctx* ctx, int64_t work_warps, int max_ctas_per_sm) {
 int check_launch() { return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA; }
 
 }  // namespace
+
+int launch_embed_gather(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
+                        const int8_t* pos, int H, int32_t* q, int8_t* r) {
+  if (T == 0) return IBERT_OK;
+  embed_gather_kernel<<<grid_for(ctx, T, 8), kThreads, 0, ctx->stream>>>(ids, T, L, word, V, pos, H, q, r,
+                                                                          ctx->d_status);
+  return check_launch();
+}
 
 int launch_gelu(ibert_ctx* ctx, const int32_t* q, int64_t n, const GeluConsts& k, int8_t* out) {
   if (n == 0) return IBERT_OK;

@@ -208,3 +208,57 @@ def layernorm_inputs(rows: int, C: int, sigma: float, tensor_id: int = 2, with_r
     q = quantize_sym(x, S, 32767).astype(np.int32)
     S_out = 4.5 * math.sqrt(1.0 * (1.0 + 0.1 ** 2) + 0.1 ** 2) / 127.0
     return q, S, r, S_r, gamma, beta, S_out
+
+
+# ---------------------------------------------------------------------------
+# the model around the layers: padded batches, INT8 embedding, classifier head
+# ---------------------------------------------------------------------------
+_T_IDS, _T_LENS, _T_WORD, _T_POS, _T_EMB_LN, _T_HEAD_W, _T_HEAD_B = 20, 21, 22, 23, 24, 25, 26
+VOCAB = 50265          # RoBERTa's vocabulary size
+N_LABELS = 4           # label dimension of the head, padded to a multiple of 4
+
+
+def make_lengths(config_id: int, B: int, L: int, shard: int = 0) -> np.ndarray:
+    """Valid tokens per sequence, a sentence-length mix: half the batch uniform in [L/8, L/2],
+    the other half uniform in [L/2, L] (mean ~0.53 L), at least one sequence of full length."""
+    rng = rng_for(config_id, 0, _T_LENS + 100 * shard)
+    short = rng.integers(max(L // 8, 1), L // 2 + 1, B)
+    long_ = rng.integers(L // 2, L + 1, B)
+    lens = np.where(rng.random(B) < 0.5, short, long_).astype(np.int32)
+    lens[0] = L
+    return lens
+
+
+def make_full_model(config_id: int, B: int, layers: int | None = None, H: int | None = None,
+                    heads: int | None = None, F: int | None = None, L: int | None = None,
+                    vocab: int = VOCAB, shard: int = 0) -> dict:
+    """Token ids, lengths, INT8 embedding tables, encoder layers and a first-token classifier.
+    Word / position rows ~ N(0, 0.02^2)-like tables quantized with one symmetric int8 scale per
+    table (Eq. 1); the embedding LayerNorm has gamma ~ N(1, 0.1), beta ~ N(0, 0.1) and an output
+    scale covering 4 standard deviations, which is the first layer's S_x."""
+    cfg = CONFIGS[config_id]
+    H = H or cfg.H
+    heads = heads or cfg.heads
+    F = F or cfg.F
+    L = L or cfg.L
+    layers = layers or cfg.layers
+    ids = rng_for(config_id, 0, _T_IDS + 100 * shard).integers(0, vocab, B * L).astype(np.int32)
+    lens = make_lengths(config_id, B, L, shard)
+    word_f = rng_for(config_id, 0, _T_WORD).standard_normal((vocab, H), dtype=np.float32).astype(np.float64) * 0.02
+    pos_f = rng_for(config_id, 0, _T_POS).standard_normal((L + 2, H), dtype=np.float32).astype(np.float64) * 0.02
+    S_word = float(np.abs(word_f).max() / 127.0)
+    S_pos = float(np.abs(pos_f).max() / 127.0)
+    rng = rng_for(config_id, 0, _T_EMB_LN)
+    emb = {"word": quantize_sym(word_f, S_word, 127).astype(np.int8), "S_word": S_word,
+           "pos": quantize_sym(pos_f, S_pos, 127).astype(np.int8), "S_pos": S_pos,
+           "gamma": 1.0 + 0.1 * rng.standard_normal(H), "beta": 0.1 * rng.standard_normal(H),
+           "S_out": 4.0 * math.sqrt(1.0 * (1.0 + 0.1 ** 2) + 0.1 ** 2) / 127.0}
+    params = []
+    s_in = emb["S_out"]
+    for l in range(layers):
+        p = make_layer(config_id, l, H, heads, F, L, s_in)
+        params.append(p)
+        s_in = p["S_out"]
+    w, S_w = _quantize_weight(rng_for(config_id, 0, _T_HEAD_W), N_LABELS, H)
+    head = {"w": w, "S_w": S_w, "bias": _quantize_bias(rng_for(config_id, 0, _T_HEAD_B), s_in, S_w)}
+    return {"ids": ids, "lens": lens, "emb": emb, "layers": params, "head": head, "B": B, "L": L, "H": H}

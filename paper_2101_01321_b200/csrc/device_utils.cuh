@@ -76,6 +76,20 @@ __device__ __forceinline__ int32_t igelu_q16_upper(int32_t q, const GeluConsts& 
   return max(requant_upper(g2, k.b2), -127);
 }
 
+// Magnitude form of the same function, taking the Q16 value BEFORE its clamp (x; q = clamp(x)):
+// with a = |q| = min(|x|, 32767) and t as above,
+//   q >= 0:  g = q ((t^2 + 2 q_c) >> s_f)                    = a ((t^2 + 2 q_c) >> s_f)
+//   q <  0:  g = q ((-t^2) >> s_f) = q (-ceil(t^2 / 2^s_f))   = a ((t^2 + 2^s_f - 1) >> s_f)
+// so one select of the addend replaces the two-sided clamp, the negation and the select of f.
+// `rnd_f` = 2^s_f - 1.  The result still needs both clamps to +-127.
+__device__ __forceinline__ int32_t igelu_magnitude_upper(int32_t x, const GeluConsts& k, int32_t rnd_f) {
+  const int32_t a = (int32_t)min((uint32_t)abs(x), 32767u);    // unsigned: |INT32_MIN| stays 2^31
+  const int32_t t = min(a >> k.s_in, k.nq_b) - k.nq_b;
+  const int32_t f = (t * t + (x >= 0 ? 2 * k.q_c : rnd_f)) >> k.s_f;
+  const int32_t g2 = (a * f + 128) >> 8;
+  return requant_upper(g2, k.b2);
+}
+
 __device__ __forceinline__ uint32_t shr_clamped(uint32_t v, uint32_t n) {
   uint32_t r;
   asm("shr.u32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(n));   // shift counts above 31 give 0

@@ -243,6 +243,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     uint32_t buf = 0;
     const GeluConsts gk = args.gelu;
     const int64_t gelu_half = rounding_half(gk.c);
+    const int32_t gelu_rnd = (1 << gk.s_f) - 1;
     uint32_t acc_empty_addr = bar_acc_empty;
     if constexpr (PAIR) acc_empty_addr = ptx::map_to_cta(bar_acc_empty, 0);
     uint32_t acc = 0, acc_phase = 0;
@@ -296,7 +297,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if constexpr (FAST) o = clamp_sym(requant_upper(a + cur_bias, cur_pb), 127);
             else o = requant_add(a, cur_pb, cur_padd, cur_pc, 127);
           } else {
-            if constexpr (FAST) o = min(igelu_q16_upper(clamp_sym(requant_upper(a + cur_bias, cur_pb), 32767), gk), 127);
+            if constexpr (FAST) o = clamp_sym(igelu_magnitude_upper(requant_upper(a + cur_bias, cur_pb), gk, gelu_rnd), 127);
             else o = igelu_q16_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
           }
           // staging tile: row = token i, column = this lane's channel

@@ -20,6 +20,7 @@ __global__ void __launch_bounds__(kThreads) gelu_kernel(const int32_t* __restric
                                                         GeluConsts k, int8_t* __restrict__ out) {
   const int64_t half = rounding_half(k.c);
   const int64_t n_vec = n >> 2;
+  const int32_t rnd_f = (1 << k.s_f) - 1;
   const int lane = threadIdx.x & 31;
   const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
   const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
@@ -38,10 +39,10 @@ __global__ void __launch_bounds__(kThreads) gelu_kernel(const int32_t* __restric
       if (idx < n_vec) {
         int32_t a, b, c, d;
         if (k.fast) {
-          a = igelu_q16_upper(clamp_sym(v[j].x, 32767), k);
-          b = igelu_q16_upper(clamp_sym(v[j].y, 32767), k);
-          c = igelu_q16_upper(clamp_sym(v[j].z, 32767), k);
-          d = igelu_q16_upper(clamp_sym(v[j].w, 32767), k);
+          a = max(igelu_magnitude_upper(v[j].x, k, rnd_f), -127);
+          b = max(igelu_magnitude_upper(v[j].y, k, rnd_f), -127);
+          c = max(igelu_magnitude_upper(v[j].z, k, rnd_f), -127);
+          d = max(igelu_magnitude_upper(v[j].w, k, rnd_f), -127);
         } else {
           a = igelu_q16_to_int8(clamp_sym(v[j].x, 32767), k, half);
           b = igelu_q16_to_int8(clamp_sym(v[j].y, 32767), k, half);

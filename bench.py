@@ -195,7 +195,7 @@ def run_reference(args):
     }))
 
 
-def workload_config(cfg, batch, n_gpus, full_model=False, valid_frac=1.0):
+def workload_config(cfg, batch, n_gpus, full_model=False, valid_frac=1.0, use_graph=False):
     what = (f"token ids -> INT8 embedding + LayerNorm -> {cfg.layers} integer-only encoder layers with a "
             f"key-padding mask ({100 * valid_frac:.0f} % of the positions valid) -> first-token classifier"
             if full_model else f"{cfg.layers}-layer integer-only encoder")
@@ -203,7 +203,8 @@ def workload_config(cfg, batch, n_gpus, full_model=False, valid_frac=1.0):
                         f"heads={cfg.heads}, FFN={cfg.F}, L={cfg.L}, B={batch} per GPU",
             "layers": cfg.layers, "hidden": cfg.H, "heads": cfg.heads, "ffn": cfg.F, "seq_len": cfg.L,
             "batch_per_gpu": batch, "global_batch": batch * n_gpus, "parallelism": f"dp{n_gpus} (batch shards, no collective)",
-            "l2": "flushed between timed steps (512 MiB write); per-step activation traffic also exceeds L2"}
+            "l2": "flushed between timed steps (512 MiB write); per-step activation traffic also exceeds L2",
+            "launch": "CUDA graph replay" if use_graph else "one C-ABI call per layer"}
 
 
 # --------------------------------------------------------------------------- our arm
@@ -249,7 +250,15 @@ def run_ours(args):
         x_stage = torch.empty((T, cfg.H), dtype=torch.int8, device=dev)
         valid_tokens = T
 
-        def forward(src):
+        graphs = {}
+
+        def forward(src, eager=False):
+            if args.graph and not eager:
+                # one captured graph per input buffer (the device-resident one and the e2e staging one)
+                g = graphs.get(src.data_ptr())
+                if g is None:
+                    g = graphs[src.data_ptr()] = binding.Graph(ctx, layers, src, batch, cfg.L, bufs[0])
+                return g.launch()
             h = src
             for i, ly in enumerate(layers):
                 h, _ = ctx.ibert_encoder_layer(ly, h, batch, cfg.L, out=bufs[i & 1])
@@ -272,7 +281,7 @@ def run_ours(args):
         S_last = m["layers"][-1]["S_out"]
         valid_tokens = int(m["lens"].sum())
 
-        def forward(src):
+        def forward(src, eager=False):
             h, _ = ctx.ibert_embedding_i8(src, cfg.L, word_d, e["S_word"], pos_d, e["S_pos"], e["gamma"], e["beta"],
                                           e["S_out"], out=emb_out)
             for i, ly in enumerate(layers):
@@ -332,7 +341,7 @@ def run_ours(args):
         prof_steps = min(args.steps, 5)
         for _ in range(prof_steps):
             flush.fill_(1)
-            forward(x_dev)
+            forward(x_dev, eager=True)          # event pairs cannot be recorded into a graph replay
         prof = ctx.ibert_profile_end()
     ctx.check()
 
@@ -392,7 +401,8 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-            "config": workload_config(cfg, batch, world, full_model, valid_tokens / T),
+            "config": workload_config(cfg, batch, world, full_model, valid_tokens / T,
+                                      args.graph and not full_model),
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_pin.numel() * x_pin.element_size(),
                     "d2h_bytes_per_step": out_pin.numel() * out_pin.element_size(),
@@ -403,6 +413,9 @@ def run_ours(args):
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
+    if not full_model:
+        for g in graphs.values():
+            g.close()
     for ly in layers:
         ly.close()
     ctx.close()
@@ -510,6 +523,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4])
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--graph", action="store_true",
+                    help="layers workload: replay the forward pass from a captured CUDA graph (ibert_encoder_graph_*)")
     ap.add_argument("--workload", choices=["layers", "model"], default="layers",
                     help="layers: the encoder layers on full-length sequences (headline); model: token ids -> "
                          "embedding -> layers with a key-padding mask on a sentence-length mix -> classifier")

@@ -211,6 +211,23 @@ int ibert_embedding_i8(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, con
 int ibert_classifier_i8(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, double S_x, const int8_t* w,
                         const double* S_w, const int32_t* bias, int N, int32_t* logits, double* S_ret);
 
+/* ---- a stack of encoder layers captured into a CUDA graph ---------------------------------------
+   No counterpart in the paper: launch-overhead removal for small batches (a 12-layer pass is 60
+   kernel launches).  ibert_encoder_graph_create runs layers[0..n_layers) once on the context's
+   stream (x -> ... -> out, every layer with the same H; lens as in ibert_encoder_layer_masked or
+   NULL) and captures the same sequence into a graph for these shapes and THESE buffers: a later
+   ibert_encoder_graph_launch reads whatever x holds then and writes out.  The graph owns its
+   workspace and intermediate activations (device memory allocated at creation, freed by
+   ibert_encoder_graph_destroy, which synchronizes the stream first).  Creation fails with
+   IBERT_ERR_ARG while ibert_profile_begin is active, and for a context created on the default
+   stream (stream capture needs a stream of its own).  x, out, lens and the layers must stay alive
+   and unmoved for the lifetime of the graph. */
+typedef struct ibert_graph ibert_graph;
+int ibert_encoder_graph_create(ibert_ctx* ctx, const ibert_layer* const* layers, int n_layers, const int8_t* x,
+                               int B, int L, const int32_t* lens, int8_t* out, ibert_graph** graph);
+int ibert_encoder_graph_launch(ibert_ctx* ctx, ibert_graph* graph);
+int ibert_encoder_graph_destroy(ibert_graph* graph);
+
 /* Per-kernel device timing (CUDA events recorded on the context's stream around every launch
    between begin and end).  No counterpart in the paper: measurement support only.
    ibert_profile_end synchronizes the stream and fills, per kernel class below, the summed

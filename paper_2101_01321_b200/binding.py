@@ -66,6 +66,9 @@ def lib():
         L.ibert_encoder_layer_masked.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
         L.ibert_embedding_i8.argtypes = [vp, vp, i64, i32, vp, i64, dbl, vp, i64, dbl, vp, vp, i32, dbl, vp, vp]
         L.ibert_classifier_i8.argtypes = [vp, vp, i32, i32, i32, dbl, vp, vp, vp, i32, vp, vp]
+        L.ibert_encoder_graph_create.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp, C.POINTER(vp)]
+        L.ibert_encoder_graph_launch.argtypes = [vp, vp]
+        L.ibert_encoder_graph_destroy.argtypes = [vp]
         L.ibert_layer_create.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(vp)]
         L.ibert_layer_destroy.argtypes = [vp]
         L.ibert_encoder_layer.argtypes = [vp, vp, vp, i32, i32, vp, vp]
@@ -81,7 +84,8 @@ def lib():
                      "ibert_linear_i8", "ibert_linear_gelu_i8", "ibert_linear_layernorm_i8", "ibert_softmax_i", "ibert_gelu_i",
                      "ibert_layernorm_i", "ibert_attention_i8", "ibert_layer_create", "ibert_layer_destroy",
                      "ibert_encoder_layer", "ibert_attention_masked_i8", "ibert_encoder_layer_masked",
-                     "ibert_embedding_i8", "ibert_classifier_i8"):
+                     "ibert_embedding_i8", "ibert_classifier_i8", "ibert_encoder_graph_create",
+                     "ibert_encoder_graph_launch", "ibert_encoder_graph_destroy"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -325,6 +329,32 @@ class Context:
         _chk(lib().ibert_encoder_layer_masked(self.h, layer.h, _dev(x, torch.int8), B, L, _dev(lens, torch.int32),
                                               _dev(out, torch.int8), C.byref(S_ret)), "ibert_encoder_layer_masked")
         return out, S_ret.value
+
+
+class Graph:
+    """``ibert_graph``: a stack of encoder layers captured into a CUDA graph for fixed shapes and
+    fixed buffers (``x`` in, ``out`` out, optional ``lens``); ``launch()`` replays it."""
+
+    def __init__(self, ctx: "Context", layers, x: torch.Tensor, B: int, L: int, out: torch.Tensor,
+                 lens: torch.Tensor | None = None):
+        self.ctx = ctx
+        self.keep = (list(layers), x, out, lens)          # the graph refers to these buffers
+        arr = (C.c_void_p * len(layers))(*[ly.h for ly in layers])
+        h = C.c_void_p()
+        _chk(lib().ibert_encoder_graph_create(ctx.h, arr, len(layers), _dev(x, torch.int8), B, L,
+                                              _dev(lens, torch.int32), _dev(out, torch.int8), C.byref(h)),
+             "ibert_encoder_graph_create")
+        self.h = h
+        self.out = out
+
+    def launch(self) -> torch.Tensor:
+        _chk(lib().ibert_encoder_graph_launch(self.ctx.h, self.h), "ibert_encoder_graph_launch")
+        return self.out
+
+    def close(self):
+        if self.h:
+            lib().ibert_encoder_graph_destroy(self.h)
+            self.h = None
 
 
 class Layer:

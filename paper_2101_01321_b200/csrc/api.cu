@@ -502,6 +502,13 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   return IBERT_OK;
 }
 
+// bytes of workspace one encoder-layer call needs for T tokens
+static size_t layer_workspace_bytes(int H, int F, int64_t T) {
+  auto up256 = [](size_t v) { return (v + 255) & ~size_t(255); };
+  return up256((size_t)T * 3 * H) + up256((size_t)T * H) + up256((size_t)T * H * 4) + up256((size_t)T * H) +
+         up256((size_t)T * F);
+}
+
 static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, int B, int L,
                                 const int32_t* lens, int8_t* out, double* S_ret) {
   if (!ctx || !ly || ly->ctx != ctx || B < 0) return IBERT_ERR_ARG;
@@ -629,6 +636,101 @@ int ibert_classifier_i8(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, do
   epi.d_bias = bias;
   ProfileScope ps(ctx, gemm_class(EPI_RAW, H));
   return launch_gemm_i8(ctx, first, w, B, N, H, epi, logits);
+}
+
+// --------------------------------------------------------------------------- captured forward pass
+// A stack of encoder layers for fixed shapes and fixed buffers, captured once into a CUDA graph:
+// small batches are bound by launch overhead (60 launches per 12-layer pass), which a graph replay
+// removes.  The graph owns its workspace and its ping-pong activation buffers.
+struct ibert_graph {
+  ibert_ctx* ctx = nullptr;
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  int8_t* bufs[2] = {nullptr, nullptr};
+};
+
+static void graph_free(ibert_graph* g) {
+  if (g->exec) cudaGraphExecDestroy(g->exec);
+  if (g->graph) cudaGraphDestroy(g->graph);
+  if (g->ws) cudaFree(g->ws);
+  for (int i = 0; i < 2; ++i) if (g->bufs[i]) cudaFree(g->bufs[i]);
+  delete g;
+}
+
+int ibert_encoder_graph_create(ibert_ctx* ctx, const ibert_layer* const* layers, int n_layers, const int8_t* x,
+                               int B, int L, const int32_t* lens, int8_t* out, ibert_graph** out_graph) {
+  if (!ctx || !layers || n_layers < 1 || !out_graph || B < 1 || !x || !out) return IBERT_ERR_ARG;
+  *out_graph = nullptr;
+  if (L < 1 || L > 512) return IBERT_ERR_SHAPE;
+  if (ctx->profiling) return IBERT_ERR_ARG;                 // events cannot be recorded into the capture
+  if (ctx->stream == nullptr) return IBERT_ERR_ARG;         // the default stream cannot be captured
+  const int H = layers[0] ? layers[0]->d.H : 0;
+  size_t need = 0;
+  for (int i = 0; i < n_layers; ++i) {
+    if (!layers[i] || layers[i]->ctx != ctx || layers[i]->d.H != H) return IBERT_ERR_ARG;
+    need = std::max(need, layer_workspace_bytes(H, layers[i]->d.F, (int64_t)B * L));
+  }
+  if (!aligned16(x) || !aligned16(out)) return IBERT_ERR_ALIGN;
+  DeviceGuard guard(ctx->device);
+  ibert_graph* g = new ibert_graph();
+  g->ctx = ctx;
+  const size_t act = (size_t)B * L * H;
+  if (cudaMalloc(&g->ws, need) != cudaSuccess ||
+      (n_layers > 1 && (cudaMalloc((void**)&g->bufs[0], act) != cudaSuccess ||
+                        cudaMalloc((void**)&g->bufs[1], act) != cudaSuccess))) {
+    cudaGetLastError();
+    graph_free(g);
+    return IBERT_ERR_NOMEM;
+  }
+  g->ws_bytes = need;
+  // the layers run against the graph's own workspace, once eagerly (function attributes, cached
+  // launch parameters, argument checks) and once under capture
+  void* saved_ws = ctx->ws;
+  const size_t saved_bytes = ctx->ws_bytes;
+  ctx->ws = g->ws;
+  ctx->ws_bytes = g->ws_bytes;
+  auto run = [&]() {
+    for (int i = 0; i < n_layers; ++i) {
+      const int8_t* in = i == 0 ? x : g->bufs[(i - 1) & 1];
+      int8_t* o = i == n_layers - 1 ? out : g->bufs[i & 1];
+      if (int rc = encoder_layer_common(ctx, layers[i], in, B, L, lens, o, nullptr)) return rc;
+    }
+    return (int)IBERT_OK;
+  };
+  int rc = run();
+  if (rc == IBERT_OK && cudaStreamSynchronize(ctx->stream) != cudaSuccess) rc = IBERT_ERR_CUDA;
+  if (rc == IBERT_OK) {
+    if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) rc = IBERT_ERR_CUDA;
+    else {
+      rc = run();
+      cudaGraph_t captured = nullptr;
+      if (cudaStreamEndCapture(ctx->stream, &captured) != cudaSuccess) { cudaGetLastError(); if (rc == IBERT_OK) rc = IBERT_ERR_CUDA; }
+      g->graph = captured;
+      if (rc == IBERT_OK && cudaGraphInstantiate(&g->exec, g->graph, 0) != cudaSuccess) { cudaGetLastError(); rc = IBERT_ERR_CUDA; }
+    }
+  }
+  ctx->ws = saved_ws;
+  ctx->ws_bytes = saved_bytes;
+  if (rc != IBERT_OK) { graph_free(g); return rc; }
+  *out_graph = g;
+  return IBERT_OK;
+}
+
+int ibert_encoder_graph_launch(ibert_ctx* ctx, ibert_graph* g) {
+  if (!ctx || !g || g->ctx != ctx || !g->exec) return IBERT_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (cudaGraphLaunch(g->exec, ctx->stream) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_CUDA; }
+  return IBERT_OK;
+}
+
+int ibert_encoder_graph_destroy(ibert_graph* g) {
+  if (!g) return IBERT_ERR_ARG;
+  DeviceGuard guard(g->ctx->device);
+  cudaStreamSynchronize(g->ctx->stream);
+  graph_free(g);
+  return IBERT_OK;
 }
 
 int ibert_selftest_exp_division(double S, int32_t* q_ln2_out) {

@@ -195,7 +195,7 @@ def run_reference(args):
     }))
 
 
-def workload_config(cfg, batch, n_gpus, full_model=False, valid_frac=1.0, use_graph=False):
+def workload_config(cfg, batch, n_gpus, full_model=False, valid_frac=1.0, use_graph=False, pow2=False):
     what = (f"token ids -> INT8 embedding + LayerNorm -> {cfg.layers} integer-only encoder layers with a "
             f"key-padding mask ({100 * valid_frac:.0f} % of the positions valid) -> first-token classifier"
             if full_model else f"{cfg.layers}-layer integer-only encoder")
@@ -204,7 +204,8 @@ def workload_config(cfg, batch, n_gpus, full_model=False, valid_frac=1.0, use_gr
             "layers": cfg.layers, "hidden": cfg.H, "heads": cfg.heads, "ffn": cfg.F, "seq_len": cfg.L,
             "batch_per_gpu": batch, "global_batch": batch * n_gpus, "parallelism": f"dp{n_gpus} (batch shards, no collective)",
             "l2": "flushed between timed steps (512 MiB write); per-step activation traffic also exceeds L2",
-            "launch": "CUDA graph replay" if use_graph else "one C-ABI call per layer"}
+            "launch": "CUDA graph replay" if use_graph else "one C-ABI call per layer",
+            "score_scales": "ln2 / 2^k" if pow2 else "calibrated"}
 
 
 # --------------------------------------------------------------------------- our arm
@@ -242,7 +243,7 @@ def run_ours(args):
     full_model = args.workload == "model"
     if not full_model:
         # the headline workload: the encoder layers on full-length sequences, int8 activations in and out
-        x_np, params = synth.make_model(args.config, batch, shard=rank)
+        x_np, params = synth.make_model(args.config, batch, shard=rank, pow2_scores=args.pow2_scores)
         layers = [ctx.ibert_layer_create(p) for p in params]
         x_dev = torch.from_numpy(x_np).to(dev)
         x_pin = torch.from_numpy(x_np).pin_memory()
@@ -402,7 +403,7 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": workload_config(cfg, batch, world, full_model, valid_tokens / T,
-                                      args.graph and not full_model),
+                                      args.graph and not full_model, args.pow2_scores and not full_model),
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_pin.numel() * x_pin.element_size(),
                     "d2h_bytes_per_step": out_pin.numel() * out_pin.element_size(),
@@ -523,6 +524,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4])
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--pow2-scores", action="store_true",
+                    help="layers workload: query scales raised so that every score scale is ln2 / 2^k "
+                         "(i-exp quotient by shift and mask)")
     ap.add_argument("--graph", action="store_true",
                     help="layers workload: replay the forward pass from a captured CUDA graph (ibert_encoder_graph_*)")
     ap.add_argument("--workload", choices=["layers", "model"], default="layers",

@@ -493,24 +493,50 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
       uint32_t sum = 0;
       if (ok) {
         for (int g = 0; g < G; ++g) mx = max(mx, s_max[g * 128 + row]);
-        for (int c0 = c_begin; c0 < c_end; c0 += 32) {
-          uint32_t v[32];
-          ptx::tmem_ld32(t_row + c0, v);
-          ptx::tmem_wait_ld();
-          if (c0 + 32 <= n) {
+        if (a.k.e.pow2_k >= 0) {
+          // score scale exactly ln2 / 2^k: quotient and remainder by shift and mask
+          const uint32_t k2 = (uint32_t)a.k.e.pow2_k, mask = (1u << k2) - 1u;
+          const uint32_t mxk = (uint32_t)mx + ((uint32_t)a.k.e.s_out << k2);
+          const int32_t q_b = a.k.e.q_b, q_c = a.k.e.q_c;
+          for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+            uint32_t v[32];
+            ptx::tmem_ld32(t_row + c0, v);
+            ptx::tmem_wait_ld();
+            if (c0 + 32 <= n) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              v[i] = iexp_dist_wide((uint32_t)mx - v[i], a.k.e);
-              sum += v[i];
-            }
-          } else {
+              for (int i = 0; i < 32; ++i) {
+                v[i] = iexp_dist_pow2(mxk - v[i], q_b, q_c, k2, mask);
+                sum += v[i];
+              }
+            } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              v[i] = (c0 + i < n) ? iexp_dist_wide((uint32_t)mx - v[i], a.k.e) : 0u;
-              sum += v[i];
+              for (int i = 0; i < 32; ++i) {
+                v[i] = (c0 + i < n) ? iexp_dist_pow2(mxk - v[i], q_b, q_c, k2, mask) : 0u;
+                sum += v[i];
+              }
             }
+            ptx::tmem_st32(t_row + c0, v);
           }
-          ptx::tmem_st32(t_row + c0, v);
+        } else {
+          for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+            uint32_t v[32];
+            ptx::tmem_ld32(t_row + c0, v);
+            ptx::tmem_wait_ld();
+            if (c0 + 32 <= n) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                v[i] = iexp_dist_wide((uint32_t)mx - v[i], a.k.e);
+                sum += v[i];
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                v[i] = (c0 + i < n) ? iexp_dist_wide((uint32_t)mx - v[i], a.k.e) : 0u;
+                sum += v[i];
+              }
+            }
+            ptx::tmem_st32(t_row + c0, v);
+          }
         }
         ptx::tmem_wait_st();
         s_sum[grp * 128 + row] = sum;

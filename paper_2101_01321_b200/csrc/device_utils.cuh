@@ -120,6 +120,12 @@ __device__ __forceinline__ uint32_t iexp_dist_wide(uint32_t d, const ExpConsts& 
   const uint32_t poly = (uint32_t)(t * t + k.q_c);
   return shr_clamped(poly, z + (uint32_t)k.s_out);
 }
+// i-exp when q_ln2 = 2^k (and no pre-shift): z and r are a shift and a mask of the distance.
+// `dk` = distance + s_out 2^k, so that dk >> k = z + s_out is the final shift count directly.
+__device__ __forceinline__ uint32_t iexp_dist_pow2(uint32_t dk, int32_t q_b, int32_t q_c, uint32_t k, uint32_t mask) {
+  const int32_t t = q_b - (int32_t)(dk & mask);                          // q_b - r
+  return shr_clamped((uint32_t)(t * t + q_c), dk >> k);
+}
 __host__ __device__ __forceinline__ int exp_div_mode(const ExpConsts& k) {
   return k.div_pre != 0 ? 2 : (k.div_post != 0 ? 1 : 0);
 }

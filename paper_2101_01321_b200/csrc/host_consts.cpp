@@ -107,6 +107,12 @@ int make_exp_consts(double S, int p_max, ExpConsts* k) {
   k->q_c = (int32_t)q_c;
   k->s_out = bl > 21 ? bl - 21 : 0;
   k->p_max = (uint32_t)p_max;
+  k->pow2_k = -1;
+  if (s_in == 0 && (k->q_ln2 & (k->q_ln2 - 1)) == 0) {
+    int lg = 0;
+    while ((1u << lg) < k->q_ln2) ++lg;
+    k->pow2_k = lg;
+  }
   return IBERT_OK;
 }
 

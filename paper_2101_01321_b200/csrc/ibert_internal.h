@@ -32,6 +32,9 @@ struct ExpConsts {
   // floor(d / q_ln2) = umulhi(d, wide_m) >> wide_post for every d < 2^21, no clamp to d_max needed
   uint32_t wide_m;
   int32_t wide_post;
+  // k when q_ln2 = 2^k and s_in = 0 (score scale exactly ln2 / 2^k): quotient and remainder of the
+  // distance are then a shift and a mask; -1 otherwise
+  int32_t pow2_k;
 };
 
 // i-GELU (Algorithm 2) followed by requantization to int8

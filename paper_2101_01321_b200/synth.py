@@ -107,6 +107,21 @@ def static_activation_scales(H: int, F: int, L: int, S_x: float, w_std: float = 
     return s
 
 
+def snap_q_scale(S_q: float, S_k: float) -> float:
+    """The smallest S_q' >= S_q for which the score scale S_q' S_k / 8 is ln2 / 2^k for an integer
+    k <= 14 (a static-quantization choice: the query scale is free as long as it covers the range).
+    With such a scale the i-exp quotient floor(d / q_ln2) has q_ln2 = 2^k exactly."""
+    ln2 = 0.6931471805599453
+    k = min(int(math.floor(math.log2(8.0 * ln2 / (S_q * S_k)))), 14)
+    S = 8.0 * ln2 / (2.0 ** k * S_k)
+    for _ in range(64):                       # a few ulps down until floor(ln2 / score scale) is 2^k
+        if math.floor(ln2 / ((S * S_k) / 8.0)) == 2 ** k:
+            break
+        S = float(np.nextafter(S, 0.0))
+    assert S >= S_q * (1.0 - 1e-12) and math.floor(ln2 / ((S * S_k) / 8.0)) == 2 ** k
+    return S
+
+
 def make_input(config_id: int, B: int, L: int, H: int, shard: int = 0):
     """x ~ N(0,1) as int8 with S_x = max|x| / 127.  Returns (x_q [B*L, H], S_x).
 
@@ -123,11 +138,14 @@ def make_input(config_id: int, B: int, L: int, H: int, shard: int = 0):
 
 
 def make_layer(config_id: int, layer: int, H: int, heads: int, F: int, L: int, S_x: float,
-               p_max: int = 255) -> dict:
-    """One layer's integer parameters and static scales (a plain dict of numpy arrays)."""
+               p_max: int = 255, pow2_scores: bool = False) -> dict:
+    """One layer's integer parameters and static scales (a plain dict of numpy arrays).
+    pow2_scores: the query scale is raised (by less than 2x) so that the score scale is ln2 / 2^k."""
     assert H == heads * 64
     p = {"H": H, "heads": heads, "F": F, "p_max": p_max}
     p.update(static_activation_scales(H, F, L, S_x))
+    if pow2_scores:
+        p["S_q"] = snap_q_scale(p["S_q"], p["S_k"])
     in_scale = {"qkv": p["S_x"], "o": p["S_ctx"], "f1": p["S_h1"], "f2": p["S_go"]}
     shapes = {"qkv": (3 * H, H), "o": (H, H), "f1": (F, H), "f2": (H, F)}
     tids = {"qkv": (_T_WQKV, _T_BQKV), "o": (_T_WO, _T_BO), "f1": (_T_WF1, _T_BF1), "f2": (_T_WF2, _T_BF2)}
@@ -145,7 +163,8 @@ def make_layer(config_id: int, layer: int, H: int, heads: int, F: int, L: int, S
 
 
 def make_model(config_id: int, B: int, layers: int | None = None, H: int | None = None,
-               heads: int | None = None, F: int | None = None, L: int | None = None, shard: int = 0):
+               heads: int | None = None, F: int | None = None, L: int | None = None, shard: int = 0,
+               pow2_scores: bool = False):
     """Input and per-layer parameters of one of the encoder configs (0, 2, 3, 4).
     Layer l+1 consumes layer l's int8 output, so its S_x is layer l's S_out."""
     cfg = CONFIGS[config_id]
@@ -158,7 +177,7 @@ def make_model(config_id: int, B: int, layers: int | None = None, H: int | None 
     params = []
     s_in = S_x
     for l in range(layers):
-        p = make_layer(config_id, l, H, heads, F, L, s_in)
+        p = make_layer(config_id, l, H, heads, F, L, s_in, pow2_scores=pow2_scores)
         params.append(p)
         s_in = p["S_out"]
     return x, params

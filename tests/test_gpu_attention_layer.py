@@ -128,3 +128,34 @@ def test_layer_error_codes():
     assert e.value.code == -2
     layer.close()
     assert ctx().ibert_last_status() == 0
+
+
+@pytest.mark.parametrize("B,L,heads", [(2, 128, 3), (3, 100, 2), (2, 256, 2), (1, 512, 1), (2, 37, 1)])
+def test_attention_power_of_two_score_scale(B, L, heads):
+    """Score scale exactly ln2 / 2^k: the kernel takes quotient and remainder of i-exp by shift and
+    mask; the oracle is the ordinary one at that scale."""
+    H = heads * 64
+    rng = np.random.default_rng(L)
+    qkv = np.clip(np.rint(rng.standard_normal((B * L, 3 * H)) * 40), -127, 127).astype(np.int8)
+    S_k = 0.02
+    S_q = synth.snap_q_scale(0.02, S_k)
+    q_ln2 = oracle.exp_consts((S_q * S_k) / 8.0)["q_ln2"]
+    assert q_ln2 & (q_ln2 - 1) == 0
+    out, _ = ctx().ibert_attention_i8(dev(qkv), B, L, H, heads, S_q, S_k, 0.02, 0.006, 255)
+    ctx().check()
+    assert_same(host(out), oracle.attention(qkv, B, L, H, heads, S_q, S_k, 0.02, 0.006, 255), f"pow2 attention L={L}")
+    lens = np.array([L, 1, max(L // 2, 1)][:B], np.int32)
+    out, _ = ctx().ibert_attention_masked_i8(dev(qkv), B, L, H, heads, dev(lens), S_q, S_k, 0.02, 0.006, 255)
+    ctx().check()
+    assert_same(host(out), oracle.attention(qkv, B, L, H, heads, S_q, S_k, 0.02, 0.006, 255, lens=lens),
+                f"pow2 masked attention L={L}")
+
+
+def test_encoder_layers_with_power_of_two_score_scales():
+    B, L, H, heads, F = 2, 128, 256, 4, 1024
+    x, params = synth.make_model(0, B, layers=2, H=H, heads=heads, F=F, L=L, pow2_scores=True)
+    outs = _run_layers(x, params, B, L)
+    h = x
+    for p, got in zip(params, outs):
+        h = oracle.encoder_layer(p, h, B, L).out
+        assert_same(got, h, "pow2-score layer")

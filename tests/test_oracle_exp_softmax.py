@@ -130,3 +130,27 @@ def test_softmax_argument_checks():
         oracle.softmax(np.zeros((1, 1025), np.int32), 1e-3, 255)
     with pytest.raises(oracle.OracleError):
         oracle.softmax(np.zeros((1, 8), np.int32), 1e-3, 200)
+
+
+def test_power_of_two_score_scale_keeps_softmax_accuracy():
+    """Raising the query scale (by < 2x) so that the score scale is ln2 / 2^k makes q_ln2 a power of
+    two (quotient and remainder of i-exp become shift and mask) without leaving the accuracy class
+    of i-softmax: compared with the float softmax of the same real scores, the error stays within
+    the same bound as at the calibrated scale."""
+    from paper_2101_01321_b200 import synth
+    rng = np.random.default_rng(11)
+    S_k = 0.0175
+    for S_q in (0.0175, 0.011, 0.03):
+        S_q2 = synth.snap_q_scale(S_q, S_k)
+        assert S_q <= S_q2 < 2 * S_q
+        S1, S2 = (S_q * S_k) / 8.0, (S_q2 * S_k) / 8.0
+        k2 = oracle.exp_consts(S2)
+        assert k2["s_in"] == 0 and k2["q_ln2"] & (k2["q_ln2"] - 1) == 0
+        x = rng.standard_normal((64, 128)) * 2.0                    # real scores
+        ref = np.exp(x - x.max(-1, keepdims=True))
+        ref /= ref.sum(-1, keepdims=True)
+        errs = []
+        for S in (S1, S2):
+            p, S_p = oracle.softmax(np.rint(x / S).astype(np.int32), S)
+            errs.append(np.abs(p * S_p - ref).max())
+        assert errs[1] <= max(errs[0] * 1.5, 2.0 / 255.0), errs

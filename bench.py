@@ -1,12 +1,13 @@
 #!/usr/bin/env python
 """Throughput of the integer-only RoBERTa-Base encoder (I-BERT) on B200.
 
-One *step* = one forward pass of the whole 12-layer integer-only encoder (7 kernels per
+One *step* = one forward pass of the whole 12-layer integer-only encoder (5 kernels per
 layer, all inside libibert_b200) over one batch of synthetic int8 activations.
 Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle instead.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--config 2|3|4] [--batch B]
+                    [--workload layers|model] [--pow2-scores] [--graph] [--only KERNEL]
 """
 from __future__ import annotations
 

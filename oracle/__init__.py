@@ -158,6 +158,16 @@ def gelu(q, S: float, S_out: float) -> tuple[np.ndarray, float]:
     return out, float(S_ret.value)
 
 
+def hgelu(q, S: float, S_out: float) -> tuple[np.ndarray, float]:
+    """Integer h-GELU (Eq. 6: x ReLU6(1.702 x + 3) / 6), the comparison function of Table 1."""
+    q = _arr(q, np.int32)
+    out = np.empty(q.shape, dtype=np.int8)
+    S_ret = C.c_double()
+    _chk(lib().orc_hgelu(_p(q), C.c_double(S), C.c_int64(q.size), C.c_double(S_out), _p(out),
+                         C.byref(S_ret)), "hgelu")
+    return out, float(S_ret.value)
+
+
 # ------------------------------------------------------------------ i-LayerNorm
 def layernorm(q, S: float, r, S_r: float, gamma, beta, S_out: float) -> tuple[np.ndarray, float]:
     q = _arr(q, np.int32)

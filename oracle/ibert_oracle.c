@@ -325,6 +325,45 @@ int orc_gelu(const int32_t* q, double S, int64_t n, double S_out, int8_t* out, d
 }
 
 /* ------------------------------------------------------------------ */
+/* Eq. 6: h-GELU(x) = x ReLU6(1.702 x + 3) / 6 -- the hard-sigmoid      */
+/* approximation the paper measures i-GELU against (Table 1, Table 3).  */
+/* The paper only remarks that it "can be computed with integer         */
+/* arithmetic"; the integer form below is this build's reading, kept    */
+/* parallel to i-GELU: the same integer q read at scale S_h = 1.702 S   */
+/* stands for 1.702 x, so                                               */
+/*   q_3 = floor(3 / S_h), q_6 = floor(6 / S_h),                        */
+/*   r = clamp(q + q_3, 0, q_6)            (ReLU6 at scale S_h),        */
+/*   g = q (r >> s_h)                      (scale S S_h 2^s_h / 6),     */
+/* with s_h keeping the product inside 32 bits, then round(g / 256)     */
+/* and the dyadic requantization to int8, exactly as for i-GELU.        */
+/* ------------------------------------------------------------------ */
+int orc_hgelu(const int32_t* q, double S, int64_t n, double S_out, int8_t* out, double* S_ret) {
+  if (!(S > 0.0) || !isfinite(S) || !(S_out > 0.0) || !isfinite(S_out) || n < 0) return ORC_ERR_SCALE_RANGE;
+  const double S_h = 1.702 * S;
+  const double q3d = floor(3.0 / S_h), q6d = floor(6.0 / S_h);
+  if (q6d < 1.0 || q6d > 1.0e9) return ORC_ERR_SCALE_RANGE;
+  const int64_t q3 = (int64_t)q3d, q6 = (int64_t)q6d;
+  const int bl = bit_length((uint64_t)q6);
+  const int s_h = bl > 15 ? bl - 15 : 0;
+  const double S_g2 = (ldexp(S * S_h, s_h) / 6.0) * 256.0;
+  int64_t b; int c;
+  int rc = orc_dyadic(S_g2 / S_out, &b, &c);
+  if (rc) return rc;
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < n; ++i) {
+    const int64_t v = clamp_sym((int64_t)q[i], 32767);
+    int64_t r = v + q3;
+    if (r < 0) r = 0;
+    if (r > q6) r = q6;
+    const int64_t g = v * shift_right_floor(r, s_h);
+    const int64_t g2 = orc_round_shift(g, 8);
+    out[i] = (int8_t)orc_requant(g2, b, c, 127);
+  }
+  if (S_ret) *S_ret = S_out;
+  return ORC_OK;
+}
+
+/* ------------------------------------------------------------------ */
 /* Sec. 3.6: i-LayerNorm (with the residual add in front of it)        */
 /* ------------------------------------------------------------------ */
 

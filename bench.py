@@ -116,14 +116,18 @@ def algorithmic_work(H: int, F: int, L: int, heads: int, T: int) -> dict:
 
 
 # --------------------------------------------------------------------------- reference arm
-def oracle_sample_run(cfg_id: int, n_seq: int, layers: int | None = None, full_model: bool = False):
+def oracle_sample_run(cfg_id: int, n_seq: int, layers: int | None = None, full_model: bool = False,
+                      L: int | None = None):
     """Runs the CPU oracle on the first n_seq sequences of the workload; returns (tokens, seconds, layers)."""
     import oracle
     from paper_2101_01321_b200 import synth
     cfg = synth.CONFIGS[cfg_id]
+    if L:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, L=L)
     oracle.lib()
     if full_model:
-        m = synth.make_full_model(cfg_id, n_seq, layers=layers)
+        m = synth.make_full_model(cfg_id, n_seq, layers=layers, L=cfg.L)
         e, hd = m["emb"], m["head"]
         t0 = time.perf_counter()
         h = oracle.embedding(m["ids"], cfg.L, e["word"], e["S_word"], e["pos"], e["S_pos"], e["gamma"], e["beta"],
@@ -133,7 +137,7 @@ def oracle_sample_run(cfg_id: int, n_seq: int, layers: int | None = None, full_m
         oracle.classifier(h, n_seq, cfg.L, m["layers"][-1]["S_out"], hd["w"], hd["S_w"], hd["bias"])
         dt = time.perf_counter() - t0
         return n_seq * cfg.L, dt, len(m["layers"])
-    x, params = synth.make_model(cfg_id, n_seq, layers=layers)
+    x, params = synth.make_model(cfg_id, n_seq, layers=layers, L=cfg.L)
     t0 = time.perf_counter()
     h = x
     for p in params:
@@ -149,12 +153,15 @@ def run_reference(args):
     import oracle
     from paper_2101_01321_b200 import synth
     cfg = synth.CONFIGS[args.config]
+    if args.seq_len:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, L=args.seq_len)
     batch = args.batch or DEFAULT_BATCH[args.config]
     n_seq = 2
     full_model = args.workload == "model"
     oracle.lib()
     if full_model:
-        m = synth.make_full_model(args.config, n_seq)
+        m = synth.make_full_model(args.config, n_seq, L=cfg.L)
         params, e, hd = m["layers"], m["emb"], m["head"]
 
         def step():
@@ -164,7 +171,7 @@ def run_reference(args):
                 h = oracle.encoder_layer(p, h, n_seq, cfg.L, lens=m["lens"]).out
             return oracle.classifier(h, n_seq, cfg.L, params[-1]["S_out"], hd["w"], hd["S_w"], hd["bias"])
     else:
-        x, params = synth.make_model(args.config, n_seq)
+        x, params = synth.make_model(args.config, n_seq, L=cfg.L)
 
         def step():
             h = x
@@ -232,6 +239,9 @@ def run_ours(args):
     build.build()
 
     cfg = synth.CONFIGS[args.config]
+    if args.seq_len:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, L=args.seq_len)
     batch = args.batch or DEFAULT_BATCH[args.config]
     T = batch * cfg.L
     # weak scaling: rank r owns sequences [r*batch, (r+1)*batch) of the global batch
@@ -244,7 +254,7 @@ def run_ours(args):
     full_model = args.workload == "model"
     if not full_model:
         # the headline workload: the encoder layers on full-length sequences, int8 activations in and out
-        x_np, params = synth.make_model(args.config, batch, shard=rank, pow2_scores=args.pow2_scores)
+        x_np, params = synth.make_model(args.config, batch, shard=rank, pow2_scores=args.pow2_scores, L=cfg.L)
         layers = [ctx.ibert_layer_create(p) for p in params]
         x_dev = torch.from_numpy(x_np).to(dev)
         x_pin = torch.from_numpy(x_np).pin_memory()
@@ -268,7 +278,7 @@ def run_ours(args):
     else:
         # the model around the layers on a padded batch: token ids in, INT8 embedding + LayerNorm,
         # the layers with a key-padding mask, first-token classifier, INT32 logits out
-        m = synth.make_full_model(args.config, batch, shard=rank)
+        m = synth.make_full_model(args.config, batch, shard=rank, L=cfg.L)
         layers = [ctx.ibert_layer_create(p) for p in m["layers"]]
         e, hd = m["emb"], m["head"]
         word_d, pos_d = torch.from_numpy(e["word"]).to(dev), torch.from_numpy(e["pos"]).to(dev)
@@ -392,7 +402,7 @@ def run_ours(args):
 
         # CPU baseline: the oracle on a bounded sample of the same workload
         n_seq = 8
-        tok_s, dt_s, n_layers = oracle_sample_run(args.config, n_seq, full_model=full_model)
+        tok_s, dt_s, n_layers = oracle_sample_run(args.config, n_seq, full_model=full_model, L=cfg.L)
         import oracle
         cpu = {"value": tok_s / dt_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                "sample": f"first {n_seq} sequences ({tok_s} tokens) through "
@@ -435,6 +445,9 @@ def run_only(args):
 
     build.build()
     cfg = synth.CONFIGS[args.config]
+    if args.seq_len:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, L=args.seq_len)
     batch = args.batch or DEFAULT_BATCH[args.config]
     T, H, F, L = batch * cfg.L, cfg.H, cfg.F, cfg.L
     dev = torch.device("cuda", 0)
@@ -460,7 +473,8 @@ def run_only(args):
         fn = lambda: ctx.ibert_linear_layernorm_i8(x, S_x, w, S_w, bias, 8 * S_acc / 32767, res, S_acc / 127,
                                                    gamma, beta, 4.5 / 127, out=out)
     elif k.startswith("gemm"):
-        N, K = {"gemm_qkv": (3 * H, H), "gemm_out": (H, H), "gemm_ffn1_gelu": (F, H), "gemm_ffn2": (H, F)}[k]
+        N, K = {"gemm_qkv": (3 * H, H), "gemm_out": (H, H), "gemm_ffn1_gelu": (F, H), "gemm_ffn1_hgelu": (F, H),
+                "gemm_ffn2": (H, F)}[k]
         x, w = i8(T, K), i8(N, K)
         bias = torch.randint(-1000, 1000, (N,), generator=g, dtype=torch.int32).to(dev)
         S_w = rng.uniform(5e-4, 7e-4, N)
@@ -469,6 +483,9 @@ def run_only(args):
         if k == "gemm_ffn1_gelu":
             out = torch.empty((T, N), dtype=torch.int8, device=dev)
             fn = lambda: ctx.ibert_linear_gelu_i8(x, S_x, w, S_w, bias, 8 * S_acc / 32767, 4 * S_acc / 127, out=out)
+        elif k == "gemm_ffn1_hgelu":
+            out = torch.empty((T, N), dtype=torch.int8, device=dev)
+            fn = lambda: ctx.ibert_linear_hgelu_i8(x, S_x, w, S_w, bias, 8 * S_acc / 32767, 4 * S_acc / 127, out=out)
         elif k == "gemm_qkv":
             out = torch.empty((T, N), dtype=torch.int8, device=dev)
             fn = lambda: ctx.ibert_linear_i8(x, S_x, w, S_w, bias, 0, 4 * S_acc / 127, out=out)
@@ -484,11 +501,12 @@ def run_only(args):
         qd, rd = torch.from_numpy(q).to(dev), torch.from_numpy(r).to(dev)
         out = torch.empty((T, H), dtype=torch.int8, device=dev)
         fn = lambda: ctx.ibert_layernorm_i(qd, S, rd, S_r, gamma, beta, S_out, out=out)
-    elif k == "gelu":
+    elif k in ("gelu", "hgelu"):
         q, S, S_out = synth.gelu_inputs(1 << 24, 1.0)
         qd = torch.from_numpy(q).to(dev)
         out = torch.empty(q.shape, dtype=torch.int8, device=dev)
-        fn = lambda: ctx.ibert_gelu_i(qd, S, S_out, out=out)
+        fn = (lambda: ctx.ibert_gelu_i(qd, S, S_out, out=out)) if k == "gelu" else \
+             (lambda: ctx.ibert_hgelu_i(qd, S, S_out, out=out))
     elif k == "softmax":
         rows = batch * cfg.heads * L
         q, S = synth.softmax_inputs(rows, L, 1.0)
@@ -525,6 +543,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4])
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--seq-len", type=int, default=0, help="override the config's sequence length (latency grids)")
     ap.add_argument("--pow2-scores", action="store_true",
                     help="layers workload: query scales raised so that every score scale is ln2 / 2^k "
                          "(i-exp quotient by shift and mask)")

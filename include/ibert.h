@@ -211,6 +211,21 @@ int ibert_embedding_i8(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, con
 int ibert_classifier_i8(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, double S_x, const int8_t* w,
                         const double* S_w, const int32_t* bias, int N, int32_t* logits, double* S_ret);
 
+/* ---- h-GELU, the comparison function of the paper (Eq. 6; Table 1, Table 3) --------------------
+   h-GELU(x) = x ReLU6(1.702 x + 3) / 6.  The paper notes that it can be computed with integers
+   but gives no integer algorithm; this library's reading keeps it parallel to i-GELU: the same
+   integer q read at scale S_h = 1.702 S stands for 1.702 x, q_3 = floor(3 / S_h),
+   q_6 = floor(6 / S_h), r = clamp(q + q_3, 0, q_6) >> s_h (s_h keeps the product in 32 bits),
+   g = q r at scale S S_h 2^s_h / 6, then round(g / 256) and a dyadic requantization to int8.
+   Not part of ibert_encoder_layer (the paper rejects h-GELU for its accuracy); provided to measure
+   what i-GELU's polynomial costs.  Arguments, layouts and errors as ibert_gelu_i and
+   ibert_linear_gelu_i8. */
+int ibert_hgelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
+                  double* S_ret);
+int ibert_linear_hgelu_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
+                          const int32_t* bias, int64_t M, int N, int K, double S_mid, double S_out,
+                          int8_t* out, double* S_ret);
+
 /* ---- a stack of encoder layers captured into a CUDA graph ---------------------------------------
    No counterpart in the paper: launch-overhead removal for small batches (a 12-layer pass is 60
    kernel launches).  ibert_encoder_graph_create runs layers[0..n_layers) once on the context's

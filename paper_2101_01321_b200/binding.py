@@ -58,6 +58,8 @@ def lib():
         L.ibert_linear_gelu_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, dbl, vp, vp]
         L.ibert_linear_layernorm_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, vp, dbl, vp, vp, dbl,
                                                 vp, vp]
+        L.ibert_hgelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
+        L.ibert_linear_hgelu_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, dbl, vp, vp]
         L.ibert_softmax_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
         L.ibert_gelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
         L.ibert_layernorm_i.argtypes = [vp, vp, dbl, vp, dbl, vp, vp, i64, i32, dbl, vp, vp]
@@ -85,7 +87,8 @@ def lib():
                      "ibert_layernorm_i", "ibert_attention_i8", "ibert_layer_create", "ibert_layer_destroy",
                      "ibert_encoder_layer", "ibert_attention_masked_i8", "ibert_encoder_layer_masked",
                      "ibert_embedding_i8", "ibert_classifier_i8", "ibert_encoder_graph_create",
-                     "ibert_encoder_graph_launch", "ibert_encoder_graph_destroy"):
+                     "ibert_encoder_graph_launch", "ibert_encoder_graph_destroy", "ibert_hgelu_i",
+                     "ibert_linear_hgelu_i8"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -177,6 +180,15 @@ class Context:
                                 C.byref(S_ret)), "ibert_gelu_i")
         return out, S_ret.value
 
+    def ibert_hgelu_i(self, q: torch.Tensor, S: float, S_out: float, out: torch.Tensor | None = None):
+        """Integer h-GELU (Eq. 6), the paper's comparison function."""
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.int8, device=q.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_hgelu_i(self.h, _dev(q, torch.int32), S, q.numel(), S_out, _dev(out, torch.int8),
+                                 C.byref(S_ret)), "ibert_hgelu_i")
+        return out, S_ret.value
+
     def ibert_softmax_i(self, q: torch.Tensor, S: float, p_max: int = 255, out: torch.Tensor | None = None):
         L = q.shape[-1]
         rows = q.numel() // L if L else 0
@@ -217,6 +229,20 @@ class Context:
                                    _dev(bias, torch.int32), M, N, K, out_kind, S_out, out.data_ptr(),
                                    S_ret.ctypes.data), "ibert_linear_i8")
         return out, (S_ret if out_kind == 2 else float(S_ret[0]))
+
+    def ibert_linear_hgelu_i8(self, x: torch.Tensor, S_x: float, w: torch.Tensor, S_w, bias: torch.Tensor | None,
+                              S_mid: float, S_out: float, out: torch.Tensor | None = None):
+        K = x.shape[-1]
+        M = x.numel() // K
+        N = w.shape[0]
+        sw = _host(S_w, np.float64)
+        if out is None:
+            out = torch.empty(x.shape[:-1] + (N,), dtype=torch.int8, device=x.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_linear_hgelu_i8(self.h, _dev(x, torch.int8), S_x, _dev(w, torch.int8), sw.ctypes.data,
+                                         _dev(bias, torch.int32), M, N, K, S_mid, S_out, _dev(out, torch.int8),
+                                         C.byref(S_ret)), "ibert_linear_hgelu_i8")
+        return out, S_ret.value
 
     def ibert_linear_layernorm_i8(self, x: torch.Tensor, S_x: float, w: torch.Tensor, S_w,
                                   bias: torch.Tensor | None, S_mid: float, res: torch.Tensor, S_res: float,

@@ -54,7 +54,7 @@ struct ProfileScope {
 
 inline int gemm_class(int kind, int K) {
   if (kind == EPI_INT8) return IBERT_K_GEMM_QKV;
-  if (kind == EPI_GELU) return IBERT_K_GEMM_GELU;
+  if (kind == EPI_GELU || kind == EPI_HGELU) return IBERT_K_GEMM_GELU;
   return K > 2048 ? IBERT_K_GEMM_Q16_WIDE : IBERT_K_GEMM_Q16;
 }
 
@@ -173,12 +173,12 @@ int ibert_last_status(ibert_ctx* ctx) {
   return st;
 }
 
-int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
-                 double* S_ret) {
+static int gelu_common(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
+                       double* S_ret, bool hard) {
   if (!ctx || n < 0 || (n > 0 && (!q || !out))) return IBERT_ERR_ARG;
   if (!aligned16(q) || !aligned16(out)) return IBERT_ERR_ALIGN;
   GeluConsts k;
-  int rc = make_gelu_consts(S, S_out, &k);
+  int rc = hard ? make_hgelu_consts(S, S_out, &k) : make_gelu_consts(S, S_out, &k);
   if (rc) return rc;
   DeviceGuard guard(ctx->device);
   {
@@ -187,6 +187,16 @@ int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S
   }
   if (rc == IBERT_OK && S_ret) *S_ret = S_out;
   return rc;
+}
+
+int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
+                 double* S_ret) {
+  return gelu_common(ctx, q, S, n, S_out, out, S_ret, false);
+}
+
+int ibert_hgelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
+                  double* S_ret) {
+  return gelu_common(ctx, q, S, n, S_out, out, S_ret, true);
 }
 
 int ibert_softmax_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
@@ -245,9 +255,9 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
                          const int32_t* bias, int64_t M, int N, int K, int kind, double S_mid,
                          double S_out, void* out, double* S_ret) {
   if (!ctx || M < 0 || !S_w) return IBERT_ERR_ARG;
-  if (kind < 0 || kind > 3) return IBERT_ERR_ARG;
+  if (kind < 0 || kind > 4) return IBERT_ERR_ARG;
   if (N < 1 || K < 1 || K % 16 != 0 || N % 4 != 0) return IBERT_ERR_SHAPE;
-  if ((kind == EPI_INT8 || kind == EPI_GELU) && N % 16 != 0) return IBERT_ERR_SHAPE;
+  if ((kind == EPI_INT8 || kind == EPI_GELU || kind == EPI_HGELU) && N % 16 != 0) return IBERT_ERR_SHAPE;
   if ((int64_t)K * 127 * 127 >= (int64_t(1) << 31)) return IBERT_ERR_SHAPE;
   if (M > 0 && (!x || !out)) return IBERT_ERR_ARG;
   if (!w) return IBERT_ERR_ARG;
@@ -260,7 +270,7 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
   epi.d_bias = bias;
   DeviceGuard guard(ctx->device);
   if (kind != EPI_RAW) {
-    const double S_acc_to = kind == EPI_GELU ? S_mid : S_out;
+    const double S_acc_to = (kind == EPI_GELU || kind == EPI_HGELU) ? S_mid : S_out;
     std::vector<int32_t> b, c;
     int rc = make_linear_tables(S_x, S_w, N, nullptr, S_acc_to, &b, &c);
     if (rc) return rc;
@@ -272,8 +282,8 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
     if (rc) return rc;
     epi.d_b = (const int32_t*)d_b;
     epi.d_c = (const int32_t*)d_c;
-    if (kind == EPI_GELU) {
-      rc = make_gelu_consts(S_mid, S_out, &epi.gelu);
+    if (kind == EPI_GELU || kind == EPI_HGELU) {
+      rc = kind == EPI_HGELU ? make_hgelu_consts(S_mid, S_out, &epi.gelu) : make_gelu_consts(S_mid, S_out, &epi.gelu);
       if (rc) return rc;
     }
   }
@@ -364,6 +374,12 @@ int ibert_linear_gelu_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
                          const int32_t* bias, int64_t M, int N, int K, double S_mid, double S_out,
                          int8_t* out, double* S_ret) {
   return linear_common(ctx, x, S_x, w, S_w, bias, M, N, K, EPI_GELU, S_mid, S_out, out, S_ret);
+}
+
+int ibert_linear_hgelu_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
+                          const int32_t* bias, int64_t M, int N, int K, double S_mid, double S_out,
+                          int8_t* out, double* S_ret) {
+  return linear_common(ctx, x, S_x, w, S_w, bias, M, N, K, EPI_HGELU, S_mid, S_out, out, S_ret);
 }
 
 static int make_attn_consts(double S_q, double S_k, double S_v, double S_ctx, int p_max, AttnConsts* k) {

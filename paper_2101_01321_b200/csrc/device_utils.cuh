@@ -90,6 +90,18 @@ __device__ __forceinline__ int32_t igelu_magnitude_upper(int32_t x, const GeluCo
   return requant_upper(g2, k.b2);
 }
 
+// Integer h-GELU (Eq. 6) of one Q16 value before its clamp: r = clamp(q + q_3, 0, q_6) >> s_h,
+// g = q r, round(g / 256), dyadic requantization (GeluConsts with hard != 0).
+__device__ __forceinline__ int32_t ihgelu_upper(int32_t x, const GeluConsts& k) {
+  const int32_t v = clamp_sym(x, 32767);
+  const int32_t r = min(max(v + k.q_c, 0), k.nq_b) >> k.s_f;
+  return requant_upper((v * r + 128) >> 8, k.b2);
+}
+__device__ __forceinline__ int32_t ihgelu_to_int8(int32_t q, const GeluConsts& k, int64_t half) {
+  const int32_t r = min(max(q + k.q_c, 0), k.nq_b) >> k.s_f;
+  return requant_add((q * r + 128) >> 8, k.b, half, k.c, 127);
+}
+
 __device__ __forceinline__ uint32_t shr_clamped(uint32_t v, uint32_t n) {
   uint32_t r;
   asm("shr.u32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(n));   // shift counts above 31 give 0

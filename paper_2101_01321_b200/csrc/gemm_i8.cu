@@ -297,8 +297,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if constexpr (FAST) o = clamp_sym(requant_upper(a + cur_bias, cur_pb), 127);
             else o = requant_add(a, cur_pb, cur_padd, cur_pc, 127);
           } else {
-            if constexpr (FAST) o = clamp_sym(igelu_magnitude_upper(requant_upper(a + cur_bias, cur_pb), gk, gelu_rnd), 127);
-            else o = igelu_q16_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
+            if constexpr (KIND == EPI_HGELU) {
+              if constexpr (FAST) o = clamp_sym(ihgelu_upper(requant_upper(a + cur_bias, cur_pb), gk), 127);
+              else o = ihgelu_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
+            } else {
+              if constexpr (FAST) o = clamp_sym(igelu_magnitude_upper(requant_upper(a + cur_bias, cur_pb), gk, gelu_rnd), 127);
+              else o = igelu_q16_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
+            }
           }
           // staging tile: row = token i, column = this lane's channel
           if constexpr (kOut32) reinterpret_cast<int32_t*>(stage)[i * 32 + lane] = o;
@@ -358,6 +363,7 @@ int launch_shape(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, c
     case EPI_INT8: return fast ? launch_inst<TOK, PAIR, EPI_INT8, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_INT8, false>(ctx, mw, mx, mo, a);
     case EPI_Q16: return fast ? launch_inst<TOK, PAIR, EPI_Q16, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_Q16, false>(ctx, mw, mx, mo, a);
     case EPI_GELU: return fast ? launch_inst<TOK, PAIR, EPI_GELU, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_GELU, false>(ctx, mw, mx, mo, a);
+    case EPI_HGELU: return fast ? launch_inst<TOK, PAIR, EPI_HGELU, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_HGELU, false>(ctx, mw, mx, mo, a);
     default: return launch_inst<TOK, PAIR, EPI_RAW, false>(ctx, mw, mx, mo, a);
   }
 }
@@ -403,7 +409,7 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
   a.b = epi.d_b; a.c = epi.d_c; a.bias = epi.d_bias; a.gelu = epi.gelu;
   a.status = ctx->d_status;
   // upper-word epilogue needs both the per-channel multipliers and (for GELU) the final one in that form
-  const bool fast = epi.fast != 0 && (epi.kind != EPI_GELU || epi.gelu.fast != 0);
+  const bool fast = epi.fast != 0 && ((epi.kind != EPI_GELU && epi.kind != EPI_HGELU) || epi.gelu.fast != 0);
   if (pair) return launch_shape<256, true>(ctx, mw, mx, mo, a, epi.kind, fast);
   return wide ? launch_shape<256, false>(ctx, mw, mx, mo, a, epi.kind, fast)
               : launch_shape<128, false>(ctx, mw, mx, mo, a, epi.kind, fast);

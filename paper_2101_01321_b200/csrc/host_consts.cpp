@@ -144,6 +144,31 @@ int make_gelu_consts(double S, double S_out, GeluConsts* k) {
   k->fast = to_upper_word_form(&b1, c1) ? 1 : 0;
   k->b2 = k->fast ? b1[0] : 0;
   k->add2 = k->fast ? (int64_t(1) << 31) : 0;                 // 2^(c-1) << (32-c)
+  k->hard = 0;
+  return IBERT_OK;
+}
+
+// Integer h-GELU (Eq. 6): the same integer q read at scale S_h = 1.702 S stands for 1.702 x;
+// r = clamp(q + q_3, 0, q_6) is ReLU6(1.702 x + 3) at that scale, g = q (r >> s_h) has scale
+// S S_h 2^s_h / 6; round(g / 256) and the dyadic step to S_out follow as for i-GELU.
+int make_hgelu_consts(double S, double S_out, GeluConsts* k) {
+  if (!good_scale(S) || !good_scale(S_out)) return IBERT_ERR_SCALE_RANGE;
+  const double S_h = 1.702 * S;
+  const double q3 = std::floor(3.0 / S_h), q6 = std::floor(6.0 / S_h);
+  if (q6 < 1.0 || q6 > 1.0e9) return IBERT_ERR_SCALE_RANGE;
+  const int bl = bit_length_u64((uint64_t)q6);
+  *k = GeluConsts{};
+  k->hard = 1;
+  k->nq_b = (int32_t)q6;
+  k->q_c = (int32_t)q3;
+  k->s_f = bl > 15 ? bl - 15 : 0;
+  const double S_g2 = (std::ldexp(S * S_h, k->s_f) / 6.0) * 256.0;
+  int rc = dyadic(S_g2 / S_out, &k->b, &k->c);
+  if (rc) return rc;
+  std::vector<int32_t> b1(1, k->b), c1(1, k->c);
+  k->fast = to_upper_word_form(&b1, c1) ? 1 : 0;
+  k->b2 = k->fast ? b1[0] : 0;
+  k->add2 = k->fast ? (int64_t(1) << 31) : 0;
   return IBERT_OK;
 }
 

@@ -48,6 +48,9 @@ struct GeluConsts {
   // (g2 * b + 2^(c-1)) >> c == (g2 * b2 + add2) >> 32 with b2 = b << (32-c); valid when fast != 0
   int32_t b2, fast;
   int64_t add2;
+  // h-GELU (Eq. 6) through the same plumbing: hard != 0 and the fields above mean
+  // nq_b = q_6 = floor(6 / S_h), q_c = q_3 = floor(3 / S_h), s_f = s_h, s_in unused (S_h = 1.702 S)
+  int32_t hard;
 };
 
 // residual add in front of i-LayerNorm
@@ -67,6 +70,7 @@ struct LnConsts {
 int dyadic(double m, int32_t* b, int32_t* c);
 int make_exp_consts(double S, int p_max, ExpConsts* k);
 int make_gelu_consts(double S, double S_out, GeluConsts* k);
+int make_hgelu_consts(double S, double S_out, GeluConsts* k);
 // per-channel multipliers b_i (int32) and addends B_i (int64, rounding constant included)
 int make_ln_tables(const double* gamma, const double* beta, int C, double S_out, LnConsts* k,
                    std::vector<int32_t>* b_i, std::vector<int64_t>* B_i);
@@ -121,7 +125,7 @@ int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t 
                      const int32_t* d_b, const int64_t* d_B, int8_t* out);
 
 // epilogue kinds of the GEMM
-enum : int { EPI_INT8 = 0, EPI_Q16 = 1, EPI_RAW = 2, EPI_GELU = 3 };
+enum : int { EPI_INT8 = 0, EPI_Q16 = 1, EPI_RAW = 2, EPI_GELU = 3, EPI_HGELU = 4 };
 
 struct GemmEpilogue {
   int kind;
@@ -129,7 +133,7 @@ struct GemmEpilogue {
   const int32_t* d_c;      // [N] dyadic shifts
   const int32_t* d_bias;   // [N] or nullptr
   int fast;                // every column's requantization fits the upper-word form
-  GeluConsts gelu;         // EPI_GELU only
+  GeluConsts gelu;         // EPI_GELU / EPI_HGELU only
 };
 
 // Upper-word form of a column set: true if for every n, c[n] >= 1 and b[n] << (32 - c[n]) fits

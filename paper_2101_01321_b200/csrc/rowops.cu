@@ -38,7 +38,12 @@ __global__ void __launch_bounds__(kThreads) gelu_kernel(const int32_t* __restric
       const int64_t idx = base + j * 32 + lane;
       if (idx < n_vec) {
         int32_t a, b, c, d;
-        if (k.fast) {
+        if (k.hard) {
+          a = k.fast ? max(ihgelu_upper(v[j].x, k), -127) : ihgelu_to_int8(clamp_sym(v[j].x, 32767), k, half);
+          b = k.fast ? max(ihgelu_upper(v[j].y, k), -127) : ihgelu_to_int8(clamp_sym(v[j].y, 32767), k, half);
+          c = k.fast ? max(ihgelu_upper(v[j].z, k), -127) : ihgelu_to_int8(clamp_sym(v[j].z, 32767), k, half);
+          d = k.fast ? max(ihgelu_upper(v[j].w, k), -127) : ihgelu_to_int8(clamp_sym(v[j].w, 32767), k, half);
+        } else if (k.fast) {
           a = max(igelu_magnitude_upper(v[j].x, k, rnd_f), -127);
           b = max(igelu_magnitude_upper(v[j].y, k, rnd_f), -127);
           c = max(igelu_magnitude_upper(v[j].z, k, rnd_f), -127);
@@ -57,7 +62,8 @@ __global__ void __launch_bounds__(kThreads) gelu_kernel(const int32_t* __restric
   const int64_t tid = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   const int64_t tail = n_vec << 2;
   if (tid < n - tail)
-    out[tail + tid] = (int8_t)igelu_q16_to_int8(clamp_sym(q[tail + tid], 32767), k, half);
+    out[tail + tid] = (int8_t)(k.hard ? ihgelu_to_int8(clamp_sym(q[tail + tid], 32767), k, half)
+                                      : igelu_q16_to_int8(clamp_sym(q[tail + tid], 32767), k, half));
 }
 
 // ----------------------------------------------------------------------------- i-softmax

@@ -1,0 +1,49 @@
+"""GPU parity (bit-exact) of the integer h-GELU (Eq. 6), standalone and as a GEMM epilogue."""
+import numpy as np
+import pytest
+
+import oracle
+from gpu_util import assert_same, ctx, dev, host
+from paper_2101_01321_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("n,sigma", [(1 << 20, 1.0), (100003, 4.0), (5, 1.0), (0, 1.0)])
+def test_hgelu_matches_oracle(n, sigma):
+    q, S, S_out = synth.gelu_inputs(max(n, 1), sigma)
+    q = q[:n]
+    out, S_ret = ctx().ibert_hgelu_i(dev(q), S, S_out)
+    ctx().check()
+    assert S_ret == S_out
+    if n:
+        want, _ = oracle.hgelu(q, S, S_out)
+        assert_same(host(out), want, "h-GELU")
+        assert (n < 1000 or want.max() > 100) and want.min() <= 0
+
+
+def test_hgelu_full_int32_range_and_odd_scales():
+    rng = np.random.default_rng(2)
+    q = np.concatenate([rng.integers(-2**31, 2**31, 100000), np.arange(-40000, 40000, 7),
+                        [2**31 - 1, -2**31, 0, 1, -1, 32767, -32767, 32768, -32768]]).astype(np.int32)
+    for S, S_out in [(1e-3, 4.0 / 127), (1.2207e-4, 0.03), (3.3e-5, 0.011), (0.02, 0.9)]:
+        out, _ = ctx().ibert_hgelu_i(dev(q), S, S_out)
+        ctx().check()
+        assert_same(host(out), oracle.hgelu(q, S, S_out)[0], f"h-GELU S={S}")
+
+
+@pytest.mark.parametrize("M,N,K", [(130, 272, 144), (300, 3072, 768), (2100, 512, 256)])
+def test_linear_hgelu_matches_oracle(M, N, K):
+    rng = np.random.default_rng(M + N)
+    x = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    w = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    bias = rng.integers(-200000, 200000, N).astype(np.int32)
+    S_w = rng.uniform(1e-4, 4e-4, N)
+    S_x = 0.03
+    amax = 127.0 * 127.0 * np.sqrt(K) * 1.2 * S_x * 2.5e-4
+    S_mid, S_out = 2.0 * amax / 32767, amax / 127
+    out, _ = ctx().ibert_linear_hgelu_i8(dev(x), S_x, dev(w), S_w, dev(bias), S_mid, S_out)
+    ctx().check()
+    mid = oracle.linear(x, S_x, w, S_w, bias, 1, S_mid)
+    want, _ = oracle.hgelu(mid, S_mid, S_out)
+    assert_same(host(out), want.reshape(M, N), "linear + h-GELU")

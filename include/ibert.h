@@ -155,14 +155,21 @@ int ibert_layer_destroy(ibert_layer* layer);
    scale S_x*S_w[n], or NULL; res: device int8 [M, N] at host scale S_res; gamma, beta: host
    double [N]; out: device int8 [M, N] at S_out (*S_ret).  The result is bit-identical to
    ibert_linear_i8(kind 1, S_mid) followed by ibert_layernorm_i.  When N is a multiple of 256 (at
-   most 2048) and the constants fit the 32-bit forms, a single kernel computes it on a cluster of
-   N/256 CTAs per 128-row tile and the Q16 tensor never reaches memory; otherwise the two kernels
-   run back to back through the context's workspace.
+   most 2048), the constants fit the 32-bit forms and M is large enough for its 128-row tiles to
+   occupy half of the SMs, a single kernel computes it on a cluster of N/256 CTAs per tile and the
+   Q16 tensor never reaches memory; otherwise the two kernels run back to back through the
+   context's workspace.
    Errors: as ibert_linear_i8 and ibert_layernorm_i. */
 int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
                               const int32_t* bias, int64_t M, int N, int K, double S_mid,
                               const int8_t* res, double S_res, const double* gamma, const double* beta,
                               double S_out, int8_t* out, double* S_ret);
+
+/* How ibert_linear_layernorm_i8 and ibert_encoder_layer choose between the single cluster kernel and
+   the two-kernel sequence (the results are identical): mode 0 (default) by problem size, 1 the
+   cluster kernel whenever shapes and constants allow it, 2 never.  No counterpart in the paper:
+   a tuning and testing switch.  Returns IBERT_ERR_ARG for another mode. */
+int ibert_set_fusion(ibert_ctx* ctx, int mode);
 
 /* The integer-only encoder layer (Fig. 1 right; post-LN order):
    QKV projection -> attention (i-softmax) -> output projection -> +x, i-LayerNorm ->

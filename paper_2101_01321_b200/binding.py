@@ -60,6 +60,7 @@ def lib():
                                                 vp, vp]
         L.ibert_hgelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
         L.ibert_linear_hgelu_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, dbl, vp, vp]
+        L.ibert_set_fusion.argtypes = [vp, i32]
         L.ibert_softmax_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
         L.ibert_gelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
         L.ibert_layernorm_i.argtypes = [vp, vp, dbl, vp, dbl, vp, vp, i64, i32, dbl, vp, vp]
@@ -88,7 +89,7 @@ def lib():
                      "ibert_encoder_layer", "ibert_attention_masked_i8", "ibert_encoder_layer_masked",
                      "ibert_embedding_i8", "ibert_classifier_i8", "ibert_encoder_graph_create",
                      "ibert_encoder_graph_launch", "ibert_encoder_graph_destroy", "ibert_hgelu_i",
-                     "ibert_linear_hgelu_i8"):
+                     "ibert_linear_hgelu_i8", "ibert_set_fusion"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -157,6 +158,10 @@ class Context:
 
     def ibert_last_status(self) -> int:
         return int(lib().ibert_last_status(self.h))
+
+    def ibert_set_fusion(self, mode: int):
+        """0: linear + LayerNorm fusion by problem size (default), 1: whenever supported, 2: never."""
+        _chk(lib().ibert_set_fusion(self.h, mode), "ibert_set_fusion")
 
     def check(self):
         _chk(self.ibert_last_status(), "ibert_last_status")

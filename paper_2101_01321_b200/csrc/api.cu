@@ -162,6 +162,12 @@ int ibert_destroy(ibert_ctx* ctx) {
   return IBERT_OK;
 }
 
+int ibert_set_fusion(ibert_ctx* ctx, int mode) {
+  if (!ctx || mode < 0 || mode > 2) return IBERT_ERR_ARG;
+  ctx->fusion_mode = mode;
+  return IBERT_OK;
+}
+
 int ibert_last_status(ibert_ctx* ctx) {
   if (!ctx) return IBERT_ERR_ARG;
   DeviceGuard guard(ctx->device);
@@ -299,6 +305,16 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
   return rc;
 }
 
+// true when T tokens give the fused GEMM + LayerNorm kernel (one cluster of H / 256 CTAs per
+// 128-token tile) enough tiles to occupy at least half of the SMs; measured crossover on config 2:
+// the two-kernel path wins up to T = 2048 (0.63 vs 0.76 ms at T = 128), the fused one from T = 4096
+static bool gemm_ln_profitable(const ibert_ctx* ctx, int64_t T, int H) {
+  if (ctx->fusion_mode == 1) return true;
+  if (ctx->fusion_mode == 2) return false;
+  const int64_t tiles = (T + 127) / 128;
+  return tiles * (H / 256) * 2 >= ctx->num_sms;
+}
+
 // grows the context's workspace to at least `need` bytes (stream-synchronizing reallocation)
 static int ensure_workspace(ibert_ctx* ctx, size_t need) {
   if (need <= ctx->ws_bytes) return IBERT_OK;
@@ -348,7 +364,7 @@ int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const
   if ((rc = cached_upload(ctx, B_i.data(), B_i.size() * sizeof(int64_t), 12, &d_Bi))) return rc;
   epi.d_b = (const int32_t*)d_b;
   epi.d_c = (const int32_t*)d_c;
-  if (gemm_ln_supported(N, K, epi, k)) {
+  if (gemm_ln_profitable(ctx, M, N) && gemm_ln_supported(N, K, epi, k)) {
     ProfileScope ps(ctx, K > 2048 ? IBERT_K_GEMM_LN_WIDE : IBERT_K_GEMM_LN);
     rc = launch_gemm_ln_i8(ctx, x, w, M, N, K, epi, res, k, (const int32_t*)d_bi, (const int64_t*)d_Bi, out);
   } else {
@@ -561,7 +577,10 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
   if (rc) return rc;
   // output projection + residual + LayerNorm: one kernel when shapes and constants allow it
   e.kind = EPI_Q16; e.d_b = ly->b_o; e.d_c = ly->c_o; e.d_bias = ly->bias_o; e.fast = ly->fast_o;
-  if (gemm_ln_supported(H, H, e, ly->ln1)) {
+  // the cluster kernel pays off once its 128-token tiles keep at least half of the SMs busy; below
+  // that the two kernels, which spread a small problem over more CTAs, are faster
+  const bool fuse = gemm_ln_profitable(ctx, T, H);
+  if (fuse && gemm_ln_supported(H, H, e, ly->ln1)) {
     ProfileScope ps(ctx, IBERT_K_GEMM_LN);
     rc = launch_gemm_ln_i8(ctx, cx, ly->w_o, T, H, H, e, x, ly->ln1, ly->ln1_b, ly->ln1_B, h1);
   } else {
@@ -574,7 +593,7 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
   { ProfileScope ps(ctx, IBERT_K_GEMM_GELU); rc = launch_gemm_i8(ctx, h1, ly->w_f1, T, F, H, e, g); }
   if (rc) return rc;
   e.kind = EPI_Q16; e.d_b = ly->b_f2; e.d_c = ly->c_f2; e.d_bias = ly->bias_f2; e.fast = ly->fast_f2;
-  if (gemm_ln_supported(H, F, e, ly->ln2)) {
+  if (fuse && gemm_ln_supported(H, F, e, ly->ln2)) {
     ProfileScope ps(ctx, F > 2048 ? IBERT_K_GEMM_LN_WIDE : IBERT_K_GEMM_LN);
     return launch_gemm_ln_i8(ctx, g, ly->w_f2, T, H, F, e, h1, ly->ln2, ly->ln2_b, ly->ln2_B, out);
   }

@@ -100,6 +100,8 @@ struct ibert_ctx {
   // workspace for the encoder layer's intermediates
   void* ws = nullptr;
   size_t ws_bytes = 0;
+  // linear + LayerNorm fusion: 0 = by problem size, 1 = whenever supported, 2 = never (ibert_set_fusion)
+  int fusion_mode = 0;
   // optional per-launch event timing (ibert_profile_begin / _end)
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;      // pairs: [2i] before, [2i+1] after launch i

@@ -58,8 +58,9 @@ def test_attention_coarse_score_scale(L, S_qk):
     ctx().check()
 
 
-def _run_layers(x, params, B, L):
+def _run_layers(x, params, B, L, fusion=0):
     c = ctx()
+    c.ibert_set_fusion(fusion)
     h = dev(x)
     outs = []
     for p in params:
@@ -69,13 +70,16 @@ def _run_layers(x, params, B, L):
         outs.append(host(h))
         c.check()
         layer.close()
+    c.ibert_set_fusion(0)
     return outs
 
 
-@pytest.mark.parametrize("B,L,H,heads,F", [(2, 16, 128, 2, 256), (1, 37, 64, 1, 64), (3, 128, 256, 4, 1024)])
-def test_small_encoder_layers_match_oracle(B, L, H, heads, F):
+@pytest.mark.parametrize("fusion", [0, 1])      # linear + LayerNorm: by size (two kernels here) / cluster kernel
+@pytest.mark.parametrize("B,L,H,heads,F", [(2, 16, 128, 2, 256), (1, 37, 64, 1, 64), (3, 128, 256, 4, 1024),
+                                           (2, 100, 768, 12, 3072)])
+def test_small_encoder_layers_match_oracle(B, L, H, heads, F, fusion):
     x, params = synth.make_model(0, B, layers=2, H=H, heads=heads, F=F, L=L)
-    outs = _run_layers(x, params, B, L)
+    outs = _run_layers(x, params, B, L, fusion)
     h = x
     for p, got in zip(params, outs):
         h = oracle.encoder_layer(p, h, B, L).out

@@ -41,17 +41,25 @@ SHAPES = [(1, 256, 64), (127, 256, 128), (300, 512, 144), (129, 768, 768), (1000
           (77, 128, 64), (300, 320, 80), (0, 768, 768)]
 
 
+@pytest.fixture(autouse=True)
+def _restore_fusion_mode():
+    yield
+    ctx().ibert_set_fusion(0)
+
+
+@pytest.mark.parametrize("mode", [1, 2, 0])       # cluster kernel forced, two kernels forced, by size
 @pytest.mark.parametrize("M,N,K", SHAPES)
-def test_linear_layernorm_matches_oracle(M, N, K):
+def test_linear_layernorm_matches_oracle(M, N, K, mode):
     p = _problem(M, N, K, M + N + K)
     x, w, bias, res, S_w, S_x, S_mid, S_res, gamma, beta, S_out = p
+    ctx().ibert_set_fusion(mode)
     out, S_ret = ctx().ibert_linear_layernorm_i8(dev(x), S_x, dev(w), S_w, dev(bias), S_mid, dev(res), S_res,
                                                  gamma, beta, S_out)
     ctx().check()
     assert S_ret == S_out
     if M:
         want = _oracle(*p)
-        assert_same(host(out), want, f"linear+LN {M}x{N}x{K}")
+        assert_same(host(out), want, f"linear+LN {M}x{N}x{K} mode {mode}")
         assert np.abs(want).max() > 20
 
 
@@ -65,6 +73,7 @@ def test_linear_layernorm_constant_rows_and_no_bias():
     p[3][:70] = 7                       # constant residual
     p[4][:] = 2e-4                      # one weight scale: every channel requantizes alike
     x, w, bias, res, S_w, S_x, S_mid, S_res, gamma, beta, S_out = p
+    ctx().ibert_set_fusion(1)
     out, _ = ctx().ibert_linear_layernorm_i8(dev(x), S_x, dev(w), S_w, dev(bias), S_mid, dev(res), S_res,
                                              gamma, beta, S_out)
     ctx().check()
@@ -80,6 +89,7 @@ def test_linear_layernorm_equals_the_two_separate_calls():
     M, N, K = 700, 768, 768
     x, w, bias, res, S_w, S_x, S_mid, S_res, gamma, beta, S_out = _problem(M, N, K, 11)
     c = ctx()
+    c.ibert_set_fusion(1)
     fused, _ = c.ibert_linear_layernorm_i8(dev(x), S_x, dev(w), S_w, dev(bias), S_mid, dev(res), S_res,
                                            gamma, beta, S_out)
     mid, _ = c.ibert_linear_i8(dev(x), S_x, dev(w), S_w, dev(bias), 1, S_mid)

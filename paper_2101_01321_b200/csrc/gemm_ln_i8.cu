@@ -130,7 +130,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(bar_acc_full + 8 * a, 1);
       ptx::mbar_init(bar_acc_empty + 8 * a, kEpiWarps);
-      ptx::mbar_init(bar_stats + 8 * a, (uint32_t)n_cta * 4u);   // 4 warps of every CTA report
+      ptx::mbar_init(bar_stats + 8 * a, (uint32_t)n_cta * kTok);   // one arrival per token from every CTA
     }
     for (int i = 0; i < 2 * kEpiWarps; ++i) ptx::mbar_init(bar_res + 8 * i, 1);
     ptx::fence_mbar_init();
@@ -285,16 +285,13 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const unsigned long long p2 = s2l[i];
         s1l[i] = 0;
         s2l[i] = 0;
+        // every thread releases its own additions (and, through the barrier that precedes this call,
+        // the clearing of this buffer two tiles ago) with its arrival: no separate fence
         for (int r = 0; r < n_cta; ++r) {
           ptx::red_add_cluster_s32(ptx::map_to_cta(ptx::smem_addr(&s1g[i]), (uint32_t)r), p1);
           ptx::red_add_cluster_u64(ptx::map_to_cta(ptx::smem_addr(&s2g[i]), (uint32_t)r), p2);
-        }
-      }
-      __syncwarp();
-      if (lane == 0 && ok) {
-        ptx::fence_acq_rel_cluster();
-        for (int r = 0; r < n_cta; ++r)
           ptx::mbar_arrive_remote_release(ptx::map_to_cta(bar_stats + 8 * par, (uint32_t)r));
+        }
       }
     };
     // mean and inverse standard deviation of the tokens of tile `it` (warps 4..7, one token per

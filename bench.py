@@ -35,6 +35,12 @@ DEFAULT_BATCH = {2: 128, 3: 32, 4: 64}
 NCU_DRAM_TRAFFIC_BYTES = {(2, 128): {"gemm_qkv": 14.5e6, "attention": 37.8e6, "gemm_out_ln": 25.8e6, "gemm_ffn1_gelu": 17.8e6, "gemm_ffn2_ln": 68.0e6, "gemm_out": 14.4e6, "layernorm": 64.1e6, "gemm_ffn2": 60.1e6}}
 
 
+# Integer-datapath instructions (ALU + IMAD pipes, which behave as one 16-lane unit per SM sub-partition)
+# per output element, from the ncu instruction counters of the same captures: what actually bounds
+# the GEMM epilogues.  Reported beside the tensor roofline of the top kernel class.
+NCU_INT_INSTR_PER_ELEMENT = {(2, 128): {"gemm_ffn1_gelu": 20.4}}
+
+
 # --------------------------------------------------------------------------- helpers
 def measured_peaks() -> tuple[dict, str]:
     p = ROOT / "MEASURED_PEAKS.json"
@@ -392,6 +398,15 @@ def run_ours(args):
                     "unit": "GB/s", "frac": kern[top]["gbs"] / peaks["hbm_gbs"], "traffic": None,
                     "peak_source": f"{peak_kind} copy bandwidth"}
         roof["ms_per_launch"] = kern[top]["ms_per_launch"]
+        ipe = NCU_INT_INSTR_PER_ELEMENT.get((args.config, batch), {}).get(top)
+        if ipe and top == "gemm_ffn1_gelu":
+            lane_ops = ipe * T * cfg.F
+            int_peak = 64.0 * torch.cuda.get_device_properties(dev).multi_processor_count * \
+                (clocks.get("sm_max_mhz") or 1965.0) * 1e6
+            roof["integer_datapath"] = {"lane_ops_per_launch": lane_ops, "peak_lane_ops_per_s": int_peak,
+                                        "frac": lane_ops / (kern[top]["ms_per_launch"] * 1e-3) / int_peak,
+                                        "note": "the epilogue's int32 work (ncu instruction counts) against 64 lanes x "
+                                                "SMs x max clock: the bound this kernel actually runs into"}
         roof["traffic"] = NCU_DRAM_TRAFFIC_BYTES.get((args.config, batch), {}).get(top)
         roof["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)"
         roof["algorithmic"] = (16.0 * T * cfg.L * cfg.heads if top == "attention"

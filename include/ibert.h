@@ -155,7 +155,7 @@ int ibert_layer_destroy(ibert_layer* layer);
    scale S_x*S_w[n], or NULL; res: device int8 [M, N] at host scale S_res; gamma, beta: host
    double [N]; out: device int8 [M, N] at S_out (*S_ret).  The result is bit-identical to
    ibert_linear_i8(kind 1, S_mid) followed by ibert_layernorm_i.  When N is a multiple of 256 (at
-   most 2048), the constants fit the 32-bit forms and M is large enough for its 128-row tiles to
+   most 1024), the constants fit the 32-bit forms and M is large enough for its 128-row tiles to
    occupy half of the SMs, a single kernel computes it on a cluster of N/256 CTAs per tile and the
    Q16 tensor never reaches memory; otherwise the two kernels run back to back through the
    context's workspace.

@@ -41,17 +41,18 @@ constexpr int kThreads = 64 + kEpiThreads;
 constexpr int kXBytes = kTok * kBK;              // 16 KB
 constexpr int kWBytes = kCh * kBK;               // 32 KB
 constexpr int kStageBytes = kXBytes + kWBytes;
-constexpr int kOutOff = kStages * kStageBytes;   // per epilogue warp: 2 x [32 tokens][32 B]
+constexpr int kMaxCta = 4;                       // cluster width the statistics buffers are sized for (H <= 1024)
+constexpr int kOutOff = kStages * kStageBytes;   // per epilogue warp: [32 tokens][32 B] output staging
 constexpr int kOutTile = 32 * 32;
-constexpr int kOutBytes = kEpiWarps * 2 * kOutTile;
+constexpr int kOutBytes = kEpiWarps * kOutTile;
 constexpr int kResOff = kOutOff + kOutBytes;     // per epilogue warp: 2 x [32 tokens][32 B] of the residual
-constexpr int kCbOff = kResOff + kOutBytes;      // int2 {multiplier, bias} per channel
+constexpr int kCbOff = kResOff + 2 * kOutBytes;  // int2 {multiplier, bias} per channel
 constexpr int kLnOff = kCbOff + kCh * 8;         // int4 {b_i, 0, B_i lo, B_i hi} per channel
-constexpr int kS1lOff = kLnOff + kCh * 16;       // [2][128] int32: this CTA's partial sums (by tile parity)
-constexpr int kS2lOff = kS1lOff + 2 * kTok * 4;  // [2][128] uint64
-constexpr int kS1gOff = kS2lOff + 2 * kTok * 8;  // [2][128] int32: cluster totals
-constexpr int kS2gOff = kS1gOff + 2 * kTok * 4;  // [2][128] uint64
-constexpr int kParOff = kS2gOff + 2 * kTok * 8;  // [2][128] int4 {mu, floor(2^31 / sigma), shift, -}
+// statistics of a tile: a block of 128 uint64 sums of squares followed by 128 int32 sums
+constexpr int kStatBytes = kTok * 12;
+constexpr int kLocOff = kLnOff + kCh * 16;       // [3]: this CTA's partial sums, by tile index mod 3
+constexpr int kGatOff = kLocOff + 3 * kStatBytes;   // [2][kMaxCta]: every CTA's partial sums, by tile parity
+constexpr int kParOff = kGatOff + 2 * kMaxCta * kStatBytes;   // [2][128] int4 {mu, floor(2^31 / sigma), shift, -}
 constexpr int kBarOff = kParOff + 2 * kTok * 16;
 constexpr int kAlloc = kBarOff + 512 + 1024;     // + slack to align the base to 1024 bytes
 static_assert(kAlloc <= 227 * 1024, "shared memory budget");
@@ -68,11 +69,12 @@ struct GemmLnArgs {
 };
 
 // floor(sqrt(floor(ss / C))) = the largest s with s^2 C <= ss, one thread per value, bit by bit.
-// Needs s < 2^24 and C < 2^12 (then s^2 C < 2^60).
+// ss / C < 2^(bits(ss) - floor(log2 C)) bounds the highest bit that can be set, so the loop runs
+// about half the bit length of the variance.  Needs s < 2^24 and C < 2^12 (then s^2 C < 2^60).
 __device__ __forceinline__ uint32_t isqrt_of_quotient(uint64_t ss, uint32_t C) {
-  const int bits = 64 - __clzll((long long)(ss | 1ull));                 // s^2 <= ss  =>  s < 2^ceil(bits / 2)
+  const int bits = 64 - __clzll((long long)(ss | 1ull)) - (31 - __clz((int)C));   // ss / C < 2^bits
   uint32_t s = 0;
-  for (int bit = min((bits + 1) >> 1, 23); bit >= 0; --bit) {
+  for (int bit = min(max((bits + 1) >> 1, 1), 24) - 1; bit >= 0; --bit) {
     const uint32_t cand = s | (1u << bit);
     const uint64_t sq = (uint64_t)cand * (uint64_t)cand;
     if (sq * (uint64_t)C <= ss) s = cand;
@@ -97,10 +99,8 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const uint32_t smem_base = ptx::smem_addr(smem);
   int2* s_cb = reinterpret_cast<int2*>(smem + kCbOff);
   int4* s_ln = reinterpret_cast<int4*>(smem + kLnOff);
-  int32_t* s1l = reinterpret_cast<int32_t*>(smem + kS1lOff);
-  unsigned long long* s2l = reinterpret_cast<unsigned long long*>(smem + kS2lOff);
-  int32_t* s1g = reinterpret_cast<int32_t*>(smem + kS1gOff);
-  unsigned long long* s2g = reinterpret_cast<unsigned long long*>(smem + kS2gOff);
+  uint8_t* s_loc = smem + kLocOff;
+  const uint8_t* s_gat = smem + kGatOff;
   int4* s_par = reinterpret_cast<int4*>(smem + kParOff);
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + kBarOff);
   // full[3], empty[3], acc_full[2], acc_empty[2], stats[2], TMEM base, then res[16 warps][2]
@@ -130,7 +130,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(bar_acc_full + 8 * a, 1);
       ptx::mbar_init(bar_acc_empty + 8 * a, kEpiWarps);
-      ptx::mbar_init(bar_stats + 8 * a, (uint32_t)n_cta * kTok);   // one arrival per token from every CTA
+      ptx::mbar_init(bar_stats + 8 * a, 1);                    // armed with the expected bytes by this CTA
     }
     for (int i = 0; i < 2 * kEpiWarps; ++i) ptx::mbar_init(bar_res + 8 * i, 1);
     ptx::fence_mbar_init();
@@ -145,7 +145,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   }
   // statistics start at zero; the per-channel constants are weights, not outputs of the previous
   // kernel, so they may be read before the grid dependency is resolved
-  for (int i = threadIdx.x; i < 2 * kTok; i += kThreads) { s1l[i] = 0; s2l[i] = 0; s1g[i] = 0; s2g[i] = 0; }
+  for (int i = threadIdx.x; i < 3 * kStatBytes / 4; i += kThreads) reinterpret_cast<uint32_t*>(s_loc)[i] = 0;
   for (int i = threadIdx.x; i < kCh; i += kThreads) {
     s_cb[i] = make_int2(__ldg(args.pb + n0 + i), args.bias ? __ldg(args.bias + n0 + i) : 0);
     const int64_t B = __ldg(args.B_i + n0 + i);
@@ -213,13 +213,12 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const int part = ew >> 2;
     const int tok = quad * 32 + lane;                  // this thread's token inside the tile
     const int e_tid = threadIdx.x - 64;                // 0..511
-    uint8_t* stage0 = smem + kOutOff + ew * 2 * kOutTile;
+    uint8_t* stage0 = smem + kOutOff + ew * kOutTile;
     const uint8_t* res0 = smem + kResOff + ew * 2 * kOutTile;
     const uint32_t my_res = bar_res + 16 * ew;
     const LnConsts ln = args.ln;
     const int C = ln.C;
     const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t buf = 0;
 
     auto tile_of = [&](uint32_t it) { return (int64_t)cluster_id + (int64_t)it * num_clusters; };
     // residual block of this warp for tile `it` (32 tokens x 64 channels) into its two private
@@ -266,48 +265,54 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           ptx::tmem_st32(t_lane + par * kCh + col, v);
         }
         ptx::tmem_wait_st();
-        atomicAdd(&s1l[par * kTok + tok], s1);
-        atomicAdd(&s2l[par * kTok + tok], (unsigned long long)s2);
+        uint8_t* loc = s_loc + (it % 3u) * kStatBytes;
+        atomicAdd(reinterpret_cast<unsigned long long*>(loc) + tok, (unsigned long long)s2);
+        atomicAdd(reinterpret_cast<int32_t*>(loc + kTok * 8) + tok, s1);
       }
       ptx::fence_proxy_async_smem();
       __syncwarp();                                    // both residual buffers are consumed
       if (lane == 0 && ok && tile_of(it + 1) < t_tiles) issue_res(it + 1);
     };
-    // sends the CTA's partial sums of tile `it` to every CTA of the cluster (warps 0..3; needs a
-    // barrier after pass A, and -- so that the totals of tile it - 2 have been read and cleared
-    // everywhere -- comes after this CTA has seen the totals of tile it - 1 complete)
+    // sends the CTA's partial sums of tile `it` to every CTA of the cluster: one bulk copy of the
+    // 1.5 KB block per destination, credited to the destination's statistics barrier (one thread;
+    // needs a barrier after pass A, and -- so that the receivers have read the block of tile
+    // it - 2 -- comes after this CTA has seen the blocks of tile it - 1 complete)
     auto exchange = [&](uint32_t it) {
-      if (ew >= 4) return;
+      if (e_tid != 0 || !ok) return;
       const uint32_t par = it & 1u;
-      const int i = par * kTok + e_tid;
-      if (ok) {
-        const int32_t p1 = s1l[i];
-        const unsigned long long p2 = s2l[i];
-        s1l[i] = 0;
-        s2l[i] = 0;
-        // every thread releases its own additions (and, through the barrier that precedes this call,
-        // the clearing of this buffer two tiles ago) with its arrival: no separate fence
-        for (int r = 0; r < n_cta; ++r) {
-          ptx::red_add_cluster_s32(ptx::map_to_cta(ptx::smem_addr(&s1g[i]), (uint32_t)r), p1);
-          ptx::red_add_cluster_u64(ptx::map_to_cta(ptx::smem_addr(&s2g[i]), (uint32_t)r), p2);
-          ptx::mbar_arrive_remote_release(ptx::map_to_cta(bar_stats + 8 * par, (uint32_t)r));
-        }
-      }
+      ptx::fence_proxy_async_smem();                   // the sums were written by ordinary atomics
+      ptx::mbar_arrive_expect_tx(bar_stats + 8 * par, (uint32_t)n_cta * kStatBytes);
+      const uint32_t src = ptx::smem_addr(s_loc + (it % 3u) * kStatBytes);
+      const uint32_t dst = ptx::smem_addr(s_gat + (par * kMaxCta + rank) * kStatBytes);
+      for (int r = 0; r < n_cta; ++r)
+        ptx::bulk_copy_to_cta(ptx::map_to_cta(dst, (uint32_t)r), src, kStatBytes,
+                              ptx::map_to_cta(bar_stats + 8 * par, (uint32_t)r));
     };
     // mean and inverse standard deviation of the tokens of tile `it` (warps 4..7, one token per
     // thread); a barrier of all epilogue warps must follow before pass B reads them
     auto params = [&](uint32_t it) {
       const uint32_t par = it & 1u, phase = (it >> 1) & 1u;
       if (ew >= 4 && ew < 8) {
-        const int i = par * kTok + (e_tid - 128);
+        const int tk = e_tid - 128;
+        const int i = par * kTok + tk;
         if (ok) ok = ptx::mbar_wait_cluster(bar_stats + 8 * par, phase);
         ok = __all_sync(0xffffffffu, ok);
         int32_t mu = 0, rho = 1 << 30, nsh = 14;
         if (ok) {
-          const int32_t sum = s1g[i];
-          const uint64_t sumsq = s2g[i];
-          s1g[i] = 0;
-          s2g[i] = 0;
+          int32_t sum = 0;
+          uint64_t sumsq = 0;
+          for (int r = 0; r < n_cta; ++r) {
+            const uint8_t* blk = s_gat + (par * kMaxCta + r) * kStatBytes;
+            sumsq += reinterpret_cast<const unsigned long long*>(blk)[tk];
+            sum += reinterpret_cast<const int32_t*>(blk + kTok * 8)[tk];
+          }
+          // every CTA has this tile's blocks, so each has read the blocks of the tile before:
+          // that tile's own partial sums can be cleared for their next use three tiles on
+          if (it > 0) {
+            uint8_t* old = s_loc + ((it - 1) % 3u) * kStatBytes;
+            reinterpret_cast<unsigned long long*>(old)[tk] = 0;
+            reinterpret_cast<int32_t*>(old + kTok * 8)[tk] = 0;
+          }
           mu = sum / C;                                // floor(sum / C)
           if (sum - mu * C < 0) mu -= 1;
           const int64_t ss = (int64_t)sumsq - 2 * (int64_t)mu * (int64_t)sum + (int64_t)C * (int64_t)mu * (int64_t)mu;
@@ -331,9 +336,9 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           uint32_t v[32];
           ptx::tmem_ld32(t_lane + par * kCh + col, v);
           ptx::tmem_wait_ld();
-          if (lane == 0) ptx::bulk_wait_read<1>();     // the store issued two chunks ago has read its tile
+          if (lane == 0) ptx::bulk_wait_read<0>();     // the previous store has read the staging tile
           __syncwarp();
-          uint8_t* stage = stage0 + buf * kOutTile;
+          uint8_t* stage = stage0;
           uint32_t w[8];
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
@@ -358,7 +363,6 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), n0 + col, t0 + quad * 32);
             ptx::bulk_commit();
           }
-          buf ^= 1;
         }
       }
       ptx::tc_fence_before_sync();
@@ -415,7 +419,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 }  // namespace
 
 bool gemm_ln_supported(int H, int K, const GemmEpilogue& epi, const LnConsts& ln) {
-  if (H % kCh != 0 || H / kCh > 8 || K % 16 != 0) return false;           // cluster of H / 256 CTAs (portable limit 8)
+  if (H % kCh != 0 || H / kCh > kMaxCta || K % 16 != 0) return false;    // cluster of H / 256 CTAs, at most 4
   if (!epi.fast || epi.kind != EPI_Q16) return false;
   if (!ln.has_res || !ln.res_fast || !ln.out_fast || ln.C != H) return false;
   // |v| = |Q16 value + rescaled residual| must stay below 2^18: sums over H <= 2048 channels then fit

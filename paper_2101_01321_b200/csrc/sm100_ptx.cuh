@@ -260,6 +260,15 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
   }
   return false;
 }
+// bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster (both
+// 16-byte aligned, size a multiple of 16); the bytes are credited to an mbarrier of the
+// destination CTA (`dst_cluster_addr`, `bar_cluster_addr` from map_to_cta).  No multicast.
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster_addr, uint32_t src_addr, uint32_t bytes,
+                                                 uint32_t bar_cluster_addr) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_cluster_addr), "r"(src_addr), "r"(bytes), "r"(bar_cluster_addr)
+               : "memory");
+}
 // named barrier among `count` threads of this CTA (ids 1..15; 0 is __syncthreads)
 __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");

@@ -34,15 +34,14 @@ namespace {
 constexpr int kTok = 128;           // tokens per tile = TMEM lanes = MMA M
 constexpr int kCh = 256;            // channels per CTA = MMA N = TMEM columns per accumulator stage
 constexpr int kBK = 128;            // K bytes per pipeline stage (one 128-byte swizzle span)
-constexpr int kStages = 3;
+constexpr int kMaxStages = 4;       // barrier slots; a kernel instance uses 3 (48 KB stages) or 4 (32 KB, CTA pairs)
 constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kThreads = 64 + kEpiThreads;
 constexpr int kXBytes = kTok * kBK;              // 16 KB
-constexpr int kWBytes = kCh * kBK;               // 32 KB
-constexpr int kStageBytes = kXBytes + kWBytes;
+constexpr int kOperandBytes = 3 * (kXBytes + kCh * kBK);   // 144 KB of operand stages either way
 constexpr int kMaxCta = 4;                       // cluster width the statistics buffers are sized for (H <= 1024)
-constexpr int kOutOff = kStages * kStageBytes;   // per epilogue warp: [32 tokens][32 B] output staging
+constexpr int kOutOff = kOperandBytes;            // per epilogue warp: [32 tokens][32 B] output staging
 constexpr int kOutTile = 32 * 32;
 constexpr int kOutBytes = kEpiWarps * kOutTile;
 constexpr int kResOff = kOutOff + kOutBytes;     // per epilogue warp: 2 x [32 tokens][32 B] of the residual
@@ -90,6 +89,10 @@ __device__ __forceinline__ int32_t sext_byte(uint32_t w, int k) {
   return r;
 }
 
+// PAIR: two CTAs (same 256 channels, adjacent 128-token tiles) share every MMA through
+// tcgen05.mma.cta_group::2 -- each loads its own token rows and half of the weight rows, which cuts
+// the bytes an SM pulls from L2 per MMA by a third (L2 bandwidth bounds the K = 3072 main loop).
+template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                const __grid_constant__ CUtensorMap map_res, const __grid_constant__ CUtensorMap map_out,
@@ -103,24 +106,35 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   const uint8_t* s_gat = smem + kGatOff;
   int4* s_par = reinterpret_cast<int4*>(smem + kParOff);
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + kBarOff);
-  // full[3], empty[3], acc_full[2], acc_empty[2], stats[2], TMEM base, then res[16 warps][2]
+  constexpr int kStages = PAIR ? 4 : 3;
+  constexpr int kWBytes = (PAIR ? kCh / 2 : kCh) * kBK;    // weight rows this CTA loads per K block
+  constexpr int kStageBytes = kXBytes + kWBytes;
+  // full[4], empty[4], acc_full[2], acc_empty[2], stats[2], TMEM base, res[16 warps][2], decision flags
   const uint32_t bar_full = ptx::smem_addr(s_bar);
-  const uint32_t bar_empty = bar_full + 8 * kStages;
-  const uint32_t bar_acc_full = bar_empty + 8 * kStages;
+  const uint32_t bar_empty = bar_full + 8 * kMaxStages;
+  const uint32_t bar_acc_full = bar_empty + 8 * kMaxStages;
   const uint32_t bar_acc_empty = bar_acc_full + 16;
   const uint32_t bar_stats = bar_acc_empty + 16;
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 2 * kStages + 8);
-  const uint32_t bar_res = bar_full + 128;                 // two per epilogue warp
-  volatile int* s_flag = reinterpret_cast<volatile int*>(s_bar + 50);   // the epilogue's next-step decision
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 20);
+  const uint32_t bar_res = bar_full + 192;                 // two per epilogue warp
+  volatile int* s_flag = reinterpret_cast<volatile int*>(s_bar + 60);   // the epilogue's next-step decision
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = ptx::cluster_ctarank();
-  const int n_cta = args.H / kCh;                          // cluster width
-  const int cluster_id = (int)blockIdx.x / n_cta;
-  const int num_clusters = (int)gridDim.x / n_cta;
+  const int n_slices = args.H / kCh;                       // CTAs that share a token tile
+  const int cl = PAIR ? 2 * n_slices : n_slices;           // cluster width
+  const int slice = PAIR ? (int)(rank >> 1) : (int)rank;   // which 256 channels
+  const int half = PAIR ? (int)(rank & 1u) : 0;            // which of the pair's two token tiles
+  const uint32_t leader = PAIR ? (rank & ~1u) : rank;      // the CTA of the pair that issues the MMAs
+  const int cluster_id = (int)blockIdx.x / cl;
+  const int num_clusters = (int)gridDim.x / cl;
   const int64_t t_tiles = (args.T + kTok - 1) / kTok;
+  const int64_t n_units = PAIR ? (t_tiles + 1) / 2 : t_tiles;   // tiles (pairs of tiles) a cluster steps through
   const int k_blocks = (args.K + kBK - 1) / kBK;
-  const int n0 = (int)rank * kCh;                          // this CTA's first channel
+  const int n0 = slice * kCh;                              // this CTA's first channel
+  // unit / token tile of this CTA at step `it` of its cluster (a tile past T reads zeros, stores nothing)
+  auto unit_of = [&](uint32_t it) { return (int64_t)cluster_id + (int64_t)it * num_clusters; };
+  auto tile_of = [&](uint32_t it) { return PAIR ? 2 * unit_of(it) + half : unit_of(it); };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -129,7 +143,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(bar_acc_full + 8 * a, 1);
-      ptx::mbar_init(bar_acc_empty + 8 * a, kEpiWarps);
+      ptx::mbar_init(bar_acc_empty + 8 * a, (PAIR ? 2 : 1) * kEpiWarps);   // the leader's is the one in use
       ptx::mbar_init(bar_stats + 8 * a, 1);                    // armed with the expected bytes by this CTA
     }
     for (int i = 0; i < 2 * kEpiWarps; ++i) ptx::mbar_init(bar_res + 8 * i, 1);
@@ -140,8 +154,8 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     ptx::tma_prefetch_desc(&map_out);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_addr(s_tmem), 2 * kCh);
-    ptx::tmem_relinquish();
+    if constexpr (PAIR) { ptx::tmem_alloc_pair(ptx::smem_addr(s_tmem), 2 * kCh); ptx::tmem_relinquish_pair(); }
+    else { ptx::tmem_alloc(ptx::smem_addr(s_tmem), 2 * kCh); ptx::tmem_relinquish(); }
   }
   // statistics start at zero; the per-channel constants are weights, not outputs of the previous
   // kernel, so they may be read before the grid dependency is resolved
@@ -163,24 +177,33 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
-      for (int64_t tile = cluster_id; tile < t_tiles && ok; tile += num_clusters) {
-        const int t0 = (int)tile * kTok;
+      for (uint32_t it = 0; unit_of(it) < n_units && ok; ++it) {
+        const int t0 = (int)tile_of(it) * kTok;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!ptx::mbar_wait(bar_empty + 8 * stage, phase ^ 1)) { ok = false; break; }
           const uint32_t sx = smem_base + stage * kStageBytes;
-          ptx::mbar_arrive_expect_tx(bar_full + 8 * stage, kStageBytes);
-          ptx::tma_load_2d(sx, &map_x, bar_full + 8 * stage, kb * kBK, t0);
-          ptx::tma_load_2d(sx + kXBytes, &map_w, bar_full + 8 * stage, kb * kBK, n0);
+          if constexpr (PAIR) {
+            // both CTAs' copies complete on the leader's barrier, which expects the bytes of both
+            const uint32_t full_leader = ptx::map_to_cta(bar_full + 8 * stage, leader);
+            if (half == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * kStageBytes);
+            ptx::tma_load_2d_pair(sx, &map_x, full_leader, kb * kBK, t0);
+            ptx::tma_load_2d_pair(sx + kXBytes, &map_w, full_leader, kb * kBK, n0 + half * (kCh / 2));
+          } else {
+            ptx::mbar_arrive_expect_tx(bar_full + 8 * stage, kStageBytes);
+            ptx::tma_load_2d(sx, &map_x, bar_full + 8 * stage, kb * kBK, t0);
+            ptx::tma_load_2d(sx + kXBytes, &map_w, bar_full + 8 * stage, kb * kBK, n0);
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = ptx::make_idesc_i8(kTok, kCh, true, true);
+    // ------------------------------------------------------------ MMA issuer (PAIR: the pair's leader only)
+    if (lane == 0 && half == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_i8(PAIR ? 2 * kTok : kTok, kCh, true, true);
+      const uint16_t pair_mask = (uint16_t)(3u << leader);
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
-      for (int64_t tile = cluster_id; tile < t_tiles && ok; tile += num_clusters) {
+      for (uint32_t it = 0; unit_of(it) < n_units && ok; ++it) {
         if (!ptx::mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * kCh;
@@ -191,13 +214,18 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           const uint64_t dx = ptx::make_kmajor_desc(sx, 1024, ptx::kSwizzle128);
           const uint64_t dw = ptx::make_kmajor_desc(sx + kXBytes, 1024, ptx::kSwizzle128);
 #pragma unroll
-          for (int k = 0; k < kBK / 32; ++k)
-            ptx::mma_i8_ss(d_tmem, dx + 2 * k, dw + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-          ptx::mma_commit(bar_empty + 8 * stage);
+          for (int k = 0; k < kBK / 32; ++k) {
+            if constexpr (PAIR) ptx::mma_i8_ss_pair(d_tmem, dx + 2 * k, dw + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            else ptx::mma_i8_ss(d_tmem, dx + 2 * k, dw + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if constexpr (PAIR) ptx::mma_commit_pair(bar_empty + 8 * stage, pair_mask);
+          else ptx::mma_commit(bar_empty + 8 * stage);
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        ptx::mma_commit(bar_acc_full + 8 * acc);
+        if constexpr (PAIR) ptx::mma_commit_pair(bar_acc_full + 8 * acc, pair_mask);
+        else ptx::mma_commit(bar_acc_full + 8 * acc);
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1;
       }
@@ -220,7 +248,6 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const int C = ln.C;
     const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
 
-    auto tile_of = [&](uint32_t it) { return (int64_t)cluster_id + (int64_t)it * num_clusters; };
     // residual block of this warp for tile `it` (32 tokens x 64 channels) into its two private
     // buffers; rows past T read as zero.  Called by lane 0 once both buffers have been consumed.
     auto issue_res = [&](uint32_t it) {
@@ -271,7 +298,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       }
       ptx::fence_proxy_async_smem();
       __syncwarp();                                    // both residual buffers are consumed
-      if (lane == 0 && ok && tile_of(it + 1) < t_tiles) issue_res(it + 1);
+      if (lane == 0 && ok && unit_of(it + 1) < n_units) issue_res(it + 1);
     };
     // sends the CTA's partial sums of tile `it` to every CTA of the cluster: one bulk copy of the
     // 1.5 KB block per destination, credited to the destination's statistics barrier (one thread;
@@ -281,12 +308,13 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       if (e_tid != 0 || !ok) return;
       const uint32_t par = it & 1u;
       ptx::fence_proxy_async_smem();                   // the sums were written by ordinary atomics
-      ptx::mbar_arrive_expect_tx(bar_stats + 8 * par, (uint32_t)n_cta * kStatBytes);
+      ptx::mbar_arrive_expect_tx(bar_stats + 8 * par, (uint32_t)n_slices * kStatBytes);
       const uint32_t src = ptx::smem_addr(s_loc + (it % 3u) * kStatBytes);
-      const uint32_t dst = ptx::smem_addr(s_gat + (par * kMaxCta + rank) * kStatBytes);
-      for (int r = 0; r < n_cta; ++r)
-        ptx::bulk_copy_to_cta(ptx::map_to_cta(dst, (uint32_t)r), src, kStatBytes,
-                              ptx::map_to_cta(bar_stats + 8 * par, (uint32_t)r));
+      const uint32_t dst = ptx::smem_addr(s_gat + (par * kMaxCta + slice) * kStatBytes);
+      for (int sl = 0; sl < n_slices; ++sl) {            // the CTAs that hold the other channels of this token tile
+        const uint32_t r = PAIR ? (uint32_t)(2 * sl + half) : (uint32_t)sl;
+        ptx::bulk_copy_to_cta(ptx::map_to_cta(dst, r), src, kStatBytes, ptx::map_to_cta(bar_stats + 8 * par, r));
+      }
     };
     // mean and inverse standard deviation of the tokens of tile `it` (warps 4..7, one token per
     // thread); a barrier of all epilogue warps must follow before pass B reads them
@@ -301,7 +329,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         if (ok) {
           int32_t sum = 0;
           uint64_t sumsq = 0;
-          for (int r = 0; r < n_cta; ++r) {
+          for (int r = 0; r < n_slices; ++r) {
             const uint8_t* blk = s_gat + (par * kMaxCta + r) * kStatBytes;
             sumsq += reinterpret_cast<const unsigned long long*>(blk)[tk];
             sum += reinterpret_cast<const int32_t*>(blk + kTok * 8)[tk];
@@ -367,14 +395,17 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       }
       ptx::tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(bar_acc_empty + 8 * par);
+      if (lane == 0) {
+        if (PAIR && half != 0) ptx::mbar_arrive_remote(ptx::map_to_cta(bar_acc_empty + 8 * par, leader));
+        else ptx::mbar_arrive(bar_acc_empty + 8 * par);
+      }
     };
 
     // decision taken by the last epilogue thread right after its pass A of tile `it`: run pass A of
     // tile it + 1 before pass B of tile it?  Only if that accumulator is complete already.
     auto decide = [&](uint32_t it) {
       if (e_tid == kEpiThreads - 1)
-        s_flag[it & 1u] = (tile_of(it + 1) < t_tiles &&
+        s_flag[it & 1u] = (unit_of(it + 1) < n_units &&
                            ptx::mbar_test_now(bar_acc_full + 8 * ((it + 1) & 1u), ((it + 1) >> 1) & 1u)) ? 1 : 0;
     };
     // One loop body for every schedule (so pass A and pass B are instantiated once -- the
@@ -383,10 +414,10 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     //   step 1: pass A of tile it + 1 if it did not run early
     // and iteration -1 only runs pass A of tile 0.  After every pass A: decision for that tile,
     // barrier (sums complete, decision and statistics visible), exchange.
-    if (tile_of(0) < t_tiles) {
+    if (unit_of(0) < n_units) {
       if (lane == 0) issue_res(0);
       for (int it = -1;; ++it) {
-        const bool has_next = tile_of((uint32_t)(it + 1)) < t_tiles;
+        const bool has_next = unit_of((uint32_t)(it + 1)) < n_units;
         const bool early = it >= 0 && s_flag[it & 1] != 0;
 #pragma unroll 1
         for (int step = 0; step < 2; ++step) {
@@ -412,7 +443,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   ptx::cluster_sync();                 // nobody leaves while a peer may still add into its shared memory
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, 2 * kCh);
+    if constexpr (PAIR) ptx::tmem_dealloc_pair(tmem_base, 2 * kCh); else ptx::tmem_dealloc(tmem_base, 2 * kCh);
   }
 }
 
@@ -459,35 +490,53 @@ int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t 
   a.pb = epi.d_b; a.bias = epi.d_bias; a.b_i = d_b_i; a.B_i = d_B_i;
   a.ln = ln;
   a.status = ctx->d_status;
-  const int n_cta = H / kCh;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_ln_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAlloc) != cudaSuccess)
-      return IBERT_ERR_CUDA;
-    attr_set = true;
-  }
-  // clusters that can be resident at once (each CTA fills an SM); cached per cluster width
-  static int max_clusters[9] = {0};
-  if (max_clusters[n_cta] == 0) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(n_cta * ctx->num_sms);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = kAlloc;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = n_cta; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_ln_kernel, &cfg) != cudaSuccess || n < 1) {
-      cudaGetLastError();
-      n = std::max(1, ctx->num_sms / (2 * n_cta));
-    }
-    max_clusters[n_cta] = n;
-  }
+  const int n_slices = H / kCh;
   const int64_t t_tiles = (T + kTok - 1) / kTok;
-  const int clusters = (int)std::min<int64_t>(t_tiles, max_clusters[n_cta]);
-  return launch_pdl(gemm_ln_kernel, dim3(clusters * n_cta), dim3(kThreads), (size_t)kAlloc, ctx->stream, n_cta,
-                    mx, mw, mr, mo, a);
+  // CTA pairs (two token tiles per cluster step) when the cluster stays within 6 CTAs and there are
+  // tiles for both halves; resident clusters from the occupancy query, cached
+  static int max_clusters[2][9] = {{0}};
+  auto resident = [&](bool pair, int cl) {
+    int& slot = max_clusters[pair ? 1 : 0][cl];
+    if (slot == 0) {
+      const void* fn = pair ? (const void*)gemm_ln_kernel<true> : (const void*)gemm_ln_kernel<false>;
+      if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kAlloc) != cudaSuccess) {
+        cudaGetLastError();
+        slot = -1;
+        return slot;
+      }
+      cudaLaunchConfig_t cfg{};
+      cfg.gridDim = dim3(cl * ctx->num_sms);
+      cfg.blockDim = dim3(kThreads);
+      cfg.dynamicSmemBytes = kAlloc;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = cl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+      int n = 0;
+      const cudaError_t e = pair ? cudaOccupancyMaxActiveClusters(&n, gemm_ln_kernel<true>, &cfg)
+                                 : cudaOccupancyMaxActiveClusters(&n, gemm_ln_kernel<false>, &cfg);
+      if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
+      slot = n >= 1 ? n : -1;
+    }
+    return slot;
+  };
+  // (clusters of 8 fit only 16 times on the 148 SMs and measured slower than clusters of 4 single CTAs)
+  const bool want_pair = 2 * n_slices <= 6 && t_tiles >= 2;
+  if (want_pair && resident(true, 2 * n_slices) > 0) {
+    const int cl = 2 * n_slices;
+    CUtensorMap mw2;
+    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)H};
+    const uint64_t str[1] = {(uint64_t)K};
+    const uint32_t box[2] = {kBK, kCh / 2};            // each CTA of a pair loads half of the weight rows
+    if ((rc = encode_tensor_map(&mw2, w, 2, dims, str, box, 128))) return rc;
+    const int clusters = (int)std::min<int64_t>((t_tiles + 1) / 2, resident(true, cl));
+    return launch_pdl(gemm_ln_kernel<true>, dim3(clusters * cl), dim3(kThreads), (size_t)kAlloc, ctx->stream, cl,
+                      mx, mw2, mr, mo, a);
+  }
+  if (resident(false, n_slices) <= 0) return IBERT_ERR_CUDA;
+  const int clusters = (int)std::min<int64_t>(t_tiles, resident(false, n_slices));
+  return launch_pdl(gemm_ln_kernel<false>, dim3(clusters * n_slices), dim3(kThreads), (size_t)kAlloc, ctx->stream,
+                    n_slices, mx, mw, mr, mo, a);
 }
 
 }  // namespace ibert

@@ -255,6 +255,8 @@ def run_ours(args):
     assert last - first == batch
     stream = torch.cuda.Stream(device=dev)
     ctx = binding.Context(local_rank, stream)
+    if args.fusion:
+        ctx.ibert_set_fusion(args.fusion)
     bufs = [torch.empty((T, cfg.H), dtype=torch.int8, device=dev) for _ in range(2)]
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     full_model = args.workload == "model"
@@ -562,6 +564,8 @@ def main():
     ap.add_argument("--pow2-scores", action="store_true",
                     help="layers workload: query scales raised so that every score scale is ln2 / 2^k "
                          "(i-exp quotient by shift and mask)")
+    ap.add_argument("--fusion", type=int, default=0, choices=[0, 1, 2],
+                    help="linear + LayerNorm: 0 by problem size (default), 1 cluster kernel whenever supported, 2 never")
     ap.add_argument("--graph", action="store_true",
                     help="layers workload: replay the forward pass from a captured CUDA graph (ibert_encoder_graph_*)")
     ap.add_argument("--workload", choices=["layers", "model"], default="layers",

@@ -672,7 +672,8 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
     int per_sm = std::min(std::min(4 / a.groups, (int)(512 / cols)), (227 * 1024) / (smem + 1024));
     if (per_sm < 1) per_sm = 1;
     const int grid = std::min(B * heads, ctx->num_sms * per_sm);
-    static int smem_set = 0;
+    static int smem_set_dev[kMaxDevices] = {0};
+    int& smem_set = smem_set_dev[ctx->device % kMaxDevices];
     if (smem > smem_set) {
       if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return IBERT_ERR_CUDA;
@@ -692,7 +693,8 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
   const int fixed_bytes = n_slabs * slab + n_slabs * 128 * 128 + 64 + 1024;
   a.stages = (2 * stage_bytes + fixed_bytes <= 112 * 1024) ? 2 : 1;     // keep at least 2 CTAs per SM
   const int smem = a.stages * stage_bytes + fixed_bytes;
-  static int smem_set = 0;
+  static int smem_set_dev[kMaxDevices] = {0};
+  int& smem_set = smem_set_dev[ctx->device % kMaxDevices];
   if (smem > smem_set) {
     if (cudaFuncSetAttribute(attention_coarse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return IBERT_ERR_CUDA;

@@ -343,7 +343,8 @@ template <int TOK, bool PAIR, int KIND, bool FAST>
 int launch_inst(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& mo,
                 const GemmArgs& args) {
   using C = Cfg<TOK, PAIR, KIND>;
-  static bool attr_set = false;
+  static bool attr_set_dev[kMaxDevices] = {false};
+  bool& attr_set = attr_set_dev[ctx->device % kMaxDevices];
   if (!attr_set) {
     if (cudaFuncSetAttribute(gemm_i8_kernel<TOK, PAIR, KIND, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::kAlloc) != cudaSuccess)

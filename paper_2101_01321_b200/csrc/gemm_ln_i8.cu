@@ -494,9 +494,9 @@ int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t 
   const int64_t t_tiles = (T + kTok - 1) / kTok;
   // CTA pairs (two token tiles per cluster step) when the cluster stays within 6 CTAs and there are
   // tiles for both halves; resident clusters from the occupancy query, cached
-  static int max_clusters[2][9] = {{0}};
+  static int max_clusters[kMaxDevices][2][9] = {{{0}}};
   auto resident = [&](bool pair, int cl) {
-    int& slot = max_clusters[pair ? 1 : 0][cl];
+    int& slot = max_clusters[ctx->device % kMaxDevices][pair ? 1 : 0][cl];
     if (slot == 0) {
       const void* fn = pair ? (const void*)gemm_ln_kernel<true> : (const void*)gemm_ln_kernel<false>;
       if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kAlloc) != cudaSuccess) {

@@ -90,6 +90,9 @@ struct DeviceTable {
 
 }  // namespace ibert
 
+// launch-time state the kernels' launchers keep per device (function attributes are per device)
+constexpr int kMaxDevices = 64;
+
 struct ibert_ctx {
   int device = 0;
   cudaStream_t stream = nullptr;

@@ -489,7 +489,8 @@ int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t 
     const int pgrid = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)ctx->num_sms * 3);
 #define IBERT_LNP(V, D)                                                                                     \
   do {                                                                                                      \
-    static bool attr = false;                                                                               \
+    static bool attr_dev[kMaxDevices] = {false};                                                            \
+    bool& attr = attr_dev[ctx->device % kMaxDevices];                                                       \
     if (!attr) {                                                                                            \
       if (cudaFuncSetAttribute(layernorm_pipe_kernel<V, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
                                100 * 1024) != cudaSuccess) return IBERT_ERR_CUDA;                           \

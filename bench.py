@@ -272,16 +272,20 @@ def run_ours(args):
 
         graphs = {}
 
-        def forward(src, eager=False):
+        def forward(src, eager=False, final_out=None):
             if args.graph and not eager:
-                # one captured graph per input buffer (the device-resident one and the e2e staging one)
-                g = graphs.get(src.data_ptr())
+                # one captured graph per (input buffer, output buffer)
+                dst = final_out if final_out is not None else bufs[(len(layers) - 1) & 1]
+                key = (src.data_ptr(), dst.data_ptr())
+                g = graphs.get(key)
                 if g is None:
-                    g = graphs[src.data_ptr()] = binding.Graph(ctx, layers, src, batch, cfg.L, bufs[0])
+                    g = graphs[key] = binding.Graph(ctx, layers, src, batch, cfg.L, dst)
                 return g.launch()
             h = src
             for i, ly in enumerate(layers):
-                h, _ = ctx.ibert_encoder_layer(ly, h, batch, cfg.L, out=bufs[i & 1])
+                last = i == len(layers) - 1
+                h, _ = ctx.ibert_encoder_layer(ly, h, batch, cfg.L,
+                                               out=final_out if (last and final_out is not None) else bufs[i & 1])
             return h
     else:
         # the model around the layers on a padded batch: token ids in, INT8 embedding + LayerNorm,
@@ -301,12 +305,13 @@ def run_ours(args):
         S_last = m["layers"][-1]["S_out"]
         valid_tokens = int(m["lens"].sum())
 
-        def forward(src, eager=False):
+        def forward(src, eager=False, final_out=None):
             h, _ = ctx.ibert_embedding_i8(src, cfg.L, word_d, e["S_word"], pos_d, e["S_pos"], e["gamma"], e["beta"],
                                           e["S_out"], out=emb_out)
             for i, ly in enumerate(layers):
                 h, _ = ctx.ibert_encoder_layer_masked(ly, h, batch, cfg.L, lens_d, out=bufs[i & 1])
-            out, _ = ctx.ibert_classifier_i8(h, batch, cfg.L, S_last, hw_d, hd["S_w"], hb_d, out=logits)
+            out, _ = ctx.ibert_classifier_i8(h, batch, cfg.L, S_last, hw_d, hd["S_w"], hb_d,
+                                             out=final_out if final_out is not None else logits)
             return out
 
     def barrier():
@@ -334,6 +339,45 @@ def run_ours(args):
         stream.synchronize()
         return [a.elapsed_time(b) for a, b in times]
 
+    def timed_e2e(n):
+        """n steps from host buffers: every step's input goes pinned host -> device and its result
+        device -> pinned host inside the timed region; the copies run on side streams over two
+        buffer sets so that step i+1's upload and step i-1's download overlap step i's kernels.
+        Returns the total milliseconds between the first upload and the last download."""
+        s_up, s_down = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        stage = [torch.empty_like(x_stage) for _ in range(2)]
+        outs = [torch.empty_like(out_pin, device=dev) for _ in range(2)]
+        pins = [torch.empty_like(out_pin).pin_memory() for _ in range(2)]
+        ev_up = [torch.cuda.Event() for _ in range(2)]
+        ev_run = [torch.cuda.Event() for _ in range(2)]
+        ev_down = [torch.cuda.Event() for _ in range(2)]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        stream.synchronize()
+        e0.record(stream)
+        s_up.wait_event(e0)
+        for i in range(n):
+            b = i & 1
+            with torch.cuda.stream(s_up):
+                if i >= 2:
+                    s_up.wait_event(ev_run[b])             # step i-2 has consumed this staging buffer
+                stage[b].copy_(x_pin, non_blocking=True)
+                ev_up[b].record(s_up)
+            with torch.cuda.stream(stream):
+                stream.wait_event(ev_up[b])
+                if i >= 2:
+                    stream.wait_event(ev_down[b])          # step i-2's result has left this output buffer
+                forward(stage[b], final_out=outs[b])
+                ev_run[b].record(stream)
+            with torch.cuda.stream(s_down):
+                s_down.wait_event(ev_run[b])
+                pins[b].copy_(outs[b], non_blocking=True)
+                ev_down[b].record(s_down)
+        for b in range(2):
+            stream.wait_event(ev_down[b])
+        e1.record(stream)
+        stream.synchronize()
+        return e0.elapsed_time(e1)
+
     with torch.cuda.stream(stream):
         for _ in range(max(args.warmup, 3)):
             forward(x_dev)
@@ -349,11 +393,10 @@ def run_ours(args):
     ctx.check()
     total_ms = sum(t_steps)
 
-    timed_steps(2, e2e=True)
+    timed_e2e(3)
     barrier()
-    t_e2e = timed_steps(args.steps, e2e=True)
+    total_e2e_ms = timed_e2e(args.steps)
     barrier()
-    total_e2e_ms = sum(t_e2e)
 
     # per-kernel device time of the same steps (separate pass: event pairs around every launch)
     with torch.cuda.stream(stream):
@@ -435,7 +478,10 @@ def run_ours(args):
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_pin.numel() * x_pin.element_size(),
                     "d2h_bytes_per_step": out_pin.numel() * out_pin.element_size(),
-                    "ms_per_step": total_e2e_ms / args.steps},
+                    "ms_per_step": total_e2e_ms / args.steps,
+                    "how": "pinned host -> device upload and device -> pinned host download of every step inside "
+                           "the timed region, on side streams over two buffer sets (overlapping the neighbouring "
+                           "steps' kernels); no L2 flush: each step's input arrives from host memory"},
             "gpu_launches": sum(v["launches_per_step"] for v in kern.values()) * args.steps,
             "roofline": roof,
             "kernels": kern,

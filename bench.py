@@ -32,7 +32,7 @@ DEFAULT_BATCH = {2: 128, 3: 32, 4: 64}
 
 # DRAM bytes (read + write) per launch from one ncu capture of each kernel class at the default
 # workload (config 2, B=128; cold L2; summaries under profiles/).  Other workloads report null.
-NCU_DRAM_TRAFFIC_BYTES = {(2, 128): {"gemm_qkv": 14.5e6, "attention": 37.8e6, "gemm_out_ln": 25.8e6, "gemm_ffn1_gelu": 17.8e6, "gemm_ffn2_ln": 68.0e6, "gemm_out": 14.4e6, "layernorm": 64.1e6, "gemm_ffn2": 60.1e6}}
+NCU_DRAM_TRAFFIC_BYTES = {(2, 128): {"gemm_qkv": 14.5e6, "attention": 37.8e6, "gemm_out_ln": 25.8e6, "gemm_ffn1_gelu": 17.5e6, "gemm_ffn2_ln": 67.4e6, "gemm_out": 13.9e6, "layernorm": 64.0e6, "gemm_ffn2": 59.5e6}}
 
 
 # Integer-datapath instructions (ALU + IMAD pipes, which behave as one 16-lane unit per SM sub-partition)

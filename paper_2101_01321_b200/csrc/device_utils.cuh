@@ -49,6 +49,14 @@ __device__ __forceinline__ uint32_t pack4_sat_s8(int32_t v0, int32_t v1, int32_t
   return r;
 }
 
+// byte k of a word as a sign-extended int32 in one permute (`prmt`: a selector nibble with bit 3
+// set replicates the sign of the byte it selects)
+__device__ __forceinline__ int32_t sext_byte(uint32_t w, int k) {
+  int32_t r;
+  asm("prmt.b32 %0, %1, 0, %2;" : "=r"(r) : "r"(w), "r"(0x8880 + k * 0x1111));
+  return r;
+}
+
 __device__ __forceinline__ int64_t rounding_half(int c) { return c > 0 ? (int64_t(1) << (c - 1)) : 0; }
 
 __device__ __forceinline__ int32_t clamp_sym(int32_t v, int32_t qmax) { return max(-qmax, min(v, qmax)); }

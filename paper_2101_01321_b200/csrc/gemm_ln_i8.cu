@@ -81,14 +81,6 @@ __device__ __forceinline__ uint32_t isqrt_of_quotient(uint64_t ss, uint32_t C) {
   return s;
 }
 
-// byte K of a word as a sign-extended int32 in one permute (`prmt`: a selector nibble with bit 3
-// set replicates the sign of the byte it selects)
-__device__ __forceinline__ int32_t sext_byte(uint32_t w, int k) {
-  int32_t r;
-  asm("prmt.b32 %0, %1, 0, %2;" : "=r"(r) : "r"(w), "r"(0x8880 + k * 0x1111));
-  return r;
-}
-
 // PAIR: two CTAs (same 256 channels, adjacent 128-token tiles) share every MMA through
 // tcgen05.mma.cta_group::2 -- each loads its own token rows and half of the weight rows, which cuts
 // the bytes an SM pulls from L2 per MMA by a third (L2 bandwidth bounds the K = 3072 main loop).

@@ -137,8 +137,10 @@ __global__ void __launch_bounds__(kThreads) softmax_kernel(const int32_t* __rest
 // each.  Needs s < 2^25 and ss < 2^61 / C.
 __device__ __forceinline__ uint32_t warp_isqrt_of_quotient(uint64_t ss, uint32_t C, int lane) {
   uint32_t base = 0;
-#pragma unroll
-  for (int shift = 20; shift >= 0; shift -= 5) {
+  // ss / C < 2^bits bounds the result below 2^ceil(bits / 2): rounds above that cannot set a digit
+  const int bits = 64 - __clzll((long long)(ss | 1ull)) - (31 - __clz((int)C));
+  const int top = 5 * ((min(max((bits + 1) >> 1, 1), 25) + 4) / 5 - 1);
+  for (int shift = top; shift >= 0; shift -= 5) {
     const uint32_t cand = base + ((uint32_t)lane << shift);
     const uint64_t sq = (uint64_t)cand * (uint64_t)cand;
     const bool le = sq * (uint64_t)C <= ss;                       // true for a prefix of the lanes
@@ -344,8 +346,7 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
     for (int j = 0; j < VPL; ++j)
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const int32_t rv = (int32_t)(int8_t)(rw[j] >> (8 * i));
-        v[j][i] += requant_upper(rv << k.res_sh, k.b_r);
+        v[j][i] += requant_upper(sext_byte(rw[j], i) << k.res_sh, k.b_r);
         sum += v[j][i];
       }
     sum = __reduce_add_sync(0xffffffffu, sum);
@@ -362,8 +363,9 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
         ss += (uint64_t)((int64_t)y * (int64_t)y);
       }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    // a lane's share is below 2^50 (|y| <= 2^21, at most 64 values): two 25-bit halves reduce as 32-bit sums
+    ss = (uint64_t)__reduce_add_sync(0xffffffffu, (uint32_t)ss & 0x1ffffffu) +
+         ((uint64_t)__reduce_add_sync(0xffffffffu, (uint32_t)(ss >> 25)) << 25);
     uint32_t sigma = warp_isqrt_of_quotient(ss, (uint32_t)C, lane);   // I-Sqrt(floor(ss / C))
     sigma = sigma < 1u ? 1u : sigma;
     // floor(2^31 / sigma) as a positive int32 multiplier: for sigma = 1 use 2^30 and shift one less
@@ -382,7 +384,9 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
         int32_t o[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int32_t nrm = (int32_t)(((int64_t)v[j][i] * (int64_t)rho) >> nsh) << k.out_sh;
+          const int64_t pr = (int64_t)v[j][i] * (int64_t)rho;
+          // floor(pr / 2^nsh) fits 32 bits: the low word of the 64-bit shift is a funnel shift
+          const int32_t nrm = (int32_t)__funnelshift_r((uint32_t)pr, (uint32_t)(pr >> 32), (uint32_t)nsh) << k.out_sh;
           o[i] = max(requant_upper_add(nrm, bv[i], Bv[i]), -127);
         }
         __stcs(reinterpret_cast<uint32_t*>(orow + col), pack4_sat_s8(o[0], o[1], o[2], o[3]));

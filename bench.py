@@ -426,7 +426,7 @@ def run_ours(args):
         top = max(kern, key=lambda k: kern[k]["share"])
         int8_peak = 2.0 * peaks["bf16_tflops_sustained"]     # nominal INT8 : BF16 dense ratio = 2
         if top == "attention":
-            # i-softmax dominates: ~16 integer instructions per score element (kernels);
+            # i-softmax dominates: ~16 integer instructions per score element (row max, i-exp, sum, quotient);
             # peak = 64 int32 lanes per SM per clock (half the issue rate of a 4-scheduler SM)
             alu_ops = 16.0 * T * cfg.L * cfg.heads
             alu_peak = 64.0 * torch.cuda.get_device_properties(dev).multi_processor_count * (clocks.get("sm_max_mhz") or 1965.0) * 1e6

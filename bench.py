@@ -564,12 +564,13 @@ def run_only(args):
         qd, rd = torch.from_numpy(q).to(dev), torch.from_numpy(r).to(dev)
         out = torch.empty((T, H), dtype=torch.int8, device=dev)
         fn = lambda: ctx.ibert_layernorm_i(qd, S, rd, S_r, gamma, beta, S_out, out=out)
-    elif k in ("gelu", "hgelu"):
+    elif k in ("gelu", "hgelu", "gelu_lut"):
         q, S, S_out = synth.gelu_inputs(1 << 24, 1.0)
         qd = torch.from_numpy(q).to(dev)
         out = torch.empty(q.shape, dtype=torch.int8, device=dev)
-        fn = (lambda: ctx.ibert_gelu_i(qd, S, S_out, out=out)) if k == "gelu" else \
-             (lambda: ctx.ibert_hgelu_i(qd, S, S_out, out=out))
+        fn = {"gelu": lambda: ctx.ibert_gelu_i(qd, S, S_out, out=out),
+              "hgelu": lambda: ctx.ibert_hgelu_i(qd, S, S_out, out=out),
+              "gelu_lut": lambda: ctx.ibert_gelu_lut_i(qd, S, S_out, out=out)}[k]
     elif k == "softmax":
         rows = batch * cfg.heads * L
         q, S = synth.softmax_inputs(rows, L, 1.0)

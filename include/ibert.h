@@ -233,6 +233,15 @@ int ibert_linear_hgelu_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int
                           const int32_t* bias, int64_t M, int N, int K, double S_mid, double S_out,
                           int8_t* out, double* S_ret);
 
+/* i-GELU by table look-up -- the alternative the paper argues against (Sec. 2, Sec. 3.4), here only
+   for a measured comparison.  A 65535-entry int8 table for the scale pair (S, S_out) is built on
+   first use by running the i-GELU kernel over every Q16 input (so its contents are Algorithm 2's
+   results bit for bit) and cached in the context; afterwards each element costs one clamp and one
+   load.  Results are identical to ibert_gelu_i.  Arguments and errors as ibert_gelu_i; the first
+   call for a scale pair allocates 64 KiB of device memory (freed by ibert_destroy). */
+int ibert_gelu_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
+                     double* S_ret);
+
 /* ---- a stack of encoder layers captured into a CUDA graph ---------------------------------------
    No counterpart in the paper: launch-overhead removal for small batches (a 12-layer pass is 60
    kernel launches).  ibert_encoder_graph_create runs layers[0..n_layers) once on the context's

@@ -59,6 +59,7 @@ def lib():
         L.ibert_linear_layernorm_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, vp, dbl, vp, vp, dbl,
                                                 vp, vp]
         L.ibert_hgelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
+        L.ibert_gelu_lut_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
         L.ibert_linear_hgelu_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, dbl, vp, vp]
         L.ibert_set_fusion.argtypes = [vp, i32]
         L.ibert_softmax_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
@@ -89,7 +90,7 @@ def lib():
                      "ibert_encoder_layer", "ibert_attention_masked_i8", "ibert_encoder_layer_masked",
                      "ibert_embedding_i8", "ibert_classifier_i8", "ibert_encoder_graph_create",
                      "ibert_encoder_graph_launch", "ibert_encoder_graph_destroy", "ibert_hgelu_i",
-                     "ibert_linear_hgelu_i8", "ibert_set_fusion"):
+                     "ibert_linear_hgelu_i8", "ibert_set_fusion", "ibert_gelu_lut_i"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -183,6 +184,15 @@ class Context:
         S_ret = C.c_double()
         _chk(lib().ibert_gelu_i(self.h, _dev(q, torch.int32), S, q.numel(), S_out, _dev(out, torch.int8),
                                 C.byref(S_ret)), "ibert_gelu_i")
+        return out, S_ret.value
+
+    def ibert_gelu_lut_i(self, q: torch.Tensor, S: float, S_out: float, out: torch.Tensor | None = None):
+        """i-GELU through a look-up table built from the integer kernel (comparison only)."""
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.int8, device=q.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_gelu_lut_i(self.h, _dev(q, torch.int32), S, q.numel(), S_out, _dev(out, torch.int8),
+                                    C.byref(S_ret)), "ibert_gelu_lut_i")
         return out, S_ret.value
 
     def ibert_hgelu_i(self, q: torch.Tensor, S: float, S_out: float, out: torch.Tensor | None = None):

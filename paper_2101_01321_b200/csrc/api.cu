@@ -155,6 +155,7 @@ int ibert_destroy(ibert_ctx* ctx) {
   DeviceGuard guard(ctx->device);
   cudaStreamSynchronize(ctx->stream);
   for (auto& kv : ctx->tables) cudaFree(kv.second.ptr);
+  for (auto& kv : ctx->gelu_luts) cudaFree(kv.second);
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   if (ctx->ws) cudaFree(ctx->ws);
   cudaFree(ctx->d_status);
@@ -198,6 +199,35 @@ static int gelu_common(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, do
 int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
                  double* S_ret) {
   return gelu_common(ctx, q, S, n, S_out, out, S_ret, false);
+}
+
+static int ensure_workspace(ibert_ctx* ctx, size_t need);
+
+int ibert_gelu_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
+                     double* S_ret) {
+  if (!ctx || n < 0 || (n > 0 && (!q || !out))) return IBERT_ERR_ARG;
+  if (!aligned16(q) || !aligned16(out)) return IBERT_ERR_ALIGN;
+  GeluConsts k{};                                   // zeroed: the bytes are hashed below
+  int rc = make_gelu_consts(S, S_out, &k);
+  if (rc) return rc;
+  DeviceGuard guard(ctx->device);
+  const uint64_t key = fnv1a(&k, sizeof(k), 0x6c7574ull);
+  int8_t* table = nullptr;
+  auto it = ctx->gelu_luts.find(key);
+  if (it != ctx->gelu_luts.end()) table = it->second;
+  else {
+    // built once per scale pair: ramp into the workspace, the i-GELU kernel over it
+    if ((rc = ensure_workspace(ctx, 65536 * sizeof(int32_t)))) return rc;
+    if (cudaMalloc((void**)&table, 65536) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_NOMEM; }
+    if ((rc = launch_gelu_table(ctx, k, static_cast<int32_t*>(ctx->ws), table))) { cudaFree(table); return rc; }
+    ctx->gelu_luts[key] = table;
+  }
+  {
+    ProfileScope ps(ctx, IBERT_K_GELU);
+    rc = launch_gelu_lut(ctx, q, n, table, out);
+  }
+  if (rc == IBERT_OK && S_ret) *S_ret = S_out;
+  return rc;
 }
 
 int ibert_hgelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,

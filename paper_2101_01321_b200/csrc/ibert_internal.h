@@ -100,6 +100,8 @@ struct ibert_ctx {
   int num_sms = 0;
   // derived constant tables already on the device, keyed by a hash of their host bytes
   std::map<uint64_t, ibert::DeviceTable> tables;
+  // look-up tables of ibert_gelu_lut_i, keyed by a hash of the GELU constants
+  std::map<uint64_t, int8_t*> gelu_luts;
   // workspace for the encoder layer's intermediates
   void* ws = nullptr;
   size_t ws_bytes = 0;
@@ -121,6 +123,10 @@ int cached_upload(ibert_ctx* ctx, const void* host, size_t bytes, uint64_t tag, 
 // ---------------------------------------------------------------------------------------
 
 int launch_gelu(ibert_ctx* ctx, const int32_t* q, int64_t n, const GeluConsts& k, int8_t* out);
+// table[i] = i-GELU(i - 32767) for i in [0, 65535), computed by the i-GELU kernel over a ramp written
+// to `ramp_scratch` (65535 int32); and the look-up kernel that uses it
+int launch_gelu_table(ibert_ctx* ctx, const GeluConsts& k, int32_t* ramp_scratch, int8_t* table);
+int launch_gelu_lut(ibert_ctx* ctx, const int32_t* q, int64_t n, const int8_t* table, int8_t* out);
 int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const ExpConsts& k, uint8_t* out);
 // rows of the word table (as int32) and of the position table (token t: position t mod L) gathered
 // into q [T, H] and r [T, H]; an id outside [0, V) records IBERT_ERR_VALUE_RANGE and reads row 0

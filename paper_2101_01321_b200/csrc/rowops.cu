@@ -66,6 +66,35 @@ __global__ void __launch_bounds__(kThreads) gelu_kernel(const int32_t* __restric
                                       : igelu_q16_to_int8(clamp_sym(q[tail + tid], 32767), k, half));
 }
 
+// ----------------------------------------------------------------------------- table look-up GELU
+// The alternative the paper argues against: a 65535-entry table of the int8 result for every Q16
+// input, built by running the i-GELU kernel once over the ramp -32767 .. 32767 (so its bits are the
+// integer function's), then one load per element.
+__global__ void __launch_bounds__(kThreads) ramp_q16_kernel(int32_t* __restrict__ q) {
+  const int i = blockIdx.x * kThreads + threadIdx.x;
+  if (i < 65535) q[i] = i - 32767;
+}
+
+__global__ void __launch_bounds__(kThreads) gelu_lut_kernel(const int32_t* __restrict__ q, int64_t n,
+                                                            const int8_t* __restrict__ table,
+                                                            int8_t* __restrict__ out) {
+  const int64_t n_vec = n >> 2;
+  const int4* q4 = reinterpret_cast<const int4*>(q);
+  uint32_t* o4 = reinterpret_cast<uint32_t*>(out);
+  const int64_t stride = (int64_t)gridDim.x * kThreads;
+  for (int64_t idx = (int64_t)blockIdx.x * kThreads + threadIdx.x; idx < n_vec; idx += stride) {
+    const int4 v = __ldcs(q4 + idx);
+    const uint32_t a = (uint8_t)__ldg(table + clamp_sym(v.x, 32767) + 32767);
+    const uint32_t b = (uint8_t)__ldg(table + clamp_sym(v.y, 32767) + 32767);
+    const uint32_t c = (uint8_t)__ldg(table + clamp_sym(v.z, 32767) + 32767);
+    const uint32_t d = (uint8_t)__ldg(table + clamp_sym(v.w, 32767) + 32767);
+    __stcs(o4 + idx, a | (b << 8) | (c << 16) | (d << 24));
+  }
+  const int64_t tid = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  const int64_t tail = n_vec << 2;
+  if (tid < n - tail) out[tail + tid] = __ldg(table + clamp_sym(q[tail + tid], 32767) + 32767);
+}
+
 // ----------------------------------------------------------------------------- i-softmax
 // One warp per row; a lane keeps VPL int4 vectors (4*VPL scores) in registers.
 // VEC: rows are 16-byte aligned (L % 4 == 0) and loaded/stored as vectors.
@@ -443,6 +472,19 @@ int launch_embed_gather(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, co
   if (T == 0) return IBERT_OK;
   embed_gather_kernel<<<grid_for(ctx, T, 8), kThreads, 0, ctx->stream>>>(ids, T, L, word, V, pos, H, q, r,
                                                                           ctx->d_status);
+  return check_launch();
+}
+
+int launch_gelu_table(ibert_ctx* ctx, const GeluConsts& k, int32_t* ramp_scratch, int8_t* table) {
+  ramp_q16_kernel<<<(65535 + kThreads - 1) / kThreads, kThreads, 0, ctx->stream>>>(ramp_scratch);
+  if (int rc = check_launch()) return rc;
+  return launch_gelu(ctx, ramp_scratch, 65535, k, table);
+}
+
+int launch_gelu_lut(ibert_ctx* ctx, const int32_t* q, int64_t n, const int8_t* table, int8_t* out) {
+  if (n == 0) return IBERT_OK;
+  const int64_t warps = ((n >> 2) + 31) / 32 / 8 + 1;          // ~8 vectors per thread
+  gelu_lut_kernel<<<grid_for(ctx, warps, 8), kThreads, 0, ctx->stream>>>(q, n, table, out);
   return check_launch();
 }
 

@@ -47,3 +47,21 @@ def test_linear_hgelu_matches_oracle(M, N, K):
     mid = oracle.linear(x, S_x, w, S_w, bias, 1, S_mid)
     want, _ = oracle.hgelu(mid, S_mid, S_out)
     assert_same(host(out), want.reshape(M, N), "linear + h-GELU")
+
+
+@pytest.mark.parametrize("sigma", [1.0, 4.0])
+def test_gelu_by_table_lookup_equals_the_integer_kernel(sigma):
+    """The look-up table is built from the i-GELU kernel, so both entry points agree bit for bit
+    (and with the oracle), for ordinary inputs and for the whole int32 range."""
+    q, S, S_out = synth.gelu_inputs(300007, sigma)
+    rng = np.random.default_rng(4)
+    q = np.concatenate([q, rng.integers(-2**31, 2**31, 5000).astype(np.int32),
+                        np.array([2**31 - 1, -2**31, 0, 32767, -32767, 32768, -32768], np.int32)])
+    a, _ = ctx().ibert_gelu_lut_i(dev(q), S, S_out)
+    b, _ = ctx().ibert_gelu_i(dev(q), S, S_out)
+    ctx().check()
+    assert_same(host(a), host(b), "table vs kernel")
+    assert_same(host(a), oracle.gelu(q, S, S_out)[0], "table vs oracle")
+    a2, _ = ctx().ibert_gelu_lut_i(dev(q), S, S_out)          # second call: cached table
+    ctx().check()
+    assert_same(host(a2), host(b), "cached table")

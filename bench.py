@@ -571,12 +571,13 @@ def run_only(args):
         fn = {"gelu": lambda: ctx.ibert_gelu_i(qd, S, S_out, out=out),
               "hgelu": lambda: ctx.ibert_hgelu_i(qd, S, S_out, out=out),
               "gelu_lut": lambda: ctx.ibert_gelu_lut_i(qd, S, S_out, out=out)}[k]
-    elif k == "softmax":
+    elif k in ("softmax", "softmax_lut"):
         rows = batch * cfg.heads * L
         q, S = synth.softmax_inputs(rows, L, 1.0)
         qd = torch.from_numpy(q).to(dev)
         out = torch.empty(q.shape, dtype=torch.uint8, device=dev)
-        fn = lambda: ctx.ibert_softmax_i(qd, S, 255, out=out)
+        fn = (lambda: ctx.ibert_softmax_i(qd, S, 255, out=out)) if k == "softmax" else \
+             (lambda: ctx.ibert_softmax_lut_i(qd, S, 255, out=out))
     else:
         raise SystemExit(f"unknown kernel class {k}")
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)

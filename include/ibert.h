@@ -88,6 +88,15 @@ int ibert_linear_gelu_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
 int ibert_softmax_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
                     uint8_t* out, double* S_ret);
 
+/* i-softmax with i-exp by table look-up -- the alternative the paper argues against (Sec. 2,
+   Sec. 3.5), here only for a measured comparison.  The table holds the i-exp of every pre-shifted
+   distance from the row maximum, 0 .. 31*q_ln2 (up to 2 MiB of uint32), filled on first use for a
+   scale by the same device function ibert_softmax_i evaluates, and cached in the context (freed by
+   ibert_destroy).  Results are identical to ibert_softmax_i; arguments and errors as there, plus
+   IBERT_ERR_NOMEM when the table cannot be allocated. */
+int ibert_softmax_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
+                        uint8_t* out, double* S_ret);
+
 /* i-GELU (Algorithm 2, Eq. 8-9), elementwise.  q int32 at scale S, clamped to Q16 first;
    out int8 at S_out (the product q*(q_erf+q_1) is requantized in-kernel); *S_ret = S_out. */
 int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,

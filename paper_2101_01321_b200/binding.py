@@ -63,6 +63,7 @@ def lib():
         L.ibert_linear_hgelu_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, dbl, vp, vp]
         L.ibert_set_fusion.argtypes = [vp, i32]
         L.ibert_softmax_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
+        L.ibert_softmax_lut_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
         L.ibert_gelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
         L.ibert_layernorm_i.argtypes = [vp, vp, dbl, vp, dbl, vp, vp, i64, i32, dbl, vp, vp]
         L.ibert_attention_i8.argtypes = [vp, vp, i32, i32, i32, i32, dbl, dbl, dbl, dbl, i32, vp, vp]
@@ -90,7 +91,7 @@ def lib():
                      "ibert_encoder_layer", "ibert_attention_masked_i8", "ibert_encoder_layer_masked",
                      "ibert_embedding_i8", "ibert_classifier_i8", "ibert_encoder_graph_create",
                      "ibert_encoder_graph_launch", "ibert_encoder_graph_destroy", "ibert_hgelu_i",
-                     "ibert_linear_hgelu_i8", "ibert_set_fusion", "ibert_gelu_lut_i"):
+                     "ibert_linear_hgelu_i8", "ibert_set_fusion", "ibert_gelu_lut_i", "ibert_softmax_lut_i"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -204,15 +205,20 @@ class Context:
                                  C.byref(S_ret)), "ibert_hgelu_i")
         return out, S_ret.value
 
-    def ibert_softmax_i(self, q: torch.Tensor, S: float, p_max: int = 255, out: torch.Tensor | None = None):
+    def ibert_softmax_i(self, q: torch.Tensor, S: float, p_max: int = 255, out: torch.Tensor | None = None,
+                        _entry: str = "ibert_softmax_i"):
         L = q.shape[-1]
         rows = q.numel() // L if L else 0
         if out is None:
             out = torch.empty(q.shape, dtype=torch.uint8, device=q.device)
         S_ret = C.c_double()
-        _chk(lib().ibert_softmax_i(self.h, _dev(q, torch.int32), S, rows, L, p_max, _dev(out, torch.uint8),
-                                   C.byref(S_ret)), "ibert_softmax_i")
+        _chk(getattr(lib(), _entry)(self.h, _dev(q, torch.int32), S, rows, L, p_max, _dev(out, torch.uint8),
+                                    C.byref(S_ret)), _entry)
         return out, S_ret.value
+
+    def ibert_softmax_lut_i(self, q: torch.Tensor, S: float, p_max: int = 255, out: torch.Tensor | None = None):
+        """i-softmax with i-exp read from a table built by the integer function (comparison only)."""
+        return self.ibert_softmax_i(q, S, p_max, out, _entry="ibert_softmax_lut_i")
 
     def ibert_layernorm_i(self, q: torch.Tensor, S: float, r: torch.Tensor | None, S_r: float, gamma, beta,
                           S_out: float, out: torch.Tensor | None = None):

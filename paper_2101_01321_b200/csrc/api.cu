@@ -156,6 +156,7 @@ int ibert_destroy(ibert_ctx* ctx) {
   cudaStreamSynchronize(ctx->stream);
   for (auto& kv : ctx->tables) cudaFree(kv.second.ptr);
   for (auto& kv : ctx->gelu_luts) cudaFree(kv.second);
+  for (auto& kv : ctx->exp_luts) cudaFree(kv.second);
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   if (ctx->ws) cudaFree(ctx->ws);
   cudaFree(ctx->d_status);
@@ -235,23 +236,48 @@ int ibert_hgelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double 
   return gelu_common(ctx, q, S, n, S_out, out, S_ret, true);
 }
 
-int ibert_softmax_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
-                    uint8_t* out, double* S_ret) {
+static int softmax_common(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
+                          uint8_t* out, double* S_ret, bool by_table) {
   if (!ctx || rows < 0) return IBERT_ERR_ARG;
   if (p_max != 255 && p_max != 127) return IBERT_ERR_ARG;
   if (L < 1 || L > 1024) return IBERT_ERR_SHAPE;
   if (rows > 0 && (!q || !out)) return IBERT_ERR_ARG;
   if (!aligned16(q) || !aligned16(out)) return IBERT_ERR_ALIGN;
-  ExpConsts k;
+  ExpConsts k{};                                    // zeroed: the bytes are hashed below
   int rc = make_exp_consts(S, p_max, &k);
   if (rc) return rc;
   DeviceGuard guard(ctx->device);
+  uint32_t* table = nullptr;
+  if (by_table) {
+    const uint64_t key = fnv1a(&k, sizeof(k), 0x657870ull);
+    auto it = ctx->exp_luts.find(key);
+    if (it != ctx->exp_luts.end()) table = it->second;
+    else {
+      // built once per scale: the i-exp of every pre-shifted distance 0 .. d_max
+      if (cudaMalloc((void**)&table, ((size_t)k.d_max + 1) * sizeof(uint32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        return IBERT_ERR_NOMEM;
+      }
+      if ((rc = launch_exp_table(ctx, k, table))) { cudaFree(table); return rc; }
+      ctx->exp_luts[key] = table;
+    }
+  }
   {
     ProfileScope ps(ctx, IBERT_K_SOFTMAX);
-    rc = launch_softmax(ctx, q, rows, L, k, out);
+    rc = launch_softmax(ctx, q, rows, L, k, out, table);
   }
   if (rc == IBERT_OK && S_ret) *S_ret = 1.0 / (double)p_max;
   return rc;
+}
+
+int ibert_softmax_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
+                    uint8_t* out, double* S_ret) {
+  return softmax_common(ctx, q, S, rows, L, p_max, out, S_ret, false);
+}
+
+int ibert_softmax_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
+                        uint8_t* out, double* S_ret) {
+  return softmax_common(ctx, q, S, rows, L, p_max, out, S_ret, true);
 }
 
 int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* r, double S_r,

@@ -102,6 +102,7 @@ struct ibert_ctx {
   std::map<uint64_t, ibert::DeviceTable> tables;
   // look-up tables of ibert_gelu_lut_i, keyed by a hash of the GELU constants
   std::map<uint64_t, int8_t*> gelu_luts;
+  std::map<uint64_t, uint32_t*> exp_luts;
   // workspace for the encoder layer's intermediates
   void* ws = nullptr;
   size_t ws_bytes = 0;
@@ -127,7 +128,9 @@ int launch_gelu(ibert_ctx* ctx, const int32_t* q, int64_t n, const GeluConsts& k
 // to `ramp_scratch` (65535 int32); and the look-up kernel that uses it
 int launch_gelu_table(ibert_ctx* ctx, const GeluConsts& k, int32_t* ramp_scratch, int8_t* table);
 int launch_gelu_lut(ibert_ctx* ctx, const int32_t* q, int64_t n, const int8_t* table, int8_t* out);
-int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const ExpConsts& k, uint8_t* out);
+int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const ExpConsts& k, uint8_t* out,
+                   const uint32_t* exp_table = nullptr);
+int launch_exp_table(ibert_ctx* ctx, const ExpConsts& k, uint32_t* table);
 // rows of the word table (as int32) and of the position table (token t: position t mod L) gathered
 // into q [T, H] and r [T, H]; an id outside [0, V) records IBERT_ERR_VALUE_RANGE and reads row 0
 int launch_embed_gather(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,

@@ -98,9 +98,22 @@ __global__ void __launch_bounds__(kThreads) gelu_lut_kernel(const int32_t* __res
 // ----------------------------------------------------------------------------- i-softmax
 // One warp per row; a lane keeps VPL int4 vectors (4*VPL scores) in registers.
 // VEC: rows are 16-byte aligned (L % 4 == 0) and loaded/stored as vectors.
+// DIV 0..2: how i-exp divides by q_ln2; DIV 3: i-exp read from `table` (comparison variant).
+constexpr int kExpByTable = 3;
+
+// table[i] = i-exp of the pre-shifted distance i, for i = 0 .. d_max
+__global__ void __launch_bounds__(kThreads) exp_table_kernel(ExpConsts k, uint32_t* __restrict__ table) {
+  const uint32_t i = blockIdx.x * kThreads + threadIdx.x;
+  if (i > k.d_max) return;
+  const uint32_t d = i << k.s_in;
+  const int mode = exp_div_mode(k);
+  table[i] = mode == 0 ? iexp_dist<0>(d, k) : (mode == 1 ? iexp_dist<1>(d, k) : iexp_dist<2>(d, k));
+}
+
 template <int VPL, bool VEC, int DIV>
 __global__ void __launch_bounds__(kThreads) softmax_kernel(const int32_t* __restrict__ q, int64_t rows,
-                                                           int L, ExpConsts k, uint8_t* __restrict__ out) {
+                                                           int L, ExpConsts k, uint8_t* __restrict__ out,
+                                                           const uint32_t* __restrict__ table) {
   const int lane = threadIdx.x & 31;
   const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
   const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
@@ -133,7 +146,12 @@ __global__ void __launch_bounds__(kThreads) softmax_kernel(const int32_t* __rest
       const int col = 4 * (j * 32 + lane);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint32_t e = (col + i < L) ? iexp_dist<DIV>((uint32_t)mx - (uint32_t)v[j][i], k) : 0u;
+        const uint32_t dist = (uint32_t)mx - (uint32_t)v[j][i];
+        uint32_t e = 0u;
+        if (col + i < L) {
+          if constexpr (DIV == kExpByTable) e = __ldg(table + min(dist >> k.s_in, k.d_max));
+          else e = iexp_dist<DIV>(dist, k);
+        }
         v[j][i] = (int32_t)e;
         sum += e;
       }
@@ -495,22 +513,29 @@ int launch_gelu(ibert_ctx* ctx, const int32_t* q, int64_t n, const GeluConsts& k
   return check_launch();
 }
 
-int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const ExpConsts& k, uint8_t* out) {
+int launch_exp_table(ibert_ctx* ctx, const ExpConsts& k, uint32_t* table) {
+  exp_table_kernel<<<(int)((k.d_max + kThreads) / kThreads), kThreads, 0, ctx->stream>>>(k, table);
+  return check_launch();
+}
+
+int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const ExpConsts& k, uint8_t* out,
+                   const uint32_t* exp_table) {
   if (rows == 0) return IBERT_OK;
   const int grid = grid_for(ctx, rows, 8);
   const bool vec = (L % 4) == 0;
   const int vpl = (L + 127) / 128;   // vectors per lane
-  const int div = exp_div_mode(k);
-#define IBERT_SM2(V, D)                                                                            \
-  do {                                                                                             \
-    if (vec) softmax_kernel<V, true, D><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out);   \
-    else softmax_kernel<V, false, D><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out);      \
+  const int div = exp_table ? kExpByTable : exp_div_mode(k);
+#define IBERT_SM2(V, D)                                                                                       \
+  do {                                                                                                        \
+    if (vec) softmax_kernel<V, true, D><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out, exp_table);   \
+    else softmax_kernel<V, false, D><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out, exp_table);      \
   } while (0)
 #define IBERT_SM(V)                 \
   do {                              \
     if (div == 0) IBERT_SM2(V, 0);  \
     else if (div == 1) IBERT_SM2(V, 1); \
-    else IBERT_SM2(V, 2);           \
+    else if (div == 2) IBERT_SM2(V, 2); \
+    else IBERT_SM2(V, kExpByTable);     \
   } while (0)
   if (vpl <= 1) IBERT_SM(1);
   else if (vpl <= 2) IBERT_SM(2);

@@ -48,6 +48,23 @@ def test_softmax_matches_oracle(rows, L, p_max):
             assert_same(host(out), want, f"softmax L={L}")
 
 
+@pytest.mark.parametrize("rows,L", [(9, 7), (96 * 8, 128), (40, 512), (12, 1024), (3, 130)])
+def test_softmax_with_exp_by_table_equals_the_integer_kernel(rows, L):
+    """The table holds the integer function's own values, so the comparison variant agrees bit for bit."""
+    for sigma, p_max in ((1.0, 255), (4.0, 127)):
+        q, S = synth.softmax_inputs(rows, L, sigma)
+        a, _ = ctx().ibert_softmax_lut_i(dev(q), S, p_max)
+        ctx().check()
+        assert_same(host(a), oracle.softmax(q, S, p_max)[0], f"softmax by table L={L}")
+    rng = np.random.default_rng(L)
+    q = rng.integers(-2 ** 31, 2 ** 31, (rows, L)).astype(np.int32)
+    q[0] = 3
+    for S in (1e-3, 2e-5, 1e-8, 0.69):
+        a, _ = ctx().ibert_softmax_lut_i(dev(q), S, 255)
+        assert_same(host(a), oracle.softmax(q, S, 255)[0], f"softmax by table S={S}")
+    ctx().check()
+
+
 def test_softmax_extreme_inputs_and_scales():
     rng = np.random.default_rng(5)
     L = 96

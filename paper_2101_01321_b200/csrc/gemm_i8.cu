@@ -87,6 +87,10 @@ constexpr int BC = 128;           // output channels per CTA = TMEM lanes
 constexpr int BK = 128;           // K bytes per pipeline stage = one 128-byte swizzle span
 constexpr int UMMA_K = 32;        // K per tcgen05.mma kind::i8
 
+// i-GELU epilogue whose results provably stay above -127 (GeluConsts::low_free): no lower clamp.
+// A kind of its own, internal to this file, so that the choice costs no instruction in the loop.
+constexpr int kEpiGeluLowFree = 16;
+
 template <int TOK, bool PAIR, int KIND>
 struct Cfg {
   static constexpr bool kOut32 = (KIND == EPI_RAW || KIND == EPI_Q16);
@@ -300,6 +304,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if constexpr (KIND == EPI_HGELU) {
               if constexpr (FAST) o = clamp_sym(ihgelu_upper(requant_upper(a + cur_bias, cur_pb), gk), 127);
               else o = ihgelu_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
+            } else if constexpr (KIND == kEpiGeluLowFree) {
+              o = min(igelu_magnitude_upper(requant_upper(a + cur_bias, cur_pb), gk, gelu_rnd), 127);
             } else {
               if constexpr (FAST) o = clamp_sym(igelu_magnitude_upper(requant_upper(a + cur_bias, cur_pb), gk, gelu_rnd), 127);
               else o = igelu_q16_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
@@ -363,7 +369,9 @@ int launch_shape(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, c
   switch (kind) {
     case EPI_INT8: return fast ? launch_inst<TOK, PAIR, EPI_INT8, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_INT8, false>(ctx, mw, mx, mo, a);
     case EPI_Q16: return fast ? launch_inst<TOK, PAIR, EPI_Q16, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_Q16, false>(ctx, mw, mx, mo, a);
-    case EPI_GELU: return fast ? launch_inst<TOK, PAIR, EPI_GELU, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_GELU, false>(ctx, mw, mx, mo, a);
+    case EPI_GELU:
+      if (fast && a.gelu.low_free) return launch_inst<TOK, PAIR, kEpiGeluLowFree, true>(ctx, mw, mx, mo, a);
+      return fast ? launch_inst<TOK, PAIR, EPI_GELU, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_GELU, false>(ctx, mw, mx, mo, a);
     case EPI_HGELU: return fast ? launch_inst<TOK, PAIR, EPI_HGELU, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_HGELU, false>(ctx, mw, mx, mo, a);
     default: return launch_inst<TOK, PAIR, EPI_RAW, false>(ctx, mw, mx, mo, a);
   }

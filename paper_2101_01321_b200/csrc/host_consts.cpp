@@ -145,6 +145,17 @@ int make_gelu_consts(double S, double S_out, GeluConsts* k) {
   k->b2 = k->fast ? b1[0] : 0;
   k->add2 = k->fast ? (int64_t(1) << 31) : 0;                 // 2^(c-1) << (32-c)
   k->hard = 0;
+  // Bound of the negative results.  For q < 0 the product is a f with a = |q| and
+  // f = ceil(t^2 / 2^s_f), t = min(a >> s_in, -q_b) + q_b; f = 0 once a >> s_in reaches -q_b, and
+  // below that, with w = (a >> s_in) + 1, a t^2 < 2^s_in w (-q_b + 1 - w)^2 <= 2^s_in (4/27) (-q_b + 1)^3.
+  // So g <= 2^s_in (4/27) (-q_b + 1)^3 / 2^s_f + 32767, and the result is at most
+  // (g / 256 + 1) |b| / 2^c + 1 in magnitude.
+  {
+    const double n1 = (double)k->nq_b + 1.0;
+    const double g = std::ldexp((4.0 / 27.0) * n1 * n1 * n1, s_in - k->s_f) + 32767.0;
+    const double out = std::ldexp((g / 256.0 + 1.0) * std::fabs((double)k->b), -k->c) + 1.0;
+    k->low_free = out * 1.001 <= 127.0 ? 1 : 0;
+  }
   return IBERT_OK;
 }
 

@@ -51,6 +51,9 @@ struct GeluConsts {
   // h-GELU (Eq. 6) through the same plumbing: hard != 0 and the fields above mean
   // nq_b = q_6 = floor(6 / S_h), q_c = q_3 = floor(3 / S_h), s_f = s_h, s_in unused (S_h = 1.702 S)
   int32_t hard;
+  // i-GELU only: the most negative result provably stays above -127 (its magnitude is bounded by
+  // the minimum of x erf-polynomial, about 0.17 in real units), so no lower clamp is needed
+  int32_t low_free;
 };
 
 // residual add in front of i-LayerNorm

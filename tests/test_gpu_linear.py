@@ -68,6 +68,23 @@ def test_linear_with_fused_gelu(M, N, K):
     assert np.abs(mid).max() > 8000 and want.max() > 60
 
 
+@pytest.mark.parametrize("S_out,low_clamp_hit", [(0.17 / 126.0, False), (0.17 / 128.0, None), (0.17 / 400.0, True),
+                                                 (6.0 / 127.0, False)])
+def test_linear_with_fused_gelu_around_the_lower_clamp(S_out, low_clamp_hit):
+    """Output scales at which the negative lobe of GELU (minimum about -0.17) stays inside int8, just
+    touches -127, or saturates: the epilogue without a lower clamp may only run where none is needed."""
+    x, w, bias, S_w, S_x, amax = _problem(256, 256, 128, 5)
+    S_mid = 6.0 / 32767.0
+    S_x = S_x * (6.0 / amax)
+    out, _ = ctx().ibert_linear_gelu_i8(dev(x), S_x, dev(w), S_w, dev(bias), S_mid, S_out)
+    ctx().check()
+    mid = oracle.linear(x, S_x, w, S_w, bias, 1, S_mid)
+    want, _ = oracle.gelu(mid, S_mid, S_out)
+    assert_same(host(out), want, f"linear+gelu S_out={S_out}")
+    if low_clamp_hit is not None:
+        assert (want.min() == -127) == low_clamp_hit
+
+
 def test_linear_odd_dyadic_shifts_and_negative_results():
     # multipliers >= 1 (small shifts) and a large-bias column block
     M, N, K = 64, 64, 64

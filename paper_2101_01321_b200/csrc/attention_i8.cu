@@ -319,10 +319,11 @@ attention_coarse_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid
 // ---------------------------------------------------------------------------------------------
 // The main kernel.  A persistent CTA owns one (batch, head) pair at a time and walks its 128-query
 // tiles, so K, V and the transposed V are loaded / built once per pair.  The CTA has 128 G threads,
-// G = ceil(L / 128) column groups: warp w works on TMEM lane quadrant w & 3 (the only lanes a warp
+// G >= ceil(L / 128) column groups: warp w works on TMEM lane quadrant w & 3 (the only lanes a warp
 // may address) and on the 32-column chunks of group w >> 2, so a score row is shared by G threads
-// that exchange their partial maximum and partial sum through shared memory.  Up to 128 keys that
-// is one thread per row and four CTAs per SM; at 512 keys one CTA of 16 warps fills the SM's TMEM.
+// that exchange their partial maximum and partial sum through shared memory.  Up to 128 keys and
+// with many pairs that is one thread per row and four CTAs per SM; at 512 keys one CTA of 16 warps
+// fills the SM's TMEM; with fewer pairs than SMs the launcher raises G to shorten the lone CTA's softmax.
 // Every operand buffer is refilled as soon as its last reader is done (V after the transpose, K
 // and a lone Q after the score MMAs), so the next pair's loads hide behind the softmax.
 // Requires the unclamped i-exp form (ExpConsts::wide_post >= 0).
@@ -663,6 +664,13 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
     AttnArgs a{};
     a.B = B; a.L = L; a.H = H; a.heads = heads;
     a.Lp = Lp; a.n_slabs = n_slabs; a.groups = n_slabs;
+    {
+      // few pairs: a score row is shared by more threads than its slabs ask for, as many as still
+      // keep every pair resident at once (the softmax of a lone CTA per SM is latency-bound)
+      const int64_t items = (int64_t)B * heads;
+      const int g = items <= ctx->num_sms ? 4 : (items <= 2 * (int64_t)ctx->num_sms ? 2 : 1);
+      a.groups = std::min(std::max(n_slabs, g), std::max(Lp / 32, n_slabs));
+    }
     a.q_bufs = n_slabs > 1 ? 2 : 1;
     a.tmem_cols = cols; a.k = k; a.lens = lens; a.out = out; a.status = ctx->d_status;
     const int smem = a.q_bufs * slab + 3 * n_slabs * slab + n_slabs * 128 * 128 + 2 * 4 * 128 * 4 + 64 + 1024;

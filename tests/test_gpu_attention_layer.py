@@ -12,7 +12,8 @@ pytestmark = pytest.mark.gpu
 
 @pytest.mark.parametrize("B,L,heads", [(1, 16, 1), (2, 37, 2), (1, 128, 12), (3, 128, 2), (2, 200, 2), (1, 256, 3),
                                        (1, 512, 2), (2, 1, 1), (1, 33, 1), (1, 300, 1), (0, 64, 1), (1, 130, 1), (1, 384, 2),
-                                       (2, 480, 1), (40, 160, 8), (20, 290, 8)])
+                                       (2, 480, 1), (40, 160, 8), (20, 290, 8), (30, 128, 12), (16, 100, 12), (38, 64, 4),
+                                       (25, 256, 8), (10, 384, 16)])
 @pytest.mark.parametrize("p_max", [255, 127])
 def test_attention_matches_oracle(B, L, heads, p_max):
     H = heads * 64

@@ -180,6 +180,14 @@ int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const
    a tuning and testing switch.  Returns IBERT_ERR_ARG for another mode. */
 int ibert_set_fusion(ibert_ctx* ctx, int mode);
 
+/* How the linear layers (ibert_linear_i8, ibert_linear_gelu_i8, ibert_linear_hgelu_i8 and the GEMMs
+   inside ibert_encoder_layer that are not taken by the cluster kernel above) treat problems with
+   fewer 128 x 128 output tiles than SMs: mode 0 (default) splits K over a cluster of 2 or 4 CTAs
+   per tile when that engages more SMs, 1 never splits, 2 and 4 force that width whenever K > 128.
+   INT32 accumulation is exact, so the results are identical in every mode.  No counterpart in the
+   paper: a tuning and testing switch.  Returns IBERT_ERR_ARG for another mode. */
+int ibert_set_split_k(ibert_ctx* ctx, int mode);
+
 /* The integer-only encoder layer (Fig. 1 right; post-LN order):
    QKV projection -> attention (i-softmax) -> output projection -> +x, i-LayerNorm ->
    FFN1 + i-GELU -> FFN2 -> +h1, i-LayerNorm.  x, out: int8 [B*L, H]; x at desc.S_x,

@@ -62,6 +62,7 @@ def lib():
         L.ibert_gelu_lut_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
         L.ibert_linear_hgelu_i8.argtypes = [vp, vp, dbl, vp, vp, vp, i64, i32, i32, dbl, dbl, vp, vp]
         L.ibert_set_fusion.argtypes = [vp, i32]
+        L.ibert_set_split_k.argtypes = [vp, i32]
         L.ibert_softmax_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
         L.ibert_softmax_lut_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
         L.ibert_gelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
@@ -91,7 +92,7 @@ def lib():
                      "ibert_encoder_layer", "ibert_attention_masked_i8", "ibert_encoder_layer_masked",
                      "ibert_embedding_i8", "ibert_classifier_i8", "ibert_encoder_graph_create",
                      "ibert_encoder_graph_launch", "ibert_encoder_graph_destroy", "ibert_hgelu_i",
-                     "ibert_linear_hgelu_i8", "ibert_set_fusion", "ibert_gelu_lut_i", "ibert_softmax_lut_i"):
+                     "ibert_linear_hgelu_i8", "ibert_set_fusion", "ibert_gelu_lut_i", "ibert_softmax_lut_i", "ibert_set_split_k"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -164,6 +165,10 @@ class Context:
     def ibert_set_fusion(self, mode: int):
         """0: linear + LayerNorm fusion by problem size (default), 1: whenever supported, 2: never."""
         _chk(lib().ibert_set_fusion(self.h, mode), "ibert_set_fusion")
+
+    def ibert_set_split_k(self, mode: int) -> None:
+        """0: split K of small GEMMs by size (default); 1: never; 2 / 4: force that cluster width."""
+        _chk(lib().ibert_set_split_k(self.h, mode), "ibert_set_split_k")
 
     def check(self):
         _chk(self.ibert_last_status(), "ibert_last_status")

@@ -9,7 +9,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libibert_b200.so"
-SOURCES = ["api.cu", "host_consts.cpp", "rowops.cu", "gemm_i8.cu", "gemm_ln_i8.cu", "attention_i8.cu", "no_alloc.cu"]
+SOURCES = ["api.cu", "host_consts.cpp", "rowops.cu", "gemm_i8.cu", "gemm_splitk_i8.cu", "gemm_ln_i8.cu", "attention_i8.cu", "no_alloc.cu"]
 
 
 def _sources():

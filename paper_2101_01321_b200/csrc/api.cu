@@ -170,6 +170,12 @@ int ibert_set_fusion(ibert_ctx* ctx, int mode) {
   return IBERT_OK;
 }
 
+int ibert_set_split_k(ibert_ctx* ctx, int mode) {
+  if (!ctx || (mode != 0 && mode != 1 && mode != 2 && mode != 4)) return IBERT_ERR_ARG;
+  ctx->splitk_mode = mode;
+  return IBERT_OK;
+}
+
 int ibert_last_status(ibert_ctx* ctx) {
   if (!ctx) return IBERT_ERR_ARG;
   DeviceGuard guard(ctx->device);

@@ -382,6 +382,14 @@ int launch_shape(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, c
 int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, int N, int K,
                    const GemmEpilogue& epi, void* out) {
   if (M == 0) return IBERT_OK;
+  {
+    // few output tiles (small batches): split K over a cluster instead of leaving most SMs idle
+    int split = ctx->splitk_mode == 1 ? 1 : gemm_splitk_width(ctx, M, N, K);
+    if ((ctx->splitk_mode == 2 || ctx->splitk_mode == 4) && K > 128 &&
+        ((M + 127) / 128) * ((N + 127) / 128) * ctx->splitk_mode <= 65535)
+      split = ctx->splitk_mode;
+    if (split > 1) return launch_gemm_splitk_i8(ctx, x, w, M, N, K, epi, out, split);
+  }
   // tile shape: 256 channels x 256 tokens on a CTA pair when that fills every pair, else one CTA
   // per 128 channels x 256 (or 128) tokens
   const int64_t t256 = (M + 255) / 256;

@@ -104,6 +104,7 @@ struct ibert_ctx {
   // derived constant tables already on the device, keyed by a hash of their host bytes
   std::map<uint64_t, ibert::DeviceTable> tables;
   // look-up tables of ibert_gelu_lut_i, keyed by a hash of the GELU constants
+  int splitk_mode = 0;     // see gemm_splitk_width
   std::map<uint64_t, int8_t*> gelu_luts;
   std::map<uint64_t, uint32_t*> exp_luts;
   // workspace for the encoder layer's intermediates
@@ -159,6 +160,14 @@ bool to_upper_word_form(std::vector<int32_t>* b, const std::vector<int32_t>& c);
 
 int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, int N, int K,
                    const GemmEpilogue& epi, void* out);
+
+// Split-K variant for problems with fewer 128 x 128 output tiles than SMs: a cluster of `split`
+// (2 or 4) CTAs per tile, each over 1/split of K, reduced through distributed shared memory.
+// gemm_splitk_width returns the width worth using (1 = do not split); ctx->splitk_mode overrides
+// it (0 = by size, 1 = never, 2 / 4 = that width whenever the shapes allow).
+int gemm_splitk_width(const ibert_ctx* ctx, int64_t M, int N, int K);
+int launch_gemm_splitk_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, int N, int K,
+                          const GemmEpilogue& epi, void* out, int split);
 
 // Launch with programmatic stream serialization (the kernel must call grid_dep_wait() before its
 // first global-memory access) and an optional cluster width.

@@ -32,13 +32,13 @@ DEFAULT_BATCH = {2: 128, 3: 32, 4: 64}
 
 # DRAM bytes (read + write) per launch from one ncu capture of each kernel class at the default
 # workload (config 2, B=128; cold L2; summaries under profiles/).  Other workloads report null.
-NCU_DRAM_TRAFFIC_BYTES = {(2, 128): {"gemm_qkv": 14.5e6, "attention": 37.8e6, "gemm_out_ln": 25.8e6, "gemm_ffn1_gelu": 17.5e6, "gemm_ffn2_ln": 67.4e6, "gemm_out": 13.9e6, "layernorm": 64.0e6, "gemm_ffn2": 59.5e6}}
+NCU_DRAM_TRAFFIC_BYTES = {(2, 128): {"gemm_qkv": 14.5e6, "attention": 37.8e6, "gemm_out_ln": 25.8e6, "gemm_ffn1_gelu": 17.2e6, "gemm_ffn2_ln": 67.6e6, "gemm_out": 13.9e6, "layernorm": 64.9e6, "gemm_ffn2": 59.8e6}}
 
 
 # Integer-datapath instructions (ALU + IMAD pipes, which behave as one 16-lane unit per SM sub-partition)
 # per output element, from the ncu instruction counters of the same captures: what actually bounds
 # the GEMM epilogues.  Reported beside the tensor roofline of the top kernel class.
-NCU_INT_INSTR_PER_ELEMENT = {(2, 128): {"gemm_ffn1_gelu": 20.4}}
+NCU_INT_INSTR_PER_ELEMENT = {(2, 128): {"gemm_ffn1_gelu": 19.4}}
 
 
 # --------------------------------------------------------------------------- helpers

@@ -20,8 +20,12 @@
  * (I-Sqrt), numpy int64 matmul (linear), float exp / erf-GELU within the
  * paper's error figures (i-exp, i-GELU; Table 1), float softmax and
  * LayerNorm within one output step, fixed-point row-sum bounds.
- * The composed encoder layer is "parity unpinned" beyond composition: its
- * only extra check is a float64 sanity comparison.
+ * The composed encoder layer is pinned twice: tap by tap to the composition
+ * of the separately pinned operators, and to a float64 textbook post-LN
+ * encoder layer on the dequantized parameters, every intermediate tensor
+ * within quantization noise -- with bounds tight enough that a planted wiring
+ * mistake (a dropped residual, K and V swapped, no 1/sqrt(d), heads
+ * interleaved, the two LayerNorms exchanged, ...) breaks them.
  */
 #include <math.h>
 #include <stdint.h>

@@ -140,46 +140,92 @@ def test_encoder_layer_is_the_composition_of_its_pinned_ops():
     assert (res.out == out).all()
 
 
-def _float_layer(p, x, B, L):
-    """float64 post-LN encoder layer on the dequantized parameters (sanity only)."""
+def _float_layer_taps(p, x, B, L, mistake=None):
+    """float64 post-LN encoder layer (Fig. 1 left) on the dequantized parameters, with its intermediate
+    tensors.  `mistake` plants one plausible wiring error, to show that the comparison below notices it."""
     H, heads = p["H"], p["heads"]
     erf = np.vectorize(math.erf)
     W = {n: p[f"w_{n}"].astype(np.float64) * p[f"S_w_{n}"][:, None] for n in ("qkv", "o", "f1", "f2")}
     sx = {"qkv": p["S_x"], "o": p["S_ctx"], "f1": p["S_h1"], "f2": p["S_go"]}
     bf = {n: p[f"bias_{n}"] * sx[n] * p[f"S_w_{n}"] for n in W}
+    if mistake == "no_bias":
+        bf = {n: 0.0 * v for n, v in bf.items()}
     xf = x.astype(np.float64) * p["S_x"]
-    qkv = (xf @ W["qkv"].T + bf["qkv"]).reshape(B, L, 3, heads, 64)
+    qkv2 = xf @ W["qkv"].T + bf["qkv"]
+    qkv = qkv2.reshape(B, L, 3, heads, 64)
+    iq, ik, iv = (0, 2, 1) if mistake == "k_and_v_swapped" else (0, 1, 2)
     ctx = np.empty((B, L, heads, 64))
     for b in range(B):
         for h in range(heads):
-            s = qkv[b, :, 0, h] @ qkv[b, :, 1, h].T / 8.0
+            s = qkv[b, :, iq, h] @ qkv[b, :, ik, h].T / (1.0 if mistake == "no_sqrt_d" else 8.0)
             e = np.exp(s - s.max(axis=1, keepdims=True))
-            ctx[b, :, h] = (e / e.sum(axis=1, keepdims=True)) @ qkv[b, :, 2, h]
-    o = ctx.reshape(B * L, H) @ W["o"].T + bf["o"]
+            ctx[b, :, h] = (e / e.sum(axis=1, keepdims=True)) @ qkv[b, :, iv, h]
+    if mistake == "heads_interleaved":
+        ctx = ctx.transpose(0, 1, 3, 2)
+    ctx2 = ctx.reshape(B * L, H)
+    o = ctx2 @ W["o"].T + bf["o"]
 
     def ln(v, g, be):
+        if mistake == "ln_without_variance":
+            return (v - v.mean(1, keepdims=True)) * g + be
         return (v - v.mean(1, keepdims=True)) / v.std(1, keepdims=True) * g + be
-    h1 = ln(xf + o, p["gamma1"], p["beta1"])
+    g1, b1, g2, b2 = p["gamma1"], p["beta1"], p["gamma2"], p["beta2"]
+    if mistake == "layernorms_swapped":
+        g1, b1, g2, b2 = g2, b2, g1, b1
+    h1 = ln((0.0 if mistake == "no_residual_1" else xf) + o, g1, b1)
     z = h1 @ W["f1"].T + bf["f1"]
-    gz = z * 0.5 * (1.0 + erf(z / math.sqrt(2.0)))
-    return ln(h1 + gz @ W["f2"].T + bf["f2"], p["gamma2"], p["beta2"])
+    gz = np.maximum(z, 0.0) if mistake == "relu" else z * 0.5 * (1.0 + erf(z / math.sqrt(2.0)))
+    res2 = {"no_residual_2": 0.0, "residual_2_from_x": xf}.get(mistake, h1)
+    out = ln(res2 + gz @ W["f2"].T + bf["f2"], g2, b2)
+    return {"qkv": qkv2, "ctx": ctx2, "h1": h1, "g": gz, "out": out}
 
 
-def test_encoder_layer_stays_close_to_a_float_layer():
-    # Not a parity pin (the composed layer is unpinned beyond composition): the
-    # integer layer should sit within a few output steps of float arithmetic, and
-    # the static scales of the synthetic recipe should clamp almost nothing.
+# mean / 99th percentile of |integer tap - float tap| in steps of the tap's scale: about twice what
+# the correct wiring shows on this input (0.25/0.49, 1.49/4.91, 0.25/0.54, 0.69/1.58, 0.35/1.03)
+_TAP_BOUNDS = {"qkv": (0.5, 1.0), "ctx": (3.0, 10.0), "h1": (0.5, 1.1), "g": (1.4, 3.2), "out": (0.7, 2.1)}
+
+
+def _tap_errors(p, x, B, L, res, mistake=None):
+    H = p["H"]
+    scales = {"qkv": np.concatenate([np.full(H, p["S_q"]), np.full(H, p["S_k"]), np.full(H, p["S_v"])]),
+              "ctx": p["S_ctx"], "h1": p["S_h1"], "g": p["S_go"], "out": p["S_out"]}
+    ft = _float_layer_taps(p, x, B, L, mistake)
+    errs = {}
+    for name, S in scales.items():
+        got = (res.out if name == "out" else res.taps[name]).astype(np.float64)
+        e = np.abs(got - np.clip(ft[name] / S, -127, 127))
+        errs[name] = (e.mean(), np.percentile(e, 99))
+    return errs
+
+
+def test_encoder_layer_tracks_a_float_layer_tap_by_tap():
+    """The pin of the composed layer against something that is not the oracle: a float64 textbook
+    post-LN encoder layer on the dequantized parameters.  Every intermediate tensor of the integer
+    layer stays within quantization noise of its float counterpart, and the static scales of the
+    synthetic recipe clamp almost nothing."""
     B, L = 2, 32
     x, p = _small_layer(B, L, H=256, heads=4, F=1024)
     res = oracle.encoder_layer(p, x, B, L, want_taps=True)
-    ref = _float_layer(p, x, B, L)
-    err = np.abs(res.out * p["S_out"] - np.clip(ref, -127 * p["S_out"], 127 * p["S_out"])) / p["S_out"]
-    assert err.mean() < 1.5 and np.percentile(err, 99) < 6.0
+    for name, (mean, p99) in _tap_errors(p, x, B, L, res).items():
+        assert mean < _TAP_BOUNDS[name][0] and p99 < _TAP_BOUNDS[name][1], (name, mean, p99)
     for name, qmax in (("qkv", 127), ("ctx", 127), ("h1", 127), ("g", 127), ("r1", 32767), ("r2", 32767)):
         frac = (np.abs(res.taps[name]) >= qmax).mean()
         assert frac < 0.01, (name, frac)
         if qmax == 127:       # (r1, r2 hold one addend at the scale of the residual *sum*)
             assert np.abs(res.taps[name]).max() > 60, name          # and the range is used
+
+
+@pytest.mark.parametrize("mistake", ["no_sqrt_d", "k_and_v_swapped", "heads_interleaved", "no_residual_1",
+                                     "no_residual_2", "residual_2_from_x", "layernorms_swapped", "relu",
+                                     "ln_without_variance", "no_bias"])
+def test_the_float_comparison_notices_a_wiring_mistake(mistake):
+    """Each plausible mistake, planted in the float layer, pushes at least one tap outside the bounds
+    the correct wiring meets -- so the same mistake inside the oracle would fail the test above."""
+    B, L = 2, 32
+    x, p = _small_layer(B, L, H=256, heads=4, F=1024)
+    res = oracle.encoder_layer(p, x, B, L, want_taps=True)
+    errs = _tap_errors(p, x, B, L, res, mistake)
+    assert any(mean > _TAP_BOUNDS[n][0] or p99 > _TAP_BOUNDS[n][1] for n, (mean, p99) in errs.items()), errs
 
 
 def test_layers_chain_through_their_scales():

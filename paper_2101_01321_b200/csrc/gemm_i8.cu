@@ -285,10 +285,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         uint32_t v[32];
         ptx::tmem_ld32(t_row + col, v);
         ptx::tmem_wait_ld();
-        // the store issued two chunks ago from this staging tile must have finished reading it
-        if (lane == 0) ptx::bulk_wait_read<1>();
-        __syncwarp();
-        uint8_t* stage = stage0 + buf * C::kOutTileBytes;
+        // GELU kinds: the warp's two 1 KB tiles form one 64-token block that leaves with a single
+        // store per output tile (one proxy fence and one TMA issue less; -1.6 us on FFN1).  The
+        // light int8 epilogue keeps two stores: it would catch up with its own previous store
+        // (+2 us on the QKV GEMM).  Otherwise a tile is reused two chunks later.  Either way the
+        // store that last read this staging tile must have finished reading it.
+        constexpr bool kOneStore = !kOut32 && C::kChunksPerWarp == 2 && KIND != EPI_INT8;
+        if (!kOneStore || ci == 0) {
+          if (lane == 0) { if constexpr (kOneStore) ptx::bulk_wait_read<0>(); else ptx::bulk_wait_read<1>(); }
+          __syncwarp();
+        }
+        uint8_t* stage = stage0 + (kOneStore ? ci : (int)buf) * C::kOutTileBytes;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const int32_t a = (int32_t)v[i];
@@ -316,11 +323,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           else  // low byte of the register, stored without a narrowing conversion
             asm volatile("st.shared.u8 [%0], %1;" ::"r"(ptx::smem_addr(stage) + i * 32 + lane), "r"(o) : "memory");
         }
-        ptx::fence_proxy_async_smem();                 // staging writes -> visible to the TMA engine
-        __syncwarp();
-        if (lane == 0) {
-          ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), ch0 * (kOut32 ? 4 : 1), t0 + ci * 32);
-          ptx::bulk_commit();
+        if (!kOneStore || ci == 1) {
+          ptx::fence_proxy_async_smem();               // staging writes -> visible to the TMA engine
+          __syncwarp();
+          if (lane == 0) {
+            if constexpr (kOneStore) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage0), ch0, t0);
+            else ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), ch0 * (kOut32 ? 4 : 1), t0 + ci * 32);
+            ptx::bulk_commit();
+          }
         }
         buf ^= 1;
       }
@@ -417,7 +427,9 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
     const uint64_t row_bytes = (uint64_t)N * (out32 ? 4 : 1);
     const uint64_t dims[2] = {row_bytes, (uint64_t)M};
     const uint64_t str[1] = {row_bytes};
-    const uint32_t box[2] = {out32 ? 128u : 32u, 32};
+    // (the GELU epilogues store a warp's 64 tokens at once)
+    const bool gelu_kind = epi.kind == EPI_GELU || epi.kind == EPI_HGELU;
+    const uint32_t box[2] = {out32 ? 128u : 32u, gelu_kind ? 64u : 32u};
     int rc = encode_tensor_map(&mo, out, 2, dims, str, box, 0);
     if (rc) return rc;
   }

@@ -461,13 +461,16 @@ def run_ours(args):
         e2e_value = tokens / (total_e2e_ms / 1e3)
 
         # CPU baseline: the oracle on a bounded sample of the same workload
-        n_seq = 8
-        tok_s, dt_s, n_layers = oracle_sample_run(args.config, n_seq, full_model=full_model, L=cfg.L)
-        import oracle
-        cpu = {"value": tok_s / dt_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-               "sample": f"first {n_seq} sequences ({tok_s} tokens) through "
-                         f"{'embedding, ' if full_model else ''}all {n_layers} layers"
-                         f"{' and the classifier' if full_model else ''}, {dt_s:.1f} s"}
+        # (single-GPU runs only: with more ranks the others would sit in the teardown meanwhile)
+        cpu = None
+        if world == 1:
+            n_seq = 8
+            tok_s, dt_s, n_layers = oracle_sample_run(args.config, n_seq, full_model=full_model, L=cfg.L)
+            import oracle
+            cpu = {"value": tok_s / dt_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                   "sample": f"first {n_seq} sequences ({tok_s} tokens) through "
+                             f"{'embedding, ' if full_model else ''}all {n_layers} layers"
+                             f"{' and the classifier' if full_model else ''}, {dt_s:.1f} s"}
 
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -62,15 +62,22 @@ inline int gemm_class(int kind, int K) {
 
 namespace ibert {
 
+// Bounds the cache of constant tables: once it holds more than 4096 entries, everything is dropped
+// after the stream has gone idle.  Called at the START of an entry point, before it looks anything
+// up -- a call holds the pointers it got from the cache until its kernels are enqueued, so the
+// cache must never shrink in the middle of one.
+int trim_tables(ibert_ctx* ctx) {
+  if (ctx->tables.size() <= 4096) return IBERT_OK;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+  for (auto& kv : ctx->tables) cudaFree(kv.second.ptr);
+  ctx->tables.clear();
+  return IBERT_OK;
+}
+
 int cached_upload(ibert_ctx* ctx, const void* host, size_t bytes, uint64_t tag, void** dev) {
   const uint64_t key = fnv1a(host, bytes, tag * 0x9e3779b97f4a7c15ull + bytes);
   auto it = ctx->tables.find(key);
   if (it != ctx->tables.end() && it->second.bytes == bytes) { *dev = it->second.ptr; return IBERT_OK; }
-  if (ctx->tables.size() > 4096) {        // bound the cache: drop everything once the stream is idle
-    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
-    for (auto& kv : ctx->tables) cudaFree(kv.second.ptr);
-    ctx->tables.clear();
-  }
   void* d = nullptr;
   if (cudaMalloc(&d, bytes ? bytes : 16) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_NOMEM; }
   if (cudaMemcpyAsync(d, host, bytes, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess) {
@@ -306,6 +313,7 @@ int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* 
   int rc = make_ln_tables(gamma, beta, C, S_out, &k, &b_i, &B_i);
   if (rc) return rc;
   DeviceGuard guard(ctx->device);
+  if ((rc = trim_tables(ctx))) return rc;
   void *d_b = nullptr, *d_B = nullptr;
   rc = cached_upload(ctx, b_i.data(), b_i.size() * sizeof(int32_t), 11, &d_b);
   if (rc) return rc;
@@ -337,6 +345,7 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
   epi.kind = kind;
   epi.d_bias = bias;
   DeviceGuard guard(ctx->device);
+  if (int rc = trim_tables(ctx)) return rc;
   if (kind != EPI_RAW) {
     const double S_acc_to = (kind == EPI_GELU || kind == EPI_HGELU) ? S_mid : S_out;
     std::vector<int32_t> b, c;
@@ -419,6 +428,7 @@ int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const
   rc = make_ln_tables(gamma, beta, N, S_out, &k, &b_i, &B_i);
   if (rc) return rc;
   DeviceGuard guard(ctx->device);
+  if ((rc = trim_tables(ctx))) return rc;
   void *d_b = nullptr, *d_c = nullptr, *d_bi = nullptr, *d_Bi = nullptr;
   if ((rc = cached_upload(ctx, b.data(), b.size() * sizeof(int32_t), 21, &d_b))) return rc;
   if ((rc = cached_upload(ctx, c.data(), c.size() * sizeof(int32_t), 22, &d_c))) return rc;
@@ -696,6 +706,7 @@ int ibert_embedding_i8(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, con
   if (S_ret) *S_ret = S_out;
   if (T == 0) return IBERT_OK;
   DeviceGuard guard(ctx->device);
+  if ((rc = trim_tables(ctx))) return rc;
   void *d_b = nullptr, *d_B = nullptr;
   if ((rc = cached_upload(ctx, b_i.data(), b_i.size() * sizeof(int32_t), 11, &d_b))) return rc;
   if ((rc = cached_upload(ctx, B_i.data(), B_i.size() * sizeof(int64_t), 12, &d_B))) return rc;

@@ -122,6 +122,7 @@ namespace ibert {
 
 // uploads `bytes` of host data once per distinct content; returns the device copy
 int cached_upload(ibert_ctx* ctx, const void* host, size_t bytes, uint64_t tag, void** dev);
+int trim_tables(ibert_ctx* ctx);   // bounds the cache; only at the start of an entry point
 
 // ---------------------------------------------------------------------------------------
 // Kernel launchers (each returns an IBERT_* code; all enqueue on ctx->stream)

@@ -116,3 +116,32 @@ def test_linear_error_codes():
         ctx().ibert_linear_i8(x, 1.0, w, np.full(16, 1e30), None, 0, 1e-30)  # multiplier >= 2^31
     assert e.value.code == -3
     assert ctx().ibert_last_status() == 0
+
+
+def test_constant_table_cache_survives_its_own_trimming():
+    """Every distinct scale set leaves constant tables in the context's cache (multipliers and shifts of
+    a linear layer: two per call here), which is dropped once it holds more than 4096 entries.  The
+    drop must not happen while a call still holds pointers into the cache: every result stays right
+    across two such drops, the second met with the other parity of the table count."""
+    M, N, K = 8, 16, 16
+    rng = np.random.default_rng(3)
+    x = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    w = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    bias = rng.integers(-2000, 2000, N).astype(np.int32)
+    base = rng.uniform(1e-3, 1.4e-3, N)
+    xd, wd, bd = dev(x), dev(w), dev(bias)
+
+    def scales(i, eps):
+        # bit j of i doubles channel j's scale: a different shift table for every i;
+        # the factor makes the multiplier table different as well
+        return base * np.array([2.0 if (i >> j) & 1 else 1.0 for j in range(N)]) * (1.0 + eps)
+
+    for i in range(4800):
+        S_w = scales(i, 1e-5 * i)
+        out, _ = ctx().ibert_linear_i8(xd, 0.03, wd, S_w, bd, 0, 0.05)
+        assert_same(host(out), oracle.linear(x, 0.03, w, S_w, bias, 0, 0.05), f"call {i}")
+        if i == 3000:       # same shifts as the call before, new multipliers: one table more, parity flips
+            S_w = scales(i, 0.5)
+            out, _ = ctx().ibert_linear_i8(xd, 0.03, wd, S_w, bd, 0, 0.05)
+            assert_same(host(out), oracle.linear(x, 0.03, w, S_w, bias, 0, 0.05), "odd call")
+    ctx().check()

@@ -1,0 +1,156 @@
+"""Seeded random shapes, scales and modes through the C ABI against the oracle, bit for bit.
+
+The fixed-shape parity tests cover the tiles, tails and degenerate cases chosen by hand; this sweep
+covers the combinations nobody chose: ragged M / N / K with every epilogue and split-K width, attention
+at arbitrary lengths with and without key lengths, score scales on and off the ln2 / 2^k grid, the
+cluster kernel forced on or off, row operators at odd widths.  One context serves all of them in
+random order, so state left behind by one call (cached constant tables, the workspace, the status
+word) meets every other call."""
+import numpy as np
+import pytest
+
+import oracle
+from gpu_util import assert_same, ctx, dev, host
+from paper_2101_01321_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _linear(rng):
+    M = int(rng.choice([1, 7, 100, 128, 129, 300, 1000, 2500]))
+    N = int(rng.choice([16, 48, 128, 272, 768, 1024, 2304, 3072]))
+    K = int(rng.choice([16, 80, 128, 144, 512, 768, 1024, 3072]))
+    if M * N * K > 3e9:
+        return
+    c = ctx()
+    c.ibert_set_split_k(int(rng.choice([0, 0, 1, 2, 4])))
+    x = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    w = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    bias = rng.integers(-200000, 200000, N).astype(np.int32)
+    S_w, S_x = rng.uniform(1e-4, 4e-4, N), 0.03
+    amax = 127.0 * 127.0 * np.sqrt(K) * 1.2 * S_x * 2.5e-4
+    kind = int(rng.integers(0, 5))
+    what = f"linear kind {kind} {M}x{N}x{K}"
+    if kind < 3:
+        S_out = [amax / 100.0, amax / 20000.0, 0.0][kind]
+        out, _ = c.ibert_linear_i8(dev(x), S_x, dev(w), S_w, dev(bias), kind, S_out)
+        assert_same(host(out), oracle.linear(x, S_x, w, S_w, bias, kind, S_out), what)
+    else:
+        S_mid, S_x2 = 6.0 / 32767.0, S_x * (6.0 / amax)
+        S_out = float(rng.choice([6.0 / 127.0, 0.17 / 300.0]))
+        mid = oracle.linear(x, S_x2, w, S_w, bias, 1, S_mid)
+        if kind == 3:
+            out, _ = c.ibert_linear_gelu_i8(dev(x), S_x2, dev(w), S_w, dev(bias), S_mid, S_out)
+            assert_same(host(out), oracle.gelu(mid, S_mid, S_out)[0], what)
+        else:
+            out, _ = c.ibert_linear_hgelu_i8(dev(x), S_x2, dev(w), S_w, dev(bias), S_mid, S_out)
+            assert_same(host(out), oracle.hgelu(mid, S_mid, S_out)[0], what)
+    c.ibert_set_split_k(0)
+
+
+def _attention(rng):
+    B = int(rng.choice([1, 2, 3, 9, 20, 40]))
+    L = int(rng.integers(1, 513))
+    heads = int(rng.choice([1, 2, 4, 12]))
+    if B * heads * L * L > 3e7:
+        return
+    H = heads * 64
+    amp = rng.choice([10, 40, 90])
+    qkv = np.clip(np.rint(rng.standard_normal((B * L, 3 * H)) * amp), -127, 127).astype(np.int8)
+    S_q, S_k = float(rng.choice([0.02, 0.005, 0.08])), 0.02
+    if rng.random() < 0.3:
+        S_q = synth.snap_q_scale(S_q, S_k)
+    lens = rng.integers(0, L + 1, B).astype(np.int32) if rng.random() < 0.5 else None
+    p_max = int(rng.choice([255, 127]))
+    c = ctx()
+    if lens is None:
+        out, _ = c.ibert_attention_i8(dev(qkv), B, L, H, heads, S_q, S_k, 0.02, 0.006, p_max)
+    else:
+        out, _ = c.ibert_attention_masked_i8(dev(qkv), B, L, H, heads, dev(lens), S_q, S_k, 0.02, 0.006, p_max)
+    want = oracle.attention(qkv, B, L, H, heads, S_q, S_k, 0.02, 0.006, p_max, lens=lens)
+    assert_same(host(out), want, f"attention B={B} L={L} heads={heads} S_q={S_q} p_max={p_max} lens={lens}")
+
+
+def _row_ops(rng):
+    c = ctx()
+    which = int(rng.integers(0, 4))
+    sigma = float(rng.choice([1.0, 4.0]))
+    if which == 0:
+        rows, C = int(rng.choice([1, 5, 64, 333, 2000])), int(rng.choice([8, 17, 260, 768, 1024, 2047]))
+        q, S, r, S_r, gamma, beta, S_out = synth.layernorm_inputs(rows, C, sigma)
+        use_r = rng.random() < 0.7
+        out, _ = c.ibert_layernorm_i(dev(q), S, dev(r) if use_r else None, S_r, gamma, beta, S_out)
+        assert_same(host(out), oracle.layernorm(q, S, r if use_r else None, S_r, gamma, beta, S_out)[0], f"layernorm {rows}x{C}")
+    elif which == 1:
+        rows, L = int(rng.choice([1, 9, 100, 700])), int(rng.integers(1, 1025))
+        q, S = synth.softmax_inputs(rows, L, sigma)
+        p_max = int(rng.choice([255, 127]))
+        fn = c.ibert_softmax_lut_i if rng.random() < 0.3 else c.ibert_softmax_i
+        out, _ = fn(dev(q), S, p_max)
+        assert_same(host(out), oracle.softmax(q, S, p_max)[0], f"softmax {rows}x{L}")
+    else:
+        n = int(rng.choice([1, 3, 1000, 4099, 70001]))
+        q, S, S_out = synth.gelu_inputs(n, sigma)
+        pick = rng.random()
+        if which == 3:
+            out, _ = c.ibert_hgelu_i(dev(q), S, S_out)
+            assert_same(host(out), oracle.hgelu(q, S, S_out)[0], f"hgelu {n}")
+        else:
+            fn = c.ibert_gelu_lut_i if pick < 0.3 else c.ibert_gelu_i
+            out, _ = fn(dev(q), S, S_out)
+            assert_same(host(out), oracle.gelu(q, S, S_out)[0], f"gelu {n}")
+
+
+def _linear_layernorm(rng):
+    T = int(rng.choice([1, 100, 128, 257, 1000, 3000]))
+    H = int(rng.choice([256, 512, 768, 1024]))
+    K = int(rng.choice([256, 768, 3072]))
+    c = ctx()
+    c.ibert_set_fusion(int(rng.choice([0, 1, 2])))
+    x = rng.integers(-127, 128, (T, K)).astype(np.int8)
+    w = rng.integers(-127, 128, (H, K)).astype(np.int8)
+    bias = rng.integers(-20000, 20000, H).astype(np.int32)
+    S_w, S_x = rng.uniform(1e-4, 4e-4, H), 0.03
+    res = rng.integers(-127, 128, (T, H)).astype(np.int8)
+    amax = 127.0 * 127.0 * np.sqrt(K) * 1.2 * S_x * 2.5e-4
+    S_mid = amax / 8000.0
+    S_res = S_mid * 100.0
+    gamma, beta, S_out = rng.normal(1, 0.1, H), rng.normal(0, 0.1, H), 4.0 / 127.0
+    out, _ = c.ibert_linear_layernorm_i8(dev(x), S_x, dev(w), S_w, dev(bias), S_mid, dev(res), S_res, gamma, beta, S_out)
+    mid = oracle.linear(x, S_x, w, S_w, bias, 1, S_mid)
+    assert_same(host(out), oracle.layernorm(mid, S_mid, res, S_res, gamma, beta, S_out)[0], f"linear+layernorm T={T} H={H} K={K}")
+    c.ibert_set_fusion(0)
+
+
+def _layer(rng):
+    B = int(rng.choice([1, 2, 5, 17]))
+    L = int(rng.choice([16, 37, 128, 200]))
+    H = 64 * int(rng.choice([2, 4, 8]))
+    heads = H // 64
+    x, params = synth.make_model(0, B, layers=1, H=H, heads=heads, F=4 * H, L=L)
+    c = ctx()
+    c.ibert_set_fusion(int(rng.choice([0, 1])))
+    ly = c.ibert_layer_create(params[0])
+    if rng.random() < 0.5:
+        lens = rng.integers(1, L + 1, B).astype(np.int32)
+        out, _ = c.ibert_encoder_layer_masked(ly, dev(x), B, L, dev(lens))
+        want = oracle.encoder_layer(params[0], x, B, L, lens=lens).out
+    else:
+        out, _ = c.ibert_encoder_layer(ly, dev(x), B, L)
+        want = oracle.encoder_layer(params[0], x, B, L).out
+    assert_same(host(out), want, f"layer B={B} L={L} H={H}")
+    ly.close()
+    c.ibert_set_fusion(0)
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_calls_in_random_order(seed):
+    rng = np.random.default_rng(seed)
+    cases = [_linear, _attention, _row_ops, _linear_layernorm, _layer]
+    try:
+        for _ in range(140):
+            cases[int(rng.choice(5, p=[0.3, 0.3, 0.15, 0.15, 0.1]))](rng)
+        ctx().check()
+    finally:
+        ctx().ibert_set_split_k(0)
+        ctx().ibert_set_fusion(0)

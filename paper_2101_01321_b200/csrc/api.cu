@@ -351,7 +351,16 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
     std::vector<int32_t> b, c;
     int rc = make_linear_tables(S_x, S_w, N, nullptr, S_acc_to, &b, &c);
     if (rc) return rc;
-    epi.fast = to_upper_word_form(&b, c) ? 1 : 0;
+    // The epilogue runs in ONE form: the upper-word form needs the per-channel multipliers AND (for
+    // the GELU kinds) the final multiplier to fit it.  The per-channel table is converted only then --
+    // the generic epilogue reads the plain (b, c) pairs.
+    bool upper_ok = true;
+    if (kind == EPI_GELU || kind == EPI_HGELU) {
+      rc = kind == EPI_HGELU ? make_hgelu_consts(S_mid, S_out, &epi.gelu) : make_gelu_consts(S_mid, S_out, &epi.gelu);
+      if (rc) return rc;
+      upper_ok = epi.gelu.fast != 0;
+    }
+    epi.fast = (upper_ok && to_upper_word_form(&b, c)) ? 1 : 0;
     void *d_b = nullptr, *d_c = nullptr;
     rc = cached_upload(ctx, b.data(), b.size() * sizeof(int32_t), 21, &d_b);
     if (rc) return rc;
@@ -359,10 +368,6 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
     if (rc) return rc;
     epi.d_b = (const int32_t*)d_b;
     epi.d_c = (const int32_t*)d_c;
-    if (kind == EPI_GELU || kind == EPI_HGELU) {
-      rc = kind == EPI_HGELU ? make_hgelu_consts(S_mid, S_out, &epi.gelu) : make_gelu_consts(S_mid, S_out, &epi.gelu);
-      if (rc) return rc;
-    }
   }
   int rc;
   {
@@ -554,13 +559,15 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   ly->d = *d;
   int rc = IBERT_OK;
   auto up = [&](const void* h, size_t bytes, void** dev) { if (rc == IBERT_OK) rc = upload_owned(ly, h, bytes, dev); };
+  // `upper_ok`: whether the rest of that GEMM's epilogue can run in the upper-word form; the table
+  // is converted to it only then (the generic epilogue reads the plain (b, c) pairs)
   auto lin = [&](double S_in, const double* S_w, int N, const double* so_cols, double so, int32_t** db, int32_t** dc,
-                 int* fast) {
+                 int* fast, bool upper_ok = true) {
     if (rc != IBERT_OK) return;
     std::vector<int32_t> b, c;
     rc = make_linear_tables(S_in, S_w, N, so_cols, so, &b, &c);
     if (rc != IBERT_OK) return;
-    *fast = to_upper_word_form(&b, c) ? 1 : 0;
+    *fast = (upper_ok && to_upper_word_form(&b, c)) ? 1 : 0;
     up(b.data(), b.size() * sizeof(int32_t), (void**)db);
     up(c.data(), c.size() * sizeof(int32_t), (void**)dc);
   };
@@ -578,7 +585,8 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
     lin(d->S_x, d->S_w_qkv, 3 * H, so.data(), 0.0, &ly->b_qkv, &ly->c_qkv, &ly->fast_qkv);
   }
   lin(d->S_ctx, d->S_w_o, H, nullptr, d->S_r1, &ly->b_o, &ly->c_o, &ly->fast_o);
-  lin(d->S_h1, d->S_w_f1, F, nullptr, d->S_gi, &ly->b_f1, &ly->c_f1, &ly->fast_f1);
+  if (rc == IBERT_OK) rc = make_gelu_consts(d->S_gi, d->S_go, &ly->gelu);
+  lin(d->S_h1, d->S_w_f1, F, nullptr, d->S_gi, &ly->b_f1, &ly->c_f1, &ly->fast_f1, ly->gelu.fast != 0);
   lin(d->S_go, d->S_w_f2, H, nullptr, d->S_r2, &ly->b_f2, &ly->c_f2, &ly->fast_f2);
   auto ln = [&](const double* g, const double* be, double S_sum, double S_res, double S_o, LnConsts* k,
                 int32_t** db, int64_t** dB) {
@@ -595,7 +603,6 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   };
   ln(d->gamma1, d->beta1, d->S_r1, d->S_x, d->S_h1, &ly->ln1, &ly->ln1_b, &ly->ln1_B);
   ln(d->gamma2, d->beta2, d->S_r2, d->S_h1, d->S_out, &ly->ln2, &ly->ln2_b, &ly->ln2_B);
-  if (rc == IBERT_OK) rc = make_gelu_consts(d->S_gi, d->S_go, &ly->gelu);
   if (rc == IBERT_OK) rc = make_attn_consts(d->S_q, d->S_k, d->S_v, d->S_ctx, d->p_max, &ly->attn);
   if (rc != IBERT_OK) { ibert_layer_destroy(ly); return rc; }
   // host arrays were pageable: make sure the copies have left them before returning

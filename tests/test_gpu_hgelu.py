@@ -65,3 +65,43 @@ def test_gelu_by_table_lookup_equals_the_integer_kernel(sigma):
     a2, _ = ctx().ibert_gelu_lut_i(dev(q), S, S_out)          # second call: cached table
     ctx().check()
     assert_same(host(a2), host(b), "cached table")
+
+
+@pytest.mark.parametrize("split", [1, 4])
+@pytest.mark.parametrize("S_mid,S_out", [(1.4e-3, 2.7e-4), (2.7e-3, 8e-4), (1.6e-3, 1e-4), (3e-4, 2e-5)])
+def test_fused_gelu_kinds_with_a_final_multiplier_above_one_half(S_mid, S_out, split):
+    """An output scale so fine that the final multiplier of the GELU epilogue does not fit the upper-word
+    form while the per-channel ones do: the whole epilogue must then run in the generic form, on the
+    plain (b, c) pairs.  (Found by a sweep over random scales: the per-channel table used to be
+    converted regardless.)"""
+    rng = np.random.default_rng(7)
+    M, N, K = 130, 272, 144
+    x = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    w = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    bias = rng.integers(-2000, 2000, N).astype(np.int32)
+    S_w, S_x = rng.uniform(1e-4, 4e-4, N), 0.02
+    c = ctx()
+    c.ibert_set_split_k(split)
+    try:
+        mid = oracle.linear(x, S_x, w, S_w, bias, 1, S_mid)
+        out, _ = c.ibert_linear_hgelu_i8(dev(x), S_x, dev(w), S_w, dev(bias), S_mid, S_out)
+        assert_same(host(out), oracle.hgelu(mid, S_mid, S_out)[0], "linear + h-GELU")
+        out, _ = c.ibert_linear_gelu_i8(dev(x), S_x, dev(w), S_w, dev(bias), S_mid, S_out)
+        assert_same(host(out), oracle.gelu(mid, S_mid, S_out)[0], "linear + i-GELU")
+        c.check()
+    finally:
+        c.ibert_set_split_k(0)
+
+
+def test_encoder_layer_with_a_fine_gelu_output_scale():
+    """The same situation inside ibert_encoder_layer: S_go small enough that FFN1's final multiplier
+    leaves the upper-word form (most outputs clamp; the bits still have to be the oracle's)."""
+    B, L = 2, 64
+    x, params = synth.make_model(0, B, layers=1, H=256, heads=4, F=1024, L=L)
+    p = dict(params[0])
+    p["S_go"] = p["S_go"] / 400.0
+    layer = ctx().ibert_layer_create(p)
+    out, _ = ctx().ibert_encoder_layer(layer, dev(x), B, L)
+    ctx().check()
+    assert_same(host(out), oracle.encoder_layer(p, x, B, L).out, "layer with a fine S_go")
+    layer.close()

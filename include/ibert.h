@@ -91,7 +91,8 @@ int ibert_softmax_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, in
 /* i-softmax with i-exp by table look-up -- the alternative the paper argues against (Sec. 2,
    Sec. 3.5), here only for a measured comparison.  The table holds the i-exp of every pre-shifted
    distance from the row maximum, 0 .. 31*q_ln2 (up to 2 MiB of uint32), filled on first use for a
-   scale by the same device function ibert_softmax_i evaluates, and cached in the context (freed by
+   scale by the same device function ibert_softmax_i evaluates, and cached in the context (at most 64
+   tables, dropped together after a stream synchronization when a 65th is needed; freed by
    ibert_destroy).  Results are identical to ibert_softmax_i; arguments and errors as there, plus
    IBERT_ERR_NOMEM when the table cannot be allocated. */
 int ibert_softmax_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
@@ -255,7 +256,8 @@ int ibert_linear_hgelu_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int
    first use by running the i-GELU kernel over every Q16 input (so its contents are Algorithm 2's
    results bit for bit) and cached in the context; afterwards each element costs one clamp and one
    load.  Results are identical to ibert_gelu_i.  Arguments and errors as ibert_gelu_i; the first
-   call for a scale pair allocates 64 KiB of device memory (freed by ibert_destroy). */
+   call for a scale pair allocates 64 KiB of device memory (the context keeps at most 64 tables and
+   drops them all, after synchronizing its stream, when a 65th is needed; ibert_destroy frees them). */
 int ibert_gelu_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
                      double* S_ret);
 

@@ -227,6 +227,11 @@ int ibert_gelu_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, doub
   DeviceGuard guard(ctx->device);
   const uint64_t key = fnv1a(&k, sizeof(k), 0x6c7574ull);
   int8_t* table = nullptr;
+  if (ctx->gelu_luts.size() >= 64) {                 // bounded: drop every table once the stream is idle
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+    for (auto& kv : ctx->gelu_luts) cudaFree(kv.second);
+    ctx->gelu_luts.clear();
+  }
   auto it = ctx->gelu_luts.find(key);
   if (it != ctx->gelu_luts.end()) table = it->second;
   else {
@@ -263,6 +268,11 @@ static int softmax_common(ibert_ctx* ctx, const int32_t* q, double S, int64_t ro
   uint32_t* table = nullptr;
   if (by_table) {
     const uint64_t key = fnv1a(&k, sizeof(k), 0x657870ull);
+    if (ctx->exp_luts.size() >= 64) {                // bounded: drop every table once the stream is idle
+      if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+      for (auto& kv : ctx->exp_luts) cudaFree(kv.second);
+      ctx->exp_luts.clear();
+    }
     auto it = ctx->exp_luts.find(key);
     if (it != ctx->exp_luts.end()) table = it->second;
     else {

@@ -105,3 +105,16 @@ def test_encoder_layer_with_a_fine_gelu_output_scale():
     ctx().check()
     assert_same(host(out), oracle.encoder_layer(p, x, B, L).out, "layer with a fine S_go")
     layer.close()
+
+
+def test_table_caches_are_bounded_and_stay_correct_past_the_bound():
+    """More distinct scale pairs than the 64 tables a context keeps, for both table look-up operators."""
+    q, S, S_out = synth.gelu_inputs(5000, 1.0)
+    sq, sS = synth.softmax_inputs(40, 96, 1.0)
+    for i in range(80):
+        f = 1.0 + 0.01 * i
+        a, _ = ctx().ibert_gelu_lut_i(dev(q), S * f, S_out * f)
+        assert_same(host(a), oracle.gelu(q, S * f, S_out * f)[0], f"gelu by table, scale pair {i}")
+        p, _ = ctx().ibert_softmax_lut_i(dev(sq), sS * f, 255)
+        assert_same(host(p), oracle.softmax(sq, sS * f, 255)[0], f"softmax by table, scale {i}")
+    ctx().check()

@@ -15,10 +15,12 @@
  *   - Work is enqueued on the stream given to ibert_create(); calls return
  *     without synchronizing (ibert_last_status() synchronizes).
  *   - Every function returns IBERT_OK (0) or a negative IBERT_ERR_* code;
- *     nothing throws, aborts, or falls back to a CPU path.  Invalid
+ *     nothing throws (a failed host allocation is IBERT_ERR_NOMEM), aborts,
+ *     or falls back to a CPU path.  Invalid
  *     arguments are rejected on the host before anything is launched.
- *   - Device-side waits are bounded; if one expires the kernel records
- *     IBERT_ERR_TIMEOUT in the context's status word and returns normally.
+ *   - Device-side waits are bounded (one second on the GPU's timer); if one
+ *     expires the kernel records IBERT_ERR_TIMEOUT in the context's status
+ *     word and returns normally.
  *   - Value formats: "int8" = [-127,127] in int8_t; "Q16" = [-32767,32767]
  *     in an int32_t container; "u8" = [0,255] in uint8_t.
  *   - Requantization (Appendix C.1, dyadic form b / 2^c):
@@ -126,11 +128,15 @@ int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* 
    device share the one array, so two calls whose GPU work may overlap (different streams without
    ordering) race on it -- serialize them; the first call on each device looks up the array's
    device address, so make that first call outside any stream capture.
-   Arguments and results are exactly those of ibert_layernorm_i. */
+   Arguments and results are exactly those of ibert_layernorm_i.  A bounded wait that runs out
+   inside the kernel is recorded in a status word inside the same array;
+   ibert_layernorm_i_static_status synchronizes `cuda_stream`, returns that word for the current
+   device (IBERT_OK or IBERT_ERR_TIMEOUT) and clears it; it allocates nothing either. */
 #define IBERT_STATIC_LN_MAX_C 2047
 int ibert_layernorm_i_static(void* cuda_stream, const int32_t* q, double S, const int8_t* r, double S_r,
                              const double* gamma, const double* beta, int64_t rows, int C, double S_out,
                              int8_t* out, double* S_ret);
+int ibert_layernorm_i_static_status(void* cuda_stream);
 
 /* Multi-head self-attention on int8 Q|K|V (Fig. 1 right: MatMul -> i-softmax -> MatMul):
    per (batch, head): s = Q K^T (int32, scale S_q*S_k/8, head size 64), p = i-softmax(s) in u8
@@ -301,6 +307,14 @@ enum {
    z = floor(d / q_ln2) equals the division.  Returns IBERT_OK, the error of the
    derivation, or IBERT_ERR_VALUE_RANGE on a mismatch.  q_ln2_out (may be NULL) receives q_ln2. */
 int ibert_selftest_exp_division(double S, int32_t* q_ln2_out);
+
+/* Self-test of the bounded device-side waits (no counterpart in the paper): enqueues a one-warp
+   kernel that waits on a barrier nobody arrives on, with a limit of limit_us microseconds
+   (1 .. 100000) on the GPU's nanosecond timer.  When the limit runs out the kernel records
+   IBERT_ERR_TIMEOUT in the context's status word -- exactly what every kernel of the library does
+   when one of its waits (limit: one second) expires -- and returns normally; the context stays
+   usable.  ibert_last_status() then returns IBERT_ERR_TIMEOUT once. */
+int ibert_selftest_wait_timeout(ibert_ctx* ctx, int64_t limit_us);
 
 int ibert_profile_begin(ibert_ctx* ctx);
 int ibert_profile_end(ibert_ctx* ctx, float* ms, int32_t* launches);

@@ -80,6 +80,10 @@ def lib():
         L.ibert_encoder_layer.argtypes = [vp, vp, vp, i32, i32, vp, vp]
         L.ibert_layernorm_i_static.argtypes = [vp, vp, dbl, vp, dbl, vp, vp, i64, i32, dbl, vp, vp]
         L.ibert_layernorm_i_static.restype = i32
+        L.ibert_layernorm_i_static_status.argtypes = [vp]
+        L.ibert_layernorm_i_static_status.restype = i32
+        L.ibert_selftest_wait_timeout.argtypes = [vp, i64]
+        L.ibert_selftest_wait_timeout.restype = i32
         L.ibert_selftest_exp_division.argtypes = [dbl, C.POINTER(C.c_int32)]
         L.ibert_selftest_exp_division.restype = i32
         L.ibert_profile_begin.argtypes = [vp]
@@ -137,6 +141,12 @@ def ibert_layernorm_i_static(q: torch.Tensor, S: float, r: torch.Tensor | None, 
     return out, S_ret.value
 
 
+def ibert_layernorm_i_static_status(stream: torch.cuda.Stream | None = None) -> int:
+    """Synchronizes `stream` and returns (then clears) the device-side status of the
+    allocation-free LayerNorm calls on the current device."""
+    return int(lib().ibert_layernorm_i_static_status(None if stream is None else stream.cuda_stream))
+
+
 class Context:
     """``ibert_ctx``: a device and the stream every call is enqueued on."""
 
@@ -172,6 +182,10 @@ class Context:
 
     def check(self):
         _chk(self.ibert_last_status(), "ibert_last_status")
+
+    def ibert_selftest_wait_timeout(self, limit_us: int) -> None:
+        """Enqueues the one-warp kernel whose bounded wait runs out after `limit_us` microseconds."""
+        _chk(lib().ibert_selftest_wait_timeout(self.h, limit_us), "ibert_selftest_wait_timeout")
 
     def ibert_profile_begin(self):
         _chk(lib().ibert_profile_begin(self.h), "ibert_profile_begin")

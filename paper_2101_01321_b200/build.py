@@ -41,15 +41,27 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC,-ffp-contract=off",
-           "--fmad=false", "-cudart", "static", "-o", str(tmp)]
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+             "-Xcompiler", "-fPIC,-ffp-contract=off", "--fmad=false"]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += [str(s) for s in _sources()]
-    subprocess.check_call(cmd)
+        flags += ["-Xptxas", "-v"]
+    # one nvcc per translation unit, side by side, then one link
+    obj_dir = PKG / "build" / f"obj{os.getpid()}"
+    obj_dir.mkdir(parents=True, exist_ok=True)
+    jobs = []
+    for src in _sources():
+        obj = obj_dir / (src.stem + ".o")
+        jobs.append((obj, subprocess.Popen([nvcc, *flags, "-c", "-o", str(obj), str(src)])))
+    failed = [str(o) for o, p in jobs if p.wait() != 0]
+    if failed:
+        raise subprocess.CalledProcessError(1, f"nvcc -c ({', '.join(failed)})")
+    tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "static",
+                           "-o", str(tmp), *[str(o) for o, _ in jobs]])
     os.replace(tmp, LIB)
+    for o, _ in jobs:
+        o.unlink()
+    obj_dir.rmdir()
     HASH_FILE.write_text(_source_hash() + "\n")
     return LIB
 

@@ -52,6 +52,19 @@ struct ProfileScope {
   }
 };
 
+// No exception leaves the C ABI: a failed host allocation becomes IBERT_ERR_NOMEM, anything else
+// IBERT_ERR_ARG (nothing in the library throws on purpose).
+template <typename F>
+inline int guarded(F&& body) noexcept {
+  try {
+    return body();
+  } catch (const std::bad_alloc&) {
+    return IBERT_ERR_NOMEM;
+  } catch (...) {
+    return IBERT_ERR_ARG;
+  }
+}
+
 inline int gemm_class(int kind, int K) {
   if (kind == EPI_INT8) return IBERT_K_GEMM_QKV;
   if (kind == EPI_GELU || kind == EPI_HGELU) return IBERT_K_GEMM_GELU;
@@ -77,14 +90,28 @@ int trim_tables(ibert_ctx* ctx) {
 int cached_upload(ibert_ctx* ctx, const void* host, size_t bytes, uint64_t tag, void** dev) {
   const uint64_t key = fnv1a(host, bytes, tag * 0x9e3779b97f4a7c15ull + bytes);
   auto it = ctx->tables.find(key);
-  if (it != ctx->tables.end() && it->second.bytes == bytes) { *dev = it->second.ptr; return IBERT_OK; }
+  if (it != ctx->tables.end()) {
+    // the hash only finds the candidate; the bytes decide
+    if (it->second.bytes == bytes && (bytes == 0 || std::memcmp(it->second.host.data(), host, bytes) == 0)) {
+      *dev = it->second.ptr;
+      return IBERT_OK;
+    }
+    // two different tables with one hash: the newer one replaces the older once the stream is idle
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+    cudaFree(it->second.ptr);
+    ctx->tables.erase(it);
+  }
   void* d = nullptr;
   if (cudaMalloc(&d, bytes ? bytes : 16) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_NOMEM; }
   if (cudaMemcpyAsync(d, host, bytes, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess) {
     cudaFree(d);
     return IBERT_ERR_CUDA;
   }
-  ctx->tables[key] = DeviceTable{d, bytes};
+  DeviceTable t;
+  t.ptr = d;
+  t.bytes = bytes;
+  t.host.assign(static_cast<const unsigned char*>(host), static_cast<const unsigned char*>(host) + bytes);
+  ctx->tables[key] = std::move(t);
   *dev = d;
   return IBERT_OK;
 }
@@ -125,11 +152,14 @@ const char* ibert_strerror(int code) {
 }
 
 int ibert_dyadic_from_double(double m, int32_t* b, int32_t* c) {
+  return guarded([&]() -> int {
   if (!b || !c) return IBERT_ERR_ARG;
   return dyadic(m, b, c);
+  });
 }
 
 int ibert_create(ibert_ctx** out, int device, void* cuda_stream) {
+  return guarded([&]() -> int {
   if (!out) return IBERT_ERR_ARG;
   *out = nullptr;
   int count = 0;
@@ -155,9 +185,11 @@ int ibert_create(ibert_ctx** out, int device, void* cuda_stream) {
   }
   *out = ctx;
   return IBERT_OK;
+  });
 }
 
 int ibert_destroy(ibert_ctx* ctx) {
+  return guarded([&]() -> int {
   if (!ctx) return IBERT_ERR_ARG;
   DeviceGuard guard(ctx->device);
   cudaStreamSynchronize(ctx->stream);
@@ -169,21 +201,27 @@ int ibert_destroy(ibert_ctx* ctx) {
   cudaFree(ctx->d_status);
   delete ctx;
   return IBERT_OK;
+  });
 }
 
 int ibert_set_fusion(ibert_ctx* ctx, int mode) {
+  return guarded([&]() -> int {
   if (!ctx || mode < 0 || mode > 2) return IBERT_ERR_ARG;
   ctx->fusion_mode = mode;
   return IBERT_OK;
+  });
 }
 
 int ibert_set_split_k(ibert_ctx* ctx, int mode) {
+  return guarded([&]() -> int {
   if (!ctx || (mode != 0 && mode != 1 && mode != 2 && mode != 4)) return IBERT_ERR_ARG;
   ctx->splitk_mode = mode;
   return IBERT_OK;
+  });
 }
 
 int ibert_last_status(ibert_ctx* ctx) {
+  return guarded([&]() -> int {
   if (!ctx) return IBERT_ERR_ARG;
   DeviceGuard guard(ctx->device);
   int32_t st = 0;
@@ -192,6 +230,7 @@ int ibert_last_status(ibert_ctx* ctx) {
   if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
   if (st != 0) cudaMemsetAsync(ctx->d_status, 0, sizeof(st), ctx->stream);
   return st;
+  });
 }
 
 static int gelu_common(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
@@ -212,13 +251,16 @@ static int gelu_common(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, do
 
 int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
                  double* S_ret) {
+  return guarded([&]() -> int {
   return gelu_common(ctx, q, S, n, S_out, out, S_ret, false);
+  });
 }
 
 static int ensure_workspace(ibert_ctx* ctx, size_t need);
 
 int ibert_gelu_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
                      double* S_ret) {
+  return guarded([&]() -> int {
   if (!ctx || n < 0 || (n > 0 && (!q || !out))) return IBERT_ERR_ARG;
   if (!aligned16(q) || !aligned16(out)) return IBERT_ERR_ALIGN;
   GeluConsts k{};                                   // zeroed: the bytes are hashed below
@@ -247,11 +289,14 @@ int ibert_gelu_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, doub
   }
   if (rc == IBERT_OK && S_ret) *S_ret = S_out;
   return rc;
+  });
 }
 
 int ibert_hgelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
                   double* S_ret) {
+  return guarded([&]() -> int {
   return gelu_common(ctx, q, S, n, S_out, out, S_ret, true);
+  });
 }
 
 static int softmax_common(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
@@ -295,17 +340,22 @@ static int softmax_common(ibert_ctx* ctx, const int32_t* q, double S, int64_t ro
 
 int ibert_softmax_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
                     uint8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   return softmax_common(ctx, q, S, rows, L, p_max, out, S_ret, false);
+  });
 }
 
 int ibert_softmax_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows, int L, int p_max,
                         uint8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   return softmax_common(ctx, q, S, rows, L, p_max, out, S_ret, true);
+  });
 }
 
 int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* r, double S_r,
                       const double* gamma, const double* beta, int64_t rows, int C, double S_out,
                       int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   if (!ctx || rows < 0 || !gamma || !beta) return IBERT_ERR_ARG;
   if (C < 1 || C > 2047) return IBERT_ERR_SHAPE;
   if (rows > 0 && (!q || !out)) return IBERT_ERR_ARG;
@@ -335,6 +385,7 @@ int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* 
   }
   if (rc == IBERT_OK && S_ret) *S_ret = S_out;
   return rc;
+  });
 }
 
 static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
@@ -345,6 +396,7 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
   if (N < 1 || K < 1 || K % 16 != 0 || N % 4 != 0) return IBERT_ERR_SHAPE;
   if ((kind == EPI_INT8 || kind == EPI_GELU || kind == EPI_HGELU) && N % 16 != 0) return IBERT_ERR_SHAPE;
   if ((int64_t)K * 127 * 127 >= (int64_t(1) << 31)) return IBERT_ERR_SHAPE;
+  if (M >= (int64_t(1) << 31) - 256) return IBERT_ERR_SHAPE;      // tile coordinates are 32-bit
   if (M > 0 && (!x || !out)) return IBERT_ERR_ARG;
   if (!w) return IBERT_ERR_ARG;
   if (!aligned16(x) || !aligned16(w) || !aligned16(out) || (bias && !aligned16(bias))) return IBERT_ERR_ALIGN;
@@ -417,9 +469,11 @@ int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const
                               const int32_t* bias, int64_t M, int N, int K, double S_mid,
                               const int8_t* res, double S_res, const double* gamma, const double* beta,
                               double S_out, int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   if (!ctx || M < 0 || !S_w || !gamma || !beta || !w) return IBERT_ERR_ARG;
   if (N < 1 || N > 2047 || K < 1 || K % 16 != 0 || N % 16 != 0) return IBERT_ERR_SHAPE;
   if ((int64_t)K * 127 * 127 >= (int64_t(1) << 31)) return IBERT_ERR_SHAPE;
+  if (M >= (int64_t(1) << 31) - 256) return IBERT_ERR_SHAPE;      // tile coordinates are 32-bit
   if (M > 0 && (!x || !out || !res)) return IBERT_ERR_ARG;
   if (!aligned16(x) || !aligned16(w) || !aligned16(out) || !aligned16(res) || (bias && !aligned16(bias)))
     return IBERT_ERR_ALIGN;
@@ -464,25 +518,32 @@ int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const
   }
   if (rc == IBERT_OK && S_ret) *S_ret = S_out;
   return rc;
+  });
 }
 
 int ibert_linear_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
                     const int32_t* bias, int64_t M, int N, int K, int out_kind, double S_out,
                     void* out, double* S_ret) {
+  return guarded([&]() -> int {
   if (out_kind < 0 || out_kind > 2) return IBERT_ERR_ARG;
   return linear_common(ctx, x, S_x, w, S_w, bias, M, N, K, out_kind, 0.0, S_out, out, S_ret);
+  });
 }
 
 int ibert_linear_gelu_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
                          const int32_t* bias, int64_t M, int N, int K, double S_mid, double S_out,
                          int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   return linear_common(ctx, x, S_x, w, S_w, bias, M, N, K, EPI_GELU, S_mid, S_out, out, S_ret);
+  });
 }
 
 int ibert_linear_hgelu_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
                           const int32_t* bias, int64_t M, int N, int K, double S_mid, double S_out,
                           int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   return linear_common(ctx, x, S_x, w, S_w, bias, M, N, K, EPI_HGELU, S_mid, S_out, out, S_ret);
+  });
 }
 
 static int make_attn_consts(double S_q, double S_k, double S_v, double S_ctx, int p_max, AttnConsts* k) {
@@ -519,14 +580,18 @@ static int attention_common(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int
 
 int ibert_attention_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads, double S_q,
                        double S_k, double S_v, double S_ctx, int p_max, int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   return attention_common(ctx, qkv, B, L, H, heads, nullptr, S_q, S_k, S_v, S_ctx, p_max, out, S_ret);
+  });
 }
 
 int ibert_attention_masked_i8(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
                               const int32_t* lens, double S_q, double S_k, double S_v, double S_ctx, int p_max,
                               int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   if (B > 0 && !lens) return IBERT_ERR_ARG;
   return attention_common(ctx, qkv, B, L, H, heads, lens, S_q, S_k, S_v, S_ctx, p_max, out, S_ret);
+  });
 }
 
 // --------------------------------------------------------------------------- encoder layer
@@ -541,15 +606,18 @@ static int upload_owned(ibert_layer* ly, const void* host, size_t bytes, void** 
 }
 
 int ibert_layer_destroy(ibert_layer* ly) {
+  return guarded([&]() -> int {
   if (!ly) return IBERT_ERR_ARG;
   DeviceGuard guard(ly->ctx->device);
   cudaStreamSynchronize(ly->ctx->stream);
   for (void* p : ly->owned) cudaFree(p);
   delete ly;
   return IBERT_OK;
+  });
 }
 
 int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** out) {
+  return guarded([&]() -> int {
   if (!ctx || !d || !out) return IBERT_ERR_ARG;
   *out = nullptr;
   const int H = d->H, F = d->F;
@@ -566,6 +634,11 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   ibert_layer* ly = new (std::nothrow) ibert_layer();
   if (!ly) return IBERT_ERR_NOMEM;
   ly->ctx = ctx;
+  // frees the half-built layer on every early exit, an exception included
+  struct Holder {
+    ibert_layer* p;
+    ~Holder() { if (p) ibert_layer_destroy(p); }
+  } holder{ly};
   ly->d = *d;
   int rc = IBERT_OK;
   auto up = [&](const void* h, size_t bytes, void** dev) { if (rc == IBERT_OK) rc = upload_owned(ly, h, bytes, dev); };
@@ -614,13 +687,15 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   ln(d->gamma1, d->beta1, d->S_r1, d->S_x, d->S_h1, &ly->ln1, &ly->ln1_b, &ly->ln1_B);
   ln(d->gamma2, d->beta2, d->S_r2, d->S_h1, d->S_out, &ly->ln2, &ly->ln2_b, &ly->ln2_B);
   if (rc == IBERT_OK) rc = make_attn_consts(d->S_q, d->S_k, d->S_v, d->S_ctx, d->p_max, &ly->attn);
-  if (rc != IBERT_OK) { ibert_layer_destroy(ly); return rc; }
+  if (rc != IBERT_OK) return rc;
   // host arrays were pageable: make sure the copies have left them before returning
-  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) { ibert_layer_destroy(ly); return IBERT_ERR_CUDA; }
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
   // scalars only from here on
   ly->d.w_qkv = ly->d.w_o = ly->d.w_f1 = ly->d.w_f2 = nullptr;
+  holder.p = nullptr;
   *out = ly;
   return IBERT_OK;
+  });
 }
 
 // bytes of workspace one encoder-layer call needs for T tokens
@@ -694,18 +769,23 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
 
 int ibert_encoder_layer(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, int B, int L,
                         int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   return encoder_layer_common(ctx, ly, x, B, L, nullptr, out, S_ret);
+  });
 }
 
 int ibert_encoder_layer_masked(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, int B, int L,
                                const int32_t* lens, int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   if (B > 0 && !lens) return IBERT_ERR_ARG;
   return encoder_layer_common(ctx, ly, x, B, L, lens, out, S_ret);
+  });
 }
 
 int ibert_embedding_i8(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
                        double S_word, const int8_t* pos, int64_t P, double S_pos, const double* gamma,
                        const double* beta, int H, double S_out, int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
   if (!ctx || T < 0 || !gamma || !beta || !word || !pos) return IBERT_ERR_ARG;
   if (L < 1 || H < 1 || H > 2047 || H % 16 != 0 || V < 1 || P < L) return IBERT_ERR_SHAPE;
   if (T > 0 && (!ids || !out)) return IBERT_ERR_ARG;
@@ -735,10 +815,12 @@ int ibert_embedding_i8(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, con
   if ((rc = launch_embed_gather(ctx, ids, T, L, word, V, pos, H, q, r))) return rc;
   ProfileScope ps(ctx, IBERT_K_LAYERNORM);
   return launch_layernorm(ctx, q, r, T, k, (const int32_t*)d_b, (const int64_t*)d_B, out);
+  });
 }
 
 int ibert_classifier_i8(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, double S_x, const int8_t* w,
                         const double* S_w, const int32_t* bias, int N, int32_t* logits, double* S_ret) {
+  return guarded([&]() -> int {
   if (!ctx || B < 0 || !S_w || !w) return IBERT_ERR_ARG;
   if (L < 1 || H < 1 || H % 16 != 0 || N < 1 || N % 4 != 0) return IBERT_ERR_SHAPE;
   if ((int64_t)H * 127 * 127 >= (int64_t(1) << 31)) return IBERT_ERR_SHAPE;
@@ -761,6 +843,7 @@ int ibert_classifier_i8(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, do
   epi.d_bias = bias;
   ProfileScope ps(ctx, gemm_class(EPI_RAW, H));
   return launch_gemm_i8(ctx, first, w, B, N, H, epi, logits);
+  });
 }
 
 // --------------------------------------------------------------------------- captured forward pass
@@ -786,6 +869,7 @@ static void graph_free(ibert_graph* g) {
 
 int ibert_encoder_graph_create(ibert_ctx* ctx, const ibert_layer* const* layers, int n_layers, const int8_t* x,
                                int B, int L, const int32_t* lens, int8_t* out, ibert_graph** out_graph) {
+  return guarded([&]() -> int {
   if (!ctx || !layers || n_layers < 1 || !out_graph || B < 1 || !x || !out) return IBERT_ERR_ARG;
   *out_graph = nullptr;
   if (L < 1 || L > 512) return IBERT_ERR_SHAPE;
@@ -799,7 +883,8 @@ int ibert_encoder_graph_create(ibert_ctx* ctx, const ibert_layer* const* layers,
   }
   if (!aligned16(x) || !aligned16(out)) return IBERT_ERR_ALIGN;
   DeviceGuard guard(ctx->device);
-  ibert_graph* g = new ibert_graph();
+  ibert_graph* g = new (std::nothrow) ibert_graph();
+  if (!g) return IBERT_ERR_NOMEM;
   g->ctx = ctx;
   const size_t act = (size_t)B * L * H;
   if (cudaMalloc(&g->ws, need) != cudaSuccess ||
@@ -841,24 +926,30 @@ int ibert_encoder_graph_create(ibert_ctx* ctx, const ibert_layer* const* layers,
   if (rc != IBERT_OK) { graph_free(g); return rc; }
   *out_graph = g;
   return IBERT_OK;
+  });
 }
 
 int ibert_encoder_graph_launch(ibert_ctx* ctx, ibert_graph* g) {
+  return guarded([&]() -> int {
   if (!ctx || !g || g->ctx != ctx || !g->exec) return IBERT_ERR_ARG;
   DeviceGuard guard(ctx->device);
   if (cudaGraphLaunch(g->exec, ctx->stream) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_CUDA; }
   return IBERT_OK;
+  });
 }
 
 int ibert_encoder_graph_destroy(ibert_graph* g) {
+  return guarded([&]() -> int {
   if (!g) return IBERT_ERR_ARG;
   DeviceGuard guard(g->ctx->device);
   cudaStreamSynchronize(g->ctx->stream);
   graph_free(g);
   return IBERT_OK;
+  });
 }
 
 int ibert_selftest_exp_division(double S, int32_t* q_ln2_out) {
+  return guarded([&]() -> int {
   ExpConsts k;
   int rc = make_exp_consts(S, 255, &k);
   if (rc) return rc;
@@ -875,16 +966,28 @@ int ibert_selftest_exp_division(double S, int32_t* q_ln2_out) {
     }
   }
   return IBERT_OK;
+  });
+}
+
+int ibert_selftest_wait_timeout(ibert_ctx* ctx, int64_t limit_us) {
+  return guarded([&]() -> int {
+  if (!ctx || limit_us < 1 || limit_us > 100000) return IBERT_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  return launch_wait_timeout(ctx, (uint64_t)limit_us * 1000ull);
+  });
 }
 
 int ibert_profile_begin(ibert_ctx* ctx) {
+  return guarded([&]() -> int {
   if (!ctx) return IBERT_ERR_ARG;
   ctx->ev_class.clear();
   ctx->profiling = true;
   return IBERT_OK;
+  });
 }
 
 int ibert_profile_end(ibert_ctx* ctx, float* ms, int32_t* launches) {
+  return guarded([&]() -> int {
   if (!ctx || !ms || !launches) return IBERT_ERR_ARG;
   DeviceGuard guard(ctx->device);
   ctx->profiling = false;
@@ -901,6 +1004,7 @@ int ibert_profile_end(ibert_ctx* ctx, float* ms, int32_t* launches) {
   }
   ctx->ev_class.clear();
   return IBERT_OK;
+  });
 }
 
 }  // extern "C"

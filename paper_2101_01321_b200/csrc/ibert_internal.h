@@ -89,6 +89,7 @@ int make_linear_tables(double S_x, const double* S_w, int N, const double* S_out
 struct DeviceTable {
   void* ptr = nullptr;
   size_t bytes = 0;
+  std::vector<unsigned char> host;   // the bytes that were uploaded: a hit must match them
 };
 
 }  // namespace ibert
@@ -128,6 +129,8 @@ int trim_tables(ibert_ctx* ctx);   // bounds the cache; only at the start of an 
 // Kernel launchers (each returns an IBERT_* code; all enqueue on ctx->stream)
 // ---------------------------------------------------------------------------------------
 
+// one warp that waits `limit_ns` on a barrier nobody arrives on, then records IBERT_ERR_TIMEOUT
+int launch_wait_timeout(ibert_ctx* ctx, uint64_t limit_ns);
 int launch_gelu(ibert_ctx* ctx, const int32_t* q, int64_t n, const GeluConsts& k, int8_t* out);
 // table[i] = i-GELU(i - 32767) for i in [0, 65535), computed by the i-GELU kernel over a ramp written
 // to `ramp_scratch` (65535 int32); and the look-up kernel that uses it

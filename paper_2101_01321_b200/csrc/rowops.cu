@@ -364,6 +364,14 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
     const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(ptx::smem_addr(bars + slot), phase));
     if (!ok) {
       if (lane == 0) atomicCAS(status, 0, IBERT_ERR_TIMEOUT);
+      // the copies already issued into the other slots must land (or run out of time as well)
+      // before this CTA's shared memory is given up
+      for (int j = 1; j < DEPTH; ++j) {
+        int s2 = slot + j;
+        uint32_t ph2 = phase;
+        if (s2 >= DEPTH) { s2 -= DEPTH; ph2 ^= 1; }
+        if (row + (int64_t)j * warp_count < rows) ptx::mbar_wait(ptx::smem_addr(bars + s2), ph2);
+      }
       break;
     }
     const uint8_t* sq = ring + (size_t)slot * slot_bytes;
@@ -475,6 +483,20 @@ __global__ void __launch_bounds__(kThreads) embed_gather_kernel(const int32_t* _
   }
 }
 
+// ----------------------------------------------------------------------------- wait self-test
+// One warp waits on an mbarrier nobody arrives on, with a short limit; when the limit runs out it
+// records IBERT_ERR_TIMEOUT like every kernel of the library does, and returns normally.
+__global__ void __launch_bounds__(32) wait_timeout_kernel(uint64_t limit_ns, int32_t* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_addr(&bar), 1);
+    ptx::fence_mbar_init();
+  }
+  __syncwarp();
+  const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait_ns(ptx::smem_addr(&bar), 0, limit_ns));
+  if (!ok && threadIdx.x == 0) atomicCAS(status, 0, IBERT_ERR_TIMEOUT);
+}
+
 int grid_for(ibert_ctx* ctx, int64_t work_warps, int max_ctas_per_sm) {
   const int64_t ctas = (work_warps + (kThreads / 32) - 1) / (kThreads / 32);
   const int64_t cap = (int64_t)ctx->num_sms * max_ctas_per_sm;
@@ -484,6 +506,11 @@ int grid_for(ibert_ctx* ctx, int64_t work_warps, int max_ctas_per_sm) {
 int check_launch() { return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA; }
 
 }  // namespace
+
+int launch_wait_timeout(ibert_ctx* ctx, uint64_t limit_ns) {
+  wait_timeout_kernel<<<1, 32, 0, ctx->stream>>>(limit_ns, ctx->d_status);
+  return check_launch();
+}
 
 int launch_embed_gather(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
                         const int8_t* pos, int H, int32_t* q, int8_t* r) {

@@ -71,14 +71,29 @@ __device__ __forceinline__ bool mbar_test_now(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after ~1 s of polling and reports failure instead of spinning forever.
-constexpr uint32_t kWaitSpinLimit = 4u << 20;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitSpinLimit; ++i) {
+// Bounded wait: polls until the phase completes or `limit_ns` of wall time (the GPU's global
+// nanosecond timer) have passed, then reports failure instead of spinning forever.  The timer is
+// only read on the slow path, after a burst of polls has failed.
+constexpr uint64_t kWaitLimitNs = 1000000000ull;       // 1 s: every wait of the kernels
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait_ns(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
+  for (int i = 0; i < 64; ++i)
     if (mbar_test(bar, parity)) return true;
-    if (i > 64) __nanosleep(64);
+  const uint64_t t0 = global_timer_ns();
+  for (;;) {
+    for (int i = 0; i < 32; ++i) {
+      if (mbar_test(bar, parity)) return true;
+      __nanosleep(64);
+    }
+    if (global_timer_ns() - t0 > limit_ns) return false;
   }
-  return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  return mbar_wait_ns(bar, parity, kWaitLimitNs);
 }
 
 // ------------------------------------------------------------------ proxies / fences
@@ -245,20 +260,28 @@ __device__ __forceinline__ void mbar_arrive_remote_release(uint32_t cluster_addr
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // bounded wait on a local mbarrier that other CTAs of the cluster arrive on; acquires their writes
+__device__ __forceinline__ bool mbar_test_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitSpinLimit; ++i) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, P;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    if (ok) return true;
-    if (i > 64) __nanosleep(64);
+  for (int i = 0; i < 64; ++i)
+    if (mbar_test_cluster(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (;;) {
+    for (int i = 0; i < 32; ++i) {
+      if (mbar_test_cluster(bar, parity)) return true;
+      __nanosleep(64);
+    }
+    if (global_timer_ns() - t0 > kWaitLimitNs) return false;
   }
-  return false;
 }
 // bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster (both
 // 16-byte aligned, size a multiple of 16); the bytes are credited to an mbarrier of the

@@ -14,6 +14,7 @@ from __future__ import annotations
 
 import math
 from dataclasses import dataclass
+from pathlib import Path
 
 import numpy as np
 
@@ -137,13 +138,36 @@ def make_input(config_id: int, B: int, L: int, H: int, shard: int = 0):
     return quantize_sym(x, S_x, 127).astype(np.int8), S_x
 
 
+CALIBRATED_SCALES_FILE = Path(__file__).resolve().parent.parent / "tests" / "golden" / "calibrated_scales.json"
+_calibrated = None
+
+
+def calibrated_scales(config_id: int, layer: int) -> dict:
+    """The ten static activation scales S_q .. S_out of one layer as calibrated offline: each site's
+    max|x| on the first sequences of the seeded input (Sec. 3.1: scales are fixed before inference).
+    The file is written by tests/golden/make_calibrated_scales.py; this module only reads it."""
+    global _calibrated
+    if _calibrated is None:
+        import json
+        if not CALIBRATED_SCALES_FILE.exists():
+            raise FileNotFoundError(f"{CALIBRATED_SCALES_FILE} is missing (run tests/golden/make_calibrated_scales.py)")
+        _calibrated = json.loads(CALIBRATED_SCALES_FILE.read_text())
+    layers = _calibrated["configs"][str(config_id)]["layers"]
+    if layer >= len(layers):
+        raise ValueError(f"no calibrated scales for config {config_id}, layer {layer}")
+    return {k: float(v) for k, v in layers[layer].items()}
+
+
 def make_layer(config_id: int, layer: int, H: int, heads: int, F: int, L: int, S_x: float,
-               p_max: int = 255, pow2_scores: bool = False) -> dict:
+               p_max: int = 255, pow2_scores: bool = False, scales: dict | None = None) -> dict:
     """One layer's integer parameters and static scales (a plain dict of numpy arrays).
-    pow2_scores: the query scale is raised (by less than 2x) so that the score scale is ln2 / 2^k."""
+    pow2_scores: the query scale is raised (by less than 2x) so that the score scale is ln2 / 2^k.
+    scales: the activation scales S_q .. S_out to use instead of the closed-form ones."""
     assert H == heads * 64
     p = {"H": H, "heads": heads, "F": F, "p_max": p_max}
     p.update(static_activation_scales(H, F, L, S_x))
+    if scales:
+        p.update({k: float(v) for k, v in scales.items() if k != "S_x"})
     if pow2_scores:
         p["S_q"] = snap_q_scale(p["S_q"], p["S_k"])
     in_scale = {"qkv": p["S_x"], "o": p["S_ctx"], "f1": p["S_h1"], "f2": p["S_go"]}
@@ -164,9 +188,11 @@ def make_layer(config_id: int, layer: int, H: int, heads: int, F: int, L: int, S
 
 def make_model(config_id: int, B: int, layers: int | None = None, H: int | None = None,
                heads: int | None = None, F: int | None = None, L: int | None = None, shard: int = 0,
-               pow2_scores: bool = False):
+               pow2_scores: bool = False, scales: str = "analytic"):
     """Input and per-layer parameters of one of the encoder configs (0, 2, 3, 4).
-    Layer l+1 consumes layer l's int8 output, so its S_x is layer l's S_out."""
+    Layer l+1 consumes layer l's int8 output, so its S_x is layer l's S_out.
+    scales: "analytic" (closed-form, any shape) or "calibrated" (the stored per-layer scales of
+    the config's own shape)."""
     cfg = CONFIGS[config_id]
     H = H or cfg.H
     heads = heads or cfg.heads
@@ -177,7 +203,8 @@ def make_model(config_id: int, B: int, layers: int | None = None, H: int | None 
     params = []
     s_in = S_x
     for l in range(layers):
-        p = make_layer(config_id, l, H, heads, F, L, s_in, pow2_scores=pow2_scores)
+        cal = calibrated_scales(config_id, l) if scales == "calibrated" else None
+        p = make_layer(config_id, l, H, heads, F, L, s_in, pow2_scores=pow2_scores, scales=cal)
         params.append(p)
         s_in = p["S_out"]
     return x, params
@@ -250,7 +277,7 @@ def make_lengths(config_id: int, B: int, L: int, shard: int = 0) -> np.ndarray:
 
 def make_full_model(config_id: int, B: int, layers: int | None = None, H: int | None = None,
                     heads: int | None = None, F: int | None = None, L: int | None = None,
-                    vocab: int = VOCAB, shard: int = 0) -> dict:
+                    vocab: int = VOCAB, shard: int = 0, scales: str = "analytic") -> dict:
     """Token ids, lengths, INT8 embedding tables, encoder layers and a first-token classifier.
     Word / position rows ~ N(0, 0.02^2)-like tables quantized with one symmetric int8 scale per
     table (Eq. 1); the embedding LayerNorm has gamma ~ N(1, 0.1), beta ~ N(0, 0.1) and an output
@@ -275,7 +302,8 @@ def make_full_model(config_id: int, B: int, layers: int | None = None, H: int | 
     params = []
     s_in = emb["S_out"]
     for l in range(layers):
-        p = make_layer(config_id, l, H, heads, F, L, s_in)
+        cal = calibrated_scales(config_id, l) if scales == "calibrated" else None
+        p = make_layer(config_id, l, H, heads, F, L, s_in, scales=cal)
         params.append(p)
         s_in = p["S_out"]
     w, S_w = _quantize_weight(rng_for(config_id, 0, _T_HEAD_W), N_LABELS, H)

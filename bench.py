@@ -644,6 +644,7 @@ def run_only(args):
     p = synth.static_activation_scales(H, F, L, 0.035)
     rng = np.random.default_rng(synth.SEED_BASE)
     k = args.only
+    alg_bytes = None
     if k in ("gemm_out_ln", "gemm_ffn2_ln"):
         N, K = (H, H) if k == "gemm_out_ln" else (H, F)
         x, w, res = i8(T, K), i8(N, K), i8(T, N)
@@ -679,15 +680,17 @@ def run_only(args):
         qkv = torch.clamp(torch.randn((T, 3 * H), generator=g) * 32, -127, 127).to(torch.int8).to(dev)
         out = torch.empty((T, H), dtype=torch.int8, device=dev)
         fn = lambda: ctx.ibert_attention_i8(qkv, batch, L, H, cfg.heads, p["S_q"], p["S_k"], p["S_v"], p["S_ctx"], 255, out=out)
-    elif k == "layernorm":
+    elif k in ("layernorm", "layernorm_i16"):
         q, S, r, S_r, gamma, beta, S_out = synth.layernorm_inputs(T, H, 1.0)
-        qd, rd = torch.from_numpy(q).to(dev), torch.from_numpy(r).to(dev)
+        qd, rd = torch.from_numpy(q.astype(np.int16) if k == "layernorm_i16" else q).to(dev), torch.from_numpy(r).to(dev)
         out = torch.empty((T, H), dtype=torch.int8, device=dev)
         fn = lambda: ctx.ibert_layernorm_i(qd, S, rd, S_r, gamma, beta, S_out, out=out)
+        alg_bytes = T * H * ((2 if k == "layernorm_i16" else 4) + 1 + 1)
     elif k in ("gelu", "hgelu", "gelu_lut"):
         q, S, S_out = synth.gelu_inputs(1 << 24, 1.0)
         qd = torch.from_numpy(q).to(dev)
         out = torch.empty(q.shape, dtype=torch.int8, device=dev)
+        alg_bytes = q.size * 5
         fn = {"gelu": lambda: ctx.ibert_gelu_i(qd, S, S_out, out=out),
               "hgelu": lambda: ctx.ibert_hgelu_i(qd, S, S_out, out=out),
               "gelu_lut": lambda: ctx.ibert_gelu_lut_i(qd, S, S_out, out=out)}[k]
@@ -696,6 +699,7 @@ def run_only(args):
         q, S = synth.softmax_inputs(rows, L, 1.0)
         qd = torch.from_numpy(q).to(dev)
         out = torch.empty(q.shape, dtype=torch.uint8, device=dev)
+        alg_bytes = q.size * 5
         fn = (lambda: ctx.ibert_softmax_i(qd, S, 255, out=out)) if k == "softmax" else \
              (lambda: ctx.ibert_softmax_lut_i(qd, S, 255, out=out))
     else:
@@ -715,8 +719,14 @@ def run_only(args):
     stream.synchronize()
     ctx.check()
     ms = [a.elapsed_time(b) for a, b in times]
-    print(json.dumps({"only": k, "tokens": T, "ms_median": statistics.median(ms), "ms_min": min(ms),
-                      "launches": args.steps}))
+    line = {"only": k, "tokens": T, "ms_median": statistics.median(ms), "ms_min": min(ms), "launches": args.steps}
+    if alg_bytes:
+        peaks, peak_kind = measured_peaks()
+        gbs = alg_bytes / statistics.median(ms) / 1e6
+        line["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                            "frac": gbs / peaks["hbm_gbs"], "algorithmic": alg_bytes,
+                            "peak_source": f"{peak_kind} copy bandwidth; the time includes the event pair (about 5 us)"}
+    print(json.dumps(line))
     ctx.close()
 
 

@@ -70,9 +70,13 @@ int ibert_dyadic_from_double(double m, int32_t* b, int32_t* c);
    x [M,K] int8, w [N,K] int8 (K contiguous), bias [N] int32 at scale S_x*S_w[n] (may be NULL),
    S_w host array [N] (per-output-channel weight scales).
    out_kind 0: out is int8 [M,N] at S_out;  1: out is Q16 in int32 [M,N] at S_out;
-            2: out is the raw int32 accumulators (S_out ignored).
-   S_ret (host, may be NULL): receives S_out (kinds 0, 1: one entry) or S_x*S_w[n] (kind 2: N entries).
-   Requires K % 16 == 0, N % 16 == 0 (kinds 0) / N % 4 == 0 (kinds 1, 2), K*127*127 + |bias| < 2^31. */
+            2: out is the raw int32 accumulators (S_out ignored);
+            3: out is Q16 in int16 [M,N] at S_out -- the values of kind 1 in half the bytes (the
+               "INT32 precision" inputs of the non-linear operations, Sec. 3.6 / Appendix C.1, are
+               brought to a per-tensor scale and then never exceed 16 bits).
+   S_ret (host, may be NULL): receives S_out (kinds 0, 1, 3: one entry) or S_x*S_w[n] (kind 2: N entries).
+   Requires K % 16 == 0, N % 16 == 0 (kind 0) / N % 4 == 0 (kinds 1, 2) / N % 8 == 0 (kind 3),
+   K*127*127 + |bias| < 2^31, M < 2^31 - 256. */
 int ibert_linear_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
                     const int32_t* bias, int64_t M, int N, int K, int out_kind, double S_out,
                     void* out, double* S_ret);
@@ -114,6 +118,14 @@ int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S
 int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* r, double S_r,
                       const double* gamma, const double* beta, int64_t rows, int C, double S_out,
                       int8_t* out, double* S_ret);
+
+/* The same operation on Q16 values stored as int16 (Sec. 3.6 / Appendix C.1: the LayerNorm input
+   is the requantized accumulator of the preceding MatMul, at a per-tensor scale; in Q16 it fits 16
+   bits): q int16 [rows,C], everything else, and every result, as ibert_layernorm_i on the same
+   values.  4 instead of 6 bytes of traffic per element. */
+int ibert_layernorm_i16(ibert_ctx* ctx, const int16_t* q, double S, const int8_t* r, double S_r,
+                        const double* gamma, const double* beta, int64_t rows, int C, double S_out,
+                        int8_t* out, double* S_ret);
 
 /* The same operation for callers that cannot allocate device memory (no counterpart in the
    paper: a deployment convenience).  ibert_layernorm_i keeps its per-channel constant tables in
@@ -174,7 +186,7 @@ int ibert_layer_destroy(ibert_layer* layer);
    most 1024), the constants fit the 32-bit forms and M is large enough for its 128-row tiles to
    occupy half of the SMs, a single kernel computes it on a cluster of N/256 CTAs per tile and the
    Q16 tensor never reaches memory; otherwise the two kernels run back to back through the
-   context's workspace.
+   context's workspace, which holds the Q16 tensor as int16.
    Errors: as ibert_linear_i8 and ibert_layernorm_i. */
 int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w, const double* S_w,
                               const int32_t* bias, int64_t M, int N, int K, double S_mid,

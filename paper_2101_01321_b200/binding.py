@@ -67,6 +67,8 @@ def lib():
         L.ibert_softmax_lut_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
         L.ibert_gelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
         L.ibert_layernorm_i.argtypes = [vp, vp, dbl, vp, dbl, vp, vp, i64, i32, dbl, vp, vp]
+        L.ibert_layernorm_i16.argtypes = [vp, vp, dbl, vp, dbl, vp, vp, i64, i32, dbl, vp, vp]
+        L.ibert_layernorm_i16.restype = i32
         L.ibert_attention_i8.argtypes = [vp, vp, i32, i32, i32, i32, dbl, dbl, dbl, dbl, i32, vp, vp]
         L.ibert_attention_masked_i8.argtypes = [vp, vp, i32, i32, i32, i32, vp, dbl, dbl, dbl, dbl, i32, vp, vp]
         L.ibert_encoder_layer_masked.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
@@ -248,6 +250,11 @@ class Context:
         if out is None:
             out = torch.empty(q.shape, dtype=torch.int8, device=q.device)
         S_ret = C.c_double()
+        if q.dtype == torch.int16:           # Q16 values in an int16 container
+            _chk(lib().ibert_layernorm_i16(self.h, _dev(q, torch.int16), S, _dev(r, torch.int8), S_r or 0.0,
+                                           g.ctypes.data, b.ctypes.data, rows, Cn, S_out, _dev(out, torch.int8),
+                                           C.byref(S_ret)), "ibert_layernorm_i16")
+            return out, S_ret.value
         _chk(lib().ibert_layernorm_i(self.h, _dev(q, torch.int32), S, _dev(r, torch.int8), S_r or 0.0,
                                      g.ctypes.data, b.ctypes.data, rows, Cn, S_out, _dev(out, torch.int8),
                                      C.byref(S_ret)), "ibert_layernorm_i")
@@ -262,8 +269,8 @@ class Context:
         sw = _host(S_w, np.float64)
         assert sw.size == N
         if out is None:
-            out = torch.empty(x.shape[:-1] + (N,), dtype=torch.int8 if out_kind == 0 else torch.int32,
-                              device=x.device)
+            out = torch.empty(x.shape[:-1] + (N,), device=x.device,
+                              dtype={0: torch.int8, 3: torch.int16}.get(out_kind, torch.int32))
         S_ret = np.zeros(N if out_kind == 2 else 1, dtype=np.float64)
         _chk(lib().ibert_linear_i8(self.h, _dev(x, torch.int8), S_x, _dev(w, torch.int8), sw.ctypes.data,
                                    _dev(bias, torch.int32), M, N, K, out_kind, S_out, out.data_ptr(),

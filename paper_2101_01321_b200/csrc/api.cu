@@ -352,10 +352,9 @@ int ibert_softmax_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t rows
   });
 }
 
-int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* r, double S_r,
-                      const double* gamma, const double* beta, int64_t rows, int C, double S_out,
-                      int8_t* out, double* S_ret) {
-  return guarded([&]() -> int {
+static int layernorm_common(ibert_ctx* ctx, const void* q, bool q_is_i16, double S, const int8_t* r, double S_r,
+                            const double* gamma, const double* beta, int64_t rows, int C, double S_out,
+                            int8_t* out, double* S_ret) {
   if (!ctx || rows < 0 || !gamma || !beta) return IBERT_ERR_ARG;
   if (C < 1 || C > 2047) return IBERT_ERR_SHAPE;
   if (rows > 0 && (!q || !out)) return IBERT_ERR_ARG;
@@ -381,10 +380,28 @@ int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* 
   if (rc) return rc;
   {
     ProfileScope ps(ctx, IBERT_K_LAYERNORM);
-    rc = launch_layernorm(ctx, q, r, rows, k, (const int32_t*)d_b, (const int64_t*)d_B, out);
+    if (q_is_i16)
+      rc = launch_layernorm_i16(ctx, static_cast<const int16_t*>(q), r, rows, k, (const int32_t*)d_b, (const int64_t*)d_B, out);
+    else
+      rc = launch_layernorm(ctx, static_cast<const int32_t*>(q), r, rows, k, (const int32_t*)d_b, (const int64_t*)d_B, out);
   }
   if (rc == IBERT_OK && S_ret) *S_ret = S_out;
   return rc;
+}
+
+int ibert_layernorm_i(ibert_ctx* ctx, const int32_t* q, double S, const int8_t* r, double S_r,
+                      const double* gamma, const double* beta, int64_t rows, int C, double S_out,
+                      int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
+  return layernorm_common(ctx, q, false, S, r, S_r, gamma, beta, rows, C, S_out, out, S_ret);
+  });
+}
+
+int ibert_layernorm_i16(ibert_ctx* ctx, const int16_t* q, double S, const int8_t* r, double S_r,
+                        const double* gamma, const double* beta, int64_t rows, int C, double S_out,
+                        int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
+  return layernorm_common(ctx, q, true, S, r, S_r, gamma, beta, rows, C, S_out, out, S_ret);
   });
 }
 
@@ -392,8 +409,9 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
                          const int32_t* bias, int64_t M, int N, int K, int kind, double S_mid,
                          double S_out, void* out, double* S_ret) {
   if (!ctx || M < 0 || !S_w) return IBERT_ERR_ARG;
-  if (kind < 0 || kind > 4) return IBERT_ERR_ARG;
+  if (kind < 0 || kind > 5) return IBERT_ERR_ARG;
   if (N < 1 || K < 1 || K % 16 != 0 || N % 4 != 0) return IBERT_ERR_SHAPE;
+  if (kind == EPI_Q16H && N % 8 != 0) return IBERT_ERR_SHAPE;      // 16-byte aligned int16 rows
   if ((kind == EPI_INT8 || kind == EPI_GELU || kind == EPI_HGELU) && N % 16 != 0) return IBERT_ERR_SHAPE;
   if ((int64_t)K * 127 * 127 >= (int64_t(1) << 31)) return IBERT_ERR_SHAPE;
   if (M >= (int64_t(1) << 31) - 256) return IBERT_ERR_SHAPE;      // tile coordinates are 32-bit
@@ -509,12 +527,14 @@ int ibert_linear_layernorm_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const
     ProfileScope ps(ctx, K > 2048 ? IBERT_K_GEMM_LN_WIDE : IBERT_K_GEMM_LN);
     rc = launch_gemm_ln_i8(ctx, x, w, M, N, K, epi, res, k, (const int32_t*)d_bi, (const int64_t*)d_Bi, out);
   } else {
-    if ((rc = ensure_workspace(ctx, (size_t)M * N * 4 + 256))) return rc;
-    int32_t* mid = static_cast<int32_t*>(ctx->ws);
+    // the Q16 tensor between the two kernels is held as int16 (value-identical, half the bytes)
+    if ((rc = ensure_workspace(ctx, (size_t)M * N * 2 + 256))) return rc;
+    int16_t* mid = static_cast<int16_t*>(ctx->ws);
+    epi.kind = EPI_Q16H;
     { ProfileScope ps(ctx, gemm_class(EPI_Q16, K)); rc = launch_gemm_i8(ctx, x, w, M, N, K, epi, mid); }
     if (rc) return rc;
     ProfileScope ps(ctx, IBERT_K_LAYERNORM);
-    rc = launch_layernorm(ctx, mid, res, M, k, (const int32_t*)d_bi, (const int64_t*)d_Bi, out);
+    rc = launch_layernorm_i16(ctx, mid, res, M, k, (const int32_t*)d_bi, (const int64_t*)d_Bi, out);
   }
   if (rc == IBERT_OK && S_ret) *S_ret = S_out;
   return rc;
@@ -525,8 +545,9 @@ int ibert_linear_i8(ibert_ctx* ctx, const int8_t* x, double S_x, const int8_t* w
                     const int32_t* bias, int64_t M, int N, int K, int out_kind, double S_out,
                     void* out, double* S_ret) {
   return guarded([&]() -> int {
-  if (out_kind < 0 || out_kind > 2) return IBERT_ERR_ARG;
-  return linear_common(ctx, x, S_x, w, S_w, bias, M, N, K, out_kind, 0.0, S_out, out, S_ret);
+  if (out_kind < 0 || out_kind > 3) return IBERT_ERR_ARG;
+  return linear_common(ctx, x, S_x, w, S_w, bias, M, N, K, out_kind == 3 ? (int)EPI_Q16H : out_kind, 0.0, S_out, out,
+                       S_ret);
   });
 }
 
@@ -728,7 +749,7 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
   char* ws = static_cast<char*>(ctx->ws);
   int8_t* qkv = (int8_t*)(ws + o_qkv);
   int8_t* cx = (int8_t*)(ws + o_ctx);
-  int32_t* r = (int32_t*)(ws + o_r);
+  int16_t* r = (int16_t*)(ws + o_r);             // Q16 residual sums as int16 (two-kernel path only)
   int8_t* h1 = (int8_t*)(ws + o_h1);
   int8_t* g = (int8_t*)(ws + o_g);
 
@@ -748,9 +769,10 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
     ProfileScope ps(ctx, IBERT_K_GEMM_LN);
     rc = launch_gemm_ln_i8(ctx, cx, ly->w_o, T, H, H, e, x, ly->ln1, ly->ln1_b, ly->ln1_B, h1);
   } else {
+    e.kind = EPI_Q16H;
     { ProfileScope ps(ctx, IBERT_K_GEMM_Q16); rc = launch_gemm_i8(ctx, cx, ly->w_o, T, H, H, e, r); }
     if (rc) return rc;
-    { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm(ctx, r, x, T, ly->ln1, ly->ln1_b, ly->ln1_B, h1); }
+    { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm_i16(ctx, r, x, T, ly->ln1, ly->ln1_b, ly->ln1_B, h1); }
   }
   if (rc) return rc;
   e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu; e.fast = ly->fast_f1;
@@ -761,9 +783,10 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
     ProfileScope ps(ctx, F > 2048 ? IBERT_K_GEMM_LN_WIDE : IBERT_K_GEMM_LN);
     return launch_gemm_ln_i8(ctx, g, ly->w_f2, T, H, F, e, h1, ly->ln2, ly->ln2_b, ly->ln2_B, out);
   }
+  e.kind = EPI_Q16H;
   { ProfileScope ps(ctx, IBERT_K_GEMM_Q16_WIDE); rc = launch_gemm_i8(ctx, g, ly->w_f2, T, H, F, e, r); }
   if (rc) return rc;
-  { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm(ctx, r, h1, T, ly->ln2, ly->ln2_b, ly->ln2_B, out); }
+  { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm_i16(ctx, r, h1, T, ly->ln2, ly->ln2_b, ly->ln2_B, out); }
   return rc;
 }
 

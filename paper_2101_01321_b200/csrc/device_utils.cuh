@@ -57,6 +57,13 @@ __device__ __forceinline__ int32_t sext_byte(uint32_t w, int k) {
   return r;
 }
 
+// 16-bit half h of a word as a sign-extended int32, likewise in one permute
+__device__ __forceinline__ int32_t sext_half(uint32_t w, int h) {
+  int32_t r;
+  asm("prmt.b32 %0, %1, 0, %2;" : "=r"(r) : "r"(w), "r"(h ? 0xBB32 : 0x9910));
+  return r;
+}
+
 __device__ __forceinline__ int64_t rounding_half(int c) { return c > 0 ? (int64_t(1) << (c - 1)) : 0; }
 
 __device__ __forceinline__ int32_t clamp_sym(int32_t v, int32_t qmax) { return max(-qmax, min(v, qmax)); }

@@ -93,7 +93,8 @@ constexpr int kEpiGeluLowFree = 16;
 
 template <int TOK, bool PAIR, int KIND>
 struct Cfg {
-  static constexpr bool kOut32 = (KIND == EPI_RAW || KIND == EPI_Q16);
+  static constexpr bool kOut32 = (KIND == EPI_RAW || KIND == EPI_Q16 || KIND == EPI_Q16H);   // light epilogue, wide output
+  static constexpr int kOutElem = (KIND == EPI_RAW || KIND == EPI_Q16) ? 4 : (KIND == EPI_Q16H ? 2 : 1);   // bytes per output value
   static constexpr int kChunks = TOK / 32;                       // 32-token chunks of a tile
   // the int8 epilogues are ALU-bound: one warp per 64 tokens; the int32 ones per 128 tokens
   static constexpr int kEpiWarps = kOut32 ? TOK / 32 : TOK / 16;
@@ -103,7 +104,7 @@ struct Cfg {
   static constexpr int kXRows = PAIR ? TOK / 2 : TOK;            // token rows this CTA loads per K block
   static constexpr int kWBytes = BC * BK;
   static constexpr int kStageBytes = kWBytes + kXRows * BK;
-  static constexpr int kOutTileBytes = kOut32 ? 32 * 128 : 32 * 32;   // 32 tokens x 32 channels
+  static constexpr int kOutTileBytes = 32 * 32 * kOutElem;            // 32 tokens x 32 channels
   static constexpr int kOutBytes = kEpiWarps * 2 * kOutTileBytes;     // double-buffered per warp
   static constexpr int kBudget = 227 * 1024 - 1024 - 512 - kOutBytes;
   static constexpr int kStages = kBudget / kStageBytes > 8 ? 8 : kBudget / kStageBytes;
@@ -304,6 +305,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           else if constexpr (KIND == EPI_Q16) {
             if constexpr (FAST) o = clamp_sym(requant_upper(a + cur_bias, cur_pb), 32767);
             else o = requant_add(a, cur_pb, cur_padd, cur_pc, 32767);
+          } else if constexpr (KIND == EPI_Q16H) {
+            if constexpr (FAST) o = clamp_sym(requant_upper(a + cur_bias, cur_pb), 32767);
+            else o = requant_add(a, cur_pb, cur_padd, cur_pc, 32767);
           } else if constexpr (KIND == EPI_INT8) {
             if constexpr (FAST) o = clamp_sym(requant_upper(a + cur_bias, cur_pb), 127);
             else o = requant_add(a, cur_pb, cur_padd, cur_pc, 127);
@@ -319,7 +323,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
           }
           // staging tile: row = token i, column = this lane's channel
-          if constexpr (kOut32) reinterpret_cast<int32_t*>(stage)[i * 32 + lane] = o;
+          if constexpr (C::kOutElem == 4) reinterpret_cast<int32_t*>(stage)[i * 32 + lane] = o;
+          else if constexpr (C::kOutElem == 2)
+            asm volatile("st.shared.u16 [%0], %1;" ::"r"(ptx::smem_addr(stage) + (i * 32 + lane) * 2), "h"((uint16_t)o) : "memory");
           else  // low byte of the register, stored without a narrowing conversion
             asm volatile("st.shared.u8 [%0], %1;" ::"r"(ptx::smem_addr(stage) + i * 32 + lane), "r"(o) : "memory");
         }
@@ -328,7 +334,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           __syncwarp();
           if (lane == 0) {
             if constexpr (kOneStore) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage0), ch0, t0);
-            else ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), ch0 * (kOut32 ? 4 : 1), t0 + ci * 32);
+            else ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), ch0 * C::kOutElem, t0 + ci * 32);
             ptx::bulk_commit();
           }
         }
@@ -379,6 +385,7 @@ int launch_shape(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, c
   switch (kind) {
     case EPI_INT8: return fast ? launch_inst<TOK, PAIR, EPI_INT8, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_INT8, false>(ctx, mw, mx, mo, a);
     case EPI_Q16: return fast ? launch_inst<TOK, PAIR, EPI_Q16, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_Q16, false>(ctx, mw, mx, mo, a);
+    case EPI_Q16H: return fast ? launch_inst<TOK, PAIR, EPI_Q16H, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_Q16H, false>(ctx, mw, mx, mo, a);
     case EPI_GELU:
       if (fast && a.gelu.low_free) return launch_inst<TOK, PAIR, kEpiGeluLowFree, true>(ctx, mw, mx, mo, a);
       return fast ? launch_inst<TOK, PAIR, EPI_GELU, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_GELU, false>(ctx, mw, mx, mo, a);
@@ -406,7 +413,7 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
   const bool pair = ctx->num_sms >= 2 && t256 * ((N + 255) / 256) >= ctx->num_sms / 2;
   const bool wide = pair || t256 * ((N + 127) / 128) >= ctx->num_sms;
   const int TOK = wide ? 256 : 128;
-  const bool out32 = epi.kind == EPI_RAW || epi.kind == EPI_Q16;
+  const uint32_t out_elem = (epi.kind == EPI_RAW || epi.kind == EPI_Q16) ? 4u : (epi.kind == EPI_Q16H ? 2u : 1u);
   CUtensorMap mw, mx, mo;
   {
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
@@ -424,12 +431,12 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
   }
   {
     // the output as a byte matrix [T, N * element size]; one box = one warp's 32-token x 32-channel block
-    const uint64_t row_bytes = (uint64_t)N * (out32 ? 4 : 1);
+    const uint64_t row_bytes = (uint64_t)N * out_elem;
     const uint64_t dims[2] = {row_bytes, (uint64_t)M};
     const uint64_t str[1] = {row_bytes};
     // (the GELU epilogues store a warp's 64 tokens at once)
     const bool gelu_kind = epi.kind == EPI_GELU || epi.kind == EPI_HGELU;
-    const uint32_t box[2] = {out32 ? 128u : 32u, gelu_kind ? 64u : 32u};
+    const uint32_t box[2] = {32u * out_elem, gelu_kind ? 64u : 32u};
     int rc = encode_tensor_map(&mo, out, 2, dims, str, box, 0);
     if (rc) return rc;
   }

@@ -63,7 +63,7 @@ template <int KIND, bool FAST>
 __device__ __forceinline__ int32_t epilogue_value(int32_t a, int32_t bias, int32_t pb, int32_t pc, int64_t padd,
                                                   const GeluConsts& gk, int64_t gelu_half, int32_t gelu_rnd) {
   if constexpr (KIND == EPI_RAW) return a + bias;
-  else if constexpr (KIND == EPI_Q16) {
+  else if constexpr (KIND == EPI_Q16 || KIND == EPI_Q16H) {
     if constexpr (FAST) return clamp_sym(requant_upper(a + bias, pb), 32767);
     else return requant_add(a, pb, padd, pc, 32767);
   } else if constexpr (KIND == EPI_INT8) {
@@ -240,6 +240,7 @@ gemm_splitk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         const int64_t t = (int64_t)t0 + col0 + j;
         if (t < args.T && n < args.N) {
           if constexpr (kOut32) static_cast<int32_t*>(args.out)[t * args.N + n] = o;
+          else if constexpr (KIND == EPI_Q16H) static_cast<int16_t*>(args.out)[t * args.N + n] = (int16_t)o;
           else static_cast<int8_t*>(args.out)[t * args.N + n] = (int8_t)o;
         }
       }
@@ -307,6 +308,7 @@ int launch_gemm_splitk_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int6
   switch (epi.kind) {
     case EPI_INT8: return fast ? launch_inst<EPI_INT8, true>(ctx, mw, mx, a, tiles) : launch_inst<EPI_INT8, false>(ctx, mw, mx, a, tiles);
     case EPI_Q16: return fast ? launch_inst<EPI_Q16, true>(ctx, mw, mx, a, tiles) : launch_inst<EPI_Q16, false>(ctx, mw, mx, a, tiles);
+    case EPI_Q16H: return fast ? launch_inst<EPI_Q16H, true>(ctx, mw, mx, a, tiles) : launch_inst<EPI_Q16H, false>(ctx, mw, mx, a, tiles);
     case EPI_GELU: return fast ? launch_inst<EPI_GELU, true>(ctx, mw, mx, a, tiles) : launch_inst<EPI_GELU, false>(ctx, mw, mx, a, tiles);
     case EPI_HGELU: return fast ? launch_inst<EPI_HGELU, true>(ctx, mw, mx, a, tiles) : launch_inst<EPI_HGELU, false>(ctx, mw, mx, a, tiles);
     default: return launch_inst<EPI_RAW, false>(ctx, mw, mx, a, tiles);

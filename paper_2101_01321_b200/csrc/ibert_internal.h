@@ -145,9 +145,13 @@ int launch_embed_gather(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, co
                         const int8_t* pos, int H, int32_t* q, int8_t* r);
 int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t rows, const LnConsts& k,
                      const int32_t* d_b, const int64_t* d_B, int8_t* out);
+// the same with the Q16 input stored as int16 (values identical, 2 bytes per element less traffic)
+int launch_layernorm_i16(ibert_ctx* ctx, const int16_t* q, const int8_t* r, int64_t rows, const LnConsts& k,
+                         const int32_t* d_b, const int64_t* d_B, int8_t* out);
 
 // epilogue kinds of the GEMM
-enum : int { EPI_INT8 = 0, EPI_Q16 = 1, EPI_RAW = 2, EPI_GELU = 3, EPI_HGELU = 4 };
+// (EPI_Q16H: the Q16 values of EPI_Q16 stored as int16 instead of int32)
+enum : int { EPI_INT8 = 0, EPI_Q16 = 1, EPI_RAW = 2, EPI_GELU = 3, EPI_HGELU = 4, EPI_Q16H = 5 };
 
 struct GemmEpilogue {
   int kind;

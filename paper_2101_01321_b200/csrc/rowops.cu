@@ -197,14 +197,28 @@ __device__ __forceinline__ uint32_t warp_isqrt_of_quotient(uint64_t ss, uint32_t
   return base;
 }
 
+// Four consecutive Q16 values of a row, from an int32 or an int16 container (16 / 8 bytes)
+template <typename QT>
+__device__ __forceinline__ void load_q4(const QT* p, int32_t (&v)[4], bool streaming) {
+  if constexpr (sizeof(QT) == 4) {
+    const int4 t = streaming ? __ldcs(reinterpret_cast<const int4*>(p)) : *reinterpret_cast<const int4*>(p);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  } else {
+    const uint2 t = streaming ? __ldcs(reinterpret_cast<const uint2*>(p)) : *reinterpret_cast<const uint2*>(p);
+    // sign-extending halves of a word: one byte permute each
+    v[0] = sext_half(t.x, 0); v[1] = sext_half(t.x, 1);
+    v[2] = sext_half(t.y, 0); v[3] = sext_half(t.y, 1);
+  }
+}
+
 // One warp per row, the whole row in registers (VPL int4 vectors per lane).
 // FAST: residual rescale and output requantization are in upper-word form (one multiply-add each).
 // Resident CTAs per SM the register budget is tuned for: the kernel is latency-bound on the row
 // loads, so short rows trade registers for more warps in flight.
 constexpr int ln_min_blocks(int vpl) { return vpl <= 4 ? 4 : (vpl <= 6 ? 3 : (vpl <= 8 ? 2 : 1)); }
 
-template <int VPL, bool VEC, bool FAST>
-__global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel(const int32_t* __restrict__ q,
+template <int VPL, bool VEC, bool FAST, typename QT>
+__global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel(const QT* __restrict__ q,
                                                              const int8_t* __restrict__ r, int64_t rows,
                                                              LnConsts k, const int32_t* __restrict__ b_i,
                                                              const int64_t* __restrict__ B_i,
@@ -215,7 +229,7 @@ __global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel
   const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
   const int64_t half_r = rounding_half(k.c_r);
   for (int64_t row = warp_global; row < rows; row += warp_count) {
-    const int32_t* qr = q + row * C;
+    const QT* qr = q + row * C;
     const int8_t* rr = r + row * C;
     int8_t* orow = out + row * C;
     int32_t v[VPL][4];
@@ -225,8 +239,7 @@ __global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel
       const int col = 4 * (j * 32 + lane);
       if (VEC) {
         if (col < C) {
-          const int4 t = __ldcs(reinterpret_cast<const int4*>(qr + col));
-          v[j][0] = t.x; v[j][1] = t.y; v[j][2] = t.z; v[j][3] = t.w;
+          load_q4(qr + col, v[j], true);
           if (k.has_res) {
             const uint32_t rw = __ldcs(reinterpret_cast<const uint32_t*>(rr + col));
 #pragma unroll
@@ -244,7 +257,7 @@ __global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel
         for (int i = 0; i < 4; ++i) {
           int32_t t = 0;
           if (col + i < C) {
-            t = qr[col + i];
+            t = (int32_t)qr[col + i];
             if (k.has_res) t += (int32_t)(((int64_t)rr[col + i] * k.b_r + half_r) >> k.c_r);
           }
           v[j][i] = t;
@@ -323,8 +336,9 @@ __global__ void __launch_bounds__(kThreads, ln_min_blocks(VPL)) layernorm_kernel
 // residual row) through a private ring of DEPTH shared-memory slots, so the loads of the next
 // rows are in flight while the current row is reduced -- the row loop no longer waits on HBM.
 // Requires C % 16 == 0 (16-byte aligned rows), upper-word constants, and a residual.
-template <int VPL, int DEPTH>
-__global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_kernel(const int32_t* __restrict__ q,
+// FULL: C == 128 VPL, no lane ever runs past the row.
+template <int VPL, int DEPTH, typename QT, bool FULL>
+__global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_kernel(const QT* __restrict__ q,
                                                                      const int8_t* __restrict__ r, int64_t rows,
                                                                      LnConsts k, const int32_t* __restrict__ b_i,
                                                                      const int64_t* __restrict__ B_i,
@@ -332,7 +346,7 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
   extern __shared__ __align__(128) uint8_t ln_smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int C = k.C;
-  const uint32_t q_bytes = (uint32_t)C * 4u, r_bytes = (uint32_t)C;
+  const uint32_t q_bytes = (uint32_t)C * (uint32_t)sizeof(QT), r_bytes = (uint32_t)C;
   const uint32_t slot_bytes = q_bytes + r_bytes;                 // multiple of 16
   uint8_t* ring = ln_smem + (size_t)warp * DEPTH * slot_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(ln_smem + (size_t)(kThreads / 32) * DEPTH * slot_bytes) + warp * DEPTH;
@@ -380,9 +394,8 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
       const int col = 4 * (j * 32 + lane);
-      if (col < C) {
-        const int4 t = *reinterpret_cast<const int4*>(sq + (size_t)col * 4);
-        v[j][0] = t.x; v[j][1] = t.y; v[j][2] = t.z; v[j][3] = t.w;
+      if (FULL || col < C) {
+        load_q4(reinterpret_cast<const QT*>(sq) + col, v[j], false);
         rw[j] = *reinterpret_cast<const uint32_t*>(sq + q_bytes + col);
       } else {
         v[j][0] = v[j][1] = v[j][2] = v[j][3] = 0;
@@ -413,7 +426,7 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
       const int col = 4 * (j * 32 + lane);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const int32_t y = (col < C) ? v[j][i] - mu : 0;
+        const int32_t y = (FULL || col < C) ? v[j][i] - mu : 0;
         v[j][i] = y;
         ss += (uint64_t)((int64_t)y * (int64_t)y);
       }
@@ -430,7 +443,7 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
       const int col = 4 * (j * 32 + lane);
-      if (col < C) {
+      if (FULL || col < C) {
         const int4 bb = __ldg(reinterpret_cast<const int4*>(b_i + col));
         const longlong2 B01 = __ldg(reinterpret_cast<const longlong2*>(B_i + col));
         const longlong2 B23 = __ldg(reinterpret_cast<const longlong2*>(B_i + col + 2));
@@ -573,8 +586,9 @@ int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const 
   return check_launch();
 }
 
-int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t rows, const LnConsts& k,
-                     const int32_t* d_b, const int64_t* d_B, int8_t* out) {
+template <typename QT>
+static int launch_layernorm_t(ibert_ctx* ctx, const QT* q, const int8_t* r, int64_t rows, const LnConsts& k,
+                              const int32_t* d_b, const int64_t* d_B, int8_t* out) {
   if (rows == 0) return IBERT_OK;
   const int grid = grid_for(ctx, rows, 8);
   const bool vec = (k.C % 4) == 0;
@@ -583,33 +597,39 @@ int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t 
   if (fast && k.has_res && k.C % 16 == 0 && k.C <= 1024) {
     // streaming variant: per-warp ring of row slots filled by bulk async copies
     const int depth = 2;
-    const size_t smem = (size_t)(kThreads / 32) * depth * (size_t)k.C * 5 + (kThreads / 32) * depth * 8;
+    const size_t smem = (size_t)(kThreads / 32) * depth * (size_t)k.C * (sizeof(QT) + 1) + (kThreads / 32) * depth * 8;
     const int pgrid = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)ctx->num_sms * 3);
-#define IBERT_LNP(V, D)                                                                                     \
+#define IBERT_LNP2(V, D, F)                                                                                 \
   do {                                                                                                      \
     static bool attr_dev[kMaxDevices] = {false};                                                            \
     bool& attr = attr_dev[ctx->device % kMaxDevices];                                                       \
     if (!attr) {                                                                                            \
-      if (cudaFuncSetAttribute(layernorm_pipe_kernel<V, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
+      if (cudaFuncSetAttribute(layernorm_pipe_kernel<V, D, QT, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                100 * 1024) != cudaSuccess) return IBERT_ERR_CUDA;                           \
       attr = true;                                                                                          \
     }                                                                                                       \
-    if (int rc_ = launch_pdl(layernorm_pipe_kernel<V, D>, dim3(pgrid), dim3(kThreads), smem, ctx->stream, 1, q, r, \
+    if (int rc_ = launch_pdl(layernorm_pipe_kernel<V, D, QT, F>, dim3(pgrid), dim3(kThreads), smem, ctx->stream, 1, q, r, \
                              rows, k, d_b, d_B, out, ctx->d_status))                                        \
       return rc_;                                                                                           \
+  } while (0)
+#define IBERT_LNP(V, D)                       \
+  do {                                        \
+    if (k.C == 128 * V) IBERT_LNP2(V, D, true); \
+    else IBERT_LNP2(V, D, false);             \
   } while (0)
     if (k.C <= 256) IBERT_LNP(2, 2);
     else if (k.C <= 512) IBERT_LNP(4, 2);
     else if (k.C <= 768) IBERT_LNP(6, 2);
     else IBERT_LNP(8, 2);
 #undef IBERT_LNP
+#undef IBERT_LNP2
     return check_launch();
   }
 #define IBERT_LN(V)                                                                                              \
   do {                                                                                                           \
-    if (fast) layernorm_kernel<V, true, true><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);  \
-    else if (vec) layernorm_kernel<V, true, false><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out); \
-    else layernorm_kernel<V, false, false><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);     \
+    if (fast) layernorm_kernel<V, true, true, QT><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);  \
+    else if (vec) layernorm_kernel<V, true, false, QT><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out); \
+    else layernorm_kernel<V, false, false, QT><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);     \
   } while (0)
   if (vpl <= 2) IBERT_LN(2);
   else if (vpl <= 4) IBERT_LN(4);
@@ -618,6 +638,16 @@ int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t 
   else IBERT_LN(16);
 #undef IBERT_LN
   return check_launch();
+}
+
+int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t rows, const LnConsts& k,
+                     const int32_t* d_b, const int64_t* d_B, int8_t* out) {
+  return launch_layernorm_t<int32_t>(ctx, q, r, rows, k, d_b, d_B, out);
+}
+
+int launch_layernorm_i16(ibert_ctx* ctx, const int16_t* q, const int8_t* r, int64_t rows, const LnConsts& k,
+                         const int32_t* d_b, const int64_t* d_B, int8_t* out) {
+  return launch_layernorm_t<int16_t>(ctx, q, r, rows, k, d_b, d_B, out);
 }
 
 }  // namespace ibert

@@ -53,6 +53,36 @@ def test_linear_requantized(M, N, K, kind):
         assert np.abs(want.astype(np.int64)).max() <= qmax
 
 
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_linear_q16_stored_as_int16(M, N, K):
+    """out_kind 3: the Q16 values of out_kind 1 in an int16 container -- same oracle, narrower store.
+    A generic (not upper-word) multiplier set and a forced split-K width are covered as well."""
+    x, w, bias, S_w, S_x, amax = _problem(M, N, K, 5)
+    for S_out in (amax / 20000.0, amax / 2.0e9):          # a few values clamp / multipliers >= 1: generic form
+        out, S_ret = ctx().ibert_linear_i8(dev(x), S_x, dev(w), S_w, dev(bias), 3, S_out)
+        ctx().check()
+        assert S_ret == S_out and out.dtype == torch.int16
+        if M:
+            want = oracle.linear(x, S_x, w, S_w, bias, 1, S_out)
+            assert_same(host(out).astype(np.int32), want, f"kind 3, S_out={S_out}")
+    if M and K > 128:
+        ctx().ibert_set_split_k(2)
+        try:
+            out, _ = ctx().ibert_linear_i8(dev(x), S_x, dev(w), S_w, dev(bias), 3, amax / 20000.0)
+            ctx().check()
+        finally:
+            ctx().ibert_set_split_k(0)
+        assert_same(host(out).astype(np.int32), oracle.linear(x, S_x, w, S_w, bias, 1, amax / 20000.0), "kind 3, split K")
+
+
+def test_linear_int16_needs_rows_of_16_bytes():
+    from paper_2101_01321_b200.binding import IbertError
+    x, w, bias, S_w, S_x, amax = _problem(8, 20, 32, 6)
+    with pytest.raises(IbertError) as e:
+        ctx().ibert_linear_i8(dev(x), S_x, dev(w), S_w, dev(bias), 3, amax / 20000.0)
+    assert e.value.code == -2
+
+
 @pytest.mark.parametrize("M,N,K", [(7, 48, 80), (300, 768, 768), (257, 3072, 768), (1000, 4096, 1024), (2500, 3072, 768)])
 def test_linear_with_fused_gelu(M, N, K):
     x, w, bias, S_w, S_x, amax = _problem(M, N, K, 3)

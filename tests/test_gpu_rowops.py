@@ -100,6 +100,28 @@ def test_layernorm_matches_oracle(rows, C, residual):
             assert_same(host(out), want, f"layernorm C={C}")
 
 
+@pytest.mark.parametrize("rows,C", [(3, 8), (5, 17), (64, 768), (33, 1024), (4, 2047), (2, 1), (9, 260), (0, 768),
+                                    (7, 1536), (300, 512), (11, 774)])
+@pytest.mark.parametrize("residual", [True, False])
+def test_layernorm_on_int16_q16_matches_oracle(rows, C, residual):
+    """ibert_layernorm_i16: the same Q16 values in an int16 container (every kernel variant: streamed
+    rows, register rows with and without vector loads) against the same oracle."""
+    for sigma in (1.0, 4.0):
+        q, S, r, S_r, gamma, beta, S_out = synth.layernorm_inputs(max(rows, 1), C, sigma, with_residual=residual)
+        q = q[:rows]
+        r = None if r is None else r[:rows]
+        assert np.abs(q).max(initial=0) <= 32767
+        gamma = gamma.copy()
+        gamma[::7] *= -1.0
+        out, S_ret = ctx().ibert_layernorm_i(dev(q.astype(np.int16)), S, None if r is None else dev(r), S_r, gamma, beta,
+                                             S_out)
+        ctx().check()
+        assert S_ret == S_out
+        if rows:
+            want, _ = oracle.layernorm(q, S, r, S_r or 0.0, gamma, beta, S_out)
+            assert_same(host(out), want, f"layernorm int16 C={C}")
+
+
 def test_layernorm_degenerate_rows():
     C = 64
     q = np.zeros((6, C), dtype=np.int32)

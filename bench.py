@@ -248,9 +248,11 @@ def run_reference(args):
 
 
 def workload_config(cfg, batch, n_gpus, full_model=False, valid_frac=1.0, use_graph=False, pow2=False,
-                    scales="analytic"):
-    what = (f"token ids -> INT8 embedding + LayerNorm -> {cfg.layers} integer-only encoder layers with a "
-            f"key-padding mask ({100 * valid_frac:.0f} % of the positions valid) -> first-token classifier"
+                    scales="analytic", packed=False):
+    layout = (f"packed batch (no padding; the sentence-length mix fills {100 * valid_frac:.0f} % of B x L)" if packed else
+              f"key-padding mask ({100 * valid_frac:.0f} % of the positions valid)")
+    what = (f"token ids -> INT8 embedding + LayerNorm -> {cfg.layers} integer-only encoder layers, {layout} "
+            f"-> first-token classifier"
             if full_model else f"{cfg.layers}-layer integer-only encoder")
     scale_note = {"analytic": "closed-form static scales (int8 sites clip at 4-5 sigma, Q16 sites at 8 sigma)",
                   "calibrated": "static scales from each site's max|x| on the first sequences of the seeded input "
@@ -339,22 +341,35 @@ def run_ours(args):
         word_d, pos_d = torch.from_numpy(e["word"]).to(dev), torch.from_numpy(e["pos"]).to(dev)
         hw_d, hb_d = torch.from_numpy(hd["w"]).to(dev), torch.from_numpy(hd["bias"]).to(dev)
         lens_d = torch.from_numpy(m["lens"]).to(dev)
-        x_dev = torch.from_numpy(m["ids"]).to(dev)
-        x_pin = torch.from_numpy(m["ids"]).pin_memory()
+        valid_tokens = int(m["lens"].sum())
+        ids_np = m["ids"]
+        if args.packed:
+            # the same sequences without their padding: valid rows in sequence order + first-row offsets
+            keep = np.concatenate([np.arange(b * cfg.L, b * cfg.L + n) for b, n in enumerate(m["lens"])])
+            ids_np = np.ascontiguousarray(m["ids"][keep])
+            cu_d = torch.from_numpy(np.concatenate([[0], np.cumsum(m["lens"])]).astype(np.int32)).to(dev)
+            bufs = [torch.empty((valid_tokens, cfg.H), dtype=torch.int8, device=dev) for _ in range(2)]
+        x_dev = torch.from_numpy(ids_np).to(dev)
+        x_pin = torch.from_numpy(ids_np).pin_memory()
         x_stage = torch.empty_like(x_dev)
         logits = torch.empty((batch, synth.N_LABELS), dtype=torch.int32, device=dev)
         out_pin = torch.empty((batch, synth.N_LABELS), dtype=torch.int32).pin_memory()
-        emb_out = torch.empty((T, cfg.H), dtype=torch.int8, device=dev)
+        emb_out = torch.empty((x_dev.numel(), cfg.H), dtype=torch.int8, device=dev)
         S_last = m["layers"][-1]["S_out"]
-        valid_tokens = int(m["lens"].sum())
 
         def forward(src, eager=False, final_out=None):
+            dst = final_out if final_out is not None else logits
+            if args.packed:
+                h, _ = ctx.ibert_embedding_packed_i8(src, cu_d, cfg.L, word_d, e["S_word"], pos_d, e["S_pos"], e["gamma"],
+                                                     e["beta"], e["S_out"], out=emb_out)
+                for i, ly in enumerate(layers):
+                    h, _ = ctx.ibert_encoder_layer_packed(ly, h, cu_d, cfg.L, out=bufs[i & 1])
+                return ctx.ibert_classifier_packed_i8(h, cu_d, S_last, hw_d, hd["S_w"], hb_d, out=dst)[0]
             h, _ = ctx.ibert_embedding_i8(src, cfg.L, word_d, e["S_word"], pos_d, e["S_pos"], e["gamma"], e["beta"],
                                           e["S_out"], out=emb_out)
             for i, ly in enumerate(layers):
                 h, _ = ctx.ibert_encoder_layer_masked(ly, h, batch, cfg.L, lens_d, out=bufs[i & 1])
-            out, _ = ctx.ibert_classifier_i8(h, batch, cfg.L, S_last, hw_d, hd["S_w"], hb_d,
-                                             out=final_out if final_out is not None else logits)
+            out, _ = ctx.ibert_classifier_i8(h, batch, cfg.L, S_last, hw_d, hd["S_w"], hb_d, out=dst)
             return out
 
     def barrier():
@@ -478,7 +493,8 @@ def run_ours(args):
         sus_ms = dp.max_over_ranks([sus_ms], device=dev)[0]
         ms_step = sus_ms / n_sus
         mhz = sus_clocks.get("sm_mhz")
-        sustained = {"value": T * n_sus * world / (sus_ms / 1e3), "unit": UNIT, "steps": n_sus,
+        n_computed = valid_tokens if (full_model and args.packed) else T
+        sustained = {"value": n_computed * n_sus * world / (sus_ms / 1e3), "unit": UNIT, "steps": n_sus,
                      "seconds": sus_ms / 1e3, "ms_per_step": ms_step, "clocks": sus_clocks,
                      "ms_per_step_at_max_clock": (ms_step * mhz / SPEC_SM_MHZ) if mhz else None,
                      "how": "steps enqueued back to back without L2 flushes, one host synchronization every "
@@ -493,7 +509,9 @@ def run_ours(args):
         figures = ncu_figures()
         n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
         sm_mhz_max = clocks.get("sm_max_mhz") or SPEC_SM_MHZ
-        work = algorithmic_work(cfg.H, cfg.F, cfg.L, cfg.heads, T)
+        # padded batches: every position is computed and counted; packed batches: only real tokens exist
+        computed = valid_tokens if (full_model and args.packed) else T
+        work = algorithmic_work(cfg.H, cfg.F, cfg.L, cfg.heads, computed)
         # Peaks.  A kernel timed by an event pair inside a step of a few milliseconds runs at burst
         # clocks, so the tensor peak is 2 x the BURST bf16 cuBLAS rate (int8 : bf16 dense = 2 nominal).
         int8_peak = 2.0 * peaks["bf16_tflops"]
@@ -557,7 +575,7 @@ def run_ours(args):
         roof["traffic"] = fig["dram_bytes"] if fig else None
         roof["traffic_unit"] = ("bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum, "
                                 "profiles/ncu_figures.md)")
-        tokens = T * args.steps * world          # padded positions count: every one of them is computed
+        tokens = computed * args.steps * world
         value = tokens / (total_ms / 1e3)
         e2e_value = tokens / (total_e2e_ms / 1e3)
 
@@ -592,7 +610,8 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": workload_config(cfg, batch, world, full_model, valid_tokens / T,
-                                      args.graph and not full_model, args.pow2_scores and not full_model, args.scales),
+                                      args.graph and not full_model, args.pow2_scores and not full_model, args.scales,
+                                      full_model and args.packed),
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_pin.numel() * x_pin.element_size(),
                     "d2h_bytes_per_step": out_pin.numel() * out_pin.element_size(),
@@ -603,6 +622,7 @@ def run_ours(args):
             "gpu_launches": sum(v["launches_per_step"] for v in kern.values()) * args.steps,
             "roofline": roof,
             "sustained": sustained,
+            "valid_tokens_per_s": valid_tokens * args.steps * world / (total_ms / 1e3),
             "parity": parity,
             "kernels": kern,
             "cpu_baseline": cpu,
@@ -761,6 +781,9 @@ def main():
     ap.add_argument("--workload", choices=["layers", "model"], default="layers",
                     help="layers: the encoder layers on full-length sequences (headline); model: token ids -> "
                          "embedding -> layers with a key-padding mask on a sentence-length mix -> classifier")
+    ap.add_argument("--packed", action="store_true",
+                    help="model workload: the same sentence-length mix stored without padding (cu_seqlens); "
+                         "tokens/s then counts real tokens only")
     ap.add_argument("--only", default="", help="run one kernel class alone (profiling aid)")
     ap.add_argument("--sustain", type=float, default=3.0,
                     help="seconds of back-to-back steps for the sustained-clock leg (0 = skip)")

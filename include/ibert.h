@@ -254,6 +254,35 @@ int ibert_embedding_i8(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, con
 int ibert_classifier_i8(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, double S_x, const int8_t* w,
                         const double* S_w, const int32_t* bias, int N, int32_t* logits, double* S_ret);
 
+/* ---- packed batches: sequences of different lengths without padding ------------------------------
+   The paper's workloads are sentence batches (GLUE), i.e. sequences of different lengths; it does
+   not treat their layout.  Here a batch may be given PACKED: all tokens of all sequences in one
+   [total_tokens, .] tensor, sequence b in rows cu_seqlens[b] .. cu_seqlens[b+1]-1 (cu_seqlens:
+   device int32 [B + 1], non-decreasing, cu_seqlens[0] = 0, cu_seqlens[B] = total_tokens, every
+   length at most max_len <= 512; total_tokens is passed on the host because it sizes the launches).
+   Linear layers, i-GELU and i-LayerNorm are per token and simply run on total_tokens rows;
+   attention (i-softmax, Algorithm 3) runs per sequence over its own rows.  The result for a
+   sequence is the one ibert_encoder_layer_masked gives on its valid rows -- padding positions
+   cost nothing instead of being computed and discarded.  A length above max_len records
+   IBERT_ERR_VALUE_RANGE in the context's status (that sequence's surplus rows are not written).
+   ibert_attention_packed_i8 returns IBERT_ERR_SCALE_RANGE for score scales so coarse that
+   floor(ln2 / (S_q S_k / 8)) <= 2 (use the padded call there). */
+int ibert_attention_packed_i8(ibert_ctx* ctx, const int8_t* qkv, const int32_t* cu_seqlens, int B, int max_len,
+                              int64_t total_tokens, int H, int heads, double S_q, double S_k, double S_v,
+                              double S_ctx, int p_max, int8_t* out, double* S_ret);
+int ibert_encoder_layer_packed(ibert_ctx* ctx, const ibert_layer* layer, const int8_t* x, const int32_t* cu_seqlens,
+                               int B, int max_len, int64_t total_tokens, int8_t* out, double* S_ret);
+/* ibert_embedding_i8 on a packed batch: the position of a token is its distance from the first row
+   of its sequence (P >= max_len).  ibert_classifier_i8 on a packed batch: the first token of
+   sequence b is row cu_seqlens[b] (every sequence must have at least one token). */
+int ibert_embedding_packed_i8(ibert_ctx* ctx, const int32_t* ids, const int32_t* cu_seqlens, int B, int max_len,
+                              int64_t total_tokens, const int8_t* word, int64_t V, double S_word, const int8_t* pos,
+                              int64_t P, double S_pos, const double* gamma, const double* beta, int H, double S_out,
+                              int8_t* out, double* S_ret);
+int ibert_classifier_packed_i8(ibert_ctx* ctx, const int8_t* x, const int32_t* cu_seqlens, int B, int H, double S_x,
+                               const int8_t* w, const double* S_w, const int32_t* bias, int N, int32_t* logits,
+                               double* S_ret);
+
 /* ---- h-GELU, the comparison function of the paper (Eq. 6; Table 1, Table 3) --------------------
    h-GELU(x) = x ReLU6(1.702 x + 3) / 6.  The paper notes that it can be computed with integers
    but gives no integer algorithm; this library's reading keeps it parallel to i-GELU: the same

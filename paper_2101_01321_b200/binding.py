@@ -74,6 +74,13 @@ def lib():
         L.ibert_encoder_layer_masked.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
         L.ibert_embedding_i8.argtypes = [vp, vp, i64, i32, vp, i64, dbl, vp, i64, dbl, vp, vp, i32, dbl, vp, vp]
         L.ibert_classifier_i8.argtypes = [vp, vp, i32, i32, i32, dbl, vp, vp, vp, i32, vp, vp]
+        L.ibert_attention_packed_i8.argtypes = [vp, vp, vp, i32, i32, i64, i32, i32, dbl, dbl, dbl, dbl, i32, vp, vp]
+        L.ibert_encoder_layer_packed.argtypes = [vp, vp, vp, vp, i32, i32, i64, vp, vp]
+        L.ibert_embedding_packed_i8.argtypes = [vp, vp, vp, i32, i32, i64, vp, i64, dbl, vp, i64, dbl, vp, vp, i32, dbl, vp, vp]
+        L.ibert_classifier_packed_i8.argtypes = [vp, vp, vp, i32, i32, dbl, vp, vp, vp, i32, vp, vp]
+        for name in ("ibert_attention_packed_i8", "ibert_encoder_layer_packed", "ibert_embedding_packed_i8",
+                     "ibert_classifier_packed_i8"):
+            getattr(L, name).restype = i32
         L.ibert_encoder_graph_create.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp, C.POINTER(vp)]
         L.ibert_encoder_graph_launch.argtypes = [vp, vp]
         L.ibert_encoder_graph_destroy.argtypes = [vp]
@@ -377,6 +384,63 @@ class Context:
         _chk(lib().ibert_classifier_i8(self.h, _dev(x, torch.int8), B, L, H, S_x, _dev(w, torch.int8), sw.ctypes.data,
                                        _dev(bias, torch.int32), N, _dev(out, torch.int32), S_ret.ctypes.data),
              "ibert_classifier_i8")
+        return out, S_ret
+
+    # ------------------------------------------------------------------ packed batches
+    def ibert_attention_packed_i8(self, qkv: torch.Tensor, cu_seqlens: torch.Tensor, max_len: int, H: int, heads: int,
+                                  S_q: float, S_k: float, S_v: float, S_ctx: float, p_max: int = 255,
+                                  out: torch.Tensor | None = None):
+        """Attention on a packed batch; ``cu_seqlens``: device int32 [B + 1], first rows of the sequences."""
+        B = cu_seqlens.numel() - 1
+        total = qkv.numel() // (3 * H)
+        if out is None:
+            out = torch.empty((total, H), dtype=torch.int8, device=qkv.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_attention_packed_i8(self.h, _dev(qkv, torch.int8), _dev(cu_seqlens, torch.int32), B, max_len,
+                                             total, H, heads, S_q, S_k, S_v, S_ctx, p_max, _dev(out, torch.int8),
+                                             C.byref(S_ret)), "ibert_attention_packed_i8")
+        return out, S_ret.value
+
+    def ibert_encoder_layer_packed(self, layer: "Layer", x: torch.Tensor, cu_seqlens: torch.Tensor, max_len: int,
+                                   out: torch.Tensor | None = None):
+        """The encoder layer on a packed batch [total tokens, H]."""
+        B = cu_seqlens.numel() - 1
+        total = x.numel() // layer.H
+        if out is None:
+            out = torch.empty((total, layer.H), dtype=torch.int8, device=x.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_encoder_layer_packed(self.h, layer.h, _dev(x, torch.int8), _dev(cu_seqlens, torch.int32), B,
+                                              max_len, total, _dev(out, torch.int8), C.byref(S_ret)),
+             "ibert_encoder_layer_packed")
+        return out, S_ret.value
+
+    def ibert_embedding_packed_i8(self, ids: torch.Tensor, cu_seqlens: torch.Tensor, max_len: int, word: torch.Tensor,
+                                  S_word: float, pos: torch.Tensor, S_pos: float, gamma, beta, S_out: float,
+                                  out: torch.Tensor | None = None):
+        T = ids.numel()
+        B = cu_seqlens.numel() - 1
+        V, H = word.shape
+        g, b = _host(gamma, np.float64), _host(beta, np.float64)
+        if out is None:
+            out = torch.empty((T, H), dtype=torch.int8, device=word.device)
+        S_ret = C.c_double()
+        _chk(lib().ibert_embedding_packed_i8(self.h, _dev(ids, torch.int32), _dev(cu_seqlens, torch.int32), B, max_len, T,
+                                             _dev(word, torch.int8), V, S_word, _dev(pos, torch.int8), pos.shape[0],
+                                             S_pos, g.ctypes.data, b.ctypes.data, H, S_out, _dev(out, torch.int8),
+                                             C.byref(S_ret)), "ibert_embedding_packed_i8")
+        return out, S_ret.value
+
+    def ibert_classifier_packed_i8(self, x: torch.Tensor, cu_seqlens: torch.Tensor, S_x: float, w: torch.Tensor, S_w,
+                                   bias: torch.Tensor | None, out: torch.Tensor | None = None):
+        N, H = w.shape
+        B = cu_seqlens.numel() - 1
+        sw = _host(S_w, np.float64)
+        if out is None:
+            out = torch.empty((B, N), dtype=torch.int32, device=x.device)
+        S_ret = np.zeros(N, dtype=np.float64)
+        _chk(lib().ibert_classifier_packed_i8(self.h, _dev(x, torch.int8), _dev(cu_seqlens, torch.int32), B, H, S_x,
+                                              _dev(w, torch.int8), sw.ctypes.data, _dev(bias, torch.int32), N,
+                                              _dev(out, torch.int32), S_ret.ctypes.data), "ibert_classifier_packed_i8")
         return out, S_ret
 
     # ------------------------------------------------------------------ encoder layer

@@ -726,12 +726,16 @@ static size_t layer_workspace_bytes(int H, int F, int64_t T) {
          up256((size_t)T * F);
 }
 
+// cu_seqlens != nullptr: packed batch of `total` rows (sequence b = rows cu_seqlens[b] .. cu_seqlens[b+1]-1,
+// at most L each); otherwise B padded sequences of L rows
 static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, int B, int L,
-                                const int32_t* lens, int8_t* out, double* S_ret) {
+                                const int32_t* lens, int8_t* out, double* S_ret, const int32_t* cu_seqlens = nullptr,
+                                int64_t total = 0) {
   if (!ctx || !ly || ly->ctx != ctx || B < 0) return IBERT_ERR_ARG;
   if (L < 1 || L > 512) return IBERT_ERR_SHAPE;
   const int H = ly->d.H, F = ly->d.F;
-  const int64_t T = (int64_t)B * L;
+  if (cu_seqlens && (total < 0 || total > (int64_t)B * L || total >= (int64_t(1) << 31) - 256)) return IBERT_ERR_SHAPE;
+  const int64_t T = cu_seqlens ? total : (int64_t)B * L;
   if (T > 0 && (!x || !out)) return IBERT_ERR_ARG;
   if (!aligned16(x) || !aligned16(out)) return IBERT_ERR_ALIGN;
   if (S_ret) *S_ret = ly->d.S_out;
@@ -758,7 +762,7 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
   e.kind = EPI_INT8; e.d_b = ly->b_qkv; e.d_c = ly->c_qkv; e.d_bias = ly->bias_qkv; e.fast = ly->fast_qkv;
   { ProfileScope ps(ctx, IBERT_K_GEMM_QKV); rc = launch_gemm_i8(ctx, x, ly->w_qkv, T, 3 * H, H, e, qkv); }
   if (rc) return rc;
-  { ProfileScope ps(ctx, IBERT_K_ATTENTION); rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, lens, cx); }
+  { ProfileScope ps(ctx, IBERT_K_ATTENTION); rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, lens, cx, cu_seqlens, T); }
   if (rc) return rc;
   // output projection + residual + LayerNorm: one kernel when shapes and constants allow it
   e.kind = EPI_Q16; e.d_b = ly->b_o; e.d_c = ly->c_o; e.d_bias = ly->bias_o; e.fast = ly->fast_o;
@@ -805,10 +809,64 @@ int ibert_encoder_layer_masked(ibert_ctx* ctx, const ibert_layer* ly, const int8
   });
 }
 
+int ibert_encoder_layer_packed(ibert_ctx* ctx, const ibert_layer* ly, const int8_t* x, const int32_t* cu_seqlens,
+                               int B, int max_len, int64_t total_tokens, int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
+  if (B > 0 && !cu_seqlens) return IBERT_ERR_ARG;
+  if (B == 0 && total_tokens != 0) return IBERT_ERR_ARG;
+  return encoder_layer_common(ctx, ly, x, B, max_len, nullptr, out, S_ret, cu_seqlens, total_tokens);
+  });
+}
+
+int ibert_attention_packed_i8(ibert_ctx* ctx, const int8_t* qkv, const int32_t* cu_seqlens, int B, int max_len,
+                              int64_t total_tokens, int H, int heads, double S_q, double S_k, double S_v,
+                              double S_ctx, int p_max, int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
+  if (!ctx || B < 0 || (B > 0 && !cu_seqlens)) return IBERT_ERR_ARG;
+  if (heads < 1 || H != heads * 64 || max_len < 1 || max_len > 512) return IBERT_ERR_SHAPE;
+  if (total_tokens < 0 || total_tokens > (int64_t)B * max_len || total_tokens >= (int64_t(1) << 31) - 256) return IBERT_ERR_SHAPE;
+  if (total_tokens > 0 && (!qkv || !out)) return IBERT_ERR_ARG;
+  if (!aligned16(qkv) || !aligned16(out)) return IBERT_ERR_ALIGN;
+  AttnConsts k{};
+  int rc = make_attn_consts(S_q, S_k, S_v, S_ctx, p_max, &k);
+  if (rc) return rc;
+  if (S_ret) *S_ret = S_ctx;
+  if (total_tokens == 0) return IBERT_OK;
+  DeviceGuard guard(ctx->device);
+  ProfileScope ps(ctx, IBERT_K_ATTENTION);
+  return launch_attention(ctx, qkv, B, max_len, H, heads, k, nullptr, out, cu_seqlens, total_tokens);
+  });
+}
+
+static int embedding_common(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
+                            double S_word, const int8_t* pos, int64_t P, double S_pos, const double* gamma,
+                            const double* beta, int H, double S_out, int8_t* out, double* S_ret,
+                            const int32_t* cu_seqlens, int B);
+
 int ibert_embedding_i8(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
                        double S_word, const int8_t* pos, int64_t P, double S_pos, const double* gamma,
                        const double* beta, int H, double S_out, int8_t* out, double* S_ret) {
   return guarded([&]() -> int {
+  return embedding_common(ctx, ids, T, L, word, V, S_word, pos, P, S_pos, gamma, beta, H, S_out, out, S_ret, nullptr, 0);
+  });
+}
+
+int ibert_embedding_packed_i8(ibert_ctx* ctx, const int32_t* ids, const int32_t* cu_seqlens, int B, int max_len,
+                              int64_t total_tokens, const int8_t* word, int64_t V, double S_word, const int8_t* pos,
+                              int64_t P, double S_pos, const double* gamma, const double* beta, int H, double S_out,
+                              int8_t* out, double* S_ret) {
+  return guarded([&]() -> int {
+  if (B < 0 || (B > 0 && !cu_seqlens) || (B == 0 && total_tokens != 0)) return IBERT_ERR_ARG;
+  if (total_tokens > (int64_t)B * max_len) return IBERT_ERR_SHAPE;
+  return embedding_common(ctx, ids, total_tokens, max_len, word, V, S_word, pos, P, S_pos, gamma, beta, H, S_out, out,
+                          S_ret, cu_seqlens, B);
+  });
+}
+
+static int embedding_common(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
+                            double S_word, const int8_t* pos, int64_t P, double S_pos, const double* gamma,
+                            const double* beta, int H, double S_out, int8_t* out, double* S_ret,
+                            const int32_t* cu_seqlens, int B) {
   if (!ctx || T < 0 || !gamma || !beta || !word || !pos) return IBERT_ERR_ARG;
   if (L < 1 || H < 1 || H > 2047 || H % 16 != 0 || V < 1 || P < L) return IBERT_ERR_SHAPE;
   if (T > 0 && (!ids || !out)) return IBERT_ERR_ARG;
@@ -835,15 +893,34 @@ int ibert_embedding_i8(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, con
   if ((rc = ensure_workspace(ctx, q_bytes + (size_t)T * H + 256))) return rc;
   int32_t* q = static_cast<int32_t*>(ctx->ws);
   int8_t* r = reinterpret_cast<int8_t*>(static_cast<char*>(ctx->ws) + q_bytes);
-  if ((rc = launch_embed_gather(ctx, ids, T, L, word, V, pos, H, q, r))) return rc;
+  if ((rc = launch_embed_gather(ctx, ids, T, L, word, V, pos, H, q, r, cu_seqlens, B))) return rc;
   ProfileScope ps(ctx, IBERT_K_LAYERNORM);
   return launch_layernorm(ctx, q, r, T, k, (const int32_t*)d_b, (const int64_t*)d_B, out);
-  });
 }
+
+static int classifier_common(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, double S_x, const int8_t* w,
+                             const double* S_w, const int32_t* bias, int N, int32_t* logits, double* S_ret,
+                             const int32_t* cu_seqlens);
 
 int ibert_classifier_i8(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, double S_x, const int8_t* w,
                         const double* S_w, const int32_t* bias, int N, int32_t* logits, double* S_ret) {
   return guarded([&]() -> int {
+  return classifier_common(ctx, x, B, L, H, S_x, w, S_w, bias, N, logits, S_ret, nullptr);
+  });
+}
+
+int ibert_classifier_packed_i8(ibert_ctx* ctx, const int8_t* x, const int32_t* cu_seqlens, int B, int H, double S_x,
+                               const int8_t* w, const double* S_w, const int32_t* bias, int N, int32_t* logits,
+                               double* S_ret) {
+  return guarded([&]() -> int {
+  if (B > 0 && !cu_seqlens) return IBERT_ERR_ARG;
+  return classifier_common(ctx, x, B, 1, H, S_x, w, S_w, bias, N, logits, S_ret, cu_seqlens);
+  });
+}
+
+static int classifier_common(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, double S_x, const int8_t* w,
+                             const double* S_w, const int32_t* bias, int N, int32_t* logits, double* S_ret,
+                             const int32_t* cu_seqlens) {
   if (!ctx || B < 0 || !S_w || !w) return IBERT_ERR_ARG;
   if (L < 1 || H < 1 || H % 16 != 0 || N < 1 || N % 4 != 0) return IBERT_ERR_SHAPE;
   if ((int64_t)H * 127 * 127 >= (int64_t(1) << 31)) return IBERT_ERR_SHAPE;
@@ -858,15 +935,16 @@ int ibert_classifier_i8(ibert_ctx* ctx, const int8_t* x, int B, int L, int H, do
   int rc = ensure_workspace(ctx, (size_t)B * H + 256);
   if (rc) return rc;
   int8_t* first = static_cast<int8_t*>(ctx->ws);
-  // first token of every sequence: B rows of H bytes, L*H bytes apart
-  if (cudaMemcpy2DAsync(first, (size_t)H, x, (size_t)L * H, (size_t)H, (size_t)B, cudaMemcpyDeviceToDevice,
-                        ctx->stream) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_CUDA; }
+  // first token of every sequence: B rows of H bytes, L*H bytes apart (packed: row cu_seqlens[b])
+  if (cu_seqlens) {
+    if ((rc = launch_gather_first_rows(ctx, x, cu_seqlens, B, H, first))) return rc;
+  } else if (cudaMemcpy2DAsync(first, (size_t)H, x, (size_t)L * H, (size_t)H, (size_t)B, cudaMemcpyDeviceToDevice,
+                               ctx->stream) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_CUDA; }
   GemmEpilogue epi{};
   epi.kind = EPI_RAW;
   epi.d_bias = bias;
   ProfileScope ps(ctx, gemm_class(EPI_RAW, H));
   return launch_gemm_i8(ctx, first, w, B, N, H, epi, logits);
-  });
 }
 
 // --------------------------------------------------------------------------- captured forward pass

@@ -141,8 +141,12 @@ int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const 
 int launch_exp_table(ibert_ctx* ctx, const ExpConsts& k, uint32_t* table);
 // rows of the word table (as int32) and of the position table (token t: position t mod L) gathered
 // into q [T, H] and r [T, H]; an id outside [0, V) records IBERT_ERR_VALUE_RANGE and reads row 0
+// (cu_seqlens != null: packed batch of B sequences, position = distance from the sequence's first row)
 int launch_embed_gather(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
-                        const int8_t* pos, int H, int32_t* q, int8_t* r);
+                        const int8_t* pos, int H, int32_t* q, int8_t* r, const int32_t* cu_seqlens = nullptr,
+                        int B = 0);
+// out[b, :] = x[cu_seqlens[b], :] for b < B (first token of every sequence of a packed batch)
+int launch_gather_first_rows(ibert_ctx* ctx, const int8_t* x, const int32_t* cu_seqlens, int B, int H, int8_t* out);
 int launch_layernorm(ibert_ctx* ctx, const int32_t* q, const int8_t* r, int64_t rows, const LnConsts& k,
                      const int32_t* d_b, const int64_t* d_B, int8_t* out);
 // the same with the Q16 input stored as int16 (values identical, 2 bytes per element less traffic)
@@ -219,7 +223,10 @@ int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t 
 
 // `lens` (device, [B], may be null): valid keys per sequence -- keys beyond take no part in the
 // softmax and get probability 0 (key-padding mask)
+// `cu_seqlens` (device, [B + 1], may be null): packed batch -- qkv and out are [total_rows, .] without
+// padding, sequence b occupies rows cu_seqlens[b] .. cu_seqlens[b+1]-1 (at most L); lens is ignored
 int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
-                     const AttnConsts& k, const int32_t* lens, int8_t* out);
+                     const AttnConsts& k, const int32_t* lens, int8_t* out, const int32_t* cu_seqlens = nullptr,
+                     int64_t total_rows = 0);
 
 }  // namespace ibert

@@ -465,11 +465,14 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
 
 // ----------------------------------------------------------------------------- embedding gather
 // One warp per token: 16 bytes of the word row and of the position row per lane and step.
+// Packed batches (cu != nullptr: [B + 1] first rows of the sequences): the position of token t is
+// its distance from the first row of its sequence, found by bisection; a position beyond the
+// position table (a sequence longer than the stated maximum) records IBERT_ERR_VALUE_RANGE.
 __global__ void __launch_bounds__(kThreads) embed_gather_kernel(const int32_t* __restrict__ ids, int64_t T, int L,
                                                                 const int8_t* __restrict__ word, int64_t V,
                                                                 const int8_t* __restrict__ pos, int H,
                                                                 int32_t* __restrict__ q, int8_t* __restrict__ r,
-                                                                int32_t* status) {
+                                                                int32_t* status, const int32_t* __restrict__ cu, int B) {
   const int lane = threadIdx.x & 31;
   const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
   const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
@@ -479,8 +482,21 @@ __global__ void __launch_bounds__(kThreads) embed_gather_kernel(const int32_t* _
       if (lane == 0) atomicCAS(status, 0, IBERT_ERR_VALUE_RANGE);
       id = 0;
     }
+    int64_t p = t % L;
+    if (cu) {
+      int lo = 0, hi = B;                    // the last sequence whose first row is <= t
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((int64_t)__ldg(cu + mid) <= t) lo = mid; else hi = mid;
+      }
+      p = t - (int64_t)__ldg(cu + lo);
+      if (p >= L) {
+        if (lane == 0) atomicCAS(status, 0, IBERT_ERR_VALUE_RANGE);
+        p = L - 1;
+      }
+    }
     const int8_t* wrow = word + id * H;
-    const int8_t* prow = pos + (t % L) * H;
+    const int8_t* prow = pos + p * H;
     for (int c = lane * 16; c < H; c += 512) {
       const uint4 wv = __ldg(reinterpret_cast<const uint4*>(wrow + c));
       const uint4 pv = __ldg(reinterpret_cast<const uint4*>(prow + c));
@@ -510,6 +526,17 @@ __global__ void __launch_bounds__(32) wait_timeout_kernel(uint64_t limit_ns, int
   if (!ok && threadIdx.x == 0) atomicCAS(status, 0, IBERT_ERR_TIMEOUT);
 }
 
+// Row cu[b] of x (the first token of sequence b of a packed batch) -> row b of out; one warp per row.
+__global__ void __launch_bounds__(kThreads) gather_first_rows_kernel(const int8_t* __restrict__ x, const int32_t* __restrict__ cu,
+                                                                     int B, int H, int8_t* __restrict__ out) {
+  const int lane = threadIdx.x & 31;
+  const int b = (int)(((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5);
+  if (b >= B) return;
+  const int8_t* src = x + (int64_t)__ldg(cu + b) * H;
+  for (int c = lane * 16; c < H; c += 512)
+    *reinterpret_cast<uint4*>(out + (int64_t)b * H + c) = __ldg(reinterpret_cast<const uint4*>(src + c));
+}
+
 int grid_for(ibert_ctx* ctx, int64_t work_warps, int max_ctas_per_sm) {
   const int64_t ctas = (work_warps + (kThreads / 32) - 1) / (kThreads / 32);
   const int64_t cap = (int64_t)ctx->num_sms * max_ctas_per_sm;
@@ -526,10 +553,16 @@ int launch_wait_timeout(ibert_ctx* ctx, uint64_t limit_ns) {
 }
 
 int launch_embed_gather(ibert_ctx* ctx, const int32_t* ids, int64_t T, int L, const int8_t* word, int64_t V,
-                        const int8_t* pos, int H, int32_t* q, int8_t* r) {
+                        const int8_t* pos, int H, int32_t* q, int8_t* r, const int32_t* cu_seqlens, int B) {
   if (T == 0) return IBERT_OK;
   embed_gather_kernel<<<grid_for(ctx, T, 8), kThreads, 0, ctx->stream>>>(ids, T, L, word, V, pos, H, q, r,
-                                                                          ctx->d_status);
+                                                                          ctx->d_status, cu_seqlens, B);
+  return check_launch();
+}
+
+int launch_gather_first_rows(ibert_ctx* ctx, const int8_t* x, const int32_t* cu_seqlens, int B, int H, int8_t* out) {
+  if (B == 0) return IBERT_OK;
+  gather_first_rows_kernel<<<(B + kThreads / 32 - 1) / (kThreads / 32), kThreads, 0, ctx->stream>>>(x, cu_seqlens, B, H, out);
   return check_launch();
 }
 

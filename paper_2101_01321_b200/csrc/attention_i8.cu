@@ -336,14 +336,17 @@ struct AttnArgs {
   int q_bufs;        // 2 when a pair has several query tiles (next tile's Q prefetched), else 1
   uint32_t tmem_cols;
   AttnConsts k;
-  const int32_t* lens;   // [B] valid keys per sequence, or nullptr: all L
-  // packed batches: [B + 1] first rows of the sequences in a [total tokens, 3H] tensor without
-  // padding (sequence b = rows cu[b] .. cu[b+1]-1, at most L of them), or nullptr: padded [B, L]
-  const int32_t* cu;
+  // padded batches: [B] valid keys per sequence, or nullptr: all L.  Packed batches (the PACKED
+  // instantiation of the kernel): [B + 1] first rows of the sequences in a [total tokens, 3H] tensor
+  // without padding -- sequence b = rows lens[b] .. lens[b+1]-1, at most L of them.  (One field for
+  // both: the size of this argument block is part of what the compiler's schedule hangs on.)
+  const int32_t* lens;
   int8_t* out;
   int32_t* status;
 };
 
+// PACKED: a.lens holds first-row offsets (a separate instantiation: the padded path compiles as without it)
+template <bool PACKED>
 __global__ void __launch_bounds__(kMaxThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_constant__ CUtensorMap map_v,
                  const AttnArgs a) {
@@ -366,7 +369,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
   const int n_threads = blockDim.x;
   const int quad = warp & 3, grp = warp >> 2, G = a.groups;
   const int row = quad * 32 + lane;                            // query row inside the tile = TMEM lane
-  const int L = a.L;
+  const int L = a.L, q_tiles_padded = a.n_slabs;
   const int total = a.B * a.heads;
 
   if (tid == 0) {
@@ -395,20 +398,20 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
   // rows loaded past its end -- the next sequence's, or zero fill past the last row -- are masked)
   auto load_q = [&](int item, int qt, int buf) {
     const int head = item % a.heads, batch = item / a.heads;
-    const int row0 = a.cu ? __ldg(a.cu + batch) : 0, zb = a.cu ? 0 : batch;
+    const int row0 = PACKED ? __ldg(a.lens + batch) : 0, zb = PACKED ? 0 : batch;
     ptx::mbar_arrive_expect_tx(bar_q0 + 8 * buf, (uint32_t)slab_bytes);
     ptx::tma_load_3d(ptx::smem_addr(sQ + buf * slab_bytes), &map_qk, bar_q0 + 8 * buf, head * kHeadDim, row0 + qt * 128, zb);
   };
   auto load_k = [&](int item) {
     const int head = item % a.heads, batch = item / a.heads;
-    const int row0 = a.cu ? __ldg(a.cu + batch) : 0, zb = a.cu ? 0 : batch;
+    const int row0 = PACKED ? __ldg(a.lens + batch) : 0, zb = PACKED ? 0 : batch;
     ptx::mbar_arrive_expect_tx(bar_k, (uint32_t)(a.n_slabs * slab_bytes));
     for (int s = 0; s < a.n_slabs; ++s)
       ptx::tma_load_3d(ptx::smem_addr(sK + s * slab_bytes), &map_qk, bar_k, a.H + head * kHeadDim, row0 + s * 128, zb);
   };
   auto load_v = [&](int item) {
     const int head = item % a.heads, batch = item / a.heads;
-    const int row0 = a.cu ? __ldg(a.cu + batch) : 0, zb = a.cu ? 0 : batch;
+    const int row0 = PACKED ? __ldg(a.lens + batch) : 0, zb = PACKED ? 0 : batch;
     ptx::mbar_arrive_expect_tx(bar_v, (uint32_t)(a.n_slabs * slab_bytes));
     for (int s = 0; s < a.n_slabs; ++s)
       ptx::tma_load_3d(ptx::smem_addr(sVs + s * slab_bytes), &map_v, bar_v, 2 * a.H + head * kHeadDim, row0 + s * 128, zb);
@@ -430,13 +433,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
     // valid keys of this sequence (key-padding mask): keys >= n take no part in max or sum and get
     // probability 0; the MMAs and the softmax only cover the 32-column chunks that hold valid keys
     // (at least one chunk, so that a sequence without valid keys yields P = 0 and context 0)
-    const int row0 = a.cu ? __ldg(a.cu + batch) : batch * L;     // first output row of this sequence
-    const int len = a.cu ? __ldg(a.cu + batch + 1) - row0 : (a.lens ? __ldg(a.lens + batch) : L);
-    if (a.cu && len > L && tid == 0) atomicCAS(a.status, 0, IBERT_ERR_VALUE_RANGE);   // longer than the stated maximum
-    const int n = min(max(len, 0), L);
+    const int row0 = PACKED ? __ldg(a.lens + batch) : 0;           // packed: first row of this sequence
+    const int len = PACKED ? __ldg(a.lens + batch + 1) - row0 : 0;
+    if (PACKED && len > L && tid == 0) atomicCAS(a.status, 0, IBERT_ERR_VALUE_RANGE);   // longer than the stated maximum
+    const int n = PACKED ? min(max(len, 0), L) : (a.lens ? min(max(__ldg(a.lens + batch), 0), L) : L);
     // query rows: all L of a padded sequence, only the existing ones of a packed one
-    const int q_rows = a.cu ? n : L;
-    const int q_tiles = a.cu ? max((n + 127) >> 7, 1) : a.n_slabs;
+    const int q_tiles = PACKED ? max((n + 127) >> 7, 1) : q_tiles_padded;
     const int Lp = max((n + 31) & ~31, 32);
     const int n_chunks = Lp >> 5, per_grp = (n_chunks + G - 1) / G;
     const int c_begin = min(grp * per_grp, n_chunks) * 32, c_end = min((grp + 1) * per_grp, n_chunks) * 32;
@@ -615,7 +617,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
         const int64_t half = rounding_half(a.k.c);
         const int q_row = qt * 128 + row;
         for (int part = grp; part < 2; part += G) {
-          int8_t* orow = a.out + ((int64_t)row0 + q_row) * a.H + head * kHeadDim + part * 32;
+          int8_t* orow = a.out + (PACKED ? (int64_t)row0 + q_row : (int64_t)batch * L + q_row) * a.H + head * kHeadDim + part * 32;
           uint32_t v[32];
           ptx::tmem_ld32(t_row + part * 32, v);
           ptx::tmem_wait_ld();
@@ -637,7 +639,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
                                     requant_add((int32_t)v[j + 3], a.k.b, half, a.k.c, 127));
               }
             }
-            if (q_row < q_rows) *reinterpret_cast<uint4*>(orow + h * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            if (q_row < (PACKED ? n : L)) *reinterpret_cast<uint4*>(orow + h * 16) = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
       }
@@ -690,7 +692,7 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
       a.groups = std::min(std::max(n_slabs, g), std::max(Lp / 32, n_slabs));
     }
     a.q_bufs = n_slabs > 1 ? 2 : 1;
-    a.tmem_cols = cols; a.k = k; a.lens = lens; a.cu = cu_seqlens; a.out = out; a.status = ctx->d_status;
+    a.tmem_cols = cols; a.k = k; a.lens = cu_seqlens ? cu_seqlens : lens; a.out = out; a.status = ctx->d_status;
     const int smem = a.q_bufs * slab + 3 * n_slabs * slab + n_slabs * 128 * 128 + 2 * 4 * 128 * 4 + 64 + 1024;
     // resident CTAs per SM: bounded by the register file (128 G threads of at most 128 registers),
     // by the 512 TMEM columns and by shared memory.  The bound must not exceed what TMEM allows:
@@ -701,12 +703,14 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
     static int smem_set_dev[kMaxDevices] = {0};
     int& smem_set = smem_set_dev[ctx->device % kMaxDevices];
     if (smem > smem_set) {
-      if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+      if (cudaFuncSetAttribute(attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+          cudaFuncSetAttribute(attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return IBERT_ERR_CUDA;
       smem_set = smem;
     }
-    if (int rc2 = launch_pdl(attention_kernel, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1,
-                             mqk, mv, a)) return rc2;
+    if (int rc2 = cu_seqlens ? launch_pdl(attention_kernel<true>, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1, mqk, mv, a)
+                             : launch_pdl(attention_kernel<false>, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1, mqk, mv, a))
+      return rc2;
     return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
   }
 

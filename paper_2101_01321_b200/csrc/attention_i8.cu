@@ -427,9 +427,22 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
     load_v(blockIdx.x);
   }
 
-  for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
+  // Packed batches: sequences differ in length, so after its first (batch, head) pair a CTA draws the
+  // following ones from a counter in global memory instead of a fixed stride -- a CTA that got short
+  // sequences takes more pairs.  The pair after the current one is drawn at the top of an iteration
+  // (its loads are issued during the current pair) and handed to the other threads through shared
+  // memory, two slots alternating.  Words 4 and 5 of the status block: the counter, and the number of
+  // CTAs that are done; the last CTA to finish zeroes both for the next launch.
+  int* s_next = reinterpret_cast<int*>(s_tmem + 1);
+  int32_t* draw = a.status + 4;
+  int next = 0;
+  for (int item = blockIdx.x, iter = 0; item < total && ok; item = next, ++iter) {
     const int head = item % a.heads, batch = item / a.heads;
-    const int next = item + gridDim.x;
+    if constexpr (PACKED) {
+      if (tid == 0) s_next[iter & 1] = (int)gridDim.x + atomicAdd(draw, 1);
+    } else {
+      next = item + gridDim.x;
+    }
     // valid keys of this sequence (key-padding mask): keys >= n take no part in max or sum and get
     // probability 0; the MMAs and the softmax only cover the 32-column chunks that hold valid keys
     // (at least one chunk, so that a sequence without valid keys yields P = 0 and context 0)
@@ -451,6 +464,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
     }
     ok = __syncthreads_and(ok);
     if (!ok) break;
+    if constexpr (PACKED) next = s_next[iter & 1];
     if (tid == 0 && next < total) load_v(next);
     ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_k, kv_phase));
     kv_phase ^= 1;
@@ -650,6 +664,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
     }
   }
   if (!ok) atomicCAS(a.status, 0, IBERT_ERR_TIMEOUT);
+  if constexpr (PACKED) {
+    if (tid == 0 && atomicAdd(draw + 1, 1) == (int)gridDim.x - 1) {   // every CTA has drawn its last pair
+      draw[0] = 0;
+      draw[1] = 0;
+    }
+  }
   ptx::tc_fence_before_sync();
   __syncthreads();
   if (warp == 0) {

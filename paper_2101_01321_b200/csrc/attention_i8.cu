@@ -519,7 +519,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
         }
         s_max[grp * 128 + row] = mx;
       }
-      __syncthreads();
+      if (G > 1) __syncthreads();                  // one thread per row: nothing to exchange
       // ---- pass 2: i-exp written back over the scores, partial sums
       uint32_t sum = 0;
       if (ok) {
@@ -572,7 +572,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
         ptx::tmem_wait_st();
         s_sum[grp * 128 + row] = sum;
       }
-      __syncthreads();
+      if (G > 1) __syncthreads();
       // ---- pass 3: u8 probabilities into the operand tile of the second MMA
       if (ok) {
         sum = 0;

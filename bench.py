@@ -787,7 +787,7 @@ def main():
     ap.add_argument("--only", default="", help="run one kernel class alone (profiling aid)")
     ap.add_argument("--sustain", type=float, default=3.0,
                     help="seconds of back-to-back steps for the sustained-clock leg (0 = skip)")
-    ap.add_argument("--scales", choices=["analytic", "calibrated"], default="analytic",
+    ap.add_argument("--scales", choices=["analytic", "calibrated"], default="calibrated",
                     help="static activation scales: closed-form from the input distributions, or the blob "
                          "calibrated with the CPU oracle (tests/golden/calibrated_scales.json)")
     args = ap.parse_args()

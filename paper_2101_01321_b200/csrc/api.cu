@@ -665,13 +665,16 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   auto up = [&](const void* h, size_t bytes, void** dev) { if (rc == IBERT_OK) rc = upload_owned(ly, h, bytes, dev); };
   // `upper_ok`: whether the rest of that GEMM's epilogue can run in the upper-word form; the table
   // is converted to it only then (the generic epilogue reads the plain (b, c) pairs)
+  // `max_acc` > 0: the largest accumulator magnitude this GEMM can produce (K 127^2 + max |bias|); a
+  // table that does not fit the upper-word form may then take the wide one (GELU epilogue only)
   auto lin = [&](double S_in, const double* S_w, int N, const double* so_cols, double so, int32_t** db, int32_t** dc,
-                 int* fast, bool upper_ok = true) {
+                 int* fast, bool upper_ok = true, int64_t max_acc = 0) {
     if (rc != IBERT_OK) return;
     std::vector<int32_t> b, c;
     rc = make_linear_tables(S_in, S_w, N, so_cols, so, &b, &c);
     if (rc != IBERT_OK) return;
     *fast = (upper_ok && to_upper_word_form(&b, c)) ? 1 : 0;
+    if (!*fast && upper_ok && max_acc > 0 && to_upper_word_wide(&b, &c, max_acc)) *fast = 2;
     up(b.data(), b.size() * sizeof(int32_t), (void**)db);
     up(c.data(), c.size() * sizeof(int32_t), (void**)dc);
   };
@@ -690,7 +693,13 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   }
   lin(d->S_ctx, d->S_w_o, H, nullptr, d->S_r1, &ly->b_o, &ly->c_o, &ly->fast_o);
   if (rc == IBERT_OK) rc = make_gelu_consts(d->S_gi, d->S_go, &ly->gelu);
-  lin(d->S_h1, d->S_w_f1, F, nullptr, d->S_gi, &ly->b_f1, &ly->c_f1, &ly->fast_f1, ly->gelu.fast != 0);
+  int64_t max_acc_f1 = (int64_t)H * 127 * 127;
+  {
+    int64_t bmax = 0;
+    for (int n = 0; n < F; ++n) bmax = std::max<int64_t>(bmax, std::llabs((int64_t)d->bias_f1[n]));
+    max_acc_f1 += bmax;
+  }
+  lin(d->S_h1, d->S_w_f1, F, nullptr, d->S_gi, &ly->b_f1, &ly->c_f1, &ly->fast_f1, ly->gelu.fast != 0, max_acc_f1);
   lin(d->S_go, d->S_w_f2, H, nullptr, d->S_r2, &ly->b_f2, &ly->c_f2, &ly->fast_f2);
   auto ln = [&](const double* g, const double* be, double S_sum, double S_res, double S_o, LnConsts* k,
                 int32_t** db, int64_t** dB) {

@@ -29,6 +29,14 @@ __device__ __forceinline__ int32_t requant_upper(int32_t v, int32_t b2) {
   return (int32_t)(t >> 32) + (int32_t)((uint32_t)t >> 31);
 }
 
+// The upper-word requantization for multipliers of 1/2 and more: b 2^(32-c) no longer fits 32 bits,
+// so it is split into w 2^32 + r with r in [-2^31, 2^31) and the product into v w + (v r >> 32).
+// Exact like the others; the host checks that v w cannot overflow.
+__device__ __forceinline__ int32_t requant_upper_wide(int32_t v, int32_t r, int32_t w) {
+  const int64_t t = (int64_t)v * (int64_t)r;
+  return v * w + (int32_t)(t >> 32) + (int32_t)((uint32_t)t >> 31);
+}
+
 // (v * b2 + add) >> 32 for a general 64-bit addend, the carry of the lower words propagated by hand
 __device__ __forceinline__ int32_t requant_upper_add(int32_t v, int32_t b2, int64_t add) {
   const int64_t t = (int64_t)v * (int64_t)b2;

@@ -90,6 +90,8 @@ constexpr int UMMA_K = 32;        // K per tcgen05.mma kind::i8
 // i-GELU epilogue whose results provably stay above -127 (GeluConsts::low_free): no lower clamp.
 // A kind of its own, internal to this file, so that the choice costs no instruction in the loop.
 constexpr int kEpiGeluLowFree = 16;
+// The same two i-GELU epilogues with per-channel multipliers of 1/2 and more (requant_upper_wide)
+constexpr int kEpiGeluWide = 17, kEpiGeluLowFreeWide = 18;
 
 template <int TOK, bool PAIR, int KIND>
 struct Cfg {
@@ -317,6 +319,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               else o = ihgelu_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
             } else if constexpr (KIND == kEpiGeluLowFree) {
               o = min(igelu_magnitude_upper(requant_upper(a + cur_bias, cur_pb), gk, gelu_rnd), 127);
+            } else if constexpr (KIND == kEpiGeluLowFreeWide) {
+              o = min(igelu_magnitude_upper(requant_upper_wide(a + cur_bias, cur_pb, cur_pc), gk, gelu_rnd), 127);
+            } else if constexpr (KIND == kEpiGeluWide) {
+              o = clamp_sym(igelu_magnitude_upper(requant_upper_wide(a + cur_bias, cur_pb, cur_pc), gk, gelu_rnd), 127);
             } else {
               if constexpr (FAST) o = clamp_sym(igelu_magnitude_upper(requant_upper(a + cur_bias, cur_pb), gk, gelu_rnd), 127);
               else o = igelu_q16_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
@@ -381,7 +387,10 @@ int launch_inst(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, co
 
 template <int TOK, bool PAIR>
 int launch_shape(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& mo, const GemmArgs& a,
-                 int kind, bool fast) {
+                 int kind, bool fast, bool wide_form) {
+  if (kind == EPI_GELU && fast && wide_form)
+    return a.gelu.low_free ? launch_inst<TOK, PAIR, kEpiGeluLowFreeWide, true>(ctx, mw, mx, mo, a)
+                           : launch_inst<TOK, PAIR, kEpiGeluWide, true>(ctx, mw, mx, mo, a);
   switch (kind) {
     case EPI_INT8: return fast ? launch_inst<TOK, PAIR, EPI_INT8, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_INT8, false>(ctx, mw, mx, mo, a);
     case EPI_Q16: return fast ? launch_inst<TOK, PAIR, EPI_Q16, true>(ctx, mw, mx, mo, a) : launch_inst<TOK, PAIR, EPI_Q16, false>(ctx, mw, mx, mo, a);
@@ -401,8 +410,8 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
   if (M == 0) return IBERT_OK;
   {
     // few output tiles (small batches): split K over a cluster instead of leaving most SMs idle
-    int split = ctx->splitk_mode == 1 ? 1 : gemm_splitk_width(ctx, M, N, K);
-    if ((ctx->splitk_mode == 2 || ctx->splitk_mode == 4) && K > 128 &&
+    int split = (ctx->splitk_mode == 1 || epi.fast == 2) ? 1 : gemm_splitk_width(ctx, M, N, K);
+    if ((ctx->splitk_mode == 2 || ctx->splitk_mode == 4) && K > 128 && epi.fast != 2 &&
         ((M + 127) / 128) * ((N + 127) / 128) * ctx->splitk_mode <= 65535)
       split = ctx->splitk_mode;
     if (split > 1) return launch_gemm_splitk_i8(ctx, x, w, M, N, K, epi, out, split);
@@ -446,9 +455,11 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
   a.status = ctx->d_status;
   // upper-word epilogue needs both the per-channel multipliers and (for GELU) the final one in that form
   const bool fast = epi.fast != 0 && ((epi.kind != EPI_GELU && epi.kind != EPI_HGELU) || epi.gelu.fast != 0);
-  if (pair) return launch_shape<256, true>(ctx, mw, mx, mo, a, epi.kind, fast);
-  return wide ? launch_shape<256, false>(ctx, mw, mx, mo, a, epi.kind, fast)
-              : launch_shape<128, false>(ctx, mw, mx, mo, a, epi.kind, fast);
+  const bool wide_form = epi.fast == 2;
+  if (wide_form && (epi.kind != EPI_GELU || !fast)) return IBERT_ERR_ARG;      // tables in a form nothing else reads
+  if (pair) return launch_shape<256, true>(ctx, mw, mx, mo, a, epi.kind, fast, wide_form);
+  return wide ? launch_shape<256, false>(ctx, mw, mx, mo, a, epi.kind, fast, wide_form)
+              : launch_shape<128, false>(ctx, mw, mx, mo, a, epi.kind, fast, wide_form);
 }
 
 }  // namespace ibert

@@ -193,6 +193,28 @@ bool to_upper_word_form(std::vector<int32_t>* b, const std::vector<int32_t>& c) 
   return true;
 }
 
+// The same for multipliers of 1/2 and more (b 2^(32-c) beyond 32 bits): b <- r, c <- w with
+// b 2^(32-c) = w 2^32 + r, r in [-2^31, 2^31).  `max_abs_v` bounds the values that will be
+// requantized; the conversion is refused (nothing changed) when v w could leave 32 bits.
+bool to_upper_word_wide(std::vector<int32_t>* b, std::vector<int32_t>* c, int64_t max_abs_v) {
+  std::vector<int32_t> r(b->size()), w(b->size());
+  for (size_t n = 0; n < b->size(); ++n) {
+    const int cn = (*c)[n];
+    if (cn < 1 || cn > 31) return false;
+    const int64_t full = (int64_t)(*b)[n] * (int64_t(1) << (32 - cn));             // |full| < 2^62
+    const int64_t wn = (full + (int64_t(1) << 31)) >> 32;                            // nearest multiple of 2^32
+    const int64_t rn = full - wn * (int64_t(1) << 32);
+    if (rn < INT32_MIN || rn > INT32_MAX || wn < -64 || wn > 64) return false;
+    // |v w| + |v r / 2^32| + 1 must stay below 2^31
+    if ((double)max_abs_v * ((double)std::llabs(wn) + 0.5) + 2.0 >= 2147483648.0) return false;
+    r[n] = (int32_t)rn;
+    w[n] = (int32_t)wn;
+  }
+  *b = r;
+  *c = w;
+  return true;
+}
+
 // LayerNorm affine + requantization folded into one dyadic step per channel: the
 // normalized value n ~ y_hat * 2^16, out = (n * b_i + B_i) >> c with a shared c.
 int make_ln_tables(const double* gamma, const double* beta, int C, double S_out, LnConsts* k,

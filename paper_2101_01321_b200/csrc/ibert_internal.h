@@ -162,13 +162,18 @@ struct GemmEpilogue {
   const int32_t* d_b;      // [N] dyadic multipliers b (fast: b << (32 - c)); unused for EPI_RAW
   const int32_t* d_c;      // [N] dyadic shifts
   const int32_t* d_bias;   // [N] or nullptr
-  int fast;                // every column's requantization fits the upper-word form
+  int fast;                // 1: every column's requantization fits the upper-word form; 2: the wide
+                           // upper-word form (d_b = low words, d_c = integer parts; GELU epilogue of
+                           // the plain GEMM only); 0: generic (b, c) pairs
   GeluConsts gelu;         // EPI_GELU / EPI_HGELU only
 };
 
 // Upper-word form of a column set: true if for every n, c[n] >= 1 and b[n] << (32 - c[n]) fits
 // int32; then b is replaced by the shifted multipliers.
 bool to_upper_word_form(std::vector<int32_t>* b, const std::vector<int32_t>& c);
+// The same for multipliers of 1/2 and more: b <- low word r, c <- integer part w of b 2^(32-c) =
+// w 2^32 + r; false (nothing changed) when a shift is 0 or |v| <= max_abs_v could overflow v w.
+bool to_upper_word_wide(std::vector<int32_t>* b, std::vector<int32_t>* c, int64_t max_abs_v);
 
 int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, int N, int K,
                    const GemmEpilogue& epi, void* out);

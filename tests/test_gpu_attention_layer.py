@@ -164,3 +164,27 @@ def test_encoder_layers_with_power_of_two_score_scales():
     for p, got in zip(params, outs):
         h = oracle.encoder_layer(p, h, B, L).out
         assert_same(got, h, "pow2-score layer")
+
+
+@pytest.mark.parametrize("shrink,S_go_scale", [(2.0, 1.0), (3.5, 1.0), (6.0, 1.0), (3.5, 0.004)])
+def test_layer_with_ffn1_multipliers_of_one_half_and_more(shrink, S_go_scale):
+    """A finer GELU-input scale makes the per-channel multipliers S_h1 S_w[n] / S_gi reach 1/2 and go
+    beyond 1: the FFN1 epilogue then takes the wide upper-word form (multiplier split into an integer
+    part and a 32-bit fraction), with and without the lower output clamp; many values clamp at Q16."""
+    B, L, H, heads, F = 5, 96, 256, 4, 1024
+    x, params = synth.make_model(0, B, layers=1, H=H, heads=heads, F=F, L=L)
+    p = dict(params[0])
+    p["S_gi"] = p["S_gi"] / shrink
+    p["S_go"] = p["S_go"] * S_go_scale
+    m = p["S_h1"] * np.asarray(p["S_w_f1"]) / p["S_gi"]
+    assert m.max() >= 0.5
+    c = ctx()
+    layer = c.ibert_layer_create(p)
+    try:
+        out, _ = c.ibert_encoder_layer(layer, dev(x), B, L)
+        c.check()
+    finally:
+        layer.close()
+    res = oracle.encoder_layer(p, x, B, L, want_taps=True)
+    assert_same(host(out), res.out, f"layer with FFN1 multipliers up to {m.max():.2f}")
+    assert np.abs(np.asarray(res.taps["g"]).astype(int)).max() > 20

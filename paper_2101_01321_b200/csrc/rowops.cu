@@ -350,8 +350,16 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
   const uint32_t slot_bytes = q_bytes + r_bytes;                 // multiple of 16
   uint8_t* ring = ln_smem + (size_t)warp * DEPTH * slot_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(ln_smem + (size_t)(kThreads / 32) * DEPTH * slot_bytes) + warp * DEPTH;
+  // the per-channel tables, copied once per CTA: every row reads all of them
+  int64_t* s_B = reinterpret_cast<int64_t*>(ln_smem + (size_t)(kThreads / 32) * DEPTH * slot_bytes + (kThreads / 32) * DEPTH * 8);
+  int32_t* s_b = reinterpret_cast<int32_t*>(s_B + C);
   const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
   const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
+  for (int i = threadIdx.x; i < C; i += kThreads) {        // constants, not outputs of the previous kernel
+    s_b[i] = __ldg(b_i + i);
+    s_B[i] = __ldg(B_i + i);
+  }
+  __syncthreads();
 
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();              // the kernel that produced q (and r) has completed
@@ -409,31 +417,25 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
     }
     if (++slot == DEPTH) { slot = 0; phase ^= 1; }
 
+    // one pass over the row: sum v and sum v^2 (columns past C hold zeros); the centred sum of squares
+    // follows exactly in integers: sum (v - mu)^2 = sum v^2 - 2 mu sum v + C mu^2
     int32_t sum = 0;
+    uint64_t s2 = 0;
 #pragma unroll
     for (int j = 0; j < VPL; ++j)
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         v[j][i] += requant_upper(sext_byte(rw[j], i) << k.res_sh, k.b_r);
         sum += v[j][i];
+        s2 += (uint64_t)((int64_t)v[j][i] * (int64_t)v[j][i]);
       }
     sum = __reduce_add_sync(0xffffffffu, sum);
+    // a lane's share is below 2^50 (|v| <= 2^21, at most 64 values): two 25-bit halves reduce as 32-bit sums
+    s2 = (uint64_t)__reduce_add_sync(0xffffffffu, (uint32_t)s2 & 0x1ffffffu) +
+         ((uint64_t)__reduce_add_sync(0xffffffffu, (uint32_t)(s2 >> 25)) << 25);
     int32_t mu = sum / C;                            // mu = floor(sum / C)
     if (sum - mu * C < 0) mu -= 1;
-    uint64_t ss = 0;
-#pragma unroll
-    for (int j = 0; j < VPL; ++j) {
-      const int col = 4 * (j * 32 + lane);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int32_t y = (FULL || col < C) ? v[j][i] - mu : 0;
-        v[j][i] = y;
-        ss += (uint64_t)((int64_t)y * (int64_t)y);
-      }
-    }
-    // a lane's share is below 2^50 (|y| <= 2^21, at most 64 values): two 25-bit halves reduce as 32-bit sums
-    ss = (uint64_t)__reduce_add_sync(0xffffffffu, (uint32_t)ss & 0x1ffffffu) +
-         ((uint64_t)__reduce_add_sync(0xffffffffu, (uint32_t)(ss >> 25)) << 25);
+    const uint64_t ss = (uint64_t)((int64_t)s2 - 2 * (int64_t)mu * (int64_t)sum + (int64_t)C * (int64_t)mu * (int64_t)mu);
     uint32_t sigma = warp_isqrt_of_quotient(ss, (uint32_t)C, lane);   // I-Sqrt(floor(ss / C))
     sigma = sigma < 1u ? 1u : sigma;
     // floor(2^31 / sigma) as a positive int32 multiplier: for sigma = 1 use 2^30 and shift one less
@@ -444,15 +446,15 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
     for (int j = 0; j < VPL; ++j) {
       const int col = 4 * (j * 32 + lane);
       if (FULL || col < C) {
-        const int4 bb = __ldg(reinterpret_cast<const int4*>(b_i + col));
-        const longlong2 B01 = __ldg(reinterpret_cast<const longlong2*>(B_i + col));
-        const longlong2 B23 = __ldg(reinterpret_cast<const longlong2*>(B_i + col + 2));
+        const int4 bb = *reinterpret_cast<const int4*>(s_b + col);
+        const longlong2 B01 = *reinterpret_cast<const longlong2*>(s_B + col);
+        const longlong2 B23 = *reinterpret_cast<const longlong2*>(s_B + col + 2);
         const int32_t bv[4] = {bb.x, bb.y, bb.z, bb.w};
         const int64_t Bv[4] = {B01.x, B01.y, B23.x, B23.y};
         int32_t o[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int64_t pr = (int64_t)v[j][i] * (int64_t)rho;
+          const int64_t pr = (int64_t)(v[j][i] - mu) * (int64_t)rho;
           // floor(pr / 2^nsh) fits 32 bits: the low word of the 64-bit shift is a funnel shift
           const int32_t nrm = (int32_t)__funnelshift_r((uint32_t)pr, (uint32_t)(pr >> 32), (uint32_t)nsh) << k.out_sh;
           o[i] = max(requant_upper_add(nrm, bv[i], Bv[i]), -127);
@@ -630,7 +632,8 @@ static int launch_layernorm_t(ibert_ctx* ctx, const QT* q, const int8_t* r, int6
   if (fast && k.has_res && k.C % 16 == 0 && k.C <= 1024) {
     // streaming variant: per-warp ring of row slots filled by bulk async copies
     const int depth = 2;
-    const size_t smem = (size_t)(kThreads / 32) * depth * (size_t)k.C * (sizeof(QT) + 1) + (kThreads / 32) * depth * 8;
+    const size_t smem = (size_t)(kThreads / 32) * depth * (size_t)k.C * (sizeof(QT) + 1) + (kThreads / 32) * depth * 8 +
+                        (size_t)k.C * 12;                  // rows in flight, barriers, the two tables
     const int pgrid = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)ctx->num_sms * 3);
 #define IBERT_LNP2(V, D, F)                                                                                 \
   do {                                                                                                      \

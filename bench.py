@@ -49,16 +49,17 @@ def _table_rows(path: Path) -> list[list[str]]:
 
 
 def ncu_figures() -> dict:
-    """{(kernel class, config, batch): {"dram_bytes": ..., "warp_instructions": ..., "int_pipe_instructions": ...}}
-    from profiles/ncu_figures.md -- the per-launch figures of the committed ncu captures, written by
-    the same step that writes the per-kernel summaries, so that this file and they cannot drift."""
+    """{(kernel class, config, batch): {"dram_bytes", "warp_instructions", "alu", "fma"}} from
+    profiles/ncu_figures.md -- the per-launch figures of the committed ncu captures (DRAM bytes, warp
+    instructions in all / on the ALU pipe / on the multiply-add pipe), written by the same step that
+    writes the per-kernel summaries, so that this file and they cannot drift."""
     out = {}
     for r in _table_rows(ROOT / "profiles" / "ncu_figures.md"):
-        if len(r) < 6:
+        if len(r) < 7:
             continue
         try:
             out[(r[0], int(r[1]), int(r[2]))] = {"dram_bytes": float(r[3]), "warp_instructions": float(r[4]),
-                                                 "int_pipe_instructions": float(r[5])}
+                                                 "alu": float(r[5]), "fma": float(r[6])}
         except ValueError:
             continue                      # header / ruler rows
     return out
@@ -69,7 +70,7 @@ def probe_peaks() -> dict:
     "i8_mma_tops": ...}; empty when the summary is absent."""
     out = {}
     for r in _table_rows(ROOT / "profiles" / "issue_probes.md"):
-        if len(r) >= 2 and r[0] in ("int32_lane_ops_per_clk_sm", "i8_mma_tops"):
+        if len(r) >= 2 and r[0] in ("int32_lane_ops_per_clk_sm", "alu_pipe_lane_ops_per_clk_sm", "i8_mma_tops"):
             try:
                 out[r[0]] = float(r[1])
             except ValueError:
@@ -515,11 +516,14 @@ def run_ours(args):
         # Peaks.  A kernel timed by an event pair inside a step of a few milliseconds runs at burst
         # clocks, so the tensor peak is 2 x the BURST bf16 cuBLAS rate (int8 : bf16 dense = 2 nominal).
         int8_peak = 2.0 * peaks["bf16_tflops"]
-        lanes = probes.get("int32_lane_ops_per_clk_sm")
-        alu_peak = (lanes or 64.0) * n_sms * sm_mhz_max * 1e6 / 1e12         # T lane-operations / s
-        alu_source = (f"{lanes:.1f} int32 lane-ops per clock and SM (measured by the issue probe, "
-                      "profiles/issue_probes.md) x SMs x max SM clock" if lanes else
-                      "64 int32 lanes x SMs x max SM clock (unit count; probe summary absent)")
+        # integer issue: 128 lane-operations per clock and SM over both integer pipes, 64 on the ALU pipe
+        # alone (shifts, min / max, selects, permutes: the pipe the epilogues and i-softmax saturate first)
+        issue_lanes = probes.get("int32_lane_ops_per_clk_sm", 128.0)
+        alu_lanes = probes.get("alu_pipe_lane_ops_per_clk_sm", 64.0)
+        issue_peak = issue_lanes * n_sms * sm_mhz_max * 1e6 / 1e12          # T lane-operations / s
+        alu_peak = alu_lanes * n_sms * sm_mhz_max * 1e6 / 1e12
+        alu_source = (f"{alu_lanes:.0f} lane-operations per clock and SM on the ALU pipe x SMs x max SM clock "
+                      f"({'measured by the issue probe, profiles/issue_probes.md' if probes else 'unit count; probe summary absent'})")
         kern = {}
         prof_total = sum(v[0] for v in prof.values())
         for k, (ms, n) in prof.items():
@@ -536,19 +540,20 @@ def run_ours(args):
             fig = figures.get((k, args.config, batch))
             if fig:
                 kern[k]["ncu_dram_bytes"] = fig["dram_bytes"]
-                kern[k]["frac_int32_issue"] = fig["int_pipe_instructions"] * 32.0 / (per * 1e-3) / (alu_peak * 1e12)
+                kern[k]["frac_alu_pipe"] = fig["alu"] * 32.0 / (per * 1e-3) / (alu_peak * 1e12)
+                kern[k]["frac_int32_issue"] = (fig["alu"] + fig["fma"]) * 32.0 / (per * 1e-3) / (issue_peak * 1e12)
         top = max(kern, key=lambda k: kern[k]["share"])
         fig = figures.get((top, args.config, batch))
         if top == "attention":
-            # i-softmax dominates: integer instructions on the ALU / multiply-add pipes per launch (ncu
-            # count when a capture of this workload is committed, else 16 per score element)
-            lane_ops = fig["int_pipe_instructions"] * 32.0 if fig else 16.0 * T * cfg.L * cfg.heads
+            # i-softmax dominates: lane-operations on the ALU pipe per launch (ncu count when a capture of
+            # this workload is committed, else 11 per score element, the count of the config-2 capture)
+            lane_ops = fig["alu"] * 32.0 if fig else 11.0 * computed * cfg.L * cfg.heads
             ach = lane_ops / (kern[top]["ms_per_launch"] * 1e-3) / 1e12
             roof = {"kernel": top, "bound": "alu", "achieved": ach, "peak": alu_peak,
-                    "unit": "Tinstr/s (int32 lane-ops)", "frac": ach / alu_peak, "peak_source": alu_source,
+                    "unit": "Tinstr/s (int32 lane-ops on the ALU pipe)", "frac": ach / alu_peak, "peak_source": alu_source,
                     "algorithmic": lane_ops,
-                    "algorithmic_source": "ncu ALU + multiply-add pipe instructions x 32" if fig else
-                                          "16 lane-ops per score element (no ncu capture of this workload committed)"}
+                    "algorithmic_source": "ncu ALU-pipe instructions of the committed capture x 32" if fig else
+                                          "11 ALU-pipe lane-ops per score element (no ncu capture of this workload committed)"}
         elif work[top]["ops"]:
             roof = {"kernel": top, "bound": "tensor", "achieved": kern[top]["tops"], "peak": int8_peak,
                     "unit": "TOP/s", "frac": kern[top]["tops"] / int8_peak,
@@ -565,13 +570,12 @@ def run_ours(args):
                     "peak_source": f"{peak_kind} copy bandwidth", "algorithmic": work[top]["bytes"]}
         roof["ms_per_launch"] = kern[top]["ms_per_launch"]
         if fig and top != "attention":
-            lane_ops = fig["int_pipe_instructions"] * 32.0
-            roof["integer_datapath"] = {"lane_ops_per_launch": lane_ops, "peak_lane_ops_per_s": alu_peak * 1e12,
+            lane_ops = fig["alu"] * 32.0
+            roof["integer_datapath"] = {"alu_lane_ops_per_launch": lane_ops, "peak_lane_ops_per_s": alu_peak * 1e12,
                                         "frac": lane_ops / (kern[top]["ms_per_launch"] * 1e-3) / (alu_peak * 1e12),
                                         "peak_source": alu_source,
-                                        "note": "the epilogue's int32 work (ncu ALU + multiply-add pipe instructions of "
-                                                "the committed capture) against the int32 issue rate: the bound this "
-                                                "kernel actually runs into"}
+                                        "note": "the epilogue's work on the ALU pipe (ncu count of the committed capture) "
+                                                "against that pipe's issue rate: the bound this kernel actually runs into"}
         roof["traffic"] = fig["dram_bytes"] if fig else None
         roof["traffic_unit"] = ("bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum, "
                                 "profiles/ncu_figures.md)")

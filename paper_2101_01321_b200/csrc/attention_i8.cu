@@ -118,7 +118,10 @@ __device__ __forceinline__ void softmax_row(uint32_t t_row, int L, int Lp, const
 __device__ __forceinline__ void transpose_v(const uint8_t* sVs, uint8_t* sVt, int n_keys, int tid,
                                             int n_threads = kAttnThreads) {
   for (int item = tid; item < (n_keys / 4) * 4; item += n_threads) {
-    const int jq = item % (n_keys / 4), dc = item / (n_keys / 4);     // key quad, 16-dim chunk
+    // consecutive lanes take the four 16-byte chunks of one key row, then the next key quad: a
+    // quarter-warp reads 128 contiguous bytes per load (no bank conflict; the 16 stores per thread
+    // then collide four ways, which costs less than the eight-way conflicts of the loads did)
+    const int dc = item & 3, jq = item >> 2;                          // 16-dim chunk, key quad
     uint32_t r[4][4];
 #pragma unroll
     for (int jj = 0; jj < 4; ++jj) {

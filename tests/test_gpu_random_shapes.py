@@ -3,7 +3,8 @@
 The fixed-shape parity tests cover the tiles, tails and degenerate cases chosen by hand; this sweep
 covers the combinations nobody chose: ragged M / N / K with every epilogue and split-K width, attention
 at arbitrary lengths with and without key lengths, score scales on and off the ln2 / 2^k grid, the
-cluster kernel forced on or off, row operators at odd widths.  One context serves all of them in
+cluster kernel forced on or off, row operators at odd widths, Q16 in int32 and int16 containers,
+packed batches, FFN1 multipliers on both sides of 1/2.  One context serves all of them in
 random order, so state left behind by one call (cached constant tables, the workspace, the status
 word) meets every other call."""
 import numpy as np
@@ -29,9 +30,13 @@ def _linear(rng):
     bias = rng.integers(-200000, 200000, N).astype(np.int32)
     S_w, S_x = rng.uniform(1e-4, 4e-4, N), 0.03
     amax = 127.0 * 127.0 * np.sqrt(K) * 1.2 * S_x * 2.5e-4
-    kind = int(rng.integers(0, 5))
+    kind = int(rng.integers(0, 6))
     what = f"linear kind {kind} {M}x{N}x{K}"
-    if kind < 3:
+    if kind == 5:                                             # Q16 in an int16 container
+        S_out = amax / 20000.0
+        out, _ = c.ibert_linear_i8(dev(x), S_x, dev(w), S_w, dev(bias), 3, S_out)
+        assert_same(host(out).astype(np.int32), oracle.linear(x, S_x, w, S_w, bias, 1, S_out), what)
+    elif kind < 3:
         S_out = [amax / 100.0, amax / 20000.0, 0.0][kind]
         out, _ = c.ibert_linear_i8(dev(x), S_x, dev(w), S_w, dev(bias), kind, S_out)
         assert_same(host(out), oracle.linear(x, S_x, w, S_w, bias, kind, S_out), what)
@@ -63,11 +68,17 @@ def _attention(rng):
     lens = rng.integers(0, L + 1, B).astype(np.int32) if rng.random() < 0.5 else None
     p_max = int(rng.choice([255, 127]))
     c = ctx()
+    want = oracle.attention(qkv, B, L, H, heads, S_q, S_k, 0.02, 0.006, p_max, lens=lens)
     if lens is None:
         out, _ = c.ibert_attention_i8(dev(qkv), B, L, H, heads, S_q, S_k, 0.02, 0.006, p_max)
+    elif rng.random() < 0.5 and lens.sum() > 0:               # the same sequences without their padding
+        rows = np.concatenate([np.arange(b * L, b * L + n) for b, n in enumerate(lens)])
+        cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        out, _ = c.ibert_attention_packed_i8(dev(np.ascontiguousarray(qkv[rows])), dev(cu), L, H, heads, S_q, S_k, 0.02,
+                                             0.006, p_max)
+        want = want[rows]
     else:
         out, _ = c.ibert_attention_masked_i8(dev(qkv), B, L, H, heads, dev(lens), S_q, S_k, 0.02, 0.006, p_max)
-    want = oracle.attention(qkv, B, L, H, heads, S_q, S_k, 0.02, 0.006, p_max, lens=lens)
     assert_same(host(out), want, f"attention B={B} L={L} heads={heads} S_q={S_q} p_max={p_max} lens={lens}")
 
 
@@ -79,7 +90,8 @@ def _row_ops(rng):
         rows, C = int(rng.choice([1, 5, 64, 333, 2000])), int(rng.choice([8, 17, 260, 768, 1024, 2047]))
         q, S, r, S_r, gamma, beta, S_out = synth.layernorm_inputs(rows, C, sigma)
         use_r = rng.random() < 0.7
-        out, _ = c.ibert_layernorm_i(dev(q), S, dev(r) if use_r else None, S_r, gamma, beta, S_out)
+        qd = dev(q.astype(np.int16)) if rng.random() < 0.5 else dev(q)      # either Q16 container
+        out, _ = c.ibert_layernorm_i(qd, S, dev(r) if use_r else None, S_r, gamma, beta, S_out)
         assert_same(host(out), oracle.layernorm(q, S, r if use_r else None, S_r, gamma, beta, S_out)[0], f"layernorm {rows}x{C}")
     elif which == 1:
         rows, L = int(rng.choice([1, 9, 100, 700])), int(rng.integers(1, 1025))
@@ -128,13 +140,24 @@ def _layer(rng):
     H = 64 * int(rng.choice([2, 4, 8]))
     heads = H // 64
     x, params = synth.make_model(0, B, layers=1, H=H, heads=heads, F=4 * H, L=L)
+    p0 = dict(params[0])
+    p0["S_gi"] = p0["S_gi"] / float(rng.choice([1.0, 1.0, 2.5, 5.0]))       # FFN1 multipliers up to and beyond 1/2
+    params = [p0]
     c = ctx()
-    c.ibert_set_fusion(int(rng.choice([0, 1])))
+    c.ibert_set_fusion(int(rng.choice([0, 1, 2])))
     ly = c.ibert_layer_create(params[0])
-    if rng.random() < 0.5:
+    mode = rng.random()
+    if mode < 0.33:
         lens = rng.integers(1, L + 1, B).astype(np.int32)
         out, _ = c.ibert_encoder_layer_masked(ly, dev(x), B, L, dev(lens))
         want = oracle.encoder_layer(params[0], x, B, L, lens=lens).out
+    elif mode < 0.66:
+        lens = rng.integers(0, L + 1, B).astype(np.int32)
+        lens[0] = max(lens[0], 1)
+        rows = np.concatenate([np.arange(b * L, b * L + n) for b, n in enumerate(lens)])
+        cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        out, _ = c.ibert_encoder_layer_packed(ly, dev(np.ascontiguousarray(x[rows])), dev(cu), L)
+        want = oracle.encoder_layer(params[0], x, B, L, lens=lens).out[rows]
     else:
         out, _ = c.ibert_encoder_layer(ly, dev(x), B, L)
         want = oracle.encoder_layer(params[0], x, B, L).out

@@ -207,6 +207,15 @@ int ibert_set_fusion(ibert_ctx* ctx, int mode);
    paper: a tuning and testing switch.  Returns IBERT_ERR_ARG for another mode. */
 int ibert_set_split_k(ibert_ctx* ctx, int mode);
 
+/* How the FFN1 GEMM inside ibert_encoder_layer (CTA-pair tiles, i.e. large batches) evaluates
+   i-GELU (Algorithm 2) and the requantization behind it: mode 0 (default) looks the int8 result up
+   in a 65535-entry table over the Q16 input, which ibert_layer_create fills by running the
+   i-GELU kernel over every Q16 value (64 KB of device memory per layer, copied into shared memory
+   by every CTA); mode 1 computes it per element.  The results are identical.  The paper names tables only
+   as the approach it avoids (Sec. 3.2: on-chip memory, look-up rate); here the table is filled by
+   the integer algorithm itself and used only where the epilogue's integer pipe is the bound.  A tuning and testing switch.  Returns IBERT_ERR_ARG for another mode. */
+int ibert_set_gelu_table(ibert_ctx* ctx, int mode);
+
 /* The integer-only encoder layer (Fig. 1 right; post-LN order):
    QKV projection -> attention (i-softmax) -> output projection -> +x, i-LayerNorm ->
    FFN1 + i-GELU -> FFN2 -> +h1, i-LayerNorm.  x, out: int8 [B*L, H]; x at desc.S_x,

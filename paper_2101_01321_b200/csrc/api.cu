@@ -130,6 +130,7 @@ struct ibert_layer {
   int64_t *ln1_B = nullptr, *ln2_B = nullptr;
   LnConsts ln1{}, ln2{};
   GeluConsts gelu{};
+  int8_t* gelu_table = nullptr;      // i-GELU of every Q16 value (FFN1 epilogue), or null
   AttnConsts attn{};
   std::vector<void*> owned;
 };
@@ -220,6 +221,14 @@ int ibert_set_split_k(ibert_ctx* ctx, int mode) {
   });
 }
 
+int ibert_set_gelu_table(ibert_ctx* ctx, int mode) {
+  return guarded([&]() -> int {
+  if (!ctx || mode < 0 || mode > 1) return IBERT_ERR_ARG;
+  ctx->gelu_table_mode = mode;
+  return IBERT_OK;
+  });
+}
+
 int ibert_last_status(ibert_ctx* ctx) {
   return guarded([&]() -> int {
   if (!ctx) return IBERT_ERR_ARG;
@@ -258,6 +267,26 @@ int ibert_gelu_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S
 
 static int ensure_workspace(ibert_ctx* ctx, size_t need);
 
+// The 65535-entry i-GELU table of one scale pair, cached in the context (built once: a ramp into the
+// workspace, the i-GELU kernel over it).  The pointer stays valid until a later entry point trims the cache.
+static int cached_gelu_table(ibert_ctx* ctx, const GeluConsts& k, const int8_t** out) {
+  const uint64_t key = fnv1a(&k, sizeof(k), 0x6c7574ull);
+  if (ctx->gelu_luts.size() >= 64) {                 // bounded: drop every table once the stream is idle
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+    for (auto& kv : ctx->gelu_luts) cudaFree(kv.second);
+    ctx->gelu_luts.clear();
+  }
+  auto it = ctx->gelu_luts.find(key);
+  if (it != ctx->gelu_luts.end()) { *out = it->second; return IBERT_OK; }
+  int8_t* table = nullptr;
+  if (int rc = ensure_workspace(ctx, 65536 * sizeof(int32_t))) return rc;
+  if (cudaMalloc((void**)&table, 65536) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_NOMEM; }
+  if (int rc = launch_gelu_table(ctx, k, static_cast<int32_t*>(ctx->ws), table)) { cudaFree(table); return rc; }
+  ctx->gelu_luts[key] = table;
+  *out = table;
+  return IBERT_OK;
+}
+
 int ibert_gelu_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, double S_out, int8_t* out,
                      double* S_ret) {
   return guarded([&]() -> int {
@@ -267,22 +296,8 @@ int ibert_gelu_lut_i(ibert_ctx* ctx, const int32_t* q, double S, int64_t n, doub
   int rc = make_gelu_consts(S, S_out, &k);
   if (rc) return rc;
   DeviceGuard guard(ctx->device);
-  const uint64_t key = fnv1a(&k, sizeof(k), 0x6c7574ull);
-  int8_t* table = nullptr;
-  if (ctx->gelu_luts.size() >= 64) {                 // bounded: drop every table once the stream is idle
-    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
-    for (auto& kv : ctx->gelu_luts) cudaFree(kv.second);
-    ctx->gelu_luts.clear();
-  }
-  auto it = ctx->gelu_luts.find(key);
-  if (it != ctx->gelu_luts.end()) table = it->second;
-  else {
-    // built once per scale pair: ramp into the workspace, the i-GELU kernel over it
-    if ((rc = ensure_workspace(ctx, 65536 * sizeof(int32_t)))) return rc;
-    if (cudaMalloc((void**)&table, 65536) != cudaSuccess) { cudaGetLastError(); return IBERT_ERR_NOMEM; }
-    if ((rc = launch_gelu_table(ctx, k, static_cast<int32_t*>(ctx->ws), table))) { cudaFree(table); return rc; }
-    ctx->gelu_luts[key] = table;
-  }
+  const int8_t* table = nullptr;
+  if ((rc = cached_gelu_table(ctx, k, &table))) return rc;
   {
     ProfileScope ps(ctx, IBERT_K_GELU);
     rc = launch_gelu_lut(ctx, q, n, table, out);
@@ -441,6 +456,9 @@ static int linear_common(ibert_ctx* ctx, const int8_t* x, double S_x, const int8
       upper_ok = epi.gelu.fast != 0;
     }
     epi.fast = (upper_ok && to_upper_word_form(&b, c)) ? 1 : 0;
+    // i-GELU by table (the tile shapes with room for it use it)
+    if (kind == EPI_GELU && epi.fast && ctx->gelu_table_mode == 0)
+      if ((rc = cached_gelu_table(ctx, epi.gelu, &epi.gelu_table))) return rc;
     void *d_b = nullptr, *d_c = nullptr;
     rc = cached_upload(ctx, b.data(), b.size() * sizeof(int32_t), 21, &d_b);
     if (rc) return rc;
@@ -718,8 +736,25 @@ int ibert_layer_create(ibert_ctx* ctx, const ibert_layer_desc* d, ibert_layer** 
   ln(d->gamma2, d->beta2, d->S_r2, d->S_h1, d->S_out, &ly->ln2, &ly->ln2_b, &ly->ln2_B);
   if (rc == IBERT_OK) rc = make_attn_consts(d->S_q, d->S_k, d->S_v, d->S_ctx, d->p_max, &ly->attn);
   if (rc != IBERT_OK) return rc;
+  // FFN1's i-GELU as a table over all Q16 inputs, written by the i-GELU kernel itself (the large-tile
+  // GEMM looks results up in it; needs the upper-word form of the requantization in front of it)
+  void* ramp = nullptr;
+  if (ly->fast_f1 != 0 && ly->gelu.fast != 0) {
+    void* t = nullptr;
+    if (cudaMalloc(&t, 65536) != cudaSuccess || cudaMalloc(&ramp, 65536 * sizeof(int32_t)) != cudaSuccess) {
+      cudaGetLastError();
+      cudaFree(t);
+      return IBERT_ERR_NOMEM;
+    }
+    ly->owned.push_back(t);
+    rc = launch_gelu_table(ctx, ly->gelu, static_cast<int32_t*>(ramp), static_cast<int8_t*>(t));
+    if (rc == IBERT_OK) ly->gelu_table = static_cast<int8_t*>(t);
+  }
   // host arrays were pageable: make sure the copies have left them before returning
-  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IBERT_ERR_CUDA;
+  const bool synced = cudaStreamSynchronize(ctx->stream) == cudaSuccess;
+  cudaFree(ramp);
+  if (rc != IBERT_OK) return rc;
+  if (!synced) return IBERT_ERR_CUDA;
   // scalars only from here on
   ly->d.w_qkv = ly->d.w_o = ly->d.w_f1 = ly->d.w_f2 = nullptr;
   holder.p = nullptr;
@@ -788,7 +823,7 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
     { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm_i16(ctx, r, x, T, ly->ln1, ly->ln1_b, ly->ln1_B, h1); }
   }
   if (rc) return rc;
-  e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu; e.fast = ly->fast_f1;
+  e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu; e.fast = ly->fast_f1; e.gelu_table = ly->gelu_table;
   { ProfileScope ps(ctx, IBERT_K_GEMM_GELU); rc = launch_gemm_i8(ctx, h1, ly->w_f1, T, F, H, e, g); }
   if (rc) return rc;
   e.kind = EPI_Q16; e.d_b = ly->b_f2; e.d_c = ly->c_f2; e.d_bias = ly->bias_f2; e.fast = ly->fast_f2;

@@ -92,6 +92,11 @@ constexpr int UMMA_K = 32;        // K per tcgen05.mma kind::i8
 constexpr int kEpiGeluLowFree = 16;
 // The same two i-GELU epilogues with per-channel multipliers of 1/2 and more (requant_upper_wide)
 constexpr int kEpiGeluWide = 17, kEpiGeluLowFreeWide = 18;
+// i-GELU and its requantization read from a table of all 65535 Q16 inputs held in shared memory:
+// the epilogue is bound by the integer ALU pipe, the load/store pipe idles, and the table (filled by
+// the i-GELU kernel itself) returns the same bits.  Costs 64 KB, i.e. two of six operand stages.
+constexpr int kEpiGeluTable = 19, kEpiGeluTableWide = 20;
+constexpr int kGeluTableBytes = 65536;
 
 template <int TOK, bool PAIR, int KIND>
 struct Cfg {
@@ -108,12 +113,15 @@ struct Cfg {
   static constexpr int kStageBytes = kWBytes + kXRows * BK;
   static constexpr int kOutTileBytes = 32 * 32 * kOutElem;            // 32 tokens x 32 channels
   static constexpr int kOutBytes = kEpiWarps * 2 * kOutTileBytes;     // double-buffered per warp
-  static constexpr int kBudget = 227 * 1024 - 1024 - 512 - kOutBytes;
+  static constexpr bool kTable = (KIND == kEpiGeluTable || KIND == kEpiGeluTableWide);
+  static constexpr int kTableBytes = kTable ? kGeluTableBytes : 0;
+  static constexpr int kBudget = 227 * 1024 - 1024 - 512 - kOutBytes - kTableBytes;
   static constexpr int kStages = kBudget / kStageBytes > 8 ? 8 : kBudget / kStageBytes;
   static constexpr int kOutOff = kStages * kStageBytes;
-  static constexpr int kBarOff = kOutOff + kOutBytes;
+  static constexpr int kTableOff = kOutOff + kOutBytes;
+  static constexpr int kBarOff = kTableOff + kTableBytes;
   static constexpr int kAlloc = kBarOff + 512 + 1024;            // + slack to align to 1024 bytes
-  static_assert(kEpiWarps % 4 == 0 && kChunks % kParts == 0 && kStages >= 3, "tile configuration");
+  static constexpr bool kValid = kEpiWarps % 4 == 0 && kChunks % kParts == 0 && kStages >= 3;
 };
 
 struct GemmArgs {
@@ -124,6 +132,7 @@ struct GemmArgs {
   const int32_t* bias;
   GeluConsts gelu;
   int32_t* status;
+  const int8_t* gelu_table;   // kEpiGeluTable kinds only
 };
 
 template <int TOK, bool PAIR, int KIND, bool FAST>
@@ -131,6 +140,7 @@ __global__ void __launch_bounds__(Cfg<TOK, PAIR, KIND>::kThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __grid_constant__ CUtensorMap map_out, const GemmArgs args) {
   using C = Cfg<TOK, PAIR, KIND>;
+  static_assert(C::kValid, "tile configuration");
   constexpr int kStages = C::kStages;
   constexpr uint32_t kTmemCols = 2 * TOK;          // two accumulator stages
   constexpr int kTileChannels = PAIR ? 2 * BC : BC;
@@ -144,6 +154,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   const uint32_t bar_acc_full = bar_empty + 8 * kStages;
   const uint32_t bar_acc_empty = bar_acc_full + 16;
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + 2 * kStages + 4);
+  const uint32_t bar_table = bar_acc_empty + 24;   // (after the TMEM base word)
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -164,6 +175,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       ptx::mbar_init(bar_acc_full + 8 * a, 1);
       ptx::mbar_init(bar_acc_empty + 8 * a, (PAIR ? 2 : 1) * C::kEpiWarps);   // one lane per epilogue warp
     }
+    if constexpr (C::kTable) ptx::mbar_init(bar_table, 1);
     ptx::fence_mbar_init();
     ptx::tma_prefetch_desc(&map_w);
     ptx::tma_prefetch_desc(&map_x);
@@ -186,6 +198,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
+      if constexpr (C::kTable) {
+        // the table may have been written by the kernel before this one: fetched after the dependency wait
+        ptx::mbar_arrive_expect_tx(bar_table, kGeluTableBytes);
+        ptx::bulk_load_1d(smem_base + C::kTableOff, args.gelu_table, kGeluTableBytes, bar_table);
+      }
       uint32_t stage = 0, phase = 0;
       for (int64_t tile = worker; tile < total_tiles && ok; tile += num_workers) {
         const int c0 = (int)(tile % c_tiles) * kTileChannels + (int)rank * BC;
@@ -206,6 +223,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           }
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
+      }
+      if constexpr (C::kTable) {
+        if (!ptx::mbar_wait(bar_table, 0)) ok = false;     // nobody leaves with the copy in flight
       }
     }
   } else if (warp == 1) {
@@ -271,6 +291,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       }
     };
     load_constants(worker);
+    // table kinds: shared-memory address of the entry of Q16 value 0, and of the two ends
+    const int32_t table_mid = (int32_t)smem_base + C::kTableOff + 32767;
+    const int32_t table_lo = table_mid - 32767, table_hi = table_mid + 32767;
+    if constexpr (C::kTable) ok = ptx::mbar_wait(bar_table, 0);
     for (int64_t tile = worker; tile < total_tiles; tile += num_workers) {
       const int ch0 = (int)(tile % c_tiles) * kTileChannels + (int)rank * BC + quarter * 32;   // this warp's channels
       const int t0 = (int)(tile / c_tiles) * TOK + part * (C::kChunksPerWarp * 32);
@@ -299,6 +323,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           __syncwarp();
         }
         uint8_t* stage = stage0 + (kOneStore ? ci : (int)buf) * C::kOutTileBytes;
+        // (all results first, then the stores: a table load may not pass an earlier store to shared
+        // memory, so element-by-element order would put the load latency between any two stores)
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const int32_t a = (int32_t)v[i];
@@ -317,6 +343,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if constexpr (KIND == EPI_HGELU) {
               if constexpr (FAST) o = clamp_sym(ihgelu_upper(requant_upper(a + cur_bias, cur_pb), gk), 127);
               else o = ihgelu_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
+            } else if constexpr (KIND == kEpiGeluTable) {
+              // |requantized value| < 2^30 (upper word of a product of two int32): the sum cannot wrap
+              const int32_t at = max(__viaddmin_s32(requant_upper(a + cur_bias, cur_pb), table_mid, table_hi), table_lo);
+              asm volatile("ld.shared.u8 %0, [%1];" : "=r"(o) : "r"(at));
+            } else if constexpr (KIND == kEpiGeluTableWide) {
+              const int32_t at = clamp_sym(requant_upper_wide(a + cur_bias, cur_pb, cur_pc), 32767) + table_mid;
+              asm volatile("ld.shared.u8 %0, [%1];" : "=r"(o) : "r"(at));
             } else if constexpr (KIND == kEpiGeluLowFree) {
               o = min(igelu_magnitude_upper(requant_upper(a + cur_bias, cur_pb), gk, gelu_rnd), 127);
             } else if constexpr (KIND == kEpiGeluLowFreeWide) {
@@ -328,6 +361,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               else o = igelu_q16_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
             }
           }
+          v[i] = (uint32_t)o;
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int32_t o = (int32_t)v[i];
           // staging tile: row = token i, column = this lane's channel
           if constexpr (C::kOutElem == 4) reinterpret_cast<int32_t*>(stage)[i * 32 + lane] = o;
           else if constexpr (C::kOutElem == 2)
@@ -388,6 +426,11 @@ int launch_inst(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, co
 template <int TOK, bool PAIR>
 int launch_shape(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& mo, const GemmArgs& a,
                  int kind, bool fast, bool wide_form) {
+  if (kind == EPI_GELU && fast && a.gelu_table) {
+    if constexpr (Cfg<TOK, PAIR, kEpiGeluTable>::kValid)          // (256 tokens on one CTA: no room for the table)
+      return wide_form ? launch_inst<TOK, PAIR, kEpiGeluTableWide, true>(ctx, mw, mx, mo, a)
+                       : launch_inst<TOK, PAIR, kEpiGeluTable, true>(ctx, mw, mx, mo, a);
+  }
   if (kind == EPI_GELU && fast && wide_form)
     return a.gelu.low_free ? launch_inst<TOK, PAIR, kEpiGeluLowFreeWide, true>(ctx, mw, mx, mo, a)
                            : launch_inst<TOK, PAIR, kEpiGeluWide, true>(ctx, mw, mx, mo, a);
@@ -444,7 +487,7 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
     const uint64_t dims[2] = {row_bytes, (uint64_t)M};
     const uint64_t str[1] = {row_bytes};
     // (the GELU epilogues store a warp's 64 tokens at once)
-    const bool gelu_kind = epi.kind == EPI_GELU || epi.kind == EPI_HGELU;
+    const bool gelu_kind = epi.kind == EPI_GELU || epi.kind == EPI_HGELU;   // (with or without the table)
     const uint32_t box[2] = {32u * out_elem, gelu_kind ? 64u : 32u};
     int rc = encode_tensor_map(&mo, out, 2, dims, str, box, 0);
     if (rc) return rc;
@@ -453,6 +496,7 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
   a.T = M; a.N = N; a.K = K;
   a.b = epi.d_b; a.c = epi.d_c; a.bias = epi.d_bias; a.gelu = epi.gelu;
   a.status = ctx->d_status;
+  a.gelu_table = ctx->gelu_table_mode == 1 ? nullptr : epi.gelu_table;
   // upper-word epilogue needs both the per-channel multipliers and (for GELU) the final one in that form
   const bool fast = epi.fast != 0 && ((epi.kind != EPI_GELU && epi.kind != EPI_HGELU) || epi.gelu.fast != 0);
   const bool wide_form = epi.fast == 2;

@@ -113,6 +113,8 @@ struct ibert_ctx {
   size_t ws_bytes = 0;
   // linear + LayerNorm fusion: 0 = by problem size, 1 = whenever supported, 2 = never (ibert_set_fusion)
   int fusion_mode = 0;
+  // i-GELU inside the large-tile GEMM epilogue: 0 = from the layer's table, 1 = computed (ibert_set_gelu_table)
+  int gelu_table_mode = 0;
   // optional per-launch event timing (ibert_profile_begin / _end)
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;      // pairs: [2i] before, [2i+1] after launch i
@@ -166,6 +168,9 @@ struct GemmEpilogue {
                            // upper-word form (d_b = low words, d_c = integer parts; GELU epilogue of
                            // the plain GEMM only); 0: generic (b, c) pairs
   GeluConsts gelu;         // EPI_GELU / EPI_HGELU only
+  // EPI_GELU, optional: table[i] = i-GELU(i - 32767) as int8 for every Q16 value (launch_gelu_table).
+  // Tile shapes with 64 KB of shared memory to spare then look the result up instead of computing it.
+  const int8_t* gelu_table = nullptr;
 };
 
 // Upper-word form of a column set: true if for every n, c[n] >= 1 and b[n] << (32 - c[n]) fits

@@ -26,3 +26,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(params=[0, 1], ids=["gelu-table", "gelu-computed"])
+def gelu_mode(request):
+    """Runs a test with FFN1's i-GELU looked up in the layer's table and computed per element."""
+    from gpu_util import ctx
+    c = ctx()
+    c.ibert_set_gelu_table(request.param)
+    yield request.param
+    c.ibert_set_gelu_table(0)

@@ -87,7 +87,7 @@ def test_small_encoder_layers_match_oracle(B, L, H, heads, F, fusion):
         assert_same(got, h, "encoder layer")
 
 
-def test_config0_roberta_base_layer_matches_oracle():
+def test_config0_roberta_base_layer_matches_oracle(gelu_mode):
     x, params = synth.make_model(0, 1)
     got = _run_layers(x, params, 1, 128)[0]
     want = oracle.encoder_layer(params[0], x, 1, 128).out
@@ -105,7 +105,7 @@ def test_config2_three_layers_batch8_match_oracle():
         assert_same(got, h, "config 2 layer")
 
 
-def test_large_shapes_one_layer_L256_and_L512():
+def test_large_shapes_one_layer_L256_and_L512(gelu_mode):
     for cfg, B in ((3, 2), (4, 1)):
         L = synth.CONFIGS[cfg].L
         x, params = synth.make_model(cfg, B, layers=1)
@@ -167,7 +167,7 @@ def test_encoder_layers_with_power_of_two_score_scales():
 
 
 @pytest.mark.parametrize("shrink,S_go_scale", [(2.0, 1.0), (3.5, 1.0), (6.0, 1.0), (3.5, 0.004)])
-def test_layer_with_ffn1_multipliers_of_one_half_and_more(shrink, S_go_scale):
+def test_layer_with_ffn1_multipliers_of_one_half_and_more(shrink, S_go_scale, gelu_mode):
     """A finer GELU-input scale makes the per-channel multipliers S_h1 S_w[n] / S_gi reach 1/2 and go
     beyond 1: the FFN1 epilogue then takes the wide upper-word form (multiplier split into an integer
     part and a 32-bit fraction), with and without the lower output clamp; many values clamp at Q16."""

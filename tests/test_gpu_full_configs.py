@@ -36,7 +36,7 @@ def _full_model_check(config_id, B, sample, scales="analytic"):
     assert got.std() > 12                      # the stack stays well scaled through all layers
 
 
-def test_config2_twelve_layers_batch128_sampled_sequences():
+def test_config2_twelve_layers_batch128_sampled_sequences(gelu_mode):
     _full_model_check(2, 128, sample=(0, 77, 127))
 
 

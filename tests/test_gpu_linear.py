@@ -84,7 +84,7 @@ def test_linear_int16_needs_rows_of_16_bytes():
 
 
 @pytest.mark.parametrize("M,N,K", [(7, 48, 80), (300, 768, 768), (257, 3072, 768), (1000, 4096, 1024), (2500, 3072, 768)])
-def test_linear_with_fused_gelu(M, N, K):
+def test_linear_with_fused_gelu(M, N, K, gelu_mode):
     x, w, bias, S_w, S_x, amax = _problem(M, N, K, 3)
     # scale the problem so the GELU input covers about [-6, 6]
     S_mid = 6.0 / 32767.0
@@ -100,7 +100,7 @@ def test_linear_with_fused_gelu(M, N, K):
 
 @pytest.mark.parametrize("S_out,low_clamp_hit", [(0.17 / 126.0, False), (0.17 / 128.0, None), (0.17 / 400.0, True),
                                                  (6.0 / 127.0, False)])
-def test_linear_with_fused_gelu_around_the_lower_clamp(S_out, low_clamp_hit):
+def test_linear_with_fused_gelu_around_the_lower_clamp(S_out, low_clamp_hit, gelu_mode):
     """Output scales at which the negative lobe of GELU (minimum about -0.17) stays inside int8, just
     touches -127, or saturates: the epilogue without a lower clamp may only run where none is needed."""
     x, w, bias, S_w, S_x, amax = _problem(256, 256, 128, 5)

@@ -119,6 +119,7 @@ def _linear_layernorm(rng):
     K = int(rng.choice([256, 768, 3072]))
     c = ctx()
     c.ibert_set_fusion(int(rng.choice([0, 1, 2])))
+    c.ibert_set_gelu_table(int(rng.choice([0, 0, 1])))
     x = rng.integers(-127, 128, (T, K)).astype(np.int8)
     w = rng.integers(-127, 128, (H, K)).astype(np.int8)
     bias = rng.integers(-20000, 20000, H).astype(np.int32)
@@ -132,6 +133,7 @@ def _linear_layernorm(rng):
     mid = oracle.linear(x, S_x, w, S_w, bias, 1, S_mid)
     assert_same(host(out), oracle.layernorm(mid, S_mid, res, S_res, gamma, beta, S_out)[0], f"linear+layernorm T={T} H={H} K={K}")
     c.ibert_set_fusion(0)
+    c.ibert_set_gelu_table(0)
 
 
 def _layer(rng):
@@ -145,6 +147,7 @@ def _layer(rng):
     params = [p0]
     c = ctx()
     c.ibert_set_fusion(int(rng.choice([0, 1, 2])))
+    c.ibert_set_gelu_table(int(rng.choice([0, 0, 1])))
     ly = c.ibert_layer_create(params[0])
     mode = rng.random()
     if mode < 0.33:
@@ -164,6 +167,7 @@ def _layer(rng):
     assert_same(host(out), want, f"layer B={B} L={L} H={H}")
     ly.close()
     c.ibert_set_fusion(0)
+    c.ibert_set_gelu_table(0)
 
 
 @pytest.mark.parametrize("seed", [11, 12, 13])
@@ -177,3 +181,4 @@ def test_random_calls_in_random_order(seed):
     finally:
         ctx().ibert_set_split_k(0)
         ctx().ibert_set_fusion(0)
+        ctx().ibert_set_gelu_table(0)

@@ -1,8 +1,9 @@
-"""Builds and runs the two issue-rate probes (``csrc/probes``): the INT32 instruction rates the
-integer epilogues depend on, and the tcgen05 kind::i8 MMA issue rate.  Both are stand-alone CUDA
+"""Builds and runs the stand-alone probes (``csrc/probes``): the INT32 instruction rates the
+integer epilogues depend on, the tcgen05 kind::i8 MMA issue rate, and the rates of the data paths of a
+GEMM epilogue (TMEM loads, shared-memory byte stores and table loads).  All are stand-alone CUDA
 programs; their output is what the ALU and INT8 peaks quoted for the kernels rest on.
 
-    python -m paper_2101_01321_b200.probes [int|mma]
+    python -m paper_2101_01321_b200.probes [int|mma|epilogue]
 """
 from __future__ import annotations
 
@@ -12,7 +13,7 @@ import sys
 from pathlib import Path
 
 PKG = Path(__file__).resolve().parent
-PROBES = {"int": "int_issue_probe.cu", "mma": "mma_issue_probe.cu"}
+PROBES = {"int": "int_issue_probe.cu", "mma": "mma_issue_probe.cu", "epilogue": "epilogue_path_probe.cu"}
 
 
 def build(name: str) -> Path:

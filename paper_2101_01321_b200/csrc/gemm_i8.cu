@@ -204,15 +204,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         ptx::bulk_load_1d(smem_base + C::kTableOff, args.gelu_table, kGeluTableBytes, bar_table);
       }
       uint32_t stage = 0, phase = 0;
+      const uint32_t full_leader0 = PAIR ? ptx::map_to_cta(bar_full, 0) : bar_full;
       for (int64_t tile = worker; tile < total_tiles && ok; tile += num_workers) {
         const int c0 = (int)(tile % c_tiles) * kTileChannels + (int)rank * BC;
         const int t0 = (int)(tile / c_tiles) * TOK + (int)rank * C::kXRows;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!ptx::mbar_wait(bar_empty + 8 * stage, phase ^ 1)) { ok = false; break; }
+          if (!ptx::mbar_wait_parked(bar_empty + 8 * stage, phase ^ 1)) { ok = false; break; }
           const uint32_t sw = smem_base + stage * C::kStageBytes;
           if constexpr (PAIR) {
             // both CTAs' copies complete on the leader's barrier, which expects the bytes of both
-            const uint32_t full_leader = ptx::map_to_cta(bar_full + 8 * stage, 0);
+            const uint32_t full_leader = full_leader0 + 8 * stage;
             if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * C::kStageBytes);
             ptx::tma_load_2d_pair(sw, &map_w, full_leader, kb * BK, c0);
             ptx::tma_load_2d_pair(sw + C::kWBytes, &map_x, full_leader, kb * BK, t0);
@@ -234,16 +235,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       constexpr uint32_t idesc = ptx::make_idesc_i8(kTileChannels, TOK, true, true);
       uint32_t stage = 0, phase = 0;
       uint32_t acc = 0, acc_phase = 0;
+      const uint64_t dw0 = ptx::make_kmajor_desc(smem_base, 1024, ptx::kSwizzle128);
+      const uint64_t dx0 = ptx::make_kmajor_desc(smem_base + C::kWBytes, 1024, ptx::kSwizzle128);
       for (int64_t tile = worker; tile < total_tiles && ok; tile += num_workers) {
-        if (!ptx::mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1)) { ok = false; break; }
+        if (!ptx::mbar_wait_parked(bar_acc_empty + 8 * acc, acc_phase ^ 1)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * TOK;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!ptx::mbar_wait(bar_full + 8 * stage, phase)) { ok = false; break; }
+          if (!ptx::mbar_wait_parked(bar_full + 8 * stage, phase)) { ok = false; break; }
           ptx::tc_fence_after_sync();
-          const uint32_t sw = smem_base + stage * C::kStageBytes;
-          const uint64_t dw = ptx::make_kmajor_desc(sw, 1024, ptx::kSwizzle128);
-          const uint64_t dx = ptx::make_kmajor_desc(sw + C::kWBytes, 1024, ptx::kSwizzle128);
+          // (descriptor start addresses count 16-byte units; a stage is a multiple of 1024 bytes)
+          const uint64_t dw = dw0 + (uint64_t)(stage * (C::kStageBytes >> 4)), dx = dx0 + (uint64_t)(stage * (C::kStageBytes >> 4));
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing K inside the swizzle span: +32 bytes = +2 in the encoded start address

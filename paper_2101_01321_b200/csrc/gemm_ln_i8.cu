@@ -172,7 +172,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       for (uint32_t it = 0; unit_of(it) < n_units && ok; ++it) {
         const int t0 = (int)tile_of(it) * kTok;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!ptx::mbar_wait(bar_empty + 8 * stage, phase ^ 1)) { ok = false; break; }
+          if (!ptx::mbar_wait_parked(bar_empty + 8 * stage, phase ^ 1)) { ok = false; break; }
           const uint32_t sx = smem_base + stage * kStageBytes;
           if constexpr (PAIR) {
             // both CTAs' copies complete on the leader's barrier, which expects the bytes of both
@@ -196,11 +196,11 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       const uint16_t pair_mask = (uint16_t)(3u << leader);
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
       for (uint32_t it = 0; unit_of(it) < n_units && ok; ++it) {
-        if (!ptx::mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1)) { ok = false; break; }
+        if (!ptx::mbar_wait_parked(bar_acc_empty + 8 * acc, acc_phase ^ 1)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * kCh;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!ptx::mbar_wait(bar_full + 8 * stage, phase)) { ok = false; break; }
+          if (!ptx::mbar_wait_parked(bar_full + 8 * stage, phase)) { ok = false; break; }
           ptx::tc_fence_after_sync();
           const uint32_t sx = smem_base + stage * kStageBytes;
           const uint64_t dx = ptx::make_kmajor_desc(sx, 1024, ptx::kSwizzle128);

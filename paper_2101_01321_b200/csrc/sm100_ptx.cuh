@@ -95,6 +95,31 @@ __device__ __forceinline__ bool mbar_wait_ns(uint32_t bar, uint32_t parity, uint
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   return mbar_wait_ns(bar, parity, kWaitLimitNs);
 }
+// The same bounded wait for the single threads that feed the tensor pipe (TMA producer, MMA issuer).
+// Such a thread shares its scheduler with busy epilogue warps and gets an issue slot only now and
+// then, so every instruction of its loop counts: try_wait is given a long suspend-time hint, which
+// parks the thread in hardware until the phase completes -- normally one instruction per wait
+// instead of a polling loop.  The timer is read only after repeated failures.
+__device__ __forceinline__ bool mbar_test_parked(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(1000000u)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_parked(uint32_t bar, uint32_t parity) {
+  for (int i = 0; i < 16; ++i)
+    if (mbar_test_parked(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (;;) {
+    if (mbar_test_parked(bar, parity)) return true;
+    if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+  }
+}
 
 // ------------------------------------------------------------------ proxies / fences
 __device__ __forceinline__ void fence_proxy_async_smem() {

@@ -174,7 +174,6 @@ attention_coarse_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid
     ptx::mbar_init(bar_mma, 1);
     ptx::fence_mbar_init();
     ptx::tma_prefetch_desc(&map_qk);
-    ptx::tma_prefetch_desc(&map_v);
   }
   if (warp == 0) {
     ptx::tmem_alloc(ptx::smem_addr(s_tmem), a.tmem_cols);
@@ -321,14 +320,16 @@ attention_coarse_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid
 
 // ---------------------------------------------------------------------------------------------
 // The main kernel.  A persistent CTA owns one (batch, head) pair at a time and walks its 128-query
-// tiles, so K, V and the transposed V are loaded / built once per pair.  The CTA has 128 G threads,
+// tiles, so K and V are loaded once per pair.  V is the B operand of the second MMA exactly as TMA
+// delivers it ([key][head dim], 64-byte swizzle): head dim contiguous is the MN-major operand form
+// (instruction-descriptor bit 16), one descriptor per 32 keys -- no transposed copy.  The CTA has 128 G threads,
 // G >= ceil(L / 128) column groups: warp w works on TMEM lane quadrant w & 3 (the only lanes a warp
 // may address) and on the 32-column chunks of group w >> 2, so a score row is shared by G threads
 // that exchange their partial maximum and partial sum through shared memory.  Up to 128 keys and
 // with many pairs that is one thread per row and four CTAs per SM; at 512 keys one CTA of 16 warps
 // fills the SM's TMEM; with fewer pairs than SMs the launcher raises G to shorten the lone CTA's softmax.
-// Every operand buffer is refilled as soon as its last reader is done (V after the transpose, K
-// and a lone Q after the score MMAs), so the next pair's loads hide behind the softmax.
+// Every operand buffer is refilled as soon as its last reader is done (K and a lone Q after the
+// score MMAs, V after the P V MMAs), so the next pair's loads hide behind the softmax and the epilogue.
 // Requires the unclamped i-exp form (ExpConsts::wide_post >= 0).
 // ---------------------------------------------------------------------------------------------
 constexpr int kMaxThreads = 512;
@@ -351,16 +352,14 @@ struct AttnArgs {
 // PACKED: a.lens holds first-row offsets (a separate instantiation: the padded path compiles as without it)
 template <bool PACKED>
 __global__ void __launch_bounds__(kMaxThreads, 1)
-attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_constant__ CUtensorMap map_v,
-                 const AttnArgs a) {
+attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int slab_bytes = 128 * kHeadDim;                       // 8 KB
   uint8_t* sQ = smem;                                          // [q_bufs][128 rows][64 B], 64-byte swizzle
   uint8_t* sK = sQ + a.q_bufs * slab_bytes;                    // [n_slabs][128][64 B], 64-byte swizzle
-  uint8_t* sVs = sK + a.n_slabs * slab_bytes;                  // [n_slabs][128][64 B], plain rows
-  uint8_t* sVt = sVs + a.n_slabs * slab_bytes;                 // [n_slabs][64 rows][128 B], swizzled
-  uint8_t* sP = sVt + a.n_slabs * slab_bytes;                  // [n_slabs][128 rows][128 B], swizzled
+  uint8_t* sVs = sK + a.n_slabs * slab_bytes;                  // [n_slabs][128][64 B], 64-byte swizzle
+  uint8_t* sP = sVs + a.n_slabs * slab_bytes;                  // [n_slabs][128 rows][128 B], swizzled
   int32_t* s_max = reinterpret_cast<int32_t*>(sP + a.n_slabs * 128 * 128);   // [4][128]
   uint32_t* s_sum = reinterpret_cast<uint32_t*>(s_max + 4 * 128);            // [4][128]
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_sum + 4 * 128);
@@ -383,7 +382,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
     ptx::mbar_init(bar_mma, 1);
     ptx::fence_mbar_init();
     ptx::tma_prefetch_desc(&map_qk);
-    ptx::tma_prefetch_desc(&map_v);
   }
   if (warp == 0) {
     ptx::tmem_alloc(ptx::smem_addr(s_tmem), a.tmem_cols);
@@ -417,7 +415,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
     const int row0 = PACKED ? __ldg(a.lens + batch) : 0, zb = PACKED ? 0 : batch;
     ptx::mbar_arrive_expect_tx(bar_v, (uint32_t)(a.n_slabs * slab_bytes));
     for (int s = 0; s < a.n_slabs; ++s)
-      ptx::tma_load_3d(ptx::smem_addr(sVs + s * slab_bytes), &map_v, bar_v, 2 * a.H + head * kHeadDim, row0 + s * 128, zb);
+      ptx::tma_load_3d(ptx::smem_addr(sVs + s * slab_bytes), &map_qk, bar_v, 2 * a.H + head * kHeadDim, row0 + s * 128, zb);
   };
 
   uint32_t q_phase[2] = {0, 0};
@@ -459,16 +457,11 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
     const int n_chunks = Lp >> 5, per_grp = (n_chunks + G - 1) / G;
     const int c_begin = min(grp * per_grp, n_chunks) * 32, c_end = min((grp + 1) * per_grp, n_chunks) * 32;
 
-    // ---- V [j][d] -> Vt [d][j] once per (batch, head); the plain copy is then free for the next pair
-    ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_v, kv_phase));
-    if (ok) {
-      transpose_v(sVs, sVt, a.n_slabs * 128, tid, n_threads);
-      ptx::fence_proxy_async_smem();
+    if constexpr (PACKED) {
+      ok = __syncthreads_and(ok);             // the draw of the next pair is visible
+      if (!ok) break;
+      next = s_next[iter & 1];
     }
-    ok = __syncthreads_and(ok);
-    if (!ok) break;
-    if constexpr (PACKED) next = s_next[iter & 1];
-    if (tid == 0 && next < total) load_v(next);
     ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_k, kv_phase));
     kv_phase ^= 1;
 
@@ -608,6 +601,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
         }
         ptx::fence_proxy_async_smem();
       }
+      // V of this pair (requested while the previous pair's epilogue ran) is needed from here on
+      if (qt == 0 && ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_v, kv_phase ^ 1));
       ptx::tc_fence_before_sync();
       ok = __syncthreads_and(ok);             // P complete; every row's exponentials have been consumed
       if (!ok) break;
@@ -615,17 +610,21 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid_consta
       // ---- ctx = P V: K = Lp in steps of 32, accumulator in columns 0..63 (scores are dead)
       if (tid == 0) {
         ptx::tc_fence_after_sync();
-        const uint32_t idesc = ptx::make_idesc_i8(128, kHeadDim, false, true);   // u8 x s8
+        // B = V as loaded ([key][head dim], head dim contiguous): the MN-major operand form (bit 16)
+        const uint32_t idesc = ptx::make_idesc_i8(128, kHeadDim, false, true) | (1u << 16);   // u8 x s8
         for (int kk = 0; kk < Lp / 32; ++kk) {
           const int kb = kk >> 2, ks = kk & 3;
           const uint64_t dp = ptx::make_kmajor_desc(ptx::smem_addr(sP + kb * 128 * 128), 1024, ptx::kSwizzle128);
-          const uint64_t dv = ptx::make_kmajor_desc(ptx::smem_addr(sVt + kb * 64 * 128), 1024, ptx::kSwizzle128);
-          ptx::mma_i8_ss(tmem_base, dp + 2 * ks, dv + 2 * ks, idesc, kk != 0 ? 1u : 0u);
+          const uint32_t va = ptx::smem_addr(sVs + kk * 32 * kHeadDim);
+          const uint64_t dv = (uint64_t)((va & 0x3FFFFu) >> 4) | ((uint64_t)(512 >> 4) << 16) | ((uint64_t)(512 >> 4) << 32) |
+                              ((uint64_t)1 << 46) | ((uint64_t)ptx::kSwizzle64 << 61);
+          ptx::mma_i8_ss(tmem_base, dp + 2 * ks, dv, idesc, kk != 0 ? 1u : 0u);
         }
         ptx::mma_commit(bar_mma);
       }
       ok = __all_sync(0xffffffffu, ptx::mbar_wait(bar_mma, mma_phase));
       mma_phase ^= 1;
+      if (ok && tid == 0 && last_tile && next < total) load_v(next);   // V was read by the MMAs that just completed
 
       // ---- epilogue: the 64 context values of a row in two halves, taken by column groups 0 and 1
       // (by group 0 alone when there is only one)
@@ -716,7 +715,7 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
     }
     a.q_bufs = n_slabs > 1 ? 2 : 1;
     a.tmem_cols = cols; a.k = k; a.lens = cu_seqlens ? cu_seqlens : lens; a.out = out; a.status = ctx->d_status;
-    const int smem = a.q_bufs * slab + 3 * n_slabs * slab + n_slabs * 128 * 128 + 2 * 4 * 128 * 4 + 64 + 1024;
+    const int smem = a.q_bufs * slab + 2 * n_slabs * slab + n_slabs * 128 * 128 + 2 * 4 * 128 * 4 + 64 + 1024;
     // resident CTAs per SM: bounded by the register file (128 G threads of at most 128 registers),
     // by the 512 TMEM columns and by shared memory.  The bound must not exceed what TMEM allows:
     // a CTA that cannot get its columns would wait for a resident one to finish.
@@ -731,8 +730,8 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
         return IBERT_ERR_CUDA;
       smem_set = smem;
     }
-    if (int rc2 = cu_seqlens ? launch_pdl(attention_kernel<true>, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1, mqk, mv, a)
-                             : launch_pdl(attention_kernel<false>, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1, mqk, mv, a))
+    if (int rc2 = cu_seqlens ? launch_pdl(attention_kernel<true>, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1, mqk, a)
+                             : launch_pdl(attention_kernel<false>, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1, mqk, a))
       return rc2;
     return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
   }

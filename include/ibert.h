@@ -358,9 +358,11 @@ enum {
    derivation, or IBERT_ERR_VALUE_RANGE on a mismatch.  q_ln2_out (may be NULL) receives q_ln2. */
 int ibert_selftest_exp_division(double S, int32_t* q_ln2_out);
 
-/* Self-test of the bounded device-side waits (no counterpart in the paper): enqueues a one-warp
-   kernel that waits on a barrier nobody arrives on, with a limit of limit_us microseconds
-   (1 .. 100000) on the GPU's nanosecond timer.  When the limit runs out the kernel records
+/* Self-test of the bounded device-side waits (no counterpart in the paper): enqueues a two-warp
+   kernel that waits on a barrier nobody arrives on -- one warp by the polling form of the wait,
+   one by the form that parks the thread in hardware between polls (the GEMM feeder threads use
+   it) -- with a limit of limit_us microseconds (1 .. 100000) on the GPU's nanosecond timer (the
+   parked form may take up to about 20 ms longer).  When both limits have run out the kernel records
    IBERT_ERR_TIMEOUT in the context's status word -- exactly what every kernel of the library does
    when one of its waits (limit: one second) expires -- and returns normally; the context stays
    usable.  ibert_last_status() then returns IBERT_ERR_TIMEOUT once. */

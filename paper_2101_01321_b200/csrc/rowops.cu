@@ -515,17 +515,24 @@ __global__ void __launch_bounds__(kThreads) embed_gather_kernel(const int32_t* _
 }
 
 // ----------------------------------------------------------------------------- wait self-test
-// One warp waits on an mbarrier nobody arrives on, with a short limit; when the limit runs out it
-// records IBERT_ERR_TIMEOUT like every kernel of the library does, and returns normally.
-__global__ void __launch_bounds__(32) wait_timeout_kernel(uint64_t limit_ns, int32_t* status) {
+// Two warps wait on an mbarrier nobody arrives on, with a short limit: one by the polling form of the
+// bounded wait (mbar_wait_ns), one by the parked form the GEMM feeder threads use (mbar_wait_parked_ns).
+// When BOTH limits have run out the kernel records IBERT_ERR_TIMEOUT like every kernel of the library
+// does, and returns normally.
+__global__ void __launch_bounds__(64) wait_timeout_kernel(uint64_t limit_ns, int32_t* status) {
   __shared__ uint64_t bar;
+  __shared__ int expired;
   if (threadIdx.x == 0) {
     ptx::mbar_init(ptx::smem_addr(&bar), 1);
     ptx::fence_mbar_init();
+    expired = 0;
   }
-  __syncwarp();
-  const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait_ns(ptx::smem_addr(&bar), 0, limit_ns));
-  if (!ok && threadIdx.x == 0) atomicCAS(status, 0, IBERT_ERR_TIMEOUT);
+  __syncthreads();
+  const bool ok = (threadIdx.x < 32) ? __all_sync(0xffffffffu, ptx::mbar_wait_ns(ptx::smem_addr(&bar), 0, limit_ns))
+                                     : __all_sync(0xffffffffu, ptx::mbar_wait_parked_ns(ptx::smem_addr(&bar), 0, limit_ns));
+  if (!ok && (threadIdx.x & 31) == 0) atomicAdd(&expired, 1);
+  __syncthreads();
+  if (threadIdx.x == 0 && expired == 2) atomicCAS(status, 0, IBERT_ERR_TIMEOUT);
 }
 
 // Row cu[b] of x (the first token of sequence b of a packed batch) -> row b of out; one warp per row.
@@ -550,7 +557,7 @@ int check_launch() { return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT
 }  // namespace
 
 int launch_wait_timeout(ibert_ctx* ctx, uint64_t limit_ns) {
-  wait_timeout_kernel<<<1, 32, 0, ctx->stream>>>(limit_ns, ctx->d_status);
+  wait_timeout_kernel<<<1, 64, 0, ctx->stream>>>(limit_ns, ctx->d_status);
   return check_launch();
 }
 

@@ -111,14 +111,17 @@ __device__ __forceinline__ bool mbar_test_parked(uint32_t bar, uint32_t parity) 
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait_parked(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_parked_ns(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
   for (int i = 0; i < 16; ++i)
     if (mbar_test_parked(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (;;) {
     if (mbar_test_parked(bar, parity)) return true;
-    if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+    if (global_timer_ns() - t0 > limit_ns) return false;
   }
+}
+__device__ __forceinline__ bool mbar_wait_parked(uint32_t bar, uint32_t parity) {
+  return mbar_wait_parked_ns(bar, parity, kWaitLimitNs);
 }
 
 // ------------------------------------------------------------------ proxies / fences

@@ -308,8 +308,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       if (!ok) continue;                               // keep walking the tiles, touch nothing
       ptx::tc_fence_after_sync();
       const uint32_t t_row = tmem_base + acc * TOK + ((uint32_t)(quarter * 32) << 16);
+      // (a warp whose token range lies past the last row -- the ragged last tile of a token count that is
+      // not a multiple of the tile -- has nothing to read or store: the tile then costs its main loop only)
 #pragma unroll 1
-      for (int ci = 0; ci < C::kChunksPerWarp; ++ci) {
+      for (int ci = 0; ci < ((int64_t)t0 < args.T ? C::kChunksPerWarp : 0); ++ci) {
         const int col = (part * C::kChunksPerWarp + ci) * 32;
         uint32_t v[32];
         ptx::tmem_ld32(t_row + col, v);

@@ -276,7 +276,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             const int2 cb = s_cb[col + i];
             const int32_t q16 = clamp_sym(requant_upper((int32_t)v[i] + cb.y, cb.x), 32767);
             const int32_t rv = sext_byte(rw[i >> 2], i & 3);
-            const int32_t val = q16 + requant_upper(rv << ln.res_sh, ln.b_r);
+            const int32_t val = q16 + ((rv * ln.res_nb + ln.res_nhalf) >> ln.res_nc);   // the residual, rescaled (narrow form)
             v[i] = (uint32_t)val;
             s1 += val;
             s2 += (uint64_t)((int64_t)val * (int64_t)val);
@@ -444,7 +444,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 bool gemm_ln_supported(int H, int K, const GemmEpilogue& epi, const LnConsts& ln) {
   if (H % kCh != 0 || H / kCh > kMaxCta || K % 16 != 0) return false;    // cluster of H / 256 CTAs, at most 4
   if (!epi.fast || epi.kind != EPI_Q16) return false;
-  if (!ln.has_res || !ln.res_fast || !ln.out_fast || ln.C != H) return false;
+  if (!ln.has_res || !ln.res_fast || !ln.res_narrow || !ln.out_fast || ln.C != H) return false;
   // |v| = |Q16 value + rescaled residual| must stay below 2^18: sums over H <= 2048 channels then fit
   // int32, sums of squares 2^47, and sigma 2^24
   const double res_max = 127.0 * std::ldexp((double)ln.b_r, ln.res_sh - 32);

@@ -259,6 +259,25 @@ int make_ln_residual(double S_r, double S, LnConsts* k) {
   // |r| <= 127 leaves 24 bits of headroom: r << (32 - c_r) fits int32 for c_r >= 8
   k->res_fast = (k->c_r >= 8 && k->c_r <= 31) ? 1 : 0;
   k->res_sh = 32 - k->c_r;
+  // narrow form: drop seven bits of the 31-bit multiplier (|r| <= 128 then keeps the product inside int32) and
+  // keep it only if every int8 value gives the exact form's result
+  k->res_narrow = 0;
+  k->res_nb = k->res_nc = k->res_nhalf = 0;
+  if (k->c_r >= 8 && k->c_r <= 31) {
+    const int nc = k->c_r - 7;
+    for (int rounding = 1; rounding >= 0 && !k->res_narrow; --rounding) {
+      const int64_t nb = ((int64_t)k->b_r + (rounding ? 64 : 0)) >> 7;
+      if (nb >= (int64_t(1) << 24)) continue;
+      const int64_t nhalf = int64_t(1) << (nc - 1);
+      bool same = true;
+      for (int r = -128; r <= 127 && same; ++r) {
+        const int64_t exact = ((int64_t)r * k->b_r + (int64_t(1) << (k->c_r - 1))) >> k->c_r;
+        const int64_t narrow = ((int64_t)r * nb + nhalf) >> nc;
+        same = exact == narrow && std::llabs((int64_t)r * nb + nhalf) < (int64_t(1) << 31);
+      }
+      if (same) { k->res_narrow = 1; k->res_nb = (int32_t)nb; k->res_nc = nc; k->res_nhalf = (int32_t)nhalf; }
+    }
+  }
   return IBERT_OK;
 }
 

@@ -68,6 +68,9 @@ struct LnConsts {
   // out_fast (the B_i table then already holds the shifted addends)
   int32_t res_sh, res_fast;
   int32_t out_sh, out_fast;
+  // the residual rescale in 32-bit arithmetic: (r * res_nb + res_nhalf) >> res_nc with a 24-bit multiplier,
+  // offered (res_narrow != 0) only when the host has checked all 256 int8 values against the exact form
+  int32_t res_nb, res_nc, res_nhalf, res_narrow;
 };
 
 int dyadic(double m, int32_t* b, int32_t* c);

@@ -425,7 +425,7 @@ __global__ void __launch_bounds__(kThreads, DEPTH == 2 ? 3 : 2) layernorm_pipe_k
     for (int j = 0; j < VPL; ++j)
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        v[j][i] += requant_upper(sext_byte(rw[j], i) << k.res_sh, k.b_r);
+        v[j][i] += (sext_byte(rw[j], i) * k.res_nb + k.res_nhalf) >> k.res_nc;   // the residual, rescaled (narrow form)
         sum += v[j][i];
         s2 += (uint64_t)((int64_t)v[j][i] * (int64_t)v[j][i]);
       }
@@ -636,7 +636,7 @@ static int launch_layernorm_t(ibert_ctx* ctx, const QT* q, const int8_t* r, int6
   const bool vec = (k.C % 4) == 0;
   const int vpl = (k.C + 127) / 128;
   const bool fast = vec && k.out_fast && (!k.has_res || k.res_fast);
-  if (fast && k.has_res && k.C % 16 == 0 && k.C <= 1024) {
+  if (fast && k.has_res && k.res_narrow && k.C % 16 == 0 && k.C <= 1024) {
     // streaming variant: per-warp ring of row slots filled by bulk async copies
     const int depth = 2;
     const size_t smem = (size_t)(kThreads / 32) * depth * (size_t)k.C * (sizeof(QT) + 1) + (kThreads / 32) * depth * 8 +

@@ -65,6 +65,8 @@ def lib():
         L.ibert_set_split_k.argtypes = [vp, i32]
         L.ibert_set_gelu_table.argtypes = [vp, i32]
         L.ibert_set_gelu_table.restype = i32
+        L.ibert_set_qkv_layout.argtypes = [vp, i32]
+        L.ibert_set_qkv_layout.restype = i32
         L.ibert_softmax_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
         L.ibert_softmax_lut_i.argtypes = [vp, vp, dbl, i64, i32, i32, vp, vp]
         L.ibert_gelu_i.argtypes = [vp, vp, dbl, i64, dbl, vp, vp]
@@ -190,6 +192,10 @@ class Context:
     def ibert_set_split_k(self, mode: int) -> None:
         """0: split K of small GEMMs by size (default); 1: never; 2 / 4: force that cluster width."""
         _chk(lib().ibert_set_split_k(self.h, mode), "ibert_set_split_k")
+
+    def ibert_set_qkv_layout(self, mode: int) -> None:
+        """0: the layer keeps Q | K | V transposed between its kernels where shapes allow (default); 1: never."""
+        _chk(lib().ibert_set_qkv_layout(self.h, mode), "ibert_set_qkv_layout")
 
     def ibert_set_gelu_table(self, mode: int) -> None:
         """0: FFN1's i-GELU from the layer's table where the tile shape has room (default); 1: computed."""

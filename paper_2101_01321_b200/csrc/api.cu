@@ -221,6 +221,14 @@ int ibert_set_split_k(ibert_ctx* ctx, int mode) {
   });
 }
 
+int ibert_set_qkv_layout(ibert_ctx* ctx, int mode) {
+  return guarded([&]() -> int {
+  if (!ctx || mode < 0 || mode > 1) return IBERT_ERR_ARG;
+  ctx->qkv_layout_mode = mode;
+  return IBERT_OK;
+  });
+}
+
 int ibert_set_gelu_table(ibert_ctx* ctx, int mode) {
   return guarded([&]() -> int {
   if (!ctx || mode < 0 || mode > 1) return IBERT_ERR_ARG;
@@ -804,9 +812,15 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
   GemmEpilogue e{};
   int rc;
   e.kind = EPI_INT8; e.d_b = ly->b_qkv; e.d_c = ly->c_qkv; e.d_bias = ly->bias_qkv; e.fast = ly->fast_qkv;
+  // Q | K | V between the two kernels: transposed ([3H][T]) where both sides take it -- a thread of the GEMM
+  // holds one channel of 32 tokens, which are contiguous bytes of that layout
+  const bool qkv_t = ctx->qkv_layout_mode == 0 && !cu_seqlens && ly->fast_qkv == 1 &&
+                     attention_takes_transposed(B, L, ly->attn);
+  e.out_transposed = qkv_t;
   { ProfileScope ps(ctx, IBERT_K_GEMM_QKV); rc = launch_gemm_i8(ctx, x, ly->w_qkv, T, 3 * H, H, e, qkv); }
+  e.out_transposed = false;
   if (rc) return rc;
-  { ProfileScope ps(ctx, IBERT_K_ATTENTION); rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, lens, cx, cu_seqlens, T); }
+  { ProfileScope ps(ctx, IBERT_K_ATTENTION); rc = launch_attention(ctx, qkv, B, L, H, ly->d.heads, ly->attn, lens, cx, cu_seqlens, T, qkv_t); }
   if (rc) return rc;
   // output projection + residual + LayerNorm: one kernel when shapes and constants allow it
   e.kind = EPI_Q16; e.d_b = ly->b_o; e.d_c = ly->c_o; e.d_bias = ly->bias_o; e.fast = ly->fast_o;

@@ -333,6 +333,9 @@ attention_coarse_kernel(const __grid_constant__ CUtensorMap map_qk, const __grid
 // Requires the unclamped i-exp form (ExpConsts::wide_post >= 0).
 // ---------------------------------------------------------------------------------------------
 constexpr int kMaxThreads = 512;
+// MN-major operand tiles [64 dims][128 tokens]: 8 KB from one 128-token tile to the next, 1 KB from one
+// group of eight dims to the next
+constexpr uint32_t kMnLbo = 8192, kMnSbo = 1024;
 
 struct AttnArgs {
   int B, L, H, heads;
@@ -350,7 +353,11 @@ struct AttnArgs {
 };
 
 // PACKED: a.lens holds first-row offsets (a separate instantiation: the padded path compiles as without it)
-template <bool PACKED>
+// QT: the input is the TRANSPOSED tensor qkv^T [3H][tokens] (token index contiguous), as the QKV GEMM
+// writes it without a transposing store: Q^T and K^T tiles [64 dims][128 tokens] are MN-major
+// operands of the score MMA (instruction-descriptor bits 15 and 16), V^T [64 dims][128 keys] is the
+// K-major B operand of the second MMA.  Padded batches with L a multiple of 16 only.
+template <bool PACKED, bool QT = false>
 __global__ void __launch_bounds__(kMaxThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
   extern __shared__ uint8_t smem_raw[];
@@ -405,21 +412,29 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
     const int head = item % a.heads, batch = item / a.heads;
     const int row0 = PACKED ? __ldg(a.lens + batch) : 0, zb = PACKED ? 0 : batch;
     ptx::mbar_arrive_expect_tx(bar_q0 + 8 * buf, (uint32_t)slab_bytes);
+    if constexpr (QT) ptx::tma_load_2d(ptx::smem_addr(sQ + buf * slab_bytes), &map_qk, bar_q0 + 8 * buf, batch * a.L + qt * 128, head * kHeadDim);
+    else
     ptx::tma_load_3d(ptx::smem_addr(sQ + buf * slab_bytes), &map_qk, bar_q0 + 8 * buf, head * kHeadDim, row0 + qt * 128, zb);
   };
   auto load_k = [&](int item) {
     const int head = item % a.heads, batch = item / a.heads;
     const int row0 = PACKED ? __ldg(a.lens + batch) : 0, zb = PACKED ? 0 : batch;
     ptx::mbar_arrive_expect_tx(bar_k, (uint32_t)(a.n_slabs * slab_bytes));
-    for (int s = 0; s < a.n_slabs; ++s)
+    for (int s = 0; s < a.n_slabs; ++s) {
+      if constexpr (QT) ptx::tma_load_2d(ptx::smem_addr(sK + s * slab_bytes), &map_qk, bar_k, batch * a.L + s * 128, a.H + head * kHeadDim);
+      else
       ptx::tma_load_3d(ptx::smem_addr(sK + s * slab_bytes), &map_qk, bar_k, a.H + head * kHeadDim, row0 + s * 128, zb);
+    }
   };
   auto load_v = [&](int item) {
     const int head = item % a.heads, batch = item / a.heads;
     const int row0 = PACKED ? __ldg(a.lens + batch) : 0, zb = PACKED ? 0 : batch;
     ptx::mbar_arrive_expect_tx(bar_v, (uint32_t)(a.n_slabs * slab_bytes));
-    for (int s = 0; s < a.n_slabs; ++s)
+    for (int s = 0; s < a.n_slabs; ++s) {
+      if constexpr (QT) ptx::tma_load_2d(ptx::smem_addr(sVs + s * slab_bytes), &map_qk, bar_v, batch * a.L + s * 128, 2 * a.H + head * kHeadDim);
+      else
       ptx::tma_load_3d(ptx::smem_addr(sVs + s * slab_bytes), &map_qk, bar_v, 2 * a.H + head * kHeadDim, row0 + s * 128, zb);
+    }
   };
 
   uint32_t q_phase[2] = {0, 0};
@@ -477,6 +492,22 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
       // ---- S = Q K^T: K = 64 bytes = two MMA K-steps; N in chunks of at most 256 columns
       if (ok && tid == 0) {
         ptx::tc_fence_after_sync();
+        if constexpr (QT) {
+          // MN-major operands: [64 dims][128 tokens] tiles, 128-byte swizzle; eight dims form a 1 KB group,
+          // a K step of 32 dims is four groups (4 KB); a second 128 keys of N is the next 8 KB tile
+          auto mn_desc = [](uint32_t addr) {
+            return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(kMnLbo >> 4) << 16) | ((uint64_t)(kMnSbo >> 4) << 32) |
+                   ((uint64_t)1 << 46) | ((uint64_t)ptx::kSwizzle128 << 61);
+          };
+          const uint64_t dq = mn_desc(ptx::smem_addr(sQ + qbuf * slab_bytes));
+          for (int n0 = 0; n0 < Lp; n0 += 256) {
+            const int nn = min(256, Lp - n0);
+            const uint32_t idesc = ptx::make_idesc_i8(128, nn, true, true) | (1u << 15) | (1u << 16);
+            const uint64_t dk = mn_desc(ptx::smem_addr(sK + (n0 >> 7) * slab_bytes));
+            ptx::mma_i8_ss(tmem_base + n0, dq, dk, idesc, 0u);
+            ptx::mma_i8_ss(tmem_base + n0, dq + (4096 >> 4), dk + (4096 >> 4), idesc, 1u);
+          }
+        } else {
         const uint64_t dq = ptx::make_kmajor_desc(ptx::smem_addr(sQ + qbuf * slab_bytes), 512, ptx::kSwizzle64);
         for (int n0 = 0; n0 < Lp; n0 += 256) {
           const int nn = min(256, Lp - n0);
@@ -484,6 +515,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
           const uint64_t dk = ptx::make_kmajor_desc(ptx::smem_addr(sK + n0 * kHeadDim), 512, ptx::kSwizzle64);
           ptx::mma_i8_ss(tmem_base + n0, dq, dk, idesc, 0u);
           ptx::mma_i8_ss(tmem_base + n0, dq + 2, dk + 2, idesc, 1u);
+        }
         }
         ptx::mma_commit(bar_mma);
         // the other Q buffer was read by the previous tile's score MMAs, which have completed
@@ -615,10 +647,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
       if (tid == 0) {
         ptx::tc_fence_after_sync();
         // B = V as loaded ([key][head dim], head dim contiguous): the MN-major operand form (bit 16)
-        const uint32_t idesc = ptx::make_idesc_i8(128, kHeadDim, false, true) | (1u << 16);   // u8 x s8
+        const uint32_t idesc = ptx::make_idesc_i8(128, kHeadDim, false, true) | (QT ? 0u : (1u << 16));   // u8 x s8
         for (int kk = 0; kk < Lp / 32; ++kk) {
           const int kb = kk >> 2, ks = kk & 3;
           const uint64_t dp = ptx::make_kmajor_desc(ptx::smem_addr(sP + kb * 128 * 128), 1024, ptx::kSwizzle128);
+          if constexpr (QT) {
+            // V^T [64 dims][128 keys]: the plain K-major operand
+            const uint64_t dvt = ptx::make_kmajor_desc(ptx::smem_addr(sVs + kb * slab_bytes), 1024, ptx::kSwizzle128);
+            ptx::mma_i8_ss(tmem_base, dp + 2 * ks, dvt + 2 * ks, idesc, kk != 0 ? 1u : 0u);
+            continue;
+          }
           const uint32_t va = ptx::smem_addr(sVs + kk * 32 * kHeadDim);
           const uint64_t dv = (uint64_t)((va & 0x3FFFFu) >> 4) | ((uint64_t)(512 >> 4) << 16) | ((uint64_t)(512 >> 4) << 32) |
                               ((uint64_t)1 << 46) | ((uint64_t)ptx::kSwizzle64 << 61);
@@ -686,10 +724,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
 
 }  // namespace
 
+bool attention_takes_transposed(int B, int L, const AttnConsts& k) {
+  // token offsets b L are the innermost TMA coordinate (16-byte aligned), B L the row pitch
+  return L % 16 == 0 && ((int64_t)B * L) % 16 == 0 && k.e.wide_post >= 0;
+}
+
 int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
                      const AttnConsts& k, const int32_t* lens, int8_t* out, const int32_t* cu_seqlens,
-                     int64_t total_rows) {
+                     int64_t total_rows, bool qkv_t) {
   if (B == 0) return IBERT_OK;
+  if (qkv_t && (cu_seqlens || !attention_takes_transposed(B, L, k))) return IBERT_ERR_ARG;
   if (cu_seqlens && k.e.wide_post < 0) return IBERT_ERR_SCALE_RANGE;   // packed batches: main kernel only
   const int Lp = (L + 31) & ~31, n_slabs = (L + 127) / 128;
   uint32_t cols = 64;
@@ -702,6 +746,13 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
   const uint32_t box[3] = {kHeadDim, 128, 1};
   int rc = encode_tensor_map(&mqk, qkv, 3, dims, str, box, 64);
   if (rc) return rc;
+  if (qkv_t) {
+    // qkv^T [3H][B L]: a tile is 64 dims x 128 tokens, rows of 128 bytes, 128-byte swizzle
+    const uint64_t tdims[2] = {(uint64_t)B * L, (uint64_t)3 * H};
+    const uint64_t tstr[1] = {(uint64_t)B * L};
+    const uint32_t tbox[2] = {128, kHeadDim};
+    if ((rc = encode_tensor_map(&mqk, qkv, 2, tdims, tstr, tbox, 128))) return rc;
+  }
   rc = encode_tensor_map(&mv, qkv, 3, dims, str, box, 0);
   if (rc) return rc;
   const int slab = 128 * kHeadDim;
@@ -729,10 +780,15 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
     static int smem_set_dev[kMaxDevices] = {0};
     int& smem_set = smem_set_dev[ctx->device % kMaxDevices];
     if (smem > smem_set) {
-      if (cudaFuncSetAttribute(attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      if (cudaFuncSetAttribute(attention_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+          cudaFuncSetAttribute(attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
           cudaFuncSetAttribute(attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return IBERT_ERR_CUDA;
       smem_set = smem;
+    }
+    if (qkv_t) {
+      if (int rc2 = launch_pdl(attention_kernel<false, true>, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1, mqk, a)) return rc2;
+      return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA;
     }
     if (int rc2 = cu_seqlens ? launch_pdl(attention_kernel<true>, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1, mqk, a)
                              : launch_pdl(attention_kernel<false>, dim3(grid), dim3(128 * a.groups), (size_t)smem, ctx->stream, 1, mqk, a))

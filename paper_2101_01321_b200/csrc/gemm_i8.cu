@@ -71,6 +71,7 @@ int encode_tensor_map(CUtensorMap* map, const void* base, int rank, const uint64
   }
   const CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                 : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                : swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
                                                       : CU_TENSOR_MAP_SWIZZLE_NONE;
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr,
                   bdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -97,6 +98,8 @@ constexpr int kEpiGeluWide = 17, kEpiGeluLowFreeWide = 18;
 // the i-GELU kernel itself) returns the same bits.  Costs 64 KB, i.e. two of six operand stages.
 constexpr int kEpiGeluTable = 19, kEpiGeluTableWide = 20;
 constexpr int kGeluTableBytes = 65536;
+// int8 results (upper-word requantization) written as the transposed tensor out[n][t]
+constexpr int kEpiInt8T = 24;
 
 template <int TOK, bool PAIR, int KIND>
 struct Cfg {
@@ -321,7 +324,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // light int8 epilogue keeps two stores: it would catch up with its own previous store
         // (+2 us on the QKV GEMM).  Otherwise a tile is reused two chunks later.  Either way the
         // store that last read this staging tile must have finished reading it.
-        constexpr bool kOneStore = !kOut32 && C::kChunksPerWarp == 2 && KIND != EPI_INT8;
+        constexpr bool kOneStore = !kOut32 && C::kChunksPerWarp == 2 && KIND != EPI_INT8 && KIND != kEpiInt8T;
         if (!kOneStore || ci == 0) {
           if (lane == 0) { if constexpr (kOneStore) ptx::bulk_wait_read<0>(); else ptx::bulk_wait_read<1>(); }
           __syncwarp();
@@ -340,6 +343,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           } else if constexpr (KIND == EPI_Q16H) {
             if constexpr (FAST) o = clamp_sym(requant_upper(a + cur_bias, cur_pb), 32767);
             else o = requant_add(a, cur_pb, cur_padd, cur_pc, 32767);
+          } else if constexpr (KIND == kEpiInt8T) {
+            o = max(requant_upper(a + cur_bias, cur_pb), -127);      // the pack below saturates the upper side
           } else if constexpr (KIND == EPI_INT8) {
             if constexpr (FAST) o = clamp_sym(requant_upper(a + cur_bias, cur_pb), 127);
             else o = requant_add(a, cur_pb, cur_padd, cur_pc, 127);
@@ -367,6 +372,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           }
           v[i] = (uint32_t)o;
         }
+        if constexpr (KIND == kEpiInt8T) {
+          // staging tile of the transposed output: row = this lane's channel, 32 tokens = 32 bytes, written as
+          // two 16-byte chunks placed by the 32-byte swizzle of the store's tensor map (chunk index XOR bit 2
+          // of the row): a quarter-warp's stores cover all banks once -- 8 wavefronts per block instead of 32
+          uint32_t w[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            w[j] = pack4_sat_s8((int32_t)v[4 * j], (int32_t)v[4 * j + 1], (int32_t)v[4 * j + 2], (int32_t)v[4 * j + 3]);
+          const uint32_t sw = ((uint32_t)lane >> 2) & 1u;
+          *reinterpret_cast<uint4*>(stage + lane * 32 + sw * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(stage + lane * 32 + (sw ^ 1u) * 16u) = make_uint4(w[4], w[5], w[6], w[7]);
+        } else
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const int32_t o = (int32_t)v[i];
@@ -382,6 +399,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           __syncwarp();
           if (lane == 0) {
             if constexpr (kOneStore) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage0), ch0, t0);
+            else if constexpr (KIND == kEpiInt8T) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), t0 + ci * 32, ch0);
             else ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), ch0 * C::kOutElem, t0 + ci * 32);
             ptx::bulk_commit();
           }
@@ -429,7 +447,8 @@ int launch_inst(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, co
 
 template <int TOK, bool PAIR>
 int launch_shape(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& mo, const GemmArgs& a,
-                 int kind, bool fast, bool wide_form) {
+                 int kind, bool fast, bool wide_form, bool transposed) {
+  if (transposed) return launch_inst<TOK, PAIR, kEpiInt8T, true>(ctx, mw, mx, mo, a);
   if (kind == EPI_GELU && fast && a.gelu_table) {
     if constexpr (Cfg<TOK, PAIR, kEpiGeluTable>::kValid)          // (256 tokens on one CTA: no room for the table)
       return wide_form ? launch_inst<TOK, PAIR, kEpiGeluTableWide, true>(ctx, mw, mx, mo, a)
@@ -457,8 +476,9 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
   if (M == 0) return IBERT_OK;
   {
     // few output tiles (small batches): split K over a cluster instead of leaving most SMs idle
-    int split = (ctx->splitk_mode == 1 || epi.fast == 2) ? 1 : gemm_splitk_width(ctx, M, N, K);
-    if ((ctx->splitk_mode == 2 || ctx->splitk_mode == 4) && K > 128 && epi.fast != 2 &&
+    if (epi.out_transposed && (epi.kind != EPI_INT8 || epi.fast != 1 || M % 16 != 0)) return IBERT_ERR_ARG;
+    int split = (ctx->splitk_mode == 1 || epi.fast == 2 || epi.out_transposed) ? 1 : gemm_splitk_width(ctx, M, N, K);
+    if ((ctx->splitk_mode == 2 || ctx->splitk_mode == 4) && K > 128 && epi.fast != 2 && !epi.out_transposed &&
         ((M + 127) / 128) * ((N + 127) / 128) * ctx->splitk_mode <= 65535)
       split = ctx->splitk_mode;
     if (split > 1) return launch_gemm_splitk_i8(ctx, x, w, M, N, K, epi, out, split);
@@ -495,6 +515,13 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
     const uint32_t box[2] = {32u * out_elem, gelu_kind ? 64u : 32u};
     int rc = encode_tensor_map(&mo, out, 2, dims, str, box, 0);
     if (rc) return rc;
+    if (epi.out_transposed) {
+      // out^T [N][M]: one box = 32 channels x 32 tokens, rows of 32 bytes, 32-byte swizzle
+      const uint64_t tdims[2] = {(uint64_t)M, (uint64_t)N};
+      const uint64_t tstr[1] = {(uint64_t)M};
+      const uint32_t tbox[2] = {32u, 32u};
+      if ((rc = encode_tensor_map(&mo, out, 2, tdims, tstr, tbox, 32))) return rc;
+    }
   }
   GemmArgs a{};
   a.T = M; a.N = N; a.K = K;
@@ -505,9 +532,9 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
   const bool fast = epi.fast != 0 && ((epi.kind != EPI_GELU && epi.kind != EPI_HGELU) || epi.gelu.fast != 0);
   const bool wide_form = epi.fast == 2;
   if (wide_form && (epi.kind != EPI_GELU || !fast)) return IBERT_ERR_ARG;      // tables in a form nothing else reads
-  if (pair) return launch_shape<256, true>(ctx, mw, mx, mo, a, epi.kind, fast, wide_form);
-  return wide ? launch_shape<256, false>(ctx, mw, mx, mo, a, epi.kind, fast, wide_form)
-              : launch_shape<128, false>(ctx, mw, mx, mo, a, epi.kind, fast, wide_form);
+  if (pair) return launch_shape<256, true>(ctx, mw, mx, mo, a, epi.kind, fast, wide_form, epi.out_transposed);
+  return wide ? launch_shape<256, false>(ctx, mw, mx, mo, a, epi.kind, fast, wide_form, epi.out_transposed)
+              : launch_shape<128, false>(ctx, mw, mx, mo, a, epi.kind, fast, wide_form, epi.out_transposed);
 }
 
 }  // namespace ibert

@@ -118,6 +118,9 @@ struct ibert_ctx {
   int fusion_mode = 0;
   // i-GELU inside the large-tile GEMM epilogue: 0 = from the layer's table, 1 = computed (ibert_set_gelu_table)
   int gelu_table_mode = 0;
+  // layout of the layer's internal Q | K | V tensor: 0 = transposed [3H][tokens] where the shapes allow it
+  // (the QKV GEMM then needs no transposing store), 1 = always [tokens][3H] (ibert_set_qkv_layout)
+  int qkv_layout_mode = 0;
   // optional per-launch event timing (ibert_profile_begin / _end)
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;      // pairs: [2i] before, [2i+1] after launch i
@@ -174,6 +177,10 @@ struct GemmEpilogue {
   // EPI_GELU, optional: table[i] = i-GELU(i - 32767) as int8 for every Q16 value (launch_gelu_table).
   // Tile shapes with 64 KB of shared memory to spare then look the result up instead of computing it.
   const int8_t* gelu_table = nullptr;
+  // EPI_INT8 in the upper-word form only: the result is written TRANSPOSED, out[n][t] (M a multiple of 16).
+  // A thread of the GEMM owns one channel and 32 tokens, so its results are contiguous bytes of the
+  // transposed tensor and leave without a transposing store; the attention kernel reads that layout.
+  bool out_transposed = false;
 };
 
 // Upper-word form of a column set: true if for every n, c[n] >= 1 and b[n] << (32 - c[n]) fits
@@ -240,6 +247,9 @@ int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t 
 // padding, sequence b occupies rows cu_seqlens[b] .. cu_seqlens[b+1]-1 (at most L); lens is ignored
 int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int heads,
                      const AttnConsts& k, const int32_t* lens, int8_t* out, const int32_t* cu_seqlens = nullptr,
-                     int64_t total_rows = 0);
+                     int64_t total_rows = 0, bool qkv_t = false);
+// true when launch_attention can read the transposed tensor qkv^T [3H][B L] (qkv_t): padded batch, L a
+// multiple of 16, a score scale the main kernel takes
+bool attention_takes_transposed(int B, int L, const AttnConsts& k);
 
 }  // namespace ibert

@@ -36,3 +36,13 @@ def gelu_mode(request):
     c.ibert_set_gelu_table(request.param)
     yield request.param
     c.ibert_set_gelu_table(0)
+
+
+@pytest.fixture(params=[0, 1], ids=["qkv-transposed", "qkv-rows"])
+def qkv_layout(request):
+    """Runs a test with the layer's internal Q | K | V tensor transposed (where shapes allow) and in rows."""
+    from gpu_util import ctx
+    c = ctx()
+    c.ibert_set_qkv_layout(request.param)
+    yield request.param
+    c.ibert_set_qkv_layout(0)

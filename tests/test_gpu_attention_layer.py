@@ -78,7 +78,7 @@ def _run_layers(x, params, B, L, fusion=0):
 @pytest.mark.parametrize("fusion", [0, 1])      # linear + LayerNorm: by size (two kernels here) / cluster kernel
 @pytest.mark.parametrize("B,L,H,heads,F", [(2, 16, 128, 2, 256), (1, 37, 64, 1, 64), (3, 128, 256, 4, 1024),
                                            (2, 100, 768, 12, 3072)])
-def test_small_encoder_layers_match_oracle(B, L, H, heads, F, fusion):
+def test_small_encoder_layers_match_oracle(B, L, H, heads, F, fusion, qkv_layout):
     x, params = synth.make_model(0, B, layers=2, H=H, heads=heads, F=F, L=L)
     outs = _run_layers(x, params, B, L, fusion)
     h = x
@@ -95,7 +95,7 @@ def test_config0_roberta_base_layer_matches_oracle(gelu_mode):
     assert want.std() > 20
 
 
-def test_config2_three_layers_batch8_match_oracle():
+def test_config2_three_layers_batch8_match_oracle(qkv_layout):
     B, L = 8, 128
     x, params = synth.make_model(2, B, layers=3)
     outs = _run_layers(x, params, B, L)
@@ -105,7 +105,7 @@ def test_config2_three_layers_batch8_match_oracle():
         assert_same(got, h, "config 2 layer")
 
 
-def test_large_shapes_one_layer_L256_and_L512(gelu_mode):
+def test_large_shapes_one_layer_L256_and_L512(gelu_mode, qkv_layout):
     for cfg, B in ((3, 2), (4, 1)):
         L = synth.CONFIGS[cfg].L
         x, params = synth.make_model(cfg, B, layers=1)

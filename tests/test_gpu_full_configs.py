@@ -45,7 +45,7 @@ def test_config2_small_batches():
         _full_model_check(2, B, sample=(0, B - 1))
 
 
-def test_config3_large_24_layers_L256_batch32_sampled_sequences():
+def test_config3_large_24_layers_L256_batch32_sampled_sequences(qkv_layout):
     _full_model_check(3, 32, sample=(0, 5, 31))
 
 

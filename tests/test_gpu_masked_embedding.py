@@ -63,7 +63,7 @@ def test_masked_attention_coarse_score_scale():
 
 
 @pytest.mark.parametrize("B,L,H,heads,F", [(4, 48, 256, 4, 512), (3, 128, 128, 2, 256)])
-def test_masked_encoder_layers_match_oracle(B, L, H, heads, F):
+def test_masked_encoder_layers_match_oracle(B, L, H, heads, F, qkv_layout):
     x, params = synth.make_model(0, B, layers=2, H=H, heads=heads, F=F, L=L)
     lens = _lens(B, L, 7)
     c = ctx()

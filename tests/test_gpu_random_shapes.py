@@ -120,6 +120,7 @@ def _linear_layernorm(rng):
     c = ctx()
     c.ibert_set_fusion(int(rng.choice([0, 1, 2])))
     c.ibert_set_gelu_table(int(rng.choice([0, 0, 1])))
+    c.ibert_set_qkv_layout(int(rng.choice([0, 0, 1])))
     x = rng.integers(-127, 128, (T, K)).astype(np.int8)
     w = rng.integers(-127, 128, (H, K)).astype(np.int8)
     bias = rng.integers(-20000, 20000, H).astype(np.int32)
@@ -134,6 +135,7 @@ def _linear_layernorm(rng):
     assert_same(host(out), oracle.layernorm(mid, S_mid, res, S_res, gamma, beta, S_out)[0], f"linear+layernorm T={T} H={H} K={K}")
     c.ibert_set_fusion(0)
     c.ibert_set_gelu_table(0)
+    c.ibert_set_qkv_layout(0)
 
 
 def _layer(rng):
@@ -148,6 +150,7 @@ def _layer(rng):
     c = ctx()
     c.ibert_set_fusion(int(rng.choice([0, 1, 2])))
     c.ibert_set_gelu_table(int(rng.choice([0, 0, 1])))
+    c.ibert_set_qkv_layout(int(rng.choice([0, 0, 1])))
     ly = c.ibert_layer_create(params[0])
     mode = rng.random()
     if mode < 0.33:
@@ -168,6 +171,7 @@ def _layer(rng):
     ly.close()
     c.ibert_set_fusion(0)
     c.ibert_set_gelu_table(0)
+    c.ibert_set_qkv_layout(0)
 
 
 @pytest.mark.parametrize("seed", [11, 12, 13])
@@ -182,3 +186,4 @@ def test_random_calls_in_random_order(seed):
         ctx().ibert_set_split_k(0)
         ctx().ibert_set_fusion(0)
         ctx().ibert_set_gelu_table(0)
+        ctx().ibert_set_qkv_layout(0)

@@ -837,13 +837,22 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
     { ProfileScope ps(ctx, IBERT_K_LAYERNORM); rc = launch_layernorm_i16(ctx, r, x, T, ly->ln1, ly->ln1_b, ly->ln1_B, h1); }
   }
   if (rc) return rc;
+  GemmEpilogue e2{};
+  e2.kind = EPI_Q16; e2.d_b = ly->b_f2; e2.d_c = ly->c_f2; e2.d_bias = ly->bias_f2; e2.fast = ly->fast_f2;
+  const bool fuse2 = fuse && gemm_ln_supported(H, F, e2, ly->ln2);
+  // the FFN1 result between its GEMM and the cluster kernel: transposed ([F][T]) where both sides take it
+  // (the table epilogue of a CTA-pair sized problem on one side, the fused kernel on the other)
+  const bool g_t = fuse2 && ctx->qkv_layout_mode == 0 && T % 16 == 0 && T >= 4096 && ly->gelu_table &&
+                   ctx->gelu_table_mode == 0 && ly->fast_f1 != 0 && ly->gelu.fast != 0;
   e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu; e.fast = ly->fast_f1; e.gelu_table = ly->gelu_table;
+  e.out_transposed = g_t;
   { ProfileScope ps(ctx, IBERT_K_GEMM_GELU); rc = launch_gemm_i8(ctx, h1, ly->w_f1, T, F, H, e, g); }
+  e.out_transposed = false;
   if (rc) return rc;
   e.kind = EPI_Q16; e.d_b = ly->b_f2; e.d_c = ly->c_f2; e.d_bias = ly->bias_f2; e.fast = ly->fast_f2;
-  if (fuse && gemm_ln_supported(H, F, e, ly->ln2)) {
+  if (fuse2) {
     ProfileScope ps(ctx, F > 2048 ? IBERT_K_GEMM_LN_WIDE : IBERT_K_GEMM_LN);
-    return launch_gemm_ln_i8(ctx, g, ly->w_f2, T, H, F, e, h1, ly->ln2, ly->ln2_b, ly->ln2_B, out);
+    return launch_gemm_ln_i8(ctx, g, ly->w_f2, T, H, F, e, h1, ly->ln2, ly->ln2_b, ly->ln2_B, out, g_t);
   }
   e.kind = EPI_Q16H;
   { ProfileScope ps(ctx, IBERT_K_GEMM_Q16_WIDE); rc = launch_gemm_i8(ctx, g, ly->w_f2, T, H, F, e, r); }

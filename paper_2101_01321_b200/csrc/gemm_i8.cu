@@ -100,6 +100,9 @@ constexpr int kEpiGeluTable = 19, kEpiGeluTableWide = 20;
 constexpr int kGeluTableBytes = 65536;
 // int8 results (upper-word requantization) written as the transposed tensor out[n][t]
 constexpr int kEpiInt8T = 24;
+// the table kinds with the transposed result (FFN1 feeding the cluster kernel, which reads it as an MN-major operand)
+constexpr int kEpiGeluTableT = 25, kEpiGeluTableWideT = 26;
+__host__ __device__ constexpr bool epi_transposed(int kind) { return kind == kEpiInt8T || kind == kEpiGeluTableT || kind == kEpiGeluTableWideT; }
 
 template <int TOK, bool PAIR, int KIND>
 struct Cfg {
@@ -116,7 +119,7 @@ struct Cfg {
   static constexpr int kStageBytes = kWBytes + kXRows * BK;
   static constexpr int kOutTileBytes = 32 * 32 * kOutElem;            // 32 tokens x 32 channels
   static constexpr int kOutBytes = kEpiWarps * 2 * kOutTileBytes;     // double-buffered per warp
-  static constexpr bool kTable = (KIND == kEpiGeluTable || KIND == kEpiGeluTableWide);
+  static constexpr bool kTable = (KIND == kEpiGeluTable || KIND == kEpiGeluTableWide || KIND == kEpiGeluTableT || KIND == kEpiGeluTableWideT);
   static constexpr int kTableBytes = kTable ? kGeluTableBytes : 0;
   static constexpr int kBudget = 227 * 1024 - 1024 - 512 - kOutBytes - kTableBytes;
   static constexpr int kStages = kBudget / kStageBytes > 8 ? 8 : kBudget / kStageBytes;
@@ -324,7 +327,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // light int8 epilogue keeps two stores: it would catch up with its own previous store
         // (+2 us on the QKV GEMM).  Otherwise a tile is reused two chunks later.  Either way the
         // store that last read this staging tile must have finished reading it.
-        constexpr bool kOneStore = !kOut32 && C::kChunksPerWarp == 2 && KIND != EPI_INT8 && KIND != kEpiInt8T;
+        constexpr bool kOneStore = !kOut32 && C::kChunksPerWarp == 2 && KIND != EPI_INT8 && !epi_transposed(KIND);
         if (!kOneStore || ci == 0) {
           if (lane == 0) { if constexpr (kOneStore) ptx::bulk_wait_read<0>(); else ptx::bulk_wait_read<1>(); }
           __syncwarp();
@@ -352,11 +355,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if constexpr (KIND == EPI_HGELU) {
               if constexpr (FAST) o = clamp_sym(ihgelu_upper(requant_upper(a + cur_bias, cur_pb), gk), 127);
               else o = ihgelu_to_int8(requant_add(a, cur_pb, cur_padd, cur_pc, 32767), gk, gelu_half);
-            } else if constexpr (KIND == kEpiGeluTable) {
+            } else if constexpr (KIND == kEpiGeluTable || KIND == kEpiGeluTableT) {
               // |requantized value| < 2^30 (upper word of a product of two int32): the sum cannot wrap
               const int32_t at = max(__viaddmin_s32(requant_upper(a + cur_bias, cur_pb), table_mid, table_hi), table_lo);
               asm volatile("ld.shared.u8 %0, [%1];" : "=r"(o) : "r"(at));
-            } else if constexpr (KIND == kEpiGeluTableWide) {
+            } else if constexpr (KIND == kEpiGeluTableWide || KIND == kEpiGeluTableWideT) {
               const int32_t at = clamp_sym(requant_upper_wide(a + cur_bias, cur_pb, cur_pc), 32767) + table_mid;
               asm volatile("ld.shared.u8 %0, [%1];" : "=r"(o) : "r"(at));
             } else if constexpr (KIND == kEpiGeluLowFree) {
@@ -372,14 +375,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           }
           v[i] = (uint32_t)o;
         }
-        if constexpr (KIND == kEpiInt8T) {
+        if constexpr (epi_transposed(KIND)) {
           // staging tile of the transposed output: row = this lane's channel, 32 tokens = 32 bytes, written as
           // two 16-byte chunks placed by the 32-byte swizzle of the store's tensor map (chunk index XOR bit 2
           // of the row): a quarter-warp's stores cover all banks once -- 8 wavefronts per block instead of 32
           uint32_t w[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j)
-            w[j] = pack4_sat_s8((int32_t)v[4 * j], (int32_t)v[4 * j + 1], (int32_t)v[4 * j + 2], (int32_t)v[4 * j + 3]);
+            w[j] = KIND == kEpiInt8T
+                       ? pack4_sat_s8((int32_t)v[4 * j], (int32_t)v[4 * j + 1], (int32_t)v[4 * j + 2], (int32_t)v[4 * j + 3])
+                       : __byte_perm(__byte_perm(v[4 * j], v[4 * j + 1], 0x0040), __byte_perm(v[4 * j + 2], v[4 * j + 3], 0x0040), 0x5410);   // table bytes
           const uint32_t sw = ((uint32_t)lane >> 2) & 1u;
           *reinterpret_cast<uint4*>(stage + lane * 32 + sw * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
           *reinterpret_cast<uint4*>(stage + lane * 32 + (sw ^ 1u) * 16u) = make_uint4(w[4], w[5], w[6], w[7]);
@@ -399,7 +404,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           __syncwarp();
           if (lane == 0) {
             if constexpr (kOneStore) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage0), ch0, t0);
-            else if constexpr (KIND == kEpiInt8T) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), t0 + ci * 32, ch0);
+            else if constexpr (epi_transposed(KIND)) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), t0 + ci * 32, ch0);
             else ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), ch0 * C::kOutElem, t0 + ci * 32);
             ptx::bulk_commit();
           }
@@ -448,7 +453,15 @@ int launch_inst(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, co
 template <int TOK, bool PAIR>
 int launch_shape(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& mo, const GemmArgs& a,
                  int kind, bool fast, bool wide_form, bool transposed) {
-  if (transposed) return launch_inst<TOK, PAIR, kEpiInt8T, true>(ctx, mw, mx, mo, a);
+  if (transposed) {
+    if (kind == EPI_INT8) return launch_inst<TOK, PAIR, kEpiInt8T, true>(ctx, mw, mx, mo, a);
+    if constexpr (Cfg<TOK, PAIR, kEpiGeluTable>::kValid) {
+      if (kind == EPI_GELU && fast && a.gelu_table)
+        return wide_form ? launch_inst<TOK, PAIR, kEpiGeluTableWideT, true>(ctx, mw, mx, mo, a)
+                         : launch_inst<TOK, PAIR, kEpiGeluTableT, true>(ctx, mw, mx, mo, a);
+    }
+    return IBERT_ERR_ARG;
+  }
   if (kind == EPI_GELU && fast && a.gelu_table) {
     if constexpr (Cfg<TOK, PAIR, kEpiGeluTable>::kValid)          // (256 tokens on one CTA: no room for the table)
       return wide_form ? launch_inst<TOK, PAIR, kEpiGeluTableWide, true>(ctx, mw, mx, mo, a)
@@ -476,7 +489,11 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
   if (M == 0) return IBERT_OK;
   {
     // few output tiles (small batches): split K over a cluster instead of leaving most SMs idle
-    if (epi.out_transposed && (epi.kind != EPI_INT8 || epi.fast != 1 || M % 16 != 0)) return IBERT_ERR_ARG;
+    if (epi.out_transposed) {
+      const bool int8_ok = epi.kind == EPI_INT8 && epi.fast == 1;
+      const bool gelu_ok = epi.kind == EPI_GELU && epi.fast != 0 && epi.gelu.fast != 0 && epi.gelu_table && ctx->gelu_table_mode == 0;
+      if ((!int8_ok && !gelu_ok) || M % 16 != 0) return IBERT_ERR_ARG;
+    }
     int split = (ctx->splitk_mode == 1 || epi.fast == 2 || epi.out_transposed) ? 1 : gemm_splitk_width(ctx, M, N, K);
     if ((ctx->splitk_mode == 2 || ctx->splitk_mode == 4) && K > 128 && epi.fast != 2 && !epi.out_transposed &&
         ((M + 127) / 128) * ((N + 127) / 128) * ctx->splitk_mode <= 65535)

@@ -84,7 +84,10 @@ __device__ __forceinline__ uint32_t isqrt_of_quotient(uint64_t ss, uint32_t C) {
 // PAIR: two CTAs (same 256 channels, adjacent 128-token tiles) share every MMA through
 // tcgen05.mma.cta_group::2 -- each loads its own token rows and half of the weight rows, which cuts
 // the bytes an SM pulls from L2 per MMA by a third (L2 bandwidth bounds the K = 3072 main loop).
-template <bool PAIR>
+// XT: x is given transposed, x^T [K][T] (token index contiguous), as the FFN1 GEMM writes it without a
+// transposing store: a stage's token tile is then [128 K rows][128 tokens], an MN-major A operand
+// (instruction-descriptor bit 15; 1 KB from one group of eight K rows to the next).
+template <bool PAIR, bool XT = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                const __grid_constant__ CUtensorMap map_res, const __grid_constant__ CUtensorMap map_out,
@@ -178,11 +181,13 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             // both CTAs' copies complete on the leader's barrier, which expects the bytes of both
             const uint32_t full_leader = ptx::map_to_cta(bar_full + 8 * stage, leader);
             if (half == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * kStageBytes);
-            ptx::tma_load_2d_pair(sx, &map_x, full_leader, kb * kBK, t0);
+            if constexpr (XT) ptx::tma_load_2d_pair(sx, &map_x, full_leader, t0, kb * kBK);
+            else ptx::tma_load_2d_pair(sx, &map_x, full_leader, kb * kBK, t0);
             ptx::tma_load_2d_pair(sx + kXBytes, &map_w, full_leader, kb * kBK, n0 + half * (kCh / 2));
           } else {
             ptx::mbar_arrive_expect_tx(bar_full + 8 * stage, kStageBytes);
-            ptx::tma_load_2d(sx, &map_x, bar_full + 8 * stage, kb * kBK, t0);
+            if constexpr (XT) ptx::tma_load_2d(sx, &map_x, bar_full + 8 * stage, t0, kb * kBK);
+            else ptx::tma_load_2d(sx, &map_x, bar_full + 8 * stage, kb * kBK, t0);
             ptx::tma_load_2d(sx + kXBytes, &map_w, bar_full + 8 * stage, kb * kBK, n0);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -192,7 +197,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (PAIR: the pair's leader only)
     if (lane == 0 && half == 0) {
-      constexpr uint32_t idesc = ptx::make_idesc_i8(PAIR ? 2 * kTok : kTok, kCh, true, true);
+      constexpr uint32_t idesc = ptx::make_idesc_i8(PAIR ? 2 * kTok : kTok, kCh, true, true) | (XT ? (1u << 15) : 0u);
       const uint16_t pair_mask = (uint16_t)(3u << leader);
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
       for (uint32_t it = 0; unit_of(it) < n_units && ok; ++it) {
@@ -205,10 +210,13 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           const uint32_t sx = smem_base + stage * kStageBytes;
           const uint64_t dx = ptx::make_kmajor_desc(sx, 1024, ptx::kSwizzle128);
           const uint64_t dw = ptx::make_kmajor_desc(sx + kXBytes, 1024, ptx::kSwizzle128);
+          // (MN-major X tile: the same fields -- 1 KB between groups of eight K rows -- and a K step of 32 rows
+          // is four groups = 4 KB further on; K-major: 32 bytes further inside the swizzle span)
+          constexpr uint64_t x_step = XT ? (4096 >> 4) : 2;
 #pragma unroll
           for (int k = 0; k < kBK / 32; ++k) {
-            if constexpr (PAIR) ptx::mma_i8_ss_pair(d_tmem, dx + 2 * k, dw + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-            else ptx::mma_i8_ss(d_tmem, dx + 2 * k, dw + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            if constexpr (PAIR) ptx::mma_i8_ss_pair(d_tmem, dx + x_step * k, dw + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            else ptx::mma_i8_ss(d_tmem, dx + x_step * k, dw + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
           if constexpr (PAIR) ptx::mma_commit_pair(bar_empty + 8 * stage, pair_mask);
@@ -453,9 +461,10 @@ bool gemm_ln_supported(int H, int K, const GemmEpilogue& epi, const LnConsts& ln
 
 int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t T, int H, int K,
                       const GemmEpilogue& epi, const int8_t* res, const LnConsts& ln, const int32_t* d_b_i,
-                      const int64_t* d_B_i, int8_t* out) {
+                      const int64_t* d_B_i, int8_t* out, bool x_transposed) {
   if (T == 0) return IBERT_OK;
   if (!gemm_ln_supported(H, K, epi, ln)) return IBERT_ERR_SHAPE;
+  if (x_transposed && T % 16 != 0) return IBERT_ERR_ARG;
   CUtensorMap mx, mw, mr, mo;
   int rc;
   {
@@ -463,6 +472,13 @@ int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t 
     const uint64_t str[1] = {(uint64_t)K};
     const uint32_t box[2] = {kBK, kTok};
     if ((rc = encode_tensor_map(&mx, x, 2, dims, str, box, 128))) return rc;
+    if (x_transposed) {
+      // x^T [K][T]: a stage's tile is 128 K rows x 128 tokens
+      const uint64_t tdims[2] = {(uint64_t)T, (uint64_t)K};
+      const uint64_t tstr[1] = {(uint64_t)T};
+      const uint32_t tbox[2] = {kTok, kBK};
+      if ((rc = encode_tensor_map(&mx, x, 2, tdims, tstr, tbox, 128))) return rc;
+    }
   }
   {
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)H};
@@ -491,7 +507,9 @@ int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t 
     int& slot = max_clusters[ctx->device % kMaxDevices][pair ? 1 : 0][cl];
     if (slot == 0) {
       const void* fn = pair ? (const void*)gemm_ln_kernel<true> : (const void*)gemm_ln_kernel<false>;
-      if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kAlloc) != cudaSuccess) {
+      const void* fnt = pair ? (const void*)gemm_ln_kernel<true, true> : (const void*)gemm_ln_kernel<false, true>;
+      if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kAlloc) != cudaSuccess ||
+          cudaFuncSetAttribute(fnt, cudaFuncAttributeMaxDynamicSharedMemorySize, kAlloc) != cudaSuccess) {
         cudaGetLastError();
         slot = -1;
         return slot;
@@ -522,11 +540,17 @@ int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t 
     const uint32_t box[2] = {kBK, kCh / 2};            // each CTA of a pair loads half of the weight rows
     if ((rc = encode_tensor_map(&mw2, w, 2, dims, str, box, 128))) return rc;
     const int clusters = (int)std::min<int64_t>((t_tiles + 1) / 2, resident(true, cl));
+    if (x_transposed)
+      return launch_pdl(gemm_ln_kernel<true, true>, dim3(clusters * cl), dim3(kThreads), (size_t)kAlloc, ctx->stream, cl,
+                        mx, mw2, mr, mo, a);
     return launch_pdl(gemm_ln_kernel<true>, dim3(clusters * cl), dim3(kThreads), (size_t)kAlloc, ctx->stream, cl,
                       mx, mw2, mr, mo, a);
   }
   if (resident(false, n_slices) <= 0) return IBERT_ERR_CUDA;
   const int clusters = (int)std::min<int64_t>(t_tiles, resident(false, n_slices));
+  if (x_transposed)
+    return launch_pdl(gemm_ln_kernel<false, true>, dim3(clusters * n_slices), dim3(kThreads), (size_t)kAlloc, ctx->stream,
+                      n_slices, mx, mw, mr, mo, a);
   return launch_pdl(gemm_ln_kernel<false>, dim3(clusters * n_slices), dim3(kThreads), (size_t)kAlloc, ctx->stream,
                     n_slices, mx, mw, mr, mo, a);
 }

@@ -239,7 +239,7 @@ struct AttnConsts {
 bool gemm_ln_supported(int H, int K, const GemmEpilogue& epi, const LnConsts& ln);
 int launch_gemm_ln_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t T, int H, int K,
                       const GemmEpilogue& epi, const int8_t* res, const LnConsts& ln, const int32_t* d_b_i,
-                      const int64_t* d_B_i, int8_t* out);
+                      const int64_t* d_B_i, int8_t* out, bool x_transposed = false);
 
 // `lens` (device, [B], may be null): valid keys per sequence -- keys beyond take no part in the
 // softmax and get probability 0 (key-padding mask)

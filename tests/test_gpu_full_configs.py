@@ -53,6 +53,29 @@ def test_config4_large_24_layers_L512_batch64_sampled_sequences():
     _full_model_check(4, 64, sample=(0, 31, 63))
 
 
+def test_config2_layers_with_ragged_token_count(qkv_layout):
+    """37 sequences of 112 tokens: 4144 tokens = 32 full 128-token tiles and a 48-token tail, large
+    enough for the transposed intermediates (Q|K|V and the FFN1 result) where the layout switch allows them."""
+    cfg = synth.CONFIGS[2]
+    B, L = 37, 112
+    x, params = synth.make_model(2, B)
+    x, params = np.ascontiguousarray(x[:B * L]), params[:2]
+    c = ctx()
+    layers = [c.ibert_layer_create(p) for p in params]
+    h = dev(x)
+    for ly in layers:
+        h, _ = c.ibert_encoder_layer(ly, h, B, L)
+    c.check()
+    got = host(h).reshape(B, L, cfg.H)
+    for ly in layers:
+        ly.close()
+    for s in (0, 36):                          # the last sequence ends in the ragged tile
+        ref = x.reshape(B, L, cfg.H)[s]
+        for p in params:
+            ref = oracle.encoder_layer(p, ref, 1, L).out
+        assert_same(got[s], ref, f"ragged batch, sequence {s}")
+
+
 def test_config2_with_oracle_calibrated_scales():
     """The same stack with the static scales calibrated from each site's max|x| (the stored blob)."""
     _full_model_check(2, 128, sample=(3, 100), scales="calibrated")

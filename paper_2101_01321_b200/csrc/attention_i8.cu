@@ -532,9 +532,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
         if (a.q_bufs == 1) load_q(next, 0, 0);      // single tile per pair: Q is as dead as K by now
       }
 
+      // packed: a warp whose 32 query rows all lie past the sequence's end computes nothing (its rows of P
+      // keep stale bytes; the context rows the second MMA makes of them are never stored)
+      const bool live = !PACKED || qt * 128 + quad * 32 < max(n, 1);
       // ---- i-softmax, pass 1: maximum of this thread's columns, then of the row
       int32_t mx = INT32_MIN;
-      if (ok) {
+      if (ok && live) {
         ptx::tc_fence_after_sync();
         for (int c0 = c_begin; c0 < c_end; c0 += kW) {
           uint32_t v[kW];
@@ -554,7 +557,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
       if (G > 1) __syncthreads();                  // one thread per row: nothing to exchange
       // ---- pass 2: i-exp written back over the scores, partial sums
       uint32_t sum = 0;
-      if (ok) {
+      if (ok && live) {
         for (int g = 0; g < G; ++g) mx = max(mx, s_max[g * 128 + row]);
         if (a.k.e.pow2_k >= 0) {
           // score scale exactly ln2 / 2^k: quotient and remainder by shift and mask
@@ -606,7 +609,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
       }
       if (G > 1) __syncthreads();
       // ---- pass 3: u8 probabilities into the operand tile of the second MMA
-      if (ok) {
+      if (ok && live) {
         sum = 0;
         for (int g = 0; g < G; ++g) sum += s_sum[g * 128 + row];
         const RowDivisor rd = make_row_divisor(max(sum, 1u), a.k.e.p_max);   // sum = 0 only without valid keys
@@ -670,7 +673,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
 
       // ---- epilogue: the 64 context values of a row in two halves, taken by column groups 0 and 1
       // (by group 0 alone when there is only one)
-      if (ok && grp < 2) {
+      if (ok && grp < 2 && live) {
         ptx::tc_fence_after_sync();
         const int64_t half = rounding_half(a.k.c);
         const int q_row = qt * 128 + row;

@@ -669,7 +669,15 @@ def run_only(args):
     rng = np.random.default_rng(synth.SEED_BASE)
     k = args.only
     alg_bytes = None
-    if k in ("gemm_out_ln", "gemm_ffn2_ln"):
+    if k == "layer":
+        # one encoder layer through the call the step makes: its five kernels in the forms the layer
+        # chooses (internal layouts included), for captures that select a kernel by name and launch index
+        x_np, params = synth.make_model(args.config, batch, scales=args.scales)
+        layer = ctx.ibert_layer_create(params[0])
+        x = torch.from_numpy(x_np).to(dev)
+        out = torch.empty_like(x)
+        fn = lambda: ctx.ibert_encoder_layer(layer, x, batch, L, out=out)
+    elif k in ("gemm_out_ln", "gemm_ffn2_ln"):
         N, K = (H, H) if k == "gemm_out_ln" else (H, F)
         x, w, res = i8(T, K), i8(N, K), i8(T, N)
         bias = torch.randint(-1000, 1000, (N,), generator=g, dtype=torch.int32).to(dev)

@@ -216,13 +216,16 @@ int ibert_set_split_k(ibert_ctx* ctx, int mode);
    the integer algorithm itself and used only where the epilogue's integer pipe is the bound.  A tuning and testing switch.  Returns IBERT_ERR_ARG for another mode. */
 int ibert_set_gelu_table(ibert_ctx* ctx, int mode);
 
-/* Layout of the Q | K | V tensor between the two first kernels of ibert_encoder_layer (an internal
-   tensor of the layer; the public attention calls always take [tokens][3H]): mode 0 (default) keeps
-   it transposed, [3H][tokens], for padded batches whose L is a multiple of 16 -- the QKV GEMM then
-   writes each thread's 32 tokens of one channel as contiguous bytes instead of transposing them
-   through shared memory, and the attention kernel reads Q and K tiles as MN-major operands; mode 1
-   keeps [tokens][3H] always.  The results are identical.  No counterpart in the paper: a tuning and
-   testing switch.  Returns IBERT_ERR_ARG for another mode. */
+/* Layout of the two tensors that never leave ibert_encoder_layer -- Q | K | V between the QKV GEMM
+   and attention, and the FFN1 result between its GEMM and the fused FFN2 + LayerNorm kernel (the
+   public calls always take and return [tokens][channels]): mode 0 (default) keeps them transposed,
+   [channels][tokens], where the shapes allow (padded batches with L a multiple of 16; for the FFN1
+   result also a token count that is a multiple of 16 and at least 4096, with the table form of
+   i-GELU and the fused kernel in use) -- the producing GEMM then writes each thread's 32 tokens of
+   one channel as contiguous bytes instead of transposing them through shared memory, and the
+   consuming kernel reads the tiles as MN-major operands; mode 1 keeps [tokens][channels] always.
+   The results are identical.  No counterpart in the paper: a tuning and testing switch.  Returns
+   IBERT_ERR_ARG for another mode. */
 int ibert_set_qkv_layout(ibert_ctx* ctx, int mode);
 
 /* The integer-only encoder layer (Fig. 1 right; post-LN order):

@@ -223,8 +223,9 @@ int ibert_set_gelu_table(ibert_ctx* ctx, int mode);
    result also a token count that is a multiple of 16 and at least 4096, with the table form of
    i-GELU and the fused kernel in use) -- the producing GEMM then writes each thread's 32 tokens of
    one channel as contiguous bytes instead of transposing them through shared memory, and the
-   consuming kernel reads the tiles as MN-major operands; mode 1 keeps [tokens][channels] always.
-   The results are identical.  No counterpart in the paper: a tuning and testing switch.  Returns
+   consuming kernel reads the tiles as MN-major operands; mode 1 keeps [tokens][channels] always;
+   mode 2 is mode 0 without the lower bound on the token count (for tests: small problems then
+   run the transposed forms too).  The results are identical.  No counterpart in the paper: a tuning and testing switch.  Returns
    IBERT_ERR_ARG for another mode. */
 int ibert_set_qkv_layout(ibert_ctx* ctx, int mode);
 

@@ -194,7 +194,7 @@ class Context:
         _chk(lib().ibert_set_split_k(self.h, mode), "ibert_set_split_k")
 
     def ibert_set_qkv_layout(self, mode: int) -> None:
-        """0: the layer keeps Q | K | V and the FFN1 result transposed between its kernels where shapes allow (default); 1: never."""
+        """0: the layer keeps Q | K | V and the FFN1 result transposed between its kernels where shapes allow and sizes make it pay (default); 1: never; 2: wherever shapes allow."""
         _chk(lib().ibert_set_qkv_layout(self.h, mode), "ibert_set_qkv_layout")
 
     def ibert_set_gelu_table(self, mode: int) -> None:

@@ -223,7 +223,7 @@ int ibert_set_split_k(ibert_ctx* ctx, int mode) {
 
 int ibert_set_qkv_layout(ibert_ctx* ctx, int mode) {
   return guarded([&]() -> int {
-  if (!ctx || mode < 0 || mode > 1) return IBERT_ERR_ARG;
+  if (!ctx || mode < 0 || mode > 2) return IBERT_ERR_ARG;
   ctx->qkv_layout_mode = mode;
   return IBERT_OK;
   });
@@ -814,7 +814,7 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
   e.kind = EPI_INT8; e.d_b = ly->b_qkv; e.d_c = ly->c_qkv; e.d_bias = ly->bias_qkv; e.fast = ly->fast_qkv;
   // Q | K | V between the two kernels: transposed ([3H][T]) where both sides take it -- a thread of the GEMM
   // holds one channel of 32 tokens, which are contiguous bytes of that layout
-  const bool qkv_t = ctx->qkv_layout_mode == 0 && !cu_seqlens && ly->fast_qkv == 1 &&
+  const bool qkv_t = ctx->qkv_layout_mode != 1 && !cu_seqlens && ly->fast_qkv == 1 &&
                      attention_takes_transposed(B, L, ly->attn);
   e.out_transposed = qkv_t;
   { ProfileScope ps(ctx, IBERT_K_GEMM_QKV); rc = launch_gemm_i8(ctx, x, ly->w_qkv, T, 3 * H, H, e, qkv); }
@@ -842,8 +842,9 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
   const bool fuse2 = fuse && gemm_ln_supported(H, F, e2, ly->ln2);
   // the FFN1 result between its GEMM and the cluster kernel: transposed ([F][T]) where both sides take it
   // (the table epilogue of a CTA-pair sized problem on one side, the fused kernel on the other)
-  const bool g_t = fuse2 && ctx->qkv_layout_mode == 0 && T % 16 == 0 && T >= 4096 && ly->gelu_table &&
-                   ctx->gelu_table_mode == 0 && ly->fast_f1 != 0 && ly->gelu.fast != 0;
+  const bool g_t = fuse2 && ctx->qkv_layout_mode != 1 && (T >= 4096 || ctx->qkv_layout_mode == 2) && ly->gelu_table &&
+                   ctx->gelu_table_mode == 0 && ly->fast_f1 != 0 && ly->gelu.fast != 0 &&
+                   gemm_gelu_takes_transposed(ctx, T, F);
   e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu; e.fast = ly->fast_f1; e.gelu_table = ly->gelu_table;
   e.out_transposed = g_t;
   { ProfileScope ps(ctx, IBERT_K_GEMM_GELU); rc = launch_gemm_i8(ctx, h1, ly->w_f1, T, F, H, e, g); }

@@ -482,7 +482,21 @@ int launch_shape(ibert_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, c
   }
 }
 
+// tile shape: 256 channels x 256 tokens on a CTA pair when that fills every pair, else one CTA
+// per 128 channels x 256 (or 128) tokens
+void tile_shape(const ibert_ctx* ctx, int64_t M, int N, bool* pair, bool* wide) {
+  const int64_t t256 = (M + 255) / 256;
+  *pair = ctx->num_sms >= 2 && t256 * ((N + 255) / 256) >= ctx->num_sms / 2;
+  *wide = *pair || t256 * ((N + 127) / 128) >= ctx->num_sms;
+}
+
 }  // namespace
+
+bool gemm_gelu_takes_transposed(const ibert_ctx* ctx, int64_t M, int N) {
+  bool pair, wide;
+  tile_shape(ctx, M, N, &pair, &wide);
+  return M % 16 == 0 && (pair || !wide);     // (256 tokens on one CTA leave no room for the table)
+}
 
 int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, int N, int K,
                    const GemmEpilogue& epi, void* out) {
@@ -500,11 +514,8 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
       split = ctx->splitk_mode;
     if (split > 1) return launch_gemm_splitk_i8(ctx, x, w, M, N, K, epi, out, split);
   }
-  // tile shape: 256 channels x 256 tokens on a CTA pair when that fills every pair, else one CTA
-  // per 128 channels x 256 (or 128) tokens
-  const int64_t t256 = (M + 255) / 256;
-  const bool pair = ctx->num_sms >= 2 && t256 * ((N + 255) / 256) >= ctx->num_sms / 2;
-  const bool wide = pair || t256 * ((N + 127) / 128) >= ctx->num_sms;
+  bool pair, wide;
+  tile_shape(ctx, M, N, &pair, &wide);
   const int TOK = wide ? 256 : 128;
   const uint32_t out_elem = (epi.kind == EPI_RAW || epi.kind == EPI_Q16) ? 4u : (epi.kind == EPI_Q16H ? 2u : 1u);
   CUtensorMap mw, mx, mo;

@@ -120,7 +120,7 @@ struct ibert_ctx {
   int gelu_table_mode = 0;
   // layout of the layer's internal Q | K | V tensor: 0 = transposed [3H][tokens] where the shapes allow it
   // (the QKV GEMM then needs no transposing store), 1 = always [tokens][3H] (ibert_set_qkv_layout)
-  int qkv_layout_mode = 0;
+  int qkv_layout_mode = 0;          // 0: transposed intermediates where they pay, 1: never, 2: wherever shapes allow
   // optional per-launch event timing (ibert_profile_begin / _end)
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;      // pairs: [2i] before, [2i+1] after launch i
@@ -251,5 +251,7 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
 // true when launch_attention can read the transposed tensor qkv^T [3H][B L] (qkv_t): padded batch, L a
 // multiple of 16, a score scale the main kernel takes
 bool attention_takes_transposed(int B, int L, const AttnConsts& k);
+// whether the table form of the FFN1 epilogue can write its result transposed for an [M, N] problem
+bool gemm_gelu_takes_transposed(const ibert_ctx* ctx, int64_t M, int N);
 
 }  // namespace ibert

@@ -38,9 +38,10 @@ def gelu_mode(request):
     c.ibert_set_gelu_table(0)
 
 
-@pytest.fixture(params=[0, 1], ids=["qkv-transposed", "qkv-rows"])
+@pytest.fixture(params=[0, 1, 2], ids=["inner-transposed", "inner-rows", "inner-transposed-any-size"])
 def qkv_layout(request):
-    """Runs a test with the layer's internal Q | K | V tensor transposed (where shapes allow) and in rows."""
+    """Runs a test with the layer's internal tensors (Q | K | V, the FFN1 result) transposed where shapes
+    allow and sizes make it pay, in rows, and transposed wherever shapes allow."""
     from gpu_util import ctx
     c = ctx()
     c.ibert_set_qkv_layout(request.param)

@@ -145,10 +145,11 @@ def test_linear_error_codes():
     with pytest.raises(IbertError) as e:
         ctx().ibert_linear_i8(x, 1.0, w, np.full(16, 1e30), None, 0, 1e-30)  # multiplier >= 2^31
     assert e.value.code == -3
-    for bad in (-1, 2):                                                  # the switches know modes 0 and 1
+    for bad in (-1, 2):                                                  # the table switch knows modes 0 and 1
         with pytest.raises(IbertError) as e:
             ctx().ibert_set_gelu_table(bad)
         assert e.value.code == -1
+    for bad in (-1, 3):                                                  # the layout switch modes 0, 1 and 2
         with pytest.raises(IbertError) as e:
             ctx().ibert_set_qkv_layout(bad)
         assert e.value.code == -1

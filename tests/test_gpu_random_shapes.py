@@ -120,7 +120,7 @@ def _linear_layernorm(rng):
     c = ctx()
     c.ibert_set_fusion(int(rng.choice([0, 1, 2])))
     c.ibert_set_gelu_table(int(rng.choice([0, 0, 1])))
-    c.ibert_set_qkv_layout(int(rng.choice([0, 0, 1])))
+    c.ibert_set_qkv_layout(int(rng.choice([0, 1, 2, 2])))
     x = rng.integers(-127, 128, (T, K)).astype(np.int8)
     w = rng.integers(-127, 128, (H, K)).astype(np.int8)
     bias = rng.integers(-20000, 20000, H).astype(np.int32)
@@ -150,7 +150,7 @@ def _layer(rng):
     c = ctx()
     c.ibert_set_fusion(int(rng.choice([0, 1, 2])))
     c.ibert_set_gelu_table(int(rng.choice([0, 0, 1])))
-    c.ibert_set_qkv_layout(int(rng.choice([0, 0, 1])))
+    c.ibert_set_qkv_layout(int(rng.choice([0, 1, 2, 2])))
     ly = c.ibert_layer_create(params[0])
     mode = rng.random()
     if mode < 0.33:

@@ -220,8 +220,8 @@ int ibert_set_gelu_table(ibert_ctx* ctx, int mode);
    and attention, and the FFN1 result between its GEMM and the fused FFN2 + LayerNorm kernel (the
    public calls always take and return [tokens][channels]): mode 0 (default) keeps them transposed,
    [channels][tokens], where the shapes allow (padded batches with L a multiple of 16; for the FFN1
-   result also a token count that is a multiple of 16 and at least 4096, with the table form of
-   i-GELU and the fused kernel in use) -- the producing GEMM then writes each thread's 32 tokens of
+   result also a token count that is a multiple of 16 and at least 4096, a tensor of at most half
+   the L2 cache, and the table form of i-GELU and the fused kernel in use) -- the producing GEMM then writes each thread's 32 tokens of
    one channel as contiguous bytes instead of transposing them through shared memory, and the
    consuming kernel reads the tiles as MN-major operands; mode 1 keeps [tokens][channels] always;
    mode 2 is mode 0 without the lower bound on the token count (for tests: small problems then

@@ -178,6 +178,7 @@ int ibert_create(ibert_ctx** out, int device, void* cuda_stream) {
   ctx->device = device;
   ctx->stream = static_cast<cudaStream_t>(cuda_stream);
   ctx->num_sms = prop.multiProcessorCount;
+  ctx->l2_bytes = prop.l2CacheSize;
   if (cudaMalloc(&ctx->d_status, 64) != cudaSuccess) { delete ctx; return IBERT_ERR_NOMEM; }
   if (cudaMemsetAsync(ctx->d_status, 0, 64, ctx->stream) != cudaSuccess) {
     cudaFree(ctx->d_status);
@@ -842,7 +843,11 @@ static int encoder_layer_common(ibert_ctx* ctx, const ibert_layer* ly, const int
   const bool fuse2 = fuse && gemm_ln_supported(H, F, e2, ly->ln2);
   // the FFN1 result between its GEMM and the cluster kernel: transposed ([F][T]) where both sides take it
   // (the table epilogue of a CTA-pair sized problem on one side, the fused kernel on the other)
-  const bool g_t = fuse2 && ctx->qkv_layout_mode != 1 && (T >= 4096 || ctx->qkv_layout_mode == 2) && ly->gelu_table &&
+  // (a tensor that no longer fits L2 comes back from HBM, where the fused kernel's channel-major tiles --
+  // 128 rows of 128 bytes, T bytes apart -- read slower than token-major ones: T = 32768, F = 4096, 128 MB,
+  // loses 1.5 % of the step)
+  const bool g_pays = T >= 4096 && (int64_t)T * F <= ctx->l2_bytes / 2;
+  const bool g_t = fuse2 && ctx->qkv_layout_mode != 1 && (g_pays || ctx->qkv_layout_mode == 2) && ly->gelu_table &&
                    ctx->gelu_table_mode == 0 && ly->fast_f1 != 0 && ly->gelu.fast != 0 &&
                    gemm_gelu_takes_transposed(ctx, T, F);
   e.kind = EPI_GELU; e.d_b = ly->b_f1; e.d_c = ly->c_f1; e.d_bias = ly->bias_f1; e.gelu = ly->gelu; e.fast = ly->fast_f1; e.gelu_table = ly->gelu_table;

@@ -105,6 +105,7 @@ struct ibert_ctx {
   cudaStream_t stream = nullptr;
   int32_t* d_status = nullptr;       // first device-side error (0 = none)
   int num_sms = 0;
+  int64_t l2_bytes = 0;             // size of the L2 cache
   // derived constant tables already on the device, keyed by a hash of their host bytes
   std::map<uint64_t, ibert::DeviceTable> tables;
   // look-up tables of ibert_gelu_lut_i, keyed by a hash of the GELU constants

@@ -260,15 +260,26 @@ int make_ln_residual(double S_r, double S, LnConsts* k) {
   k->res_fast = (k->c_r >= 8 && k->c_r <= 31) ? 1 : 0;
   k->res_sh = 32 - k->c_r;
   // narrow form: drop seven bits of the 31-bit multiplier (|r| <= 128 then keeps the product inside int32) and
-  // keep it only if every int8 value gives the exact form's result
+  // keep it only if every int8 value gives the exact form's result.  For a candidate multiplier nb the
+  // addend may be any value that puts all 256 results on the right side of their floors: each r bounds it
+  // to an interval, and the candidate serves if the intervals intersect.
   k->res_narrow = 0;
   k->res_nb = k->res_nc = k->res_nhalf = 0;
   if (k->c_r >= 8 && k->c_r <= 31) {
     const int nc = k->c_r - 7;
-    for (int rounding = 1; rounding >= 0 && !k->res_narrow; --rounding) {
-      const int64_t nb = ((int64_t)k->b_r + (rounding ? 64 : 0)) >> 7;
-      if (nb >= (int64_t(1) << 24)) continue;
-      const int64_t nhalf = int64_t(1) << (nc - 1);
+    const int64_t base = (int64_t)k->b_r >> 7;
+    static const int kTry[4] = {0, 1, -1, 2};
+    for (int t = 0; t < 4 && !k->res_narrow; ++t) {
+      const int64_t nb = base + kTry[t];
+      if (nb <= 0 || nb >= (int64_t(1) << 24)) continue;
+      int64_t lo = INT64_MIN, hi = INT64_MAX;
+      for (int r = -128; r <= 127; ++r) {
+        const int64_t exact = ((int64_t)r * k->b_r + (int64_t(1) << (k->c_r - 1))) >> k->c_r;
+        lo = std::max(lo, exact * (int64_t(1) << nc) - (int64_t)r * nb);
+        hi = std::min(hi, (exact + 1) * (int64_t(1) << nc) - 1 - (int64_t)r * nb);
+      }
+      if (lo > hi) continue;
+      const int64_t nhalf = std::min(std::max(int64_t(1) << (nc - 1), lo), hi);   // the usual half where it serves
       bool same = true;
       for (int r = -128; r <= 127 && same; ++r) {
         const int64_t exact = ((int64_t)r * k->b_r + (int64_t(1) << (k->c_r - 1))) >> k->c_r;

@@ -357,6 +357,8 @@ struct AttnArgs {
 // writes it without a transposing store: Q^T and K^T tiles [64 dims][128 tokens] are MN-major
 // operands of the score MMA (instruction-descriptor bits 15 and 16), V^T [64 dims][128 keys] is the
 // K-major B operand of the second MMA.  Padded batches with L a multiple of 16 only.
+constexpr int kMaxSorted = 256;    // packed batches up to this many sequences are walked longest first
+
 template <bool PACKED, bool QT = false>
 __global__ void __launch_bounds__(kMaxThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
@@ -394,6 +396,26 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
     ptx::fence_mbar_init();
     ptx::tma_prefetch_desc(&map_qk);
   }
+  // Packed batches of up to 256 sequences are walked longest first: with work items of unequal length the
+  // order decides how evenly the CTAs finish (the sentence mix: -6 % per launch).  Every CTA ranks the
+  // sequences by length itself (the offsets are an input of the call, not a product of the kernel before
+  // this one, so this runs ahead of the dependency wait): s_order[rank] = sequence.
+  uint16_t* s_order = reinterpret_cast<uint16_t*>(s_tmem + 4);
+  const bool sorted = PACKED && a.B <= kMaxSorted;
+  if constexpr (PACKED) {
+    if (sorted) {
+      for (int i = tid; i < a.B; i += n_threads) {
+        const int len_i = __ldg(a.lens + i + 1) - __ldg(a.lens + i);
+        int rank = 0, prev = __ldg(a.lens);
+        for (int j = 0; j < a.B; ++j) {
+          const int cur = __ldg(a.lens + j + 1), len_j = cur - prev;
+          prev = cur;
+          rank += (len_j > len_i || (len_j == len_i && j < i)) ? 1 : 0;
+        }
+        s_order[rank] = (uint16_t)i;
+      }
+    }
+  }
   if (warp == 0) {
     ptx::tmem_alloc(ptx::smem_addr(s_tmem), a.tmem_cols);
     ptx::tmem_relinquish();
@@ -405,11 +427,17 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
   const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();              // the kernel that wrote qkv has completed
+  // sequence of a work item (items of one sequence are consecutive: its heads)
+  auto seq_of = [&](int item) {
+    const int s0 = item / a.heads;
+    if constexpr (PACKED) return sorted ? (int)s_order[s0] : s0;
+    else return s0;
+  };
 
   // (packed: the tensor maps see one "batch" of all rows; a sequence starts at row cu[batch], and
   // rows loaded past its end -- the next sequence's, or zero fill past the last row -- are masked)
   auto load_q = [&](int item, int qt, int buf) {
-    const int head = item % a.heads, batch = item / a.heads;
+    const int head = item % a.heads, batch = seq_of(item);
     const int row0 = PACKED ? __ldg(a.lens + batch) : 0, zb = PACKED ? 0 : batch;
     ptx::mbar_arrive_expect_tx(bar_q0 + 8 * buf, (uint32_t)slab_bytes);
     if constexpr (QT) ptx::tma_load_2d(ptx::smem_addr(sQ + buf * slab_bytes), &map_qk, bar_q0 + 8 * buf, batch * a.L + qt * 128, head * kHeadDim);
@@ -417,7 +445,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
     ptx::tma_load_3d(ptx::smem_addr(sQ + buf * slab_bytes), &map_qk, bar_q0 + 8 * buf, head * kHeadDim, row0 + qt * 128, zb);
   };
   auto load_k = [&](int item) {
-    const int head = item % a.heads, batch = item / a.heads;
+    const int head = item % a.heads, batch = seq_of(item);
     const int row0 = PACKED ? __ldg(a.lens + batch) : 0, zb = PACKED ? 0 : batch;
     ptx::mbar_arrive_expect_tx(bar_k, (uint32_t)(a.n_slabs * slab_bytes));
     for (int s = 0; s < a.n_slabs; ++s) {
@@ -427,7 +455,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
     }
   };
   auto load_v = [&](int item) {
-    const int head = item % a.heads, batch = item / a.heads;
+    const int head = item % a.heads, batch = seq_of(item);
     const int row0 = PACKED ? __ldg(a.lens + batch) : 0, zb = PACKED ? 0 : batch;
     ptx::mbar_arrive_expect_tx(bar_v, (uint32_t)(a.n_slabs * slab_bytes));
     for (int s = 0; s < a.n_slabs; ++s) {
@@ -457,7 +485,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_qk, const AttnArgs a) {
   int32_t* draw = a.status + 4;
   int next = 0;
   for (int item = blockIdx.x, iter = 0; item < total && ok; item = next, ++iter) {
-    const int head = item % a.heads, batch = item / a.heads;
+    const int head = item % a.heads, batch = seq_of(item);
     if constexpr (PACKED) {
       if (tid == 0) s_next[iter & 1] = (int)gridDim.x + atomicAdd(draw, 1);
     } else {
@@ -773,7 +801,8 @@ int launch_attention(ibert_ctx* ctx, const int8_t* qkv, int B, int L, int H, int
     }
     a.q_bufs = n_slabs > 1 ? 2 : 1;
     a.tmem_cols = cols; a.k = k; a.lens = cu_seqlens ? cu_seqlens : lens; a.out = out; a.status = ctx->d_status;
-    const int smem = a.q_bufs * slab + 2 * n_slabs * slab + n_slabs * 128 * 128 + 2 * 4 * 128 * 4 + 64 + 1024;
+    const int smem = a.q_bufs * slab + 2 * n_slabs * slab + n_slabs * 128 * 128 + 2 * 4 * 128 * 4 + 64 + 1024 +
+                     (cu_seqlens ? 2 * kMaxSorted : 0);      // (packed: the sequence order)
     // resident CTAs per SM: bounded by the register file (128 G threads of at most 128 registers),
     // by the 512 TMEM columns and by shared memory.  The bound must not exceed what TMEM allows:
     // a CTA that cannot get its columns would wait for a resident one to finish.

@@ -641,7 +641,10 @@ static int launch_layernorm_t(ibert_ctx* ctx, const QT* q, const int8_t* r, int6
     const int depth = 2;
     const size_t smem = (size_t)(kThreads / 32) * depth * (size_t)k.C * (sizeof(QT) + 1) + (kThreads / 32) * depth * 8 +
                         (size_t)k.C * 12;                  // rows in flight, barriers, the two tables
-    const int pgrid = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)ctx->num_sms * 3);
+    // one wave of resident CTAs: three per SM by registers, fewer when the row slots take more shared memory
+    // (C = 1024 with int32 input: two -- a grid of three per SM ran as a wave and a half)
+    const int per_sm = (int)std::min<size_t>(3, (size_t)(227 * 1024) / (smem + 1024));
+    const int pgrid = (int)std::min<int64_t>((rows + 7) / 8, (int64_t)ctx->num_sms * std::max(per_sm, 1));
 #define IBERT_LNP2(V, D, F)                                                                                 \
   do {                                                                                                      \
     static bool attr_dev[kMaxDevices] = {false};                                                            \

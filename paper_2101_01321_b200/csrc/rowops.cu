@@ -546,6 +546,69 @@ __global__ void __launch_bounds__(kThreads) gather_first_rows_kernel(const int8_
     *reinterpret_cast<uint4*>(out + (int64_t)b * H + c) = __ldg(reinterpret_cast<const uint4*>(src + c));
 }
 
+// Short rows (L <= 128, a multiple of 4: one 16-byte vector per lane): a warp takes R rows at a time.  The one
+// true division a row needs (Algorithm 3's quotient by the row sum, made a multiplication for its elements)
+// costs about as much as the rest of a 128-element row; lane r performs it for row r, so one division
+// instruction stream serves R rows, and the R loads of a lane are in flight together.
+template <int R, int DIV>
+__global__ void __launch_bounds__(kThreads, 4) softmax_short_kernel(const int32_t* __restrict__ q, int64_t rows,
+                                                                 int L, ExpConsts k, uint8_t* __restrict__ out,
+                                                                 const uint32_t* __restrict__ table) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp_global = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int64_t warp_count = ((int64_t)gridDim.x * kThreads) >> 5;
+  const int col = 4 * lane;
+  const bool in_row = col < L;
+  for (int64_t row0 = warp_global * R; row0 < rows; row0 += warp_count * R) {
+    int32_t v[R][4];
+    uint32_t sums[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      if (in_row && row0 + r < rows) {
+        const int4 t = __ldcs(reinterpret_cast<const int4*>(q + (row0 + r) * L + col));
+        v[r][0] = t.x; v[r][1] = t.y; v[r][2] = t.z; v[r][3] = t.w;
+      } else {
+        v[r][0] = v[r][1] = v[r][2] = v[r][3] = INT32_MIN;
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      int32_t mx = max(max(v[r][0], v[r][1]), max(v[r][2], v[r][3]));
+      mx = __reduce_max_sync(0xffffffffu, mx);
+      uint32_t sum = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t dist = (uint32_t)mx - (uint32_t)v[r][i];
+        uint32_t e = 0u;
+        if (in_row && row0 + r < rows) {
+          if constexpr (DIV == kExpByTable) e = __ldg(table + min(dist >> k.s_in, k.d_max));
+          else e = iexp_dist<DIV>(dist, k);
+        }
+        v[r][i] = (int32_t)e;
+        sum += e;
+      }
+      sums[r] = max(__reduce_add_sync(0xffffffffu, sum), 1u);     // (0 only for a row past the end)
+    }
+    uint32_t my_sum = sums[0];
+#pragma unroll
+    for (int r = 1; r < R; ++r) my_sum = lane == r ? sums[r] : my_sum;
+    const uint32_t my_m = make_row_divisor(my_sum, k.p_max).m;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      RowDivisor rd;
+      rd.m = __shfl_sync(0xffffffffu, my_m, r);
+      const int K = 21 + 32 - __clz(sums[r]);
+      rd.pre = K < 32 ? 32 - K : 0;
+      rd.post = K < 32 ? 0 : K - 32;
+      uint32_t p[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) p[i] = softmax_quotient((uint32_t)v[r][i], rd);
+      if (in_row && row0 + r < rows)
+        __stcs(reinterpret_cast<uint32_t*>(out + (row0 + r) * L + col), p[0] | (p[1] << 8) | (p[2] << 16) | (p[3] << 24));
+    }
+  }
+}
+
 int grid_for(ibert_ctx* ctx, int64_t work_warps, int max_ctas_per_sm) {
   const int64_t ctas = (work_warps + (kThreads / 32) - 1) / (kThreads / 32);
   const int64_t cap = (int64_t)ctx->num_sms * max_ctas_per_sm;
@@ -619,7 +682,15 @@ int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const 
     else if (div == 2) IBERT_SM2(V, 2); \
     else IBERT_SM2(V, kExpByTable);     \
   } while (0)
-  if (vpl <= 1) IBERT_SM(1);
+  if (vpl <= 1 && vec) {
+    constexpr int R = 4;
+    const int sgrid = grid_for(ctx, (rows + R - 1) / R, 4);      // (one wave: four CTAs are resident per SM)
+    if (div == 0) softmax_short_kernel<R, 0><<<sgrid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out, exp_table);
+    else if (div == 1) softmax_short_kernel<R, 1><<<sgrid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out, exp_table);
+    else if (div == 2) softmax_short_kernel<R, 2><<<sgrid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out, exp_table);
+    else softmax_short_kernel<R, kExpByTable><<<sgrid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out, exp_table);
+  }
+  else if (vpl <= 1) IBERT_SM(1);
   else if (vpl <= 2) IBERT_SM(2);
   else if (vpl <= 4) IBERT_SM(4);
   else IBERT_SM(8);

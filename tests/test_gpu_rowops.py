@@ -34,7 +34,8 @@ def test_gelu_full_int32_range_and_odd_scales():
 
 
 @pytest.mark.parametrize("rows,L", [(5, 1), (9, 7), (33, 64), (17, 65), (96 * 8, 128), (64, 256), (40, 512),
-                                    (7, 1000), (12, 1024), (3, 130), (0, 128)])
+                                    (7, 1000), (12, 1024), (3, 130), (0, 128),
+                                    (6, 4), (1, 128), (1027, 100), (2, 124)])   # short rows: four rows per warp
 @pytest.mark.parametrize("p_max", [255, 127])
 def test_softmax_matches_oracle(rows, L, p_max):
     for sigma in (1.0, 4.0):

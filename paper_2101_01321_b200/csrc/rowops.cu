@@ -615,6 +615,15 @@ int grid_for(ibert_ctx* ctx, int64_t work_warps, int max_ctas_per_sm) {
   return (int)(ctas < 1 ? 1 : (ctas > cap ? cap : ctas));
 }
 
+// grid of at most one wave of resident CTAs of `kernel` (its registers decide how many an SM holds: a larger
+// grid of grid-stride CTAs runs as a full wave plus a partial one)
+template <typename Kernel>
+int wave_grid(ibert_ctx* ctx, Kernel kernel, int64_t work_warps) {
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+  return grid_for(ctx, work_warps, std::min(per_sm, 8));
+}
+
 int check_launch() { return cudaGetLastError() == cudaSuccess ? IBERT_OK : IBERT_ERR_CUDA; }
 
 }  // namespace
@@ -647,14 +656,14 @@ int launch_gelu_table(ibert_ctx* ctx, const GeluConsts& k, int32_t* ramp_scratch
 int launch_gelu_lut(ibert_ctx* ctx, const int32_t* q, int64_t n, const int8_t* table, int8_t* out) {
   if (n == 0) return IBERT_OK;
   const int64_t warps = ((n >> 2) + 31) / 32 / 8 + 1;          // ~8 vectors per thread
-  gelu_lut_kernel<<<grid_for(ctx, warps, 8), kThreads, 0, ctx->stream>>>(q, n, table, out);
+  gelu_lut_kernel<<<wave_grid(ctx, gelu_lut_kernel, warps), kThreads, 0, ctx->stream>>>(q, n, table, out);
   return check_launch();
 }
 
 int launch_gelu(ibert_ctx* ctx, const int32_t* q, int64_t n, const GeluConsts& k, int8_t* out) {
   if (n == 0) return IBERT_OK;
   const int64_t warps = ((n >> 2) + 127) / 128 + 1;
-  gelu_kernel<<<grid_for(ctx, warps, 8), kThreads, 0, ctx->stream>>>(q, n, k, out);
+  gelu_kernel<<<wave_grid(ctx, gelu_kernel, warps), kThreads, 0, ctx->stream>>>(q, n, k, out);
   return check_launch();
 }
 
@@ -666,14 +675,13 @@ int launch_exp_table(ibert_ctx* ctx, const ExpConsts& k, uint32_t* table) {
 int launch_softmax(ibert_ctx* ctx, const int32_t* q, int64_t rows, int L, const ExpConsts& k, uint8_t* out,
                    const uint32_t* exp_table) {
   if (rows == 0) return IBERT_OK;
-  const int grid = grid_for(ctx, rows, 8);
   const bool vec = (L % 4) == 0;
   const int vpl = (L + 127) / 128;   // vectors per lane
   const int div = exp_table ? kExpByTable : exp_div_mode(k);
 #define IBERT_SM2(V, D)                                                                                       \
   do {                                                                                                        \
-    if (vec) softmax_kernel<V, true, D><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out, exp_table);   \
-    else softmax_kernel<V, false, D><<<grid, kThreads, 0, ctx->stream>>>(q, rows, L, k, out, exp_table);      \
+    if (vec) softmax_kernel<V, true, D><<<wave_grid(ctx, softmax_kernel<V, true, D>, rows), kThreads, 0, ctx->stream>>>(q, rows, L, k, out, exp_table);   \
+    else softmax_kernel<V, false, D><<<wave_grid(ctx, softmax_kernel<V, false, D>, rows), kThreads, 0, ctx->stream>>>(q, rows, L, k, out, exp_table);      \
   } while (0)
 #define IBERT_SM(V)                 \
   do {                              \
@@ -703,7 +711,6 @@ template <typename QT>
 static int launch_layernorm_t(ibert_ctx* ctx, const QT* q, const int8_t* r, int64_t rows, const LnConsts& k,
                               const int32_t* d_b, const int64_t* d_B, int8_t* out) {
   if (rows == 0) return IBERT_OK;
-  const int grid = grid_for(ctx, rows, 8);
   const bool vec = (k.C % 4) == 0;
   const int vpl = (k.C + 127) / 128;
   const bool fast = vec && k.out_fast && (!k.has_res || k.res_fast);
@@ -744,9 +751,9 @@ static int launch_layernorm_t(ibert_ctx* ctx, const QT* q, const int8_t* r, int6
   }
 #define IBERT_LN(V)                                                                                              \
   do {                                                                                                           \
-    if (fast) layernorm_kernel<V, true, true, QT><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);  \
-    else if (vec) layernorm_kernel<V, true, false, QT><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out); \
-    else layernorm_kernel<V, false, false, QT><<<grid, kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);     \
+    if (fast) layernorm_kernel<V, true, true, QT><<<wave_grid(ctx, layernorm_kernel<V, true, true, QT>, rows), kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);  \
+    else if (vec) layernorm_kernel<V, true, false, QT><<<wave_grid(ctx, layernorm_kernel<V, true, false, QT>, rows), kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out); \
+    else layernorm_kernel<V, false, false, QT><<<wave_grid(ctx, layernorm_kernel<V, false, false, QT>, rows), kThreads, 0, ctx->stream>>>(q, r, rows, k, d_b, d_B, out);     \
   } while (0)
   if (vpl <= 2) IBERT_LN(2);
   else if (vpl <= 4) IBERT_LN(4);

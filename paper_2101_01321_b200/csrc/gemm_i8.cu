@@ -328,8 +328,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // (+2 us on the QKV GEMM).  Otherwise a tile is reused two chunks later.  Either way the
         // store that last read this staging tile must have finished reading it.
         constexpr bool kOneStore = !kOut32 && C::kChunksPerWarp == 2 && KIND != EPI_INT8 && !epi_transposed(KIND);
-        if (!kOneStore || ci == 0) {
-          if (lane == 0) { if constexpr (kOneStore) ptx::bulk_wait_read<0>(); else ptx::bulk_wait_read<1>(); }
+        // the same for the transposed GELU kinds: the warp's 32 channels x 64 tokens leave as one 2 KB block
+        constexpr bool kOneStoreT = C::kChunksPerWarp == 2 && (KIND == kEpiGeluTableT || KIND == kEpiGeluTableWideT);
+        if (!(kOneStore || kOneStoreT) || ci == 0) {
+          if (lane == 0) { if constexpr (kOneStore || kOneStoreT) ptx::bulk_wait_read<0>(); else ptx::bulk_wait_read<1>(); }
           __syncwarp();
         }
         uint8_t* stage = stage0 + (kOneStore ? ci : (int)buf) * C::kOutTileBytes;
@@ -385,9 +387,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             w[j] = KIND == kEpiInt8T
                        ? pack4_sat_s8((int32_t)v[4 * j], (int32_t)v[4 * j + 1], (int32_t)v[4 * j + 2], (int32_t)v[4 * j + 3])
                        : __byte_perm(__byte_perm(v[4 * j], v[4 * j + 1], 0x0040), __byte_perm(v[4 * j + 2], v[4 * j + 3], 0x0040), 0x5410);   // table bytes
+          if constexpr (kOneStoreT) {
+            // rows of 64 tokens = four 16-byte chunks, placed by the 64-byte swizzle (chunk index XOR bits 1..2
+            // of the row); this 32-token chunk fills chunks 2 ci and 2 ci + 1
+            const uint32_t sw = ((uint32_t)lane >> 1) & 3u, c0 = 2u * (uint32_t)ci;
+            *reinterpret_cast<uint4*>(stage0 + lane * 64 + ((c0 ^ sw) * 16u)) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(stage0 + lane * 64 + (((c0 + 1u) ^ sw) * 16u)) = make_uint4(w[4], w[5], w[6], w[7]);
+          } else {
           const uint32_t sw = ((uint32_t)lane >> 2) & 1u;
           *reinterpret_cast<uint4*>(stage + lane * 32 + sw * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
           *reinterpret_cast<uint4*>(stage + lane * 32 + (sw ^ 1u) * 16u) = make_uint4(w[4], w[5], w[6], w[7]);
+          }
         } else
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
@@ -399,11 +409,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           else  // low byte of the register, stored without a narrowing conversion
             asm volatile("st.shared.u8 [%0], %1;" ::"r"(ptx::smem_addr(stage) + i * 32 + lane), "r"(o) : "memory");
         }
-        if (!kOneStore || ci == 1) {
+        if (!(kOneStore || kOneStoreT) || ci == 1) {
           ptx::fence_proxy_async_smem();               // staging writes -> visible to the TMA engine
           __syncwarp();
           if (lane == 0) {
-            if constexpr (kOneStore) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage0), ch0, t0);
+            if constexpr (kOneStoreT) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage0), t0, ch0);
+            else if constexpr (kOneStore) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage0), ch0, t0);
             else if constexpr (epi_transposed(KIND)) ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), t0 + ci * 32, ch0);
             else ptx::tma_store_2d(&map_out, ptx::smem_addr(stage), ch0 * C::kOutElem, t0 + ci * 32);
             ptx::bulk_commit();
@@ -547,8 +558,9 @@ int launch_gemm_i8(ibert_ctx* ctx, const int8_t* x, const int8_t* w, int64_t M, 
       // out^T [N][M]: one box = 32 channels x 32 tokens, rows of 32 bytes, 32-byte swizzle
       const uint64_t tdims[2] = {(uint64_t)M, (uint64_t)N};
       const uint64_t tstr[1] = {(uint64_t)M};
-      const uint32_t tbox[2] = {32u, 32u};
-      if ((rc = encode_tensor_map(&mo, out, 2, tdims, tstr, tbox, 32))) return rc;
+      // (the GELU kinds store a warp's 64 tokens at once: rows of 64 bytes, 64-byte swizzle)
+      const uint32_t tbox[2] = {gelu_kind ? 64u : 32u, 32u};
+      if ((rc = encode_tensor_map(&mo, out, 2, tdims, tstr, tbox, gelu_kind ? 64 : 32))) return rc;
     }
   }
   GemmArgs a{};
